@@ -1,0 +1,244 @@
+/*
+ * edg_moe.h -- C ABI of the streaming-MoE per-layer decode step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one thing: the routed-expert block of a streaming mixture-of-experts
+ * decoder as the paper states it (Sec. 3 "System Design" and Appendix A "Routing Math"):
+ *
+ *   a1  prerouter logits       l = W_pre . s                       (Sec. 3.2 "Head", linear path)
+ *   a2  softmax top-k          g = softmax(l), inds = top-k(g, K),
+ *                              w = g[inds] / sum g[inds]            (Appendix A, softmax-topk)
+ *   a3  slot map + staging     slots = take(slot_table, inds); only missing experts are copied
+ *                              into a fixed pool of sticky slots     (Sec. 3.1, "staged" path)
+ *   a4  gate/up                h = silu(gate(x)) * up(x)            (Sec. 3.1 "Math contract")
+ *   a5  down                   o = down(h)
+ *       every projection is  W_int4(x) + (alpha/r) B A x,  W dequantised on the fly and the
+ *       LoRA delta added as a parallel branch, never merged          (Sec. 3.3, Fig. 1 caption)
+ *   a6  reduce                 y = sum_k w_k o_k                    (Appendix A weights)
+ *
+ * Conventions
+ *   - Plain C: pointers and sizes only.  "dev" = device (HBM) pointer, "host" = host pointer,
+ *     "pinned" = page-locked host memory.  Streams are cudaStream_t passed as void*.
+ *   - Every call returns an int32 status: EDG_OK or a negative EDG_E_* code.  Nothing throws.
+ *   - The caller owns every buffer and every stream.  The library owns only the opaque store
+ *     handle (allocator state, CUDA events, a small pinned ring for slot-table updates).
+ *   - Device work is asynchronous on the stream given.  The hot calls (prerouter_topk,
+ *     moe_expert_ffn_int4_lora, moe_layer_decode) neither allocate nor synchronise with the host.
+ *   - Device pointers must be 16-byte aligned; slot records must be 256-byte aligned (the record
+ *     size is always a multiple of 256).
+ *   - bf16 and fp16 values are passed as their 16-bit patterns.
+ *
+ * Quantised weight format (Sec. 3.1: int4, group-wise affine, one scale and one second parameter
+ * per group of `group` consecutive input elements):  w[n][k] = scale[n][k/group] * (q[n][k] -
+ * zero[n][k/group]),  q in 0..15, scale and zero stored as fp16.  Canonical interchange layout:
+ * row-major [out][in]; byte j of a row holds q[2j] in its low nibble and q[2j+1] in its high nibble.
+ * One expert = gate [I][H], up [I][H], down [H][I].  edg_pack_expert turns canonical tensors into
+ * the record the kernels read; its size is edg_record_bytes (1,769,472 B at H=2048, I=512,
+ * group 64 -- the paper's 1.77 MB per expert).
+ */
+#ifndef EDG_MOE_H
+#define EDG_MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define EDG_OK          0
+#define EDG_E_INVAL    -1   /* null pointer, misaligned pointer, bad enum, bad handle            */
+#define EDG_E_SHAPE    -2   /* a dimension the kernels do not support (see edg_check_desc)     */
+#define EDG_E_SLOTS    -3   /* more experts to stage than slots in the pool                     */
+#define EDG_E_RANGE    -4   /* expert / layer / slot index out of range, or duplicate expert    */
+#define EDG_E_CUDA     -5   /* a CUDA runtime call failed; see edg_last_cuda_error              */
+#define EDG_E_TIMEOUT  -6   /* a bounded host wait ran out                                      */
+#define EDG_E_WORKSPACE -7  /* workspace too small or misaligned                                */
+
+/* dtypes */
+#define EDG_F32   0
+#define EDG_F16   1
+#define EDG_BF16  2
+
+/* Shape of one MoE layer: the paper's model spec (expert count, K, quantisation, ...), Sec. 3. */
+typedef struct edg_layer_desc {
+    int32_t H;           /* hidden size                                                          */
+    int32_t I;           /* expert intermediate size                                             */
+    int32_t E;           /* experts per layer                                                    */
+    int32_t K;           /* experts routed per token (top-k)                                     */
+    int32_t group;       /* quantisation group size along the input dimension                    */
+    int32_t rank;        /* LoRA rank r (0 = no adapter)                                         */
+    int32_t n_adapters;  /* 1: one adapter shared by all experts of the layer; E: one per expert */
+    int32_t n_slots;     /* slots per layer in the HBM pool                                      */
+    int32_t pre_dtype;   /* storage type of the prerouter head: EDG_F32 or EDG_F16               */
+    int32_t out_dtype;   /* type of y: EDG_F32, EDG_F16 or EDG_BF16                              */
+    float   lora_scale;  /* alpha / r                                                            */
+} edg_layer_desc;
+
+/* Unmerged LoRA factors of one layer, bf16, all dev.  Leading dimension n_adapters.
+ * A maps the projection's input to rank r, B maps rank r to its output (Sec. 3.3). */
+typedef struct edg_lora {
+    const void* A_gate;  /* [n_adapters][rank][H] */
+    const void* B_gate;  /* [n_adapters][I][rank] */
+    const void* A_up;    /* [n_adapters][rank][H] */
+    const void* B_up;    /* [n_adapters][I][rank] */
+    const void* A_down;  /* [n_adapters][rank][I] */
+    const void* B_down;  /* [n_adapters][H][rank] */
+} edg_lora;
+
+typedef struct edg_store edg_store;   /* opaque slot-pool expert store */
+
+typedef struct edg_store_stats {
+    int64_t stage_calls;    /* calls of stage_experts_to_slots                     */
+    int64_t hits;           /* staged experts already resident (nothing copied)    */
+    int64_t misses;         /* staged experts copied host -> HBM                   */
+    int64_t bytes_copied;   /* misses * record bytes                               */
+    int64_t table_updates;  /* device slot-table rows rewritten                    */
+} edg_store_stats;
+
+/* ---------------------------------------------------------------- utilities (host, synchronous) */
+
+/* Version of this ABI (major * 1000 + minor). */
+int32_t edg_version(void);
+
+/* Last cudaError_t seen by this library on the calling thread (0 = none), and its text. */
+int32_t edg_last_cuda_error(void);
+const char* edg_last_cuda_error_string(void);
+
+/* Checks a descriptor against what the kernels support: H and I multiples of 128 and at most
+ * 4096 with H/32 and I/32 a power of two; group a multiple of 32 dividing H and I; 1 <= K <= 32;
+ * K <= E <= 1024; 0 <= rank <= 64; n_adapters 1 or E; n_slots >= 1.  Returns EDG_OK or EDG_E_SHAPE. */
+int32_t edg_check_desc(const edg_layer_desc* desc);
+
+/* Bytes of one expert record: 3*H*I/2 code bytes + 3*(H*I/group) (scale, zero) fp16 pairs. */
+int32_t edg_record_bytes(const edg_layer_desc* desc, size_t* bytes);
+
+/* One-time host repack of canonical tensors (layout above; scales/zeros as fp16 bit patterns,
+ * [out][in/group]) into the record the kernels read.  `record` is host memory of
+ * edg_record_bytes bytes.  Never on the hot path.  edg_unpack_expert is its exact inverse. */
+int32_t edg_pack_expert(const edg_layer_desc* desc,
+                        const uint8_t* codes_gate, const uint16_t* scales_gate, const uint16_t* zeros_gate,
+                        const uint8_t* codes_up,   const uint16_t* scales_up,   const uint16_t* zeros_up,
+                        const uint8_t* codes_down, const uint16_t* scales_down, const uint16_t* zeros_down,
+                        void* record);
+int32_t edg_unpack_expert(const edg_layer_desc* desc, const void* record,
+                          uint8_t* codes_gate, uint16_t* scales_gate, uint16_t* zeros_gate,
+                          uint8_t* codes_up,   uint16_t* scales_up,   uint16_t* zeros_up,
+                          uint8_t* codes_down, uint16_t* scales_down, uint16_t* zeros_down);
+
+/* Bytes of device scratch the FFN calls need for T tokens (T = 1 for batch-1 decode). */
+int32_t edg_ffn_workspace_bytes(const edg_layer_desc* desc, int32_t T, size_t* bytes);
+
+/* Reads the device-side status word that the kernels keep at the start of a workspace: 0, or an
+ * EDG_E_RANGE raised by a slot or expert index outside its range (the kernel skips that access
+ * instead of faulting).  Synchronises `stream`. */
+int32_t edg_workspace_status(const void* workspace, void* stream, int32_t* status);
+
+/* ---------------------------------------------------------------- a1 + a2: prerouter */
+
+/* Prerouter head + routing (Sec. 3.2; Appendix A softmax-topk), for n_heads independent
+ * (head, hidden state) pairs in one launch -- the "single flush per step" that predicts every
+ * staged layer at once.
+ *   W_pre   dev [n_heads][E][H], pre_dtype           s       dev bf16 [n_heads][H]
+ *   inds    dev int32 [n_heads][K], ascending expert index, distinct
+ *   gates   dev float [n_heads][K], aligned with inds, sum to 1
+ *   logits_opt  dev float [n_heads][E] or NULL: the fp32 logits the selection was made on
+ * Equal logits go to the lower expert index. */
+int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
+                       int32_t* inds, float* gates, float* logits_opt, void* stream);
+
+/* a2 alone on given logits (a router's own gate at prefill): logits dev float [T][E] ->
+ * inds dev int32 [T][K], gates dev float [T][K].  Same ordering and tie rule. */
+int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,
+                          int32_t* inds, float* gates, void* stream);
+
+/* ---------------------------------------------------------------- a3: slot-pool expert store */
+
+/* Creates the store of n_layers layers (Sec. 3.1 "staged" path; Fig. 1: bounded streaming pool
+ * with fixed staged slots).
+ *   host_layers  host array of n_layers pointers, each to pinned [E][record bytes] (the tier that
+ *                stands in for the paper's SSD); layers may alias
+ *   dev_slots    dev [n_layers][n_slots][record bytes]
+ *   dev_tables   dev int32 [n_layers][E]: slot of each expert, -1 if not resident; the store
+ *                initialises it and keeps it current
+ *   loras        host array of n_layers edg_lora (copied), or NULL for no adapter
+ *   copy_stream  side stream the staging copies run on
+ * Allocates events and a small pinned ring; not a hot call. */
+int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
+                         void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
+                         void* copy_stream, edg_store** out);
+int32_t edg_store_destroy(edg_store* store);
+int32_t edg_store_get_stats(const edg_store* store, edg_store_stats* out);
+
+/* Host side of a3.  `inds_host` holds n distinct experts (n <= n_slots; n = K for one token, up to
+ * the union of a batch).  Experts already resident keep their slot and copy nothing (sticky slots);
+ * each missing expert, in the order given, replaces the least recently used slot that this call
+ * does not need.  For every miss one cudaMemcpyAsync host->HBM is enqueued on the copy stream,
+ * after the layer's last compute (ordered by an event), followed by the slot-table row update and
+ * the layer's copy-done event.  Hits enqueue nothing.  Returns the slots (aligned with inds_host)
+ * and the number of misses.  The prediction is consumed as the routing, so the staged set equals
+ * the routed set by construction (Sec. 3.2 "Prediction-as-routing"). */
+int32_t stage_experts_to_slots(edg_store* store, int32_t layer, const int32_t* inds_host, int32_t n,
+                               int32_t* slots_host_out, int32_t* n_miss_out);
+
+/* Host copy of a layer's tables, for inspection: expert_of_slot [n_slots], slot_of_expert [E]
+ * (either may be NULL). */
+int32_t edg_store_snapshot(const edg_store* store, int32_t layer, int32_t* expert_of_slot, int32_t* slot_of_expert);
+
+/* Ordering hooks for callers that run the FFN themselves instead of through moe_layer_decode
+ * (batched decode, prefill): edg_store_wait_staged makes `stream` wait for the layer's pending
+ * staging copies (no-op when none are pending); edg_store_mark_computed tells the store that
+ * everything enqueued on `stream` so far must finish before the layer's slots may be overwritten
+ * (no-op for a pool that never evicts, n_slots == E). */
+int32_t edg_store_wait_staged(edg_store* store, int32_t layer, void* stream);
+int32_t edg_store_mark_computed(edg_store* store, int32_t layer, void* stream);
+
+/* ---------------------------------------------------------------- a4-a6: expert FFN */
+
+/* y = sum_k gates[k] * down_k( silu(gate_k(x)) * up_k(x) ), each projection = int4 base
+ * dequantised on the fly + lora_scale * B (A .) (Sec. 3.1 "Math contract", Sec. 3.3), over
+ * exactly the K given slots, summed in the order given.
+ *   slot_pool   dev: n_slots records of one layer
+ *   slot_table  dev int32 [E] or NULL.  NULL: `slots` holds slot indices in [0, n_slots).
+ *               Non-NULL: `slots` holds expert ids, mapped on the device through the table
+ *               (the paper's take; the indices never leave the GPU)
+ *   slots       dev int32 [T][K]
+ *   experts     dev int32 [T][K] expert ids, read only to pick per-expert adapters when
+ *               n_adapters == E and slot_table is NULL; may be NULL otherwise
+ *   gates       dev float [T][K]                        x       dev bf16 [T][H]
+ *   lora        host struct of dev pointers, or NULL for no adapter
+ *   y           dev [T][H] of out_dtype
+ *   workspace   dev, edg_ffn_workspace_bytes(desc, T) bytes, 256-byte aligned; holds the
+ *               intermediate h and the rank-r projections.  Its first 256 bytes are a control
+ *               block (sticky status word, see edg_workspace_status) that the caller zeroes once
+ *               before first use; the rest needs no initialisation.  Calls that share a
+ *               workspace must be ordered on the device.
+ * An index outside its range makes the kernels skip that expert and raise the status word; no
+ * out-of-range address is ever formed.
+ * T = 1 is batch-1 decode (fused dequant GEMV kernels).  T > 1 is batched decode / prefill. */
+int32_t moe_expert_ffn_int4_lora(const edg_layer_desc* desc, const void* slot_pool, const int32_t* slot_table,
+                                 int32_t T, const int32_t* slots, const int32_t* experts, const float* gates,
+                                 const void* x, const edg_lora* lora, void* y,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------- the whole layer-step */
+
+/* One layer-step of batch-1 decode (Sec. 3.2 "Motivation": the double shift).  On `stream`:
+ * waits for the layer's staging copies, maps inds_cur through the layer's device slot table (take;
+ * the indices never leave the GPU), runs a4-a6 for the current token with the routing predicted one
+ * token earlier, and evaluates the head W_pre_next on the same hidden state to predict the next
+ * layer-step's routing (a1-a2); then marks the layer's slots free for restaging.
+ *   x dev bf16 [H]; inds_cur dev int32 [K]; gates_cur dev float [K];
+ *   W_pre_next dev [E][H] (NULL skips the prediction); inds_next dev int32 [K];
+ *   gates_next dev float [K]; logits_next_opt dev float [E] or NULL; y dev [H] of out_dtype;
+ *   workspace as for moe_expert_ffn_int4_lora with T = 1. */
+int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
+                         const int32_t* inds_cur, const float* gates_cur,
+                         const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                         float* logits_next_opt, void* y,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EDG_MOE_H */

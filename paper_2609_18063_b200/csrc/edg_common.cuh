@@ -1,0 +1,183 @@
+// Shared host/device helpers of the streaming-MoE decode library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/edg_moe.h"
+
+namespace edg {
+
+// ---------------------------------------------------------------- host: errors
+
+void set_cuda_error(cudaError_t e);            // records the error for edg_last_cuda_error
+#define EDG_CUDA_TRY(expr)                                                   \
+    do {                                                                     \
+        cudaError_t _e = (expr);                                             \
+        if (_e != cudaSuccess) { ::edg::set_cuda_error(_e); return EDG_E_CUDA; } \
+    } while (0)
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// ---------------------------------------------------------------- record layout
+// One expert record: [gate codes][up codes][down codes][gate sz][up sz][down sz].
+// Codes are row-major int4, low nibble first; sz is one (scale, zero) fp16 pair per group,
+// row-major [out][in/group].  All section offsets are multiples of 256 bytes for the shapes
+// edg_check_desc admits.
+struct RecordLayout {
+    uint32_t codes_gate, codes_up, codes_down;   // byte offsets
+    uint32_t sz_gate, sz_up, sz_down;
+    uint32_t bytes;
+};
+
+__host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
+    RecordLayout L;
+    const uint32_t c = (uint32_t)H * (uint32_t)I / 2u;
+    const uint32_t s = (uint32_t)H * (uint32_t)I / (uint32_t)group * 4u;
+    L.codes_gate = 0;
+    L.codes_up = c;
+    L.codes_down = 2 * c;
+    L.sz_gate = 3 * c;
+    L.sz_up = 3 * c + s;
+    L.sz_down = 3 * c + 2 * s;
+    L.bytes = 3 * c + 3 * s;
+    return L;
+}
+
+// Workspace layout for T tokens (floats unless noted).  The first 256 bytes are a control block
+// whose first int32 is the device-side status word.
+struct WorkspaceLayout {
+    size_t ctrl;      // 256 B control block
+    size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
+    size_t h;         // [T][K][I] float            : silu(gate) * up
+    size_t u_d;       // [T][K][rank] float         : A_down h
+    size_t bytes;
+};
+
+__host__ __device__ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
+    WorkspaceLayout W;
+    const size_t n_sets = d.n_adapters == 1 ? 1 : (size_t)d.K;
+    const size_t r = d.rank > 0 ? (size_t)d.rank : 1;
+    W.ctrl = 0;
+    W.u_gu = 256;
+    W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
+    W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
+    W.bytes = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
+    return W;
+}
+
+int32_t check_desc(const edg_layer_desc* d);   // EDG_OK or EDG_E_INVAL / EDG_E_SHAPE
+
+// ---------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+// bf16 pair packed in one 32-bit word (low half = first element)
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Sum over aligned groups of LPR lanes (LPR a power of two <= 32).
+template <int LPR>
+__device__ __forceinline__ float group_sum(float v) {
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// ---- int4 -> fp32 without conversion instructions.
+//
+// A float whose exponent field is 0 or 1 has the value (bit pattern) * 2^-149, so masking one
+// nibble of a packed word in place gives q * 2^(4p - 149) exactly for nibble positions p = 0..5
+// (bits 0..23).  Nibbles 6 and 7 are brought to positions 4 and 5 by one shift.  The matching
+// activation is pre-multiplied by 2^(XS - 4p), so every product is q * x * 2^(XS - 149) and the
+// running sum is an ordinary fp32 dot product of exact integer codes with x, scaled by a power
+// of two.  The zero point and the scale are applied per 32-code chunk on the fp32 partial sum:
+//     sum_k s (q_k - z) x_k = s * (sum_k q_k x_k - z * sum_k x_k).
+// Requires subnormal inputs to be honoured (no -ftz, no --use_fast_math).
+constexpr int XS = 100;                                  // activation pre-scale exponent
+__device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }
+
+// position of nibble j (0..7) after the masks below, and the exponent its activation carries
+__device__ __forceinline__ int nibble_pos(int j) { return j < 6 ? j : j - 2; }
+
+// xs[j] for a 32-code chunk: x_j * 2^(XS - 4 pos(j % 8)).  Returns sum_j x_j * 2^(XS - 149).
+__device__ __forceinline__ float scale_chunk(const float (&x)[32], float (&xs)[32]) {
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        xs[j] = x[j] * pow2f(XS - 4 * nibble_pos(j & 7));
+        sum += x[j];
+    }
+    return sum * pow2f(XS - 149);
+}
+
+__device__ __forceinline__ void word_fma(uint32_t w, const float* xs, float& a, float& b) {
+    const uint32_t w2 = w >> 8;
+    a = fmaf(__uint_as_float(w & 0x0000000Fu), xs[0], a);
+    b = fmaf(__uint_as_float(w & 0x000000F0u), xs[1], b);
+    a = fmaf(__uint_as_float(w & 0x00000F00u), xs[2], a);
+    b = fmaf(__uint_as_float(w & 0x0000F000u), xs[3], b);
+    a = fmaf(__uint_as_float(w & 0x000F0000u), xs[4], a);
+    b = fmaf(__uint_as_float(w & 0x00F00000u), xs[5], b);
+    a = fmaf(__uint_as_float(w2 & 0x000F0000u), xs[6], a);
+    b = fmaf(__uint_as_float(w2 & 0x00F00000u), xs[7], b);
+}
+
+// 2^(XS-149) * sum_{j<32} q_j x_j for one 16-byte chunk of codes.
+__device__ __forceinline__ float chunk_dot(const uint4& c, const float (&xs)[32]) {
+    float a = 0.f, b = 0.f;
+    word_fma(c.x, xs + 0, a, b);
+    word_fma(c.y, xs + 8, a, b);
+    word_fma(c.z, xs + 16, a, b);
+    word_fma(c.w, xs + 24, a, b);
+    return a + b;
+}
+
+// s * (qx - z * xsum): one chunk's contribution, still scaled by 2^(XS-149).  sz = (scale, zero) fp16 pair.
+__device__ __forceinline__ float chunk_affine(float qx, float xsum, uint32_t sz) {
+    const __half2 h = *reinterpret_cast<const __half2*>(&sz);
+    const float2 f = __half22float2(h);
+    return f.x * fmaf(-f.y, xsum, qx);
+}
+
+constexpr float kUnscale = 562949953421312.0f;           // 2^(149 - XS) = 2^49
+
+__device__ __forceinline__ float silu_f(float v) { return v / (1.f + __expf(-v)); }
+
+// read-only 16-byte / 4-byte loads that do not pollute L1 (weights are streamed once)
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_stream4(const void* p) {
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+template <typename T> __device__ __forceinline__ void store_out(T* y, size_t i, float v);
+template <> __device__ __forceinline__ void store_out<float>(float* y, size_t i, float v) { y[i] = v; }
+template <> __device__ __forceinline__ void store_out<__half>(__half* y, size_t i, float v) { y[i] = __float2half_rn(v); }
+struct bf16_t { uint16_t bits; };
+template <> __device__ __forceinline__ void store_out<bf16_t>(bf16_t* y, size_t i, float v) {
+    uint32_t u = __float_as_uint(v);
+    u += 0x7FFFu + ((u >> 16) & 1u);                      // round to nearest even (finite inputs)
+    y[i].bits = (uint16_t)(u >> 16);
+}
+
+#endif  // __CUDACC__
+
+}  // namespace edg

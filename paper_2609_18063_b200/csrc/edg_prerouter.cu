@@ -1,0 +1,196 @@
+// a1 + a2: prerouter head logits, softmax, top-k and renormalised gate weights
+// (Sec. 3.2 "Head" linear path; Appendix A softmax-topk).
+//
+// One thread-block cluster per head: the E rows of the head are split over the CTAs of the
+// cluster, every CTA writes its logits straight into the leader CTA's shared memory
+// (distributed shared memory), and after one cluster barrier a single warp of the leader does
+// softmax + top-k with warp shuffles.  No global scratch, no atomics, one launch.
+#include <cooperative_groups.h>
+#include <math_constants.h>
+
+#include "edg_common.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace edg {
+
+constexpr int kPreCluster = 8;      // CTAs per head (portable cluster size)
+constexpr int kPreWarps = 8;
+
+struct PreParams {
+    const void* W;          // [n_heads][E][H]
+    const uint16_t* s;      // [n_heads][H] bf16
+    int32_t* inds;          // [n_heads][K]
+    float* gates;           // [n_heads][K]
+    float* logits;          // [n_heads][E] or null
+    int H, E, K;
+};
+
+// Top-k of work[0..E) by one warp, ties to the lower index; the K winners are written in
+// ascending index with gate weights exp(l - max) / sum over the winners (which equals
+// softmax(l)[inds] / sum softmax(l)[inds]: the full-softmax denominator cancels).
+// `work` is overwritten.
+__device__ void warp_softmax_topk(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    const unsigned full = 0xFFFFFFFFu;
+    float myv = 0.f;
+    int myi = 0x7FFFFFFF;
+    for (int j = 0; j < K; ++j) {
+        float bv = -CUDART_INF_F;
+        int bi = 0x7FFFFFFF;
+        for (int e = lane; e < E; e += 32) {
+            const float v = work[e];
+            if (v > bv || (v == bv && e < bi)) { bv = v; bi = e; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(full, bv, o);
+            const int oi = __shfl_xor_sync(full, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == j) { myv = bv; myi = bi; }
+        if (bi != 0x7FFFFFFF && (bi & 31) == lane) work[bi] = CUDART_NAN_F;   // taken: never compares true again
+        __syncwarp();
+    }
+    const float m = __shfl_sync(full, myv, 0);
+    const float ex = lane < K ? expf(myv - m) : 0.f;
+    const float sum = warp_sum(ex);
+    int rank = 0;
+    for (int i = 0; i < K; ++i) {
+        const int oi = __shfl_sync(full, myi, i);
+        rank += (oi < myi) ? 1 : 0;
+    }
+    if (lane < K) {
+        inds[rank] = myi;
+        gates[rank] = ex / sum;
+    }
+}
+
+template <typename WT> struct RowDot;
+
+// fp16 head: 8 weights (16 bytes) per lane per step
+template <> struct RowDot<__half> {
+    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+        const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const __half*>(W) + row * H);
+        float acc = 0.f;
+#pragma unroll 4
+        for (int c = lane; c < H / 8; c += 32) {
+            const uint4 w = ld_stream16(wp + c);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+            const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
+            const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
+            const float* x = sx + c * 8;
+            acc = fmaf(a.x, x[0], acc); acc = fmaf(a.y, x[1], acc);
+            acc = fmaf(b.x, x[2], acc); acc = fmaf(b.y, x[3], acc);
+            acc = fmaf(d.x, x[4], acc); acc = fmaf(d.y, x[5], acc);
+            acc = fmaf(e.x, x[6], acc); acc = fmaf(e.y, x[7], acc);
+        }
+        return warp_sum(acc);
+    }
+};
+
+// fp32 head: 4 weights (16 bytes) per lane per step
+template <> struct RowDot<float> {
+    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+        const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const float*>(W) + row * H);
+        float acc = 0.f;
+#pragma unroll 4
+        for (int c = lane; c < H / 4; c += 32) {
+            const uint4 w = ld_stream16(wp + c);
+            const float* x = sx + c * 4;
+            acc = fmaf(__uint_as_float(w.x), x[0], acc); acc = fmaf(__uint_as_float(w.y), x[1], acc);
+            acc = fmaf(__uint_as_float(w.z), x[2], acc); acc = fmaf(__uint_as_float(w.w), x[3], acc);
+        }
+        return warp_sum(acc);
+    }
+};
+
+template <typename WT>
+__global__ void __launch_bounds__(kPreWarps * 32) prerouter_kernel(PreParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
+    const int csize = (int)cluster.num_blocks();
+    const int head = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    extern __shared__ float smem[];
+    float* s_logits = smem;             // [E]   (the leader's copy collects every CTA's rows)
+    float* s_x = smem + p.E;            // [H]   hidden state widened to fp32
+
+    const uint16_t* sv = p.s + (size_t)head * p.H;
+    for (int i = threadIdx.x; i < p.H; i += blockDim.x) s_x[i] = bf16_bits_to_float(sv[i]);
+    __syncthreads();
+
+    float* leader = cluster.map_shared_rank(s_logits, 0);
+    const int per = (p.E + csize - 1) / csize;
+    const int e0 = crank * per, e1 = min(p.E, e0 + per);
+    const size_t wbase = (size_t)head * p.E;
+    for (int e = e0 + warp; e < e1; e += kPreWarps) {
+        const float l = RowDot<WT>::run(p.W, wbase + e, s_x, p.H, lane);
+        if (lane == 0) leader[e] = l;
+    }
+    cluster.sync();                     // every CTA's logits have landed in the leader
+    if (crank != 0) return;
+
+    if (p.logits != nullptr)
+        for (int e = threadIdx.x; e < p.E; e += blockDim.x) p.logits[(size_t)head * p.E + e] = s_logits[e];
+    __syncthreads();
+    if (warp == 0)
+        warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds + (size_t)head * p.K, p.gates + (size_t)head * p.K);
+}
+
+// a2 alone: one warp per row of given logits.
+__global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* logits, int T, int E, int K,
+                                                                int32_t* inds, float* gates) {
+    extern __shared__ float smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * 4 + warp;
+    if (t >= T) return;
+    float* work = smem + warp * E;
+    for (int e = lane; e < E; e += 32) work[e] = logits[(size_t)t * E + e];
+    __syncwarp();
+    warp_softmax_topk(work, E, K, lane, inds + (size_t)t * K, gates + (size_t)t * K);
+}
+
+int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st) {
+    int32_t rc = check_desc(d);
+    if (rc != EDG_OK) return rc;
+    if (!W_pre || !s || !inds || !gates || n_heads < 1 || n_heads > 65535) return EDG_E_INVAL;
+    if (!aligned(W_pre, 16) || !aligned(s, 16)) return EDG_E_INVAL;
+    PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K};
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kPreCluster, n_heads, 1);
+    cfg.blockDim = dim3(kPreWarps * 32, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)(d->E + d->H) * sizeof(float);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = kPreCluster;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (d->pre_dtype == EDG_F16) EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_kernel<__half>, p));
+    else EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_kernel<float>, p));
+    return EDG_OK;
+}
+
+}  // namespace edg
+
+extern "C" int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
+                                  int32_t* inds, float* gates, float* logits_opt, void* stream) {
+    return edg::run_prerouter(desc, W_pre, s, n_heads, inds, gates, logits_opt, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,
+                                     int32_t* inds, float* gates, void* stream) {
+    int32_t rc = edg::check_desc(desc);
+    if (rc != EDG_OK) return rc;
+    if (!logits || !inds || !gates || T < 1) return EDG_E_INVAL;
+    const size_t sm = 4 * (size_t)desc->E * sizeof(float);
+    edg::softmax_topk_rows_kernel<<<(T + 3) / 4, 128, sm, static_cast<cudaStream_t>(stream)>>>(
+        logits, T, desc->E, desc->K, inds, gates);
+    EDG_CUDA_TRY(cudaGetLastError());
+    return EDG_OK;
+}

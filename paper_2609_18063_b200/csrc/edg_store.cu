@@ -1,0 +1,254 @@
+// a3: the slot-pool expert store (Sec. 3.1 "staged" executor path; Fig. 1 streaming pool) and
+// the whole layer-step (Sec. 3.2, the double shift).
+//
+// A pinned-host tier holds every expert record of every layer and stands in for the paper's
+// SSD.  Each layer owns a fixed pool of HBM slots.  Staging is host-driven: the allocator below
+// is pure integer logic; for each missing expert one cudaMemcpyAsync is enqueued on a side
+// stream, ordered after the layer's last compute by an event, so that the copies of the next
+// token overlap the compute of the current one.  Slots are sticky: an expert that stays routed
+// is never copied again, and a step rewrites only the slots whose expert changed.
+#include <new>
+#include <vector>
+
+#include "edg_common.cuh"
+
+namespace edg {
+int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots,
+                const int32_t* table, const int32_t* experts, const float* gates, const void* x,
+                const edg_lora* lora, void* y, void* workspace, size_t workspace_bytes, cudaStream_t st);
+int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st);
+}  // namespace edg
+
+namespace {
+
+constexpr uint32_t kMagic = 0x45444731u;   // "EDG1"
+constexpr int kRing = 64;                  // pinned staging rows for slot-table updates
+
+struct LayerState {
+    std::vector<int32_t> expert_of_slot, slot_of_expert;
+    std::vector<int64_t> last_use;
+    std::vector<uint8_t> taken;
+    int64_t n = 0;                         // stage calls so far (the LRU clock)
+    cudaEvent_t copy_done = nullptr, compute_done = nullptr;
+    bool copy_pending = false;             // copy_done recorded and not yet waited on by compute
+    bool compute_recorded = false;
+};
+
+}  // namespace
+
+struct edg_store {
+    uint32_t magic = kMagic;
+    edg_layer_desc d{};
+    int n_layers = 0;
+    size_t R = 0;
+    std::vector<const uint8_t*> host_layers;
+    uint8_t* dev_slots = nullptr;
+    int32_t* dev_tables = nullptr;
+    std::vector<edg_lora> loras;
+    cudaStream_t copy_stream = nullptr;
+    std::vector<LayerState> layers;
+    int32_t* ring = nullptr;               // pinned [kRing][E]
+    cudaEvent_t ring_ev[kRing] = {};
+    bool ring_used[kRing] = {};
+    int ring_pos = 0;
+    edg_store_stats stats{};
+};
+
+static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
+
+extern "C" int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
+                                    void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
+                                    void* copy_stream, edg_store** out) {
+    int32_t rc = edg::check_desc(desc);
+    if (rc != EDG_OK) return rc;
+    if (!host_layers || !dev_slots || !dev_tables || !out || n_layers < 1) return EDG_E_INVAL;
+    if (!edg::aligned(dev_slots, 256) || !edg::aligned(dev_tables, 16)) return EDG_E_INVAL;
+    for (int l = 0; l < n_layers; ++l)
+        if (!host_layers[l] || !edg::aligned(host_layers[l], 16)) return EDG_E_INVAL;
+    edg_store* s = new (std::nothrow) edg_store();
+    if (!s) return EDG_E_INVAL;
+    s->d = *desc;
+    s->n_layers = n_layers;
+    s->R = edg::record_layout(desc->H, desc->I, desc->group).bytes;
+    s->host_layers.assign(reinterpret_cast<const uint8_t* const*>(host_layers),
+                          reinterpret_cast<const uint8_t* const*>(host_layers) + n_layers);
+    s->dev_slots = static_cast<uint8_t*>(dev_slots);
+    s->dev_tables = dev_tables;
+    if (loras) s->loras.assign(loras, loras + n_layers);
+    s->copy_stream = static_cast<cudaStream_t>(copy_stream);
+    s->layers.resize(n_layers);
+    auto fail = [&](cudaError_t e) { edg::set_cuda_error(e); edg_store_destroy(s); return EDG_E_CUDA; };
+    for (auto& L : s->layers) {
+        L.expert_of_slot.assign(desc->n_slots, -1);
+        L.slot_of_expert.assign(desc->E, -1);
+        L.last_use.assign(desc->n_slots, -1);
+        L.taken.assign(desc->n_slots, 0);
+        cudaError_t e = cudaEventCreateWithFlags(&L.copy_done, cudaEventDisableTiming);
+        if (e != cudaSuccess) return fail(e);
+        e = cudaEventCreateWithFlags(&L.compute_done, cudaEventDisableTiming);
+        if (e != cudaSuccess) return fail(e);
+    }
+    cudaError_t e = cudaHostAlloc(reinterpret_cast<void**>(&s->ring), (size_t)kRing * desc->E * sizeof(int32_t), cudaHostAllocDefault);
+    if (e != cudaSuccess) return fail(e);
+    for (int i = 0; i < kRing; ++i) {
+        e = cudaEventCreateWithFlags(&s->ring_ev[i], cudaEventDisableTiming);
+        if (e != cudaSuccess) return fail(e);
+    }
+    // every expert starts non-resident
+    e = cudaMemsetAsync(dev_tables, 0xFF, (size_t)n_layers * desc->E * sizeof(int32_t), s->copy_stream);
+    if (e != cudaSuccess) return fail(e);
+    e = cudaStreamSynchronize(s->copy_stream);
+    if (e != cudaSuccess) return fail(e);
+    *out = s;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_destroy(edg_store* s) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    cudaStreamSynchronize(s->copy_stream);
+    for (auto& L : s->layers) {
+        if (L.copy_done) cudaEventDestroy(L.copy_done);
+        if (L.compute_done) cudaEventDestroy(L.compute_done);
+    }
+    for (int i = 0; i < kRing; ++i)
+        if (s->ring_ev[i]) cudaEventDestroy(s->ring_ev[i]);
+    if (s->ring) cudaFreeHost(s->ring);
+    s->magic = 0;
+    delete s;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_get_stats(const edg_store* s, edg_store_stats* out) {
+    if (!store_ok(s) || !out) return EDG_E_INVAL;
+    *out = s->stats;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_snapshot(const edg_store* s, int32_t layer, int32_t* expert_of_slot, int32_t* slot_of_expert) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    const LayerState& L = s->layers[layer];
+    if (expert_of_slot) for (int i = 0; i < s->d.n_slots; ++i) expert_of_slot[i] = L.expert_of_slot[i];
+    if (slot_of_expert) for (int i = 0; i < s->d.E; ++i) slot_of_expert[i] = L.slot_of_expert[i];
+    return EDG_OK;
+}
+
+extern "C" int32_t stage_experts_to_slots(edg_store* s, int32_t layer, const int32_t* inds, int32_t n,
+                                          int32_t* slots_out, int32_t* n_miss_out) {
+    if (!store_ok(s) || !inds || !slots_out) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    const int S = s->d.n_slots, E = s->d.E;
+    if (n < 0) return EDG_E_INVAL;
+    if (n > S) return EDG_E_SLOTS;
+    LayerState& L = s->layers[layer];
+
+    // validate before touching any state: in range and distinct
+    for (int i = 0; i < n; ++i) {
+        if (inds[i] < 0 || inds[i] >= E) return EDG_E_RANGE;
+        for (int j = 0; j < i; ++j) if (inds[j] == inds[i]) return EDG_E_RANGE;
+    }
+
+    // (i) residents keep their slot and are touched
+    for (int i = 0; i < S; ++i) L.taken[i] = 0;
+    for (int i = 0; i < n; ++i) {
+        const int sl = L.slot_of_expert[inds[i]];
+        if (sl >= 0) { L.taken[sl] = 1; L.last_use[sl] = L.n; }
+    }
+    // (ii) each missing expert takes the least recently used slot this call does not need
+    int n_miss = 0;
+    bool waited = false;
+    for (int i = 0; i < n; ++i) {
+        const int e = inds[i];
+        if (L.slot_of_expert[e] >= 0) continue;
+        int victim = -1;
+        for (int sl = 0; sl < S; ++sl)
+            if (!L.taken[sl] && (victim < 0 || L.last_use[sl] < L.last_use[victim])) victim = sl;
+        // n <= S guarantees a free slot
+        const int old = L.expert_of_slot[victim];
+        if (old >= 0) L.slot_of_expert[old] = -1;
+        L.expert_of_slot[victim] = e;
+        L.slot_of_expert[e] = victim;
+        L.last_use[victim] = L.n;
+        L.taken[victim] = 1;
+        if (!waited && L.compute_recorded) {
+            // do not overwrite a slot the layer's last compute may still be reading
+            EDG_CUDA_TRY(cudaStreamWaitEvent(s->copy_stream, L.compute_done, 0));
+            waited = true;
+        }
+        EDG_CUDA_TRY(cudaMemcpyAsync(s->dev_slots + ((size_t)layer * S + victim) * s->R,
+                                     s->host_layers[layer] + (size_t)e * s->R, s->R,
+                                     cudaMemcpyHostToDevice, s->copy_stream));
+        ++n_miss;
+    }
+    L.n += 1;
+    for (int i = 0; i < n; ++i) slots_out[i] = L.slot_of_expert[inds[i]];
+    if (n_miss_out) *n_miss_out = n_miss;
+    s->stats.stage_calls += 1;
+    s->stats.hits += n - n_miss;
+    s->stats.misses += n_miss;
+    s->stats.bytes_copied += (int64_t)n_miss * (int64_t)s->R;
+
+    if (n_miss > 0) {
+        // publish the new expert -> slot row to the device table, after the record copies
+        const int r = s->ring_pos;
+        s->ring_pos = (r + 1) % kRing;
+        if (s->ring_used[r]) EDG_CUDA_TRY(cudaEventSynchronize(s->ring_ev[r]));
+        int32_t* row = s->ring + (size_t)r * E;
+        for (int e = 0; e < E; ++e) row[e] = L.slot_of_expert[e];
+        EDG_CUDA_TRY(cudaMemcpyAsync(s->dev_tables + (size_t)layer * E, row, (size_t)E * sizeof(int32_t),
+                                     cudaMemcpyHostToDevice, s->copy_stream));
+        EDG_CUDA_TRY(cudaEventRecord(s->ring_ev[r], s->copy_stream));
+        s->ring_used[r] = true;
+        EDG_CUDA_TRY(cudaEventRecord(L.copy_done, s->copy_stream));
+        L.copy_pending = true;
+        s->stats.table_updates += 1;
+    }
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_wait_staged(edg_store* s, int32_t layer, void* stream) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    LayerState& L = s->layers[layer];
+    if (L.copy_pending) {
+        EDG_CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), L.copy_done, 0));
+        L.copy_pending = false;
+    }
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* stream) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    // Only a pool that can evict needs the ordering: with n_slots == E nothing is ever overwritten.
+    if (s->d.n_slots < s->d.E) {
+        LayerState& L = s->layers[layer];
+        EDG_CUDA_TRY(cudaEventRecord(L.compute_done, static_cast<cudaStream_t>(stream)));
+        L.compute_recorded = true;
+    }
+    return EDG_OK;
+}
+
+extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
+                                    const int32_t* inds_cur, const float* gates_cur,
+                                    const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                                    float* logits_next_opt, void* y,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+    if (!store_ok(s) || !x || !inds_cur || !gates_cur || !y) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t rc = edg_store_wait_staged(s, layer, stream);
+    if (rc != EDG_OK) return rc;
+    const edg_lora* lora = s->loras.empty() ? nullptr : &s->loras[layer];
+    rc = edg::run_ffn(&s->d, s->dev_slots + (size_t)layer * s->d.n_slots * s->R, 1, inds_cur,
+                      s->dev_tables + (size_t)layer * s->d.E, nullptr, gates_cur, x, lora, y,
+                      workspace, workspace_bytes, st);
+    if (rc != EDG_OK) return rc;
+    if (W_pre_next != nullptr) {
+        if (!inds_next || !gates_next) return EDG_E_INVAL;
+        rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st);
+        if (rc != EDG_OK) return rc;
+    }
+    return edg_store_mark_computed(s, layer, stream);
+}

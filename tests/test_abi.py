@@ -1,0 +1,84 @@
+"""The C-ABI library: it builds, loads without a GPU, exports every function the header declares,
+and its host-side entry points behave (descriptor checks, record size, repacking)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import moe_oracle as orc
+from workloads import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_18063_b200 import build
+    build.build()
+    import paper_2609_18063_b200 as m
+    return m
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "edg_moe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"^\s*(?:int32_t|const char\*)\s+(\w+)\s*\(", text, flags=re.M)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared_functions()
+    assert {"prerouter_topk", "stage_experts_to_slots", "moe_expert_ffn_int4_lora", "moe_layer_decode"} <= set(names)
+    raw = ctypes.CDLL(lib.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), f"{n} is declared in edg_moe.h but not exported"
+    assert set(lib.EXPORTS) == set(names), "binding and header disagree"
+    assert lib.version() >= 1000
+
+
+def test_record_bytes_and_desc_checks(lib):
+    d2 = lib.make_desc(synth.CONFIGS["cfg2"])
+    d1 = lib.make_desc(synth.CONFIGS["cfg1"])
+    assert lib.record_bytes(d2) == orc.record_bytes(2048, 512, 64) == 1_769_472
+    assert lib.record_bytes(d1) == orc.record_bytes(1024, 256, 32) == 491_520
+    assert lib.check_desc(d2) == 0
+    for field, bad in [("H", 2000), ("I", 96), ("group", 48), ("K", 33), ("E", 4), ("rank", 65),
+                       ("n_adapters", 3), ("n_slots", 0), ("H", 8192)]:
+        d = lib.make_desc(synth.CONFIGS["cfg2"])
+        setattr(d, field, bad)
+        assert lib.check_desc(d) == -2, field
+    d = lib.make_desc(synth.CONFIGS["cfg2"]); d.out_dtype = 7
+    assert lib.check_desc(d) == -1
+    with pytest.raises(lib.EdgError):
+        lib.record_bytes(d)
+    assert lib.ffn_workspace_bytes(d2, 1) % 256 == 0
+    assert lib.ffn_workspace_bytes(d2, 64) > lib.ffn_workspace_bytes(d2, 1)
+
+
+def test_pack_unpack_identity_and_layout(lib):
+    cfg = synth.CONFIGS["cfg1"]
+    d = lib.make_desc(cfg)
+    ex = synth.expert_tensors(cfg, 0, 5)
+    rec = lib.pack_expert(d, ex)
+    assert rec.nbytes == cfg.record_bytes
+    back = lib.unpack_expert(d, rec)
+    for proj in ("gate", "up", "down"):
+        for a, b in zip(ex[proj], back[proj]):
+            assert np.array_equal(np.asarray(a).view(np.uint8), np.asarray(b).view(np.uint8))
+    # the record's code sections are the canonical nibble order the oracle unpacks
+    half = cfg.H * cfg.I // 2
+    assert np.array_equal(orc.unpack_codes(rec[:half].reshape(cfg.I, cfg.H // 2)), orc.unpack_codes(ex["gate"][0]))
+    # (scale, zero) pairs interleaved after the codes
+    sz = rec[3 * half:3 * half + 8].view(np.float16)
+    assert sz[0] == ex["gate"][1][0, 0] and sz[1] == ex["gate"][2][0, 0] and sz[2] == ex["gate"][1][0, 1]
+    with pytest.raises(ValueError):
+        lib.pack_expert(lib.make_desc(synth.CONFIGS["cfg2"]), ex)
+
+
+def test_host_calls_reject_bad_handles(lib):
+    import paper_2609_18063_b200.binding as b
+    assert b._lib.edg_store_destroy(None) == -1
+    assert b._lib.stage_experts_to_slots(None, 0, None, 0, None, None) == -1
+    st = b.StoreStats()
+    assert b._lib.edg_store_get_stats(None, ctypes.byref(st)) == -1
