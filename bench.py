@@ -1,0 +1,427 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE layer decode step at batch 1 on the 35B-class layer shape.
+
+One "step" is one layer-step: the prerouter head scores the next step's experts from this step's
+hidden state (logits, softmax, top-k, renormalised gates), the routing predicted one step earlier
+is mapped through the slot table, the K int4 SwiGLU experts with their unmerged LoRA delta run
+over those slots, and the K outputs are reduced by their gate weights -- all through the C-ABI
+call ``moe_layer_decode``.
+
+Default arm (``--impl b200``):
+  value : layer-steps per second with everything resident in HBM.  The workload rotates over
+          several independently seeded instances of the layer (each with all E experts resident),
+          so the bytes a step streams are far outside the L2 and come from HBM.  Steps are chained
+          through the routing (step t+1 consumes the top-k that step t produced) and launched from
+          CUDA graphs; timed with CUDA events on the launching stream.
+  e2e   : the same metric with HOST buffers: the experts live in a pinned-host store, the HBM pool
+          has the configuration's 8 slots, every step copies its hidden state host->device, stages
+          the missing experts with cudaMemcpyAsync, runs the layer-step and reads y back.
+  roofline / cpu_baseline / clocks: see the keys of the JSON line.
+Reference arm (``--impl reference``): the fp64 CPU oracle, as it stands, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import synth  # noqa: E402
+
+METRIC = "moe_layer_decode_tok_per_s_batch1"
+UNIT = "tok/s"
+WORKLOAD = "cfg2: one 35B-class MoE layer (H2048 I512 E256 top-8 int4 g64 LoRA r16), batch-1 decode"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until captured).
+NCU_TRAFFIC_BYTES = None
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the GPU is under load."""
+
+    def __init__(self, index: int, period_s: float = 0.01):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        self.period = period_s
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "sw_power_cap": 0x4, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr is not None:
+            self._thr.join()
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ workload
+
+def _physical_device(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def build_instances(edg, layer_io, cfg, desc, n_inst, first_layer):
+    """Pinned host layers for `n_inst` independently seeded instances of the layer."""
+    R = edg.record_bytes(desc)
+    import torch
+    hosts = [torch.empty((cfg.E, R), dtype=torch.uint8, pin_memory=True) for _ in range(n_inst)]
+
+    def fill(job):
+        i, e = job
+        edg.pack_expert(desc, synth.expert_tensors(cfg, first_layer + i, e), hosts[i].numpy()[e])
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        list(ex.map(fill, [(i, e) for i in range(n_inst) for e in range(cfg.E)]))
+    return hosts
+
+
+def run_b200(args):
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    from paper_2609_18063_b200 import build
+    build.build()
+    import paper_2609_18063_b200 as edg
+    from paper_2609_18063_b200 import layer_io
+
+    cfg = synth.CONFIGS["cfg2"]
+    n_inst = args.instances
+    first_layer = rank * n_inst            # replicas: every rank serves its own layer instances
+    desc = edg.make_desc(cfg, n_slots=cfg.E, out_dtype="f32")
+    R = edg.record_bytes(desc)
+    K, E, H = cfg.K, cfg.E, cfg.H
+
+    hosts = build_instances(edg, layer_io, cfg, desc, n_inst, first_layer)
+    loras, keep = [], []
+    for i in range(n_inst):
+        lo, k = layer_io.lora_to_device(desc, [synth.lora_tensors(cfg, first_layer + i, 0)])
+        loras.append(lo); keep.append(k)
+    W = torch.from_numpy(np.stack([synth.prerouter_weights(cfg, first_layer + i) for i in range(n_inst)])).cuda()
+
+    # ---- resident arm: all experts of all instances in HBM, slot e of instance i holds expert e
+    pool = torch.empty((n_inst, E, R), dtype=torch.uint8, device="cuda")
+    tables = torch.empty((n_inst, E), dtype=torch.int32, device="cuda")
+    copy_stream = torch.cuda.Stream()
+    store = edg.Store(desc, hosts, pool, tables, loras, copy_stream)
+    for i in range(n_inst):
+        for e0 in range(0, E, 64):
+            edg.stage_experts_to_slots(store, i, np.arange(e0, min(E, e0 + 64), dtype=np.int32))
+    copy_stream.synchronize()
+    assert store.stats()["misses"] == n_inst * E
+
+    NX = 256
+    X_bits = synth.hidden_states(cfg, NX, layer=first_layer, stream=100)
+    xd = layer_io.bits_to_device(X_bits, torch.bfloat16)
+    y = torch.zeros((NX, H), dtype=torch.float32, device="cuda")
+    inds = torch.zeros((2, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((2, K), dtype=torch.float32, device="cuda")
+    ws = layer_io.new_workspace(desc)
+
+    def step(s):
+        i = s % n_inst
+        edg.moe_layer_decode(store, i, xd[s % NX], inds[s % 2], gates[s % 2], W[(s + 1) % n_inst],
+                             inds[(s + 1) % 2], gates[(s + 1) % 2], None, y[s % NX], ws)
+
+    # routing of step 0 comes from a "last prompt token" state
+    edg.prerouter_topk(desc, W[0], xd[NX - 1], 1, inds[0], gates[0], None)
+    torch.cuda.synchronize()
+
+    G = NX                                 # steps per CUDA graph
+    if G % n_inst or n_inst % 2 and n_inst != 1:
+        raise SystemExit("--instances must be even (or 1) and divide 256")
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+
+    def capture(n_steps):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            # touch every instance once outside capture (an even count keeps the two-entry routing
+            # ring in phase), so that no staging event is waited on inside the graph
+            for s in range(2 * n_inst):
+                step(s)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                for s in range(n_steps):
+                    step(s)
+        return g
+
+    steps, warmup = args.steps, max(args.warmup, 3)
+    full, rem = divmod(steps, G)
+    if rem % 2:                            # the inds ring has two entries: keep graph lengths even
+        raise SystemExit("--steps must be even")
+    g_full = capture(G) if full or warmup else None
+    g_rem = capture(rem) if rem else None
+
+    sampler = ClockSampler(_physical_device(local_rank))
+    with torch.cuda.stream(stream):
+        for _ in range((warmup + G - 1) // G):
+            g_full.replay()
+        stream.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(full):
+            g_full.replay()
+        if g_rem is not None:
+            g_rem.replay()
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1)
+        # keep the GPU under the same load a little longer so the clock sampler sees it
+        t_end = time.time() + 0.3
+        while time.time() < t_end and g_full is not None:
+            g_full.replay()
+        stream.synchronize()
+    clocks = sampler.stop()
+    torch.cuda.synchronize()
+    status = edg.workspace_status(ws)
+    if status != 0 or not bool(torch.isfinite(y).all()):
+        raise SystemExit(f"bench: bad device status {status} or non-finite output")
+
+    t_ms = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_max = float(t_ms.item())
+    value = world * steps / (ms_max * 1e-3)
+    ms_per_step = ms_max / steps
+
+    # ---- e2e arm: pinned-host store, 8 slots, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(edg, layer_io, cfg, hosts[0], loras[0], W[0], X_bits, args, world)
+
+    # ---- roofline of the dominant work: the int4 expert bytes one step streams
+    peak, how = _peaks()
+    alg_bytes = K * R
+    launches_per_step = 5                  # lora-A(x), gate/up, lora-A(h), down+reduce, prerouter
+    achieved = alg_bytes / (ms_per_step * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES, "peak_kind": how + " (burst copy)",
+                "kernel": "all kernels of one layer-step (their summed duration)",
+                "algorithmic_bytes_per_launch": alg_bytes}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(cfg, args.cpu_seconds)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": round(ms_per_step, 6), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int4 weights, bf16 activations, fp32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "resident_instances": n_inst,
+                       "hbm_working_set_bytes": n_inst * E * R,
+                       "l2": "inputs larger than L2: steps rotate over the instances, routing iid from the prerouter",
+                       "routing": "redrawn every step from the prerouter (step t+1 consumes step t's top-k)",
+                       "launch": f"CUDA graphs of {G} steps", "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps,
+            "roofline": roofline, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    store.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
+    """Config 2 as written: pinned-host expert store, 8 slots, one layer; per step the hidden state
+    goes host->device, the routed experts that are not resident are staged, the layer-step runs and
+    y comes back to the host."""
+    import torch
+    import torch.distributed as dist
+    K, E, H = cfg.K, cfg.E, cfg.H
+    desc = edg.make_desc(cfg, n_slots=cfg.n_slots, out_dtype="f32")
+    R = edg.record_bytes(desc)
+    slots = torch.empty((1, cfg.n_slots, R), dtype=torch.uint8, device="cuda")
+    tables = torch.empty((1, E), dtype=torch.int32, device="cuda")
+    cs = torch.cuda.Stream()
+    store = edg.Store(desc, [host_layer], slots, tables, [lora], cs)
+    ws = layer_io.new_workspace(desc)
+    NX = X_bits.shape[0]
+    x_host = torch.from_numpy(X_bits.view(np.int16).copy()).pin_memory()
+    x_dev = torch.empty((H,), dtype=torch.int16, device="cuda")
+    y_dev = torch.empty((H,), dtype=torch.float32, device="cuda")
+    y_host = torch.empty((H,), dtype=torch.float32).pin_memory()
+    inds = torch.zeros((2, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((2, K), dtype=torch.float32, device="cuda")
+    inds_host = torch.empty((K,), dtype=torch.int32).pin_memory()
+    st = torch.cuda.current_stream()
+    edg.prerouter_topk(desc, W, layer_io.bits_to_device(X_bits[NX - 1], torch.bfloat16), 1, inds[0], gates[0], None)
+
+    def step(s):
+        x_dev.copy_(x_host[s % NX], non_blocking=True)
+        inds_host.copy_(inds[s % 2], non_blocking=True)           # the prediction made one step earlier
+        st.synchronize()
+        edg.stage_experts_to_slots(store, 0, inds_host.numpy())
+        edg.moe_layer_decode(store, 0, x_dev, inds[s % 2], gates[s % 2], W, inds[(s + 1) % 2], gates[(s + 1) % 2],
+                             None, y_dev, ws)
+        y_host.copy_(y_dev, non_blocking=True)
+        st.synchronize()
+
+    n = min(args.steps, args.e2e_steps)
+    n -= n % 2
+    for s in range(max(4, min(args.warmup, 20) // 2 * 2)):
+        step(s)
+    base = store.stats()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(n):
+        step(s)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    after = store.stats()
+    miss_bytes = (after["bytes_copied"] - base["bytes_copied"]) / n
+    table_bytes = (after["table_updates"] - base["table_updates"]) * E * 4 / n
+    out = {"value": round(world * n / (float(t.item()) * 1e-3), 1), "unit": UNIT,
+           "h2d_bytes_per_step": int(H * 2 + miss_bytes + table_bytes), "d2h_bytes_per_step": H * 4 + K * 4,
+           "steps": n, "slots": cfg.n_slots,
+           "misses_per_step": round((after["misses"] - base["misses"]) / n, 3),
+           "note": "pinned-host expert store, 8 slots, experts staged on demand by cudaMemcpyAsync: bound by host->device copy bandwidth"}
+    store.close()
+    return out
+
+
+# ------------------------------------------------------------------ CPU oracle timing
+
+def _oracle_steps(cfg, n_steps, budget_s):
+    """Times the oracle's layer-step on pre-generated inputs; returns (steps done, seconds, threads)."""
+    from oracle import moe_oracle as orc
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        threads = 1
+    W = synth.prerouter_weights(cfg, 0)
+    X = synth.hidden_states(cfg, n_steps + 1, stream=100)
+    lora = synth.lora_tensors(cfg, 0, 0)
+    inds, gates = orc.softmax_topk(orc.prerouter_logits(W, X[n_steps]), cfg.K)
+    done, spent = 0, 0.0
+    for t in range(n_steps):
+        experts = {int(e): synth.expert_tensors(cfg, 0, int(e)) for e in inds}      # input generation: untimed
+        t0 = time.perf_counter()
+        _, _, _, inds, gates, _ = orc.moe_layer_decode(X[t], inds, gates, W, cfg.K, experts.__getitem__,
+                                                       lambda e: lora, cfg.lora_scale, cfg.group)
+        spent += time.perf_counter() - t0
+        done += 1
+        if spent >= budget_s:
+            break
+    return done, spent, threads
+
+
+def cpu_baseline(cfg, budget_s):
+    done, spent, threads = _oracle_steps(cfg, 1000, budget_s)
+    return {"value": round(done / spent, 3), "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"{done} consecutive layer-steps of the same workload (fp64 numpy oracle, {spent:.1f} s)"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS["cfg2"]
+    _oracle_steps(cfg, max(1, min(args.warmup, 2)), 5.0)
+    done, spent, threads = _oracle_steps(cfg, args.steps, 120.0)
+    value = done / spent
+    sample = (f"{done} of the {args.steps} requested layer-steps were run (time-bounded sample); "
+              "each is one full oracle layer-step")
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 / value, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "parallelism": "host cores"},
+            "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "kind": "oracle", "cores": threads, "sample": sample},
+            "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10000)
+    ap.add_argument("--warmup", type=int, default=100)
+    ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
+    ap.add_argument("--instances", type=int, default=8, help="independently seeded resident layer instances")
+    ap.add_argument("--e2e-steps", type=int, default=400)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_b200(args)
+
+
+if __name__ == "__main__":
+    main()
