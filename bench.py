@@ -255,11 +255,11 @@ def run_b200(args):
     # ---- roofline of the dominant work: the int4 expert bytes one step streams
     peak, how = _peaks()
     alg_bytes = K * R
-    launches_per_step = 5                  # lora-A(x), gate/up, lora-A(h), down+reduce, prerouter
+    launches_per_step = 1                  # one fused kernel: prerouter + take + FFN + reduce
     achieved = alg_bytes / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                 "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES, "peak_kind": how + " (burst copy)",
-                "kernel": "all kernels of one layer-step (their summed duration)",
+                "kernel": "fused_layer_kernel (one launch per layer-step; duration = timed region / launches)",
                 "algorithmic_bytes_per_launch": alg_bytes}
 
     cpu = None

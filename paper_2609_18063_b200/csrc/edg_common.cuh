@@ -47,12 +47,14 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 }
 
 // Workspace layout for T tokens (floats unless noted).  The first 256 bytes are a control block
-// whose first int32 is the device-side status word.
+// whose first int32 is the device-side status word; bytes 64..127 hold the per-slice arrival
+// counters of the fused kernel's reduce (zero between launches).
 struct WorkspaceLayout {
     size_t ctrl;      // 256 B control block
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
+    size_t partial;   // [K][H] float               : gate-weighted expert outputs of the fused batch-1 kernel
     size_t bytes;
 };
 
@@ -66,7 +68,8 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_gu = 256;
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
-    W.bytes = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
+    W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
+    W.bytes = round_up(W.partial + (size_t)d.K * d.H * sizeof(float), 256);
     return W;
 }
 
@@ -166,6 +169,45 @@ __device__ __forceinline__ uint32_t ld_stream4(const void* p) {
     uint32_t v;
     asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
     return v;
+}
+
+// Top-k of work[0..E) by one warp, ties to the lower index; the K winners are written in
+// ascending index with gate weights exp(l - max) / sum over the winners (which equals
+// softmax(l)[inds] / sum softmax(l)[inds]: the full-softmax denominator cancels).
+// `work` is overwritten.
+__device__ __forceinline__ void warp_softmax_topk(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    const unsigned full = 0xFFFFFFFFu;
+    float myv = 0.f;
+    int myi = 0x7FFFFFFF;
+    for (int j = 0; j < K; ++j) {
+        float bv = -__int_as_float(0x7f800000);
+        int bi = 0x7FFFFFFF;
+        for (int e = lane; e < E; e += 32) {
+            const float v = work[e];
+            if (v > bv || (v == bv && e < bi)) { bv = v; bi = e; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(full, bv, o);
+            const int oi = __shfl_xor_sync(full, bi, o);
+            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == j) { myv = bv; myi = bi; }
+        if (bi != 0x7FFFFFFF && (bi & 31) == lane) work[bi] = __int_as_float(0x7fffffff);   // taken: never compares true again
+        __syncwarp();
+    }
+    const float m = __shfl_sync(full, myv, 0);
+    const float ex = lane < K ? expf(myv - m) : 0.f;
+    const float sum = warp_sum(ex);
+    int rank = 0;
+    for (int i = 0; i < K; ++i) {
+        const int oi = __shfl_sync(full, myi, i);
+        rank += (oi < myi) ? 1 : 0;
+    }
+    if (lane < K) {
+        inds[rank] = myi;
+        gates[rank] = ex / sum;
+    }
 }
 
 template <typename T> __device__ __forceinline__ void store_out(T* y, size_t i, float v);

@@ -8,6 +8,12 @@
 
 namespace edg {
 
+bool fused_supported(const edg_layer_desc& d);
+int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
+                        const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
+                        const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
+                        void* workspace, cudaStream_t st);
+
 struct FfnParams {
     const uint8_t* pool;        // slot records of one layer
     const int32_t* slots;       // [T][K] slot per routed expert, or expert ids when `table` is set
@@ -284,6 +290,11 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
         if (!lora->A_gate || !lora->B_gate || !lora->A_up || !lora->B_up || !lora->A_down || !lora->B_down) return EDG_E_INVAL;
         if (d->n_adapters != 1 && table == nullptr && experts == nullptr) return EDG_E_INVAL;
     }
+
+    // batch-1 decode on the shapes the fused kernel covers: one launch for the whole FFN
+    if (T == 1 && fused_supported(*d))
+        return run_fused_layer(d, slot_pool, slots, table, experts, gates, x, has_lora ? lora : nullptr, y,
+                               nullptr, nullptr, nullptr, nullptr, workspace, st);
 
     FfnParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);

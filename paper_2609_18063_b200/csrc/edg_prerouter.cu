@@ -26,45 +26,6 @@ struct PreParams {
     int H, E, K;
 };
 
-// Top-k of work[0..E) by one warp, ties to the lower index; the K winners are written in
-// ascending index with gate weights exp(l - max) / sum over the winners (which equals
-// softmax(l)[inds] / sum softmax(l)[inds]: the full-softmax denominator cancels).
-// `work` is overwritten.
-__device__ void warp_softmax_topk(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
-    const unsigned full = 0xFFFFFFFFu;
-    float myv = 0.f;
-    int myi = 0x7FFFFFFF;
-    for (int j = 0; j < K; ++j) {
-        float bv = -CUDART_INF_F;
-        int bi = 0x7FFFFFFF;
-        for (int e = lane; e < E; e += 32) {
-            const float v = work[e];
-            if (v > bv || (v == bv && e < bi)) { bv = v; bi = e; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(full, bv, o);
-            const int oi = __shfl_xor_sync(full, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (lane == j) { myv = bv; myi = bi; }
-        if (bi != 0x7FFFFFFF && (bi & 31) == lane) work[bi] = CUDART_NAN_F;   // taken: never compares true again
-        __syncwarp();
-    }
-    const float m = __shfl_sync(full, myv, 0);
-    const float ex = lane < K ? expf(myv - m) : 0.f;
-    const float sum = warp_sum(ex);
-    int rank = 0;
-    for (int i = 0; i < K; ++i) {
-        const int oi = __shfl_sync(full, myi, i);
-        rank += (oi < myi) ? 1 : 0;
-    }
-    if (lane < K) {
-        inds[rank] = myi;
-        gates[rank] = ex / sum;
-    }
-}
-
 template <typename WT> struct RowDot;
 
 // fp16 head: 8 weights (16 bytes) per lane per step

@@ -16,6 +16,11 @@ namespace edg {
 int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots,
                 const int32_t* table, const int32_t* experts, const float* gates, const void* x,
                 const edg_lora* lora, void* y, void* workspace, size_t workspace_bytes, cudaStream_t st);
+bool fused_supported(const edg_layer_desc& d);
+int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
+                        const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
+                        const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
+                        void* workspace, cudaStream_t st);
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
                       int32_t* inds, float* gates, float* logits_opt, cudaStream_t st);
 }  // namespace edg
@@ -241,14 +246,27 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
     int32_t rc = edg_store_wait_staged(s, layer, stream);
     if (rc != EDG_OK) return rc;
     const edg_lora* lora = s->loras.empty() ? nullptr : &s->loras[layer];
-    rc = edg::run_ffn(&s->d, s->dev_slots + (size_t)layer * s->d.n_slots * s->R, 1, inds_cur,
-                      s->dev_tables + (size_t)layer * s->d.E, nullptr, gates_cur, x, lora, y,
-                      workspace, workspace_bytes, st);
-    if (rc != EDG_OK) return rc;
-    if (W_pre_next != nullptr) {
-        if (!inds_next || !gates_next) return EDG_E_INVAL;
-        rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st);
+    if (W_pre_next != nullptr && (!inds_next || !gates_next)) return EDG_E_INVAL;
+    const void* pool = s->dev_slots + (size_t)layer * s->d.n_slots * s->R;
+    const int32_t* table = s->dev_tables + (size_t)layer * s->d.E;
+    if (edg::fused_supported(s->d)) {
+        // one launch: prerouter for the next step, take, FFN and reduce for this one
+        rc = edg::check_desc(&s->d);
         if (rc != EDG_OK) return rc;
+        if (!workspace || !edg::aligned(workspace, 256) || workspace_bytes < edg::workspace_layout(s->d, 1).bytes)
+            return EDG_E_WORKSPACE;
+        if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
+        rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
+                                  (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
+                                  logits_next_opt, workspace, st);
+        if (rc != EDG_OK) return rc;
+    } else {
+        rc = edg::run_ffn(&s->d, pool, 1, inds_cur, table, nullptr, gates_cur, x, lora, y, workspace, workspace_bytes, st);
+        if (rc != EDG_OK) return rc;
+        if (W_pre_next != nullptr) {
+            rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st);
+            if (rc != EDG_OK) return rc;
+        }
     }
     return edg_store_mark_computed(s, layer, stream);
 }
