@@ -134,6 +134,13 @@ int32_t edg_ffn_workspace_bytes(const edg_layer_desc* desc, int32_t T, size_t* b
  * instead of faulting).  Synchronises `stream`. */
 int32_t edg_workspace_status(const void* workspace, void* stream, int32_t* status);
 
+/* Tracing: with a dev buffer of (CTAs in the grid) x 16 uint64 (the batch-1 layer kernel launches
+ * (K + 1) x 16 CTAs), every CTA stamps the GPU's nanosecond timer at its phase boundaries, in slot
+ * 0 start, 1 copies issued, 2 adapter projections sent, 3 first weights landed, 4 gate/up done,
+ * 5 peers' projections in, 6 h sent, 7 whole h in, 8 down done, 9 end.  NULL switches it off
+ * (the default).  Process-wide; set it while no launch is in flight. */
+int32_t edg_set_trace_buffer(void* dev_buffer);
+
 /* ---------------------------------------------------------------- a1 + a2: prerouter */
 
 /* Prerouter head + routing (Sec. 3.2; Appendix A softmax-topk), for n_heads independent

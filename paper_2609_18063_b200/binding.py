@@ -15,7 +15,7 @@ import numpy as np
 __all__ = [
     "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
-    "ffn_workspace_bytes", "workspace_status", "prerouter_topk", "softmax_topk_rows",
+    "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "softmax_topk_rows",
     "moe_expert_ffn_int4_lora", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
 ]
 
@@ -65,6 +65,7 @@ _SIG = {
     "edg_unpack_expert": ([_D] + [_P] * 10, C.c_int32),
     "edg_ffn_workspace_bytes": ([_D, C.c_int32, C.POINTER(C.c_size_t)], C.c_int32),
     "edg_workspace_status": ([_P, _P, C.POINTER(C.c_int32)], C.c_int32),
+    "edg_set_trace_buffer": ([_P], C.c_int32),
     "prerouter_topk": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "softmax_topk_rows": ([_D, _P, C.c_int32, _P, _P, _P], C.c_int32),
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
@@ -203,6 +204,11 @@ def workspace_status(workspace, stream=None) -> int:
     st = C.c_int32()
     _check(_lib.edg_workspace_status(_ptr(workspace), _stream(stream), C.byref(st)), "edg_workspace_status")
     return st.value
+
+
+def set_trace_buffer(dev_buffer) -> None:
+    """Phase timestamps of the batch-1 layer kernel into `dev_buffer` (uint64 [CTAs][16]); None = off."""
+    _check(_lib.edg_set_trace_buffer(_ptr(dev_buffer)), "edg_set_trace_buffer")
 
 
 def prerouter_topk(desc, W_pre, s, n_heads, inds, gates, logits_opt=None, stream=None) -> None:

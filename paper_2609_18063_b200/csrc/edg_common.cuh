@@ -23,14 +23,29 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ---------------------------------------------------------------- record layout
 // One expert record: [gate codes][up codes][down codes][gate sz][up sz][down sz].
-// Codes are row-major int4, low nibble first; sz is one (scale, zero) fp16 pair per group,
-// row-major [out][in/group].  All section offsets are multiples of 256 bytes for the shapes
-// edg_check_desc admits.
+// Codes are int4, low nibble first; sz is one (scale, zero) fp16 pair per group.  gate and up are
+// row-major [out][in].  down is stored as kDownSlices column slices, each row-major
+// [H][I/kDownSlices]: the batch-1 kernel splits the down projection over the intermediate
+// dimension, and a (slice, block of rows) is then one contiguous run of bytes.  All section
+// offsets are multiples of 256 bytes for the shapes edg_check_desc admits.
 struct RecordLayout {
     uint32_t codes_gate, codes_up, codes_down;   // byte offsets
     uint32_t sz_gate, sz_up, sz_down;
     uint32_t bytes;
 };
+
+constexpr int kDownSlices = 4;
+
+// byte offset, inside the down code section, of the 16-byte chunk c (codes 32c .. 32c+31) of row n
+__host__ __device__ inline size_t down_code_off(int H, int I, int n, int c) {
+    const int sw = I / kDownSlices, cps = sw / 32;            // slice width in codes, chunks per row-slice
+    return ((size_t)(c / cps) * H + n) * (sw / 2) + (size_t)(c % cps) * 16;
+}
+// byte offset, inside the down sz section, of the (scale, zero) pair of group gi of row n
+__host__ __device__ inline size_t down_sz_off(int H, int I, int group, int n, int gi) {
+    const int gps = (I / kDownSlices) / group;                // groups per row-slice
+    return (((size_t)(gi / gps) * H + n) * gps + (gi % gps)) * 4;
+}
 
 __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
     RecordLayout L;
@@ -48,13 +63,15 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 
 // Workspace layout for T tokens (floats unless noted).  The first 256 bytes are a control block
 // whose first int32 is the device-side status word; bytes 64..127 hold the per-slice arrival
-// counters of the fused kernel's reduce (zero between launches).
+// counters of the fused kernel's reduce, byte 128 the count of head rows delivered (all zero
+// between launches) and bytes 160..175 the routing-ready flags of chained layer-steps.
 struct WorkspaceLayout {
     size_t ctrl;      // 256 B control block
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
-    size_t partial;   // [K][H] float               : gate-weighted expert outputs of the fused batch-1 kernel
+    size_t partial;   // [K*kDownSlices][H] float   : gate-weighted partial expert outputs of the fused batch-1 kernel
+    size_t logits;    // [E] float                  : next-step head logits gathered across CTAs
     size_t bytes;
 };
 
@@ -69,7 +86,8 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.bytes = round_up(W.partial + (size_t)d.K * d.H * sizeof(float), 256);
+    W.logits = round_up(W.partial + (size_t)d.K * 4 * d.H * sizeof(float), 256);
+    W.bytes = round_up(W.logits + (size_t)d.E * sizeof(float), 256);
     return W;
 }
 
@@ -125,26 +143,26 @@ __device__ __forceinline__ float scale_chunk(const float (&x)[32], float (&xs)[3
     return sum * pow2f(XS - 149);
 }
 
-__device__ __forceinline__ void word_fma(uint32_t w, const float* xs, float& a, float& b) {
+__device__ __forceinline__ void word_fma(uint32_t w, const float* xs, float& a, float& b, float& c, float& d) {
     const uint32_t w2 = w >> 8;
     a = fmaf(__uint_as_float(w & 0x0000000Fu), xs[0], a);
     b = fmaf(__uint_as_float(w & 0x000000F0u), xs[1], b);
-    a = fmaf(__uint_as_float(w & 0x00000F00u), xs[2], a);
-    b = fmaf(__uint_as_float(w & 0x0000F000u), xs[3], b);
+    c = fmaf(__uint_as_float(w & 0x00000F00u), xs[2], c);
+    d = fmaf(__uint_as_float(w & 0x0000F000u), xs[3], d);
     a = fmaf(__uint_as_float(w & 0x000F0000u), xs[4], a);
     b = fmaf(__uint_as_float(w & 0x00F00000u), xs[5], b);
-    a = fmaf(__uint_as_float(w2 & 0x000F0000u), xs[6], a);
-    b = fmaf(__uint_as_float(w2 & 0x00F00000u), xs[7], b);
+    c = fmaf(__uint_as_float(w2 & 0x000F0000u), xs[6], c);
+    d = fmaf(__uint_as_float(w2 & 0x00F00000u), xs[7], d);
 }
 
-// 2^(XS-149) * sum_{j<32} q_j x_j for one 16-byte chunk of codes.
-__device__ __forceinline__ float chunk_dot(const uint4& c, const float (&xs)[32]) {
-    float a = 0.f, b = 0.f;
-    word_fma(c.x, xs + 0, a, b);
-    word_fma(c.y, xs + 8, a, b);
-    word_fma(c.z, xs + 16, a, b);
-    word_fma(c.w, xs + 24, a, b);
-    return a + b;
+// 2^(XS-149) * sum_{j<32} q_j x_j for one 16-byte chunk of codes (four independent chains).
+__device__ __forceinline__ float chunk_dot(const uint4& q, const float (&xs)[32]) {
+    float a = 0.f, b = 0.f, c = 0.f, d = 0.f;
+    word_fma(q.x, xs + 0, a, b, c, d);
+    word_fma(q.y, xs + 8, a, b, c, d);
+    word_fma(q.z, xs + 16, a, b, c, d);
+    word_fma(q.w, xs + 24, a, b, c, d);
+    return (a + b) + (c + d);
 }
 
 // s * (qx - z * xsum): one chunk's contribution, still scaled by 2^(XS-149).  sz = (scale, zero) fp16 pair.

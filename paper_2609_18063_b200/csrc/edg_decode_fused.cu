@@ -1,19 +1,29 @@
 // The batch-1 layer-step as ONE kernel (a1-a2 for the next step, a3 take, a4-a6 for this step).
 //
-// Work split.  Every routed expert k gets one thread-block cluster of kC = 16 CTAs; one more
-// cluster evaluates the prerouter head.  Inside an expert's cluster:
-//   * each CTA owns I/16 rows of gate and up and H/16 rows of down.  At kernel start one thread
-//     issues bulk asynchronous copies (cp.async.bulk, completion on mbarriers) that bring the
-//     CTA's whole slice of the record -- codes and (scale, zero) pairs -- into shared memory, so
-//     all of the expert's bytes are in flight from the first microsecond and the down weights
-//     arrive while gate/up is being computed;
-//   * the rank-r LoRA projections A.x are split over the CTAs and all-gathered through
-//     distributed shared memory; so is h = silu(gate) * up and the per-slice partial of A_down.h;
-//   * two cluster barriers order the exchange (the first one is split into arrive / wait around
-//     the gate/up GEMV so nobody waits on it).
-// Across experts the reduce y = sum_k w_k o_k goes through a [K][H] fp32 scratch: each CTA writes
-// its gate-weighted slice, and the last CTA to arrive for a slice (one atomic counter per slice)
-// sums the K partials in ascending k, so the result does not depend on arrival order.
+// Work split.  Every routed expert is handled by 16 CTAs, arranged as four thread-block clusters
+// of kC = 4 CTAs (clusters of 4 can all be placed one CTA per SM on a B200; eight clusters of 16
+// cannot, and a cluster that shares SMs finishes last).  Cluster c of an expert owns a quarter of
+// the intermediate dimension: its CTAs compute the gate/up rows of that quarter, exchange
+// h = silu(gate) * up inside the cluster, and then compute a partial of the down projection over
+// that quarter of the columns for all H rows (a K-split) -- so no exchange ever crosses a cluster.
+//   * At kernel start every CTA issues bulk asynchronous copies (cp.async.bulk, completion on
+//     mbarriers) that bring its gate/up slice of the record into shared memory in four stages; its
+//     block of the down matrix follows into the space of the first two stages as soon as every
+//     warp is done with them, and lands while the rest of gate/up is being computed.
+//   * The rank-r LoRA projections A.x are split over the CTAs of a cluster and exchanged through
+//     distributed shared memory, as is h and the partial of A_down.h; the down adapter is applied
+//     per quarter (B (A h) is linear in h).  The exchanges are remote stores that count their bytes
+//     on an mbarrier of the receiving CTA (st.async); the only cluster barrier is a handshake at
+//     start-up, before any copy is issued, because a cluster-scope fence also waits for every bulk
+//     copy in flight into the SM.
+//   * The rows of the prerouter head are dealt over all CTAs of the grid and finished by whichever
+//     warp delivers the last logits.
+// The reduce y = sum_k w_k o_k goes through a [4K][H] fp32 scratch: each CTA writes its
+// gate-weighted partial, and the last CTA to arrive for a block of rows (one atomic counter per
+// block) sums the 4K partials in a fixed order, so the result does not depend on arrival order.
+// Consecutive layer-steps are chained by programmatic dependent launch: the next step's kernel
+// starts early, waits for a flag raised by this step's top-k, and streams its weights while this
+// step is still computing.
 #include <cooperative_groups.h>
 
 #include "edg_common.cuh"
@@ -22,10 +32,12 @@ namespace cg = cooperative_groups;
 
 namespace edg {
 
-constexpr int kC = 16;            // CTAs per cluster
+constexpr int kC = 4;             // CTAs per cluster
+constexpr int kE16 = kC * kDownSlices;   // CTAs per expert
 constexpr int kFW = 8;            // warps per CTA
 constexpr int kStages = 4;        // gate/up copy stages per CTA
 constexpr int kMaxRank = 64;
+constexpr int kTraceMarks = 16;
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
 
 struct FusedParams {
@@ -38,8 +50,10 @@ struct FusedParams {
     edg_lora lora;
     void* y;                      // [H]
     int32_t* status;
-    int32_t* counters;            // [kC], zero between launches
-    float* partial;               // [K][H]
+    int32_t* counters;            // [kC] one per block of output rows, zero between launches
+    int32_t* pre_counter;         // rows of the head delivered so far, zero between launches
+    float* partial;               // [K * kDownSlices][H]
+    float* logits_ws;             // [E] logits of the next step's head, gathered across CTAs
     const void* W_pre;            // [E][H] or null
     int32_t* inds_next;
     float* gates_next;
@@ -47,6 +61,10 @@ struct FusedParams {
     int H, I, E, K, group, rank, n_adapters, n_slots, pre_dtype, out_dtype;
     float sigma;
     RecordLayout L;
+    unsigned long long* trace;    // optional [grid CTAs][kTraceMarks] globaltimer stamps, or null
+    int32_t* flags;               // [0..1] routing-ready flags, [2..3] CTAs that have consumed them
+    int flag_in;                  // -1: the routing is already in memory; 0/1: wait for flags[flag_in]
+    int flag_out;                 // -1 or the flag to raise once inds_next / gates_next are written
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -59,9 +77,32 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// L2 policies: expert weights are read once per step and must not push the small tensors that
+// every step reuses (adapters, head, hidden state) out of the L2.
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s_hint(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
+// 16-byte load of data that later steps read again: ask the L2 to keep it
+__device__ __forceinline__ uint4 ld_keep16(const void* p) {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    uint4 v;
+    asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    return v;
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
@@ -76,8 +117,45 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_
         if (mbar_try_wait(bar, parity)) return;
     atomicExch(status, EDG_E_TIMEOUT);
 }
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(const void* local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(local)), "r"(rank));
+    return r;
+}
+// Remote shared-memory stores that count their bytes on an mbarrier of the receiving CTA: the
+// receiver waits on its own barrier, so no cluster-wide fence (which would also wait for every
+// bulk copy in flight into the SM) is needed.
+__device__ __forceinline__ void st_async_f32(uint32_t raddr, float v, uint32_t rbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                 ::"r"(raddr), "r"(__float_as_uint(v)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ void st_async_f32x4(uint32_t raddr, float4 v, uint32_t rbar) {
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1,%2,%3,%4}, [%5];"
+                 ::"r"(raddr), "r"(__float_as_uint(v.x)), "r"(__float_as_uint(v.y)), "r"(__float_as_uint(v.z)),
+                   "r"(__float_as_uint(v.w)), "r"(rbar) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release_gpu(int32_t* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// programmatic dependent launch: let the next kernel in the stream start / wait for the previous one
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ void trace_mark(const FusedParams& p, int m) {
+    if (p.trace != nullptr && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[(size_t)blockIdx.x * kTraceMarks + m] = t;
+    }
+}
 
 __device__ __forceinline__ void store_y(void* y, int out_dtype, size_t i, float v) {
     if (out_dtype == EDG_F32) store_out<float>(static_cast<float*>(y), i, v);
@@ -85,182 +163,356 @@ __device__ __forceinline__ void store_y(void* y, int out_dtype, size_t i, float 
     else store_out<bf16_t>(static_cast<bf16_t*>(y), i, v);
 }
 
-// dot of a bf16 row with the bf16 hidden state, both read from global (L2), one warp
-__device__ __forceinline__ float warp_dot_bf16(const uint16_t* a, const uint16_t* b, int n, int lane) {
-    float acc = 0.f;
-    for (int c = lane * 8; c < n; c += 256) {
-        const uint4 u = *reinterpret_cast<const uint4*>(a + c);
-        const uint4 v = *reinterpret_cast<const uint4*>(b + c);
-        acc = fmaf(bf16_lo(u.x), bf16_lo(v.x), acc); acc = fmaf(bf16_hi(u.x), bf16_hi(v.x), acc);
-        acc = fmaf(bf16_lo(u.y), bf16_lo(v.y), acc); acc = fmaf(bf16_hi(u.y), bf16_hi(v.y), acc);
-        acc = fmaf(bf16_lo(u.z), bf16_lo(v.z), acc); acc = fmaf(bf16_hi(u.z), bf16_hi(v.z), acc);
-        acc = fmaf(bf16_lo(u.w), bf16_lo(v.w), acc); acc = fmaf(bf16_hi(u.w), bf16_hi(v.w), acc);
+// sum_j B[j] * u[j] over a bf16 row in shared memory, r a multiple of 8
+__device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, int r) {
+    float d = 0.f;
+    for (int j = 0; j < r; j += 8) {
+        const uint4 b = *reinterpret_cast<const uint4*>(B + j);
+        d = fmaf(bf16_lo(b.x), u[j + 0], d); d = fmaf(bf16_hi(b.x), u[j + 1], d);
+        d = fmaf(bf16_lo(b.y), u[j + 2], d); d = fmaf(bf16_hi(b.y), u[j + 3], d);
+        d = fmaf(bf16_lo(b.z), u[j + 4], d); d = fmaf(bf16_hi(b.z), u[j + 5], d);
+        d = fmaf(bf16_lo(b.w), u[j + 6], d); d = fmaf(bf16_hi(b.w), u[j + 7], d);
     }
-    return warp_sum(acc);
+    return d;
 }
 
-// shared-memory carve-up of an expert CTA (byte offsets), identical on host and device
+// ---------------------------------------------------------------- shared-memory carve-up
+// Byte offsets, identical on host and device.  The four gate/up stages come first; the down block
+// later reuses stages 0 and 1 (it is exactly half the size of the gate/up slice), which keeps a
+// CTA under half an SM's shared memory so two CTAs -- of this launch or of the next one -- can
+// share an SM.
 struct FusedSmem {
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, flag;
-    uint32_t c_gate, c_up, z_gate, z_up, c_down, z_down, total;
+    uint32_t stage0, stage_bytes;                      // stage s at stage0 + s * stage_bytes
+    uint32_t g_codes, u_codes, g_sz, u_sz;             // offsets inside a stage
+    uint32_t d_codes, d_sz;                            // down block, from stage0
+    uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, flag, total;
 };
-__host__ __device__ inline FusedSmem fused_smem(int H, int I, int group) {
+__host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
-    const uint32_t rows_gu = I / kC, rows_d = H / kC;
+    const uint32_t rows_gu = I / kE16, rows_d = H / kC, rs = rows_gu / kStages, sw = I / kDownSlices;
+    const uint32_t row_b = H / 2, grp_b = (H / group) * 4;
+    S.g_codes = 0;
+    S.u_codes = rs * row_b;
+    S.g_sz = 2 * rs * row_b;
+    S.u_sz = 2 * rs * row_b + rs * grp_b;
+    S.stage_bytes = 2 * rs * (row_b + grp_b);
     uint32_t o = 0;
-    S.bars = o;       o += 8 * (kStages + 1);
+    S.stage0 = o;     o += kStages * S.stage_bytes;
+    S.d_codes = S.stage0;
+    S.d_sz = S.stage0 + rows_d * sw / 2;               // rows_d * (sw/2 + sw/group*4) == 2 * stage_bytes
+    S.b_gate = o;     o += rows_gu * (uint32_t)rank * 2;      // B_gate[n0 .. n0+rows_gu][rank]
+    S.b_up = o;       o += rows_gu * (uint32_t)rank * 2;
+    S.b_down = o;     o += rows_d * (uint32_t)rank * 2;       // B_down[n0 .. n0+rows_d][rank]
+    S.a_down = o;     o += (uint32_t)rank * rows_gu * 2;      // A_down[rank][my rows of h]
+    o = (o + 15) / 16 * 16;
+    S.bars = o;       o += 8 * (kStages + 5);
     o = (o + 15) / 16 * 16;
     S.s_u = o;        o += 2 * kMaxRank * 4;
-    S.s_h = o;        o += (uint32_t)I * 4;
+    S.s_h = o;        o += sw * 4;                    // the cluster's quarter of h
     S.s_ud_part = o;  o += kC * kMaxRank * 4;
     S.s_ud = o;       o += kMaxRank * 4;
     S.s_gu = o;       o += 2 * rows_gu * 4;
     S.s_o = o;        o += rows_d * 4;
+    S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
+    S.s_hloc = o;     o += 32 * 4;
+    S.s_topk = o;     o += (uint32_t)E * 4;           // logits gathered by the warp that finishes the routing
     S.flag = o;       o += 16;
-    o = (o + 127) / 128 * 128;
-    S.c_gate = o;     o += rows_gu * (uint32_t)H / 2;
-    S.c_up = o;       o += rows_gu * (uint32_t)H / 2;
-    S.z_gate = o;     o += rows_gu * (uint32_t)(H / group) * 4;
-    S.z_up = o;       o += rows_gu * (uint32_t)(H / group) * 4;
-    S.c_down = o;     o += rows_d * (uint32_t)I / 2;
-    S.z_down = o;     o += rows_d * (uint32_t)(I / group) * 4;
-    S.total = o;
+    S.total = (o + 15) / 16 * 16;
     return S;
 }
 
-// ---------------------------------------------------------------- prerouter role (one cluster)
+enum { BAR_DOWN = kStages, BAR_LORA = kStages + 1, BAR_FREE = kStages + 2, BAR_U = kStages + 3, BAR_H = kStages + 4 };
 
-template <typename WT>
-__device__ __forceinline__ float pre_row_dot(const void* W, size_t row, const float* sx, int H, int lane);
-template <>
-__device__ __forceinline__ float pre_row_dot<__half>(const void* W, size_t row, const float* sx, int H, int lane) {
-    const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const __half*>(W) + row * H);
+// ---------------------------------------------------------------- prerouter rows (a1) and top-k (a2)
+// The E rows of the head are dealt round-robin to the CTAs of the grid; a row is split over all
+// threads of its CTA (one 16-byte read each), so it costs one trip to memory.  The warp that
+// delivers the last logits (an atomic counter) gathers all E and does softmax + top-k.
+
+// Partial dot of one head row with the hidden state over this thread's elements (8 per sweep of
+// kFW*32*8).  `w0` / `x0` are the values of the first sweep when the caller loaded them early.
+__device__ __forceinline__ float pre_row_partial(const FusedParams& p, int e, int tid, bool preloaded, uint4 w0, uint4 x0) {
     float acc = 0.f;
-#pragma unroll 4
-    for (int c = lane; c < H / 8; c += 32) {
-        const uint4 w = ld_stream16(wp + c);
-        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
-        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
-        const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
-        const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
-        const float* x = sx + c * 8;
-        acc = fmaf(a.x, x[0], acc); acc = fmaf(a.y, x[1], acc);
-        acc = fmaf(b.x, x[2], acc); acc = fmaf(b.y, x[3], acc);
-        acc = fmaf(d.x, x[4], acc); acc = fmaf(d.y, x[5], acc);
-        acc = fmaf(e.x, x[6], acc); acc = fmaf(e.y, x[7], acc);
+    if (p.pre_dtype == EDG_F16) {
+        const __half* wr = static_cast<const __half*>(p.W_pre) + (size_t)e * p.H;
+        for (int c = tid * 8; c < p.H; c += kFW * 32 * 8) {
+            const bool first = preloaded && c == tid * 8;
+            const uint4 w = first ? w0 : ld_keep16(wr + c);
+            const uint4 x = first ? x0 : ld_keep16(p.x + c);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+            const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
+            acc = fmaf(a.x, bf16_lo(x.x), acc); acc = fmaf(a.y, bf16_hi(x.x), acc);
+            acc = fmaf(b.x, bf16_lo(x.y), acc); acc = fmaf(b.y, bf16_hi(x.y), acc);
+            acc = fmaf(d.x, bf16_lo(x.z), acc); acc = fmaf(d.y, bf16_hi(x.z), acc);
+            acc = fmaf(f.x, bf16_lo(x.w), acc); acc = fmaf(f.y, bf16_hi(x.w), acc);
+        }
+    } else {
+        const float* wr = static_cast<const float*>(p.W_pre) + (size_t)e * p.H;
+        for (int c = tid * 4; c < p.H; c += kFW * 32 * 4) {
+            const uint4 w = ld_keep16(wr + c);
+            const uint2 x = *reinterpret_cast<const uint2*>(p.x + c);
+            acc = fmaf(__uint_as_float(w.x), bf16_lo(x.x), acc); acc = fmaf(__uint_as_float(w.y), bf16_hi(x.x), acc);
+            acc = fmaf(__uint_as_float(w.z), bf16_lo(x.y), acc); acc = fmaf(__uint_as_float(w.w), bf16_hi(x.y), acc);
+        }
     }
-    return warp_sum(acc);
-}
-template <>
-__device__ __forceinline__ float pre_row_dot<float>(const void* W, size_t row, const float* sx, int H, int lane) {
-    const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const float*>(W) + row * H);
-    float acc = 0.f;
-#pragma unroll 4
-    for (int c = lane; c < H / 4; c += 32) {
-        const uint4 w = ld_stream16(wp + c);
-        const float* x = sx + c * 4;
-        acc = fmaf(__uint_as_float(w.x), x[0], acc); acc = fmaf(__uint_as_float(w.y), x[1], acc);
-        acc = fmaf(__uint_as_float(w.z), x[2], acc); acc = fmaf(__uint_as_float(w.w), x[3], acc);
-    }
-    return warp_sum(acc);
+    return acc;
 }
 
-__device__ void prerouter_role(const FusedParams& p, uint8_t* smem, int crank) {
-    cg::cluster_group cluster = cg::this_cluster();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float* s_logits = reinterpret_cast<float*>(smem);     // [E]
-    float* s_x = s_logits + p.E;                          // [H]
-    cluster_arrive();                                     // (#0) every CTA of the cluster is running ...
-    for (int i = threadIdx.x; i < p.H; i += blockDim.x) s_x[i] = bf16_bits_to_float(p.x[i]);
-    __syncthreads();
-    cluster_wait();                                       // ... before anyone writes into a peer's shared memory
-    float* leader = cluster.map_shared_rank(s_logits, 0);
-    const int per = (p.E + kC - 1) / kC;
-    const int e0 = crank * per, e1 = min(p.E, e0 + per);
-    for (int e = e0 + warp; e < e1; e += kFW) {
-        const float l = p.pre_dtype == EDG_F16 ? pre_row_dot<__half>(p.W_pre, e, s_x, p.H, lane)
-                                               : pre_row_dot<float>(p.W_pre, e, s_x, p.H, lane);
-        if (lane == 0) leader[e] = l;
+// One warp: publish this CTA's logits (summed from the per-warp partials in s_pre), and if they were
+// the last ones of the head, gather all E, do softmax + top-k and raise the routing-ready flag.
+__device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const FusedSmem& S,
+                                                 const float* s_pre, int n_rows, int lane) {
+    const int ncta = gridDim.x;
+    int mine = 0;
+    if (lane < n_rows) {
+        const int e = blockIdx.x + lane * ncta;
+        if (e < p.E) {
+            float v = 0.f;
+            for (int w = 0; w < kFW; ++w) v += s_pre[lane * kFW + w];
+            p.logits_ws[e] = v;
+            mine = 1;
+        }
     }
-    cluster_arrive();
-    cluster_wait();
-    if (crank != 0) return;
-    if (p.logits_next != nullptr)
-        for (int e = threadIdx.x; e < p.E; e += blockDim.x) p.logits_next[e] = s_logits[e];
-    __syncthreads();
-    if (warp == 0) warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds_next, p.gates_next);
+    const int n_mine = __popc(__ballot_sync(0xFFFFFFFFu, mine));
+    __threadfence();
+    int last = 0;
+    if (lane == 0) last = (atomicAdd(p.pre_counter, n_mine) + n_mine == p.E) ? 1 : 0;
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (last) {
+        __threadfence();
+        float* work = reinterpret_cast<float*>(smem + S.s_topk);
+        for (int i0 = 0; i0 < p.E; i0 += 256) {                 // 8 independent loads per lane and pass
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * 32 + lane;
+                v[u] = i < p.E ? __ldcg(&p.logits_ws[i]) : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * 32 + lane;
+                if (i < p.E) {
+                    work[i] = v[u];
+                    if (p.logits_next != nullptr) p.logits_next[i] = v[u];
+                }
+            }
+        }
+        __syncwarp();
+        warp_softmax_topk(work, p.E, p.K, lane, p.inds_next, p.gates_next);
+        __syncwarp();
+        if (lane == 0) {
+            *p.pre_counter = 0;
+            __threadfence();
+            if (p.flag_out >= 0) st_release_gpu(&p.flags[p.flag_out], 1);
+            if (p.trace != nullptr) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.trace[(size_t)blockIdx.x * kTraceMarks + 15] = t; }
+        }
+    }
 }
 
 // ---------------------------------------------------------------- the fused kernel
-// NCH = H / 1024 (chunks of a gate/up row per lane), LPR_I = I / 32 (lanes per down row).
+// NCH = H / 1024 (chunks of a gate/up row per lane), LPR_D = I / 128 (lanes per down row-slice).
 
-template <int NCH, int LPR_I>
-__global__ void __launch_bounds__(kFW * 32, 1) fused_layer_kernel(FusedParams p) {
+constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
+
+template <int NCH, int LPR_D>
+__global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    cg::cluster_group cluster = cg::this_cluster();
-    const int crank = (int)cluster.block_rank();
-    const int k = blockIdx.x / kC;                 // cluster index: expert position, or K = prerouter
+    const int b16 = blockIdx.x % kE16;             // CTA of the expert
+    const int k = blockIdx.x / kE16;               // position of the expert in the routing
+    const int c = b16 / kC;                        // quarter of the intermediate dimension (cluster of the expert)
+    const int crank = b16 % kC;                    // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
 
-    if (k == p.K) { prerouter_role(p, smem, crank); return; }
-
-    const FusedSmem S = fused_smem(p.H, p.I, p.group);
+    const FusedSmem S = fused_smem(p.H, p.I, p.E, p.group, p.rank);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars);
     float* s_u = reinterpret_cast<float*>(smem + S.s_u);            // [2][kMaxRank]
-    float* s_h = reinterpret_cast<float*>(smem + S.s_h);            // [I]
+    float* s_h = reinterpret_cast<float*>(smem + S.s_h);            // [I/4]
     float* s_ud_part = reinterpret_cast<float*>(smem + S.s_ud_part);// [kC][kMaxRank]
     float* s_ud = reinterpret_cast<float*>(smem + S.s_ud);          // [kMaxRank]
     float* s_gu = reinterpret_cast<float*>(smem + S.s_gu);          // [2][rows_gu]
     float* s_o = reinterpret_cast<float*>(smem + S.s_o);            // [rows_d]
+    float* s_red = reinterpret_cast<float*>(smem + S.s_red);        // [40][kFW]
+    float* s_hloc = reinterpret_cast<float*>(smem + S.s_hloc);      // [rows_gu]
     int* s_flag = reinterpret_cast<int*>(smem + S.flag);
 
-    const int rows_gu = p.I / kC, rows_d = p.H / kC;
-    const int n0_gu = crank * rows_gu, n0_d = crank * rows_d;
+    const int rows_gu = p.I / kE16, rows_d = p.H / kC, sw = p.I / kDownSlices;
+    const int n0_gu = b16 * rows_gu;               // first gate/up row of this CTA (= c * sw + crank * rows_gu)
+    const int n0_d = crank * rows_d;               // first down row of this CTA
     const int r = p.rank;
+    trace_mark(p, 0);
 
-    // ---- a3: take.  The decision is the same in every CTA of the cluster.
-    int slot = p.slots[k];
-    int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
+    // ---- barriers first: peers will count bytes on BAR_U / BAR_H of this CTA, so they must exist
+    //      (and every CTA of the cluster must be running) before anyone sends.  The cluster
+    //      handshake completes while the routing loads below are in flight, and it happens before
+    //      any bulk copy is issued: a cluster-scope fence waits for every copy in flight into the
+    //      SM, so none is used after this point.
+    if (tid == 0) {
+        for (int s = 0; s <= BAR_LORA; ++s) mbar_init(&bars[s], 1);
+        mbar_init(&bars[BAR_FREE], kFW);
+        mbar_init(&bars[BAR_U], 1);
+        mbar_init(&bars[BAR_H], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // bytes this CTA will receive: 2r adapter projections; then the cluster's quarter of h and kC partials of A_down.h
+        if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
+        mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
+    }
+    __syncthreads();
+    cluster_arrive();
+
+    // ---- loads that do not depend on the routing: the hidden state chunks this lane multiplies with
+    uint4 xraw[NCH][4];
+#pragma unroll
+    for (int i = 0; i < NCH; ++i) {
+        const uint4* xp = reinterpret_cast<const uint4*>(p.x + (lane + 32 * i) * 32);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) xraw[i][q] = xp[q];
+    }
+
+    // ---- a1 for the next step: this CTA's rows of the head, every thread 8 elements of each.  They
+    //      depend on nothing but x, so their loads go out first of all.
+    const int n_pre = p.W_pre != nullptr ? (p.E + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const bool pre_fast = n_pre > 0 && n_pre <= 2 && p.pre_dtype == EDG_F16 && p.H == kFW * 32 * 8;
+    uint4 lw[2], lx = make_uint4(0, 0, 0, 0);
+    if (pre_fast) {
+        lx = ld_keep16(p.x + tid * 8);
+#pragma unroll
+        for (int ri = 0; ri < 2; ++ri) {
+            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * (int)gridDim.x, p.E - 1);
+            lw[ri] = ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8);
+        }
+    }
+
+    // ---- the routing may still be on its way: the previous layer-step raises a flag when its top-k
+    //      is written, long before that kernel ends (bounded wait; on a time-out fall back to
+    //      waiting for the whole previous kernel, which is always sufficient)
+    if (p.flag_in >= 0) {
+        if (tid == 0) {
+            uint32_t it = 0;
+            while (ld_acquire_gpu(&p.flags[p.flag_in]) == 0 && ++it < kSpinLimit) {}
+            if (it >= kSpinLimit) { atomicExch(p.status, EDG_E_TIMEOUT); pdl_wait_prior_grid(); }
+        }
+        __syncthreads();
+    }
+    trace_mark(p, 14);
+
+    // ---- a3: take.  The decision is the same in every CTA of the expert.
+    int slot = __ldcg(&p.slots[k]);
+    const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
     if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? p.table[slot] : -1;
     int ad = 0;
     if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
     const bool valid = slot >= 0 && slot < p.n_slots && ad >= 0;
+    const float gate_k = __ldcg(&p.gates[k]);
+    trace_mark(p, 10);
+    if (p.flag_in >= 0) {
+        // the CTA that is last to have read the routing re-arms the flag for the step after next
+        if (tid == 0 && atomicAdd(&p.flags[2 + p.flag_in], 1) == (int)gridDim.x - 1) {
+            p.flags[2 + p.flag_in] = 0;
+            st_release_gpu(&p.flags[p.flag_in], 0);
+        }
+        __syncthreads();
+    }
+    pdl_launch_dependents();              // the next layer-step may start its own prologue now
+    cluster_wait();                       // nothing is in flight yet: this returns at once
+    trace_mark(p, 11);
 
     if (valid) {
-        cluster_arrive();                 // (#0) a peer's shared memory may be written only once it runs
         const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
         const int row_b = p.H / 2, grp_b = (p.H / p.group) * 4;
         const int rs = rows_gu / kStages;                            // gate/up rows per stage
+        const int drow_b = sw / 2, gps = sw / p.group, dgrp_b = gps * 4;   // one row of the down block
 
-        // ---- issue every copy of this CTA's slice
-        if (tid == 0) {
-            for (int s = 0; s <= kStages; ++s) mbar_init(&bars[s], 1);
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            for (int s = 0; s < kStages; ++s) {
-                const int lr = s * rs;                               // local row
-                const size_t gr = (size_t)(n0_gu + lr);              // row in the expert
-                mbar_expect_tx(&bars[s], 2u * rs * (row_b + grp_b));
-                bulk_g2s(smem + S.c_gate + lr * row_b, rec + p.L.codes_gate + gr * row_b, rs * row_b, &bars[s]);
-                bulk_g2s(smem + S.c_up + lr * row_b, rec + p.L.codes_up + gr * row_b, rs * row_b, &bars[s]);
-                bulk_g2s(smem + S.z_gate + lr * grp_b, rec + p.L.sz_gate + gr * grp_b, rs * grp_b, &bars[s]);
-                bulk_g2s(smem + S.z_up + lr * grp_b, rec + p.L.sz_up + gr * grp_b, rs * grp_b, &bars[s]);
+        // ---- issue the copies of this CTA's gate/up slice and adapter rows, one warp per barrier
+        if (lane == 0) {
+            const uint64_t pol = policy_evict_first();       // weights stream through L2 once
+            if (warp < kStages) {
+                const int s = warp;
+                uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+                const size_t gr = (size_t)(n0_gu + s * rs);          // first row of the stage in the expert
+                mbar_expect_tx(&bars[s], S.stage_bytes);
+                bulk_g2s_hint(st + S.g_codes, rec + p.L.codes_gate + gr * row_b, rs * row_b, &bars[s], pol);
+                bulk_g2s_hint(st + S.u_codes, rec + p.L.codes_up + gr * row_b, rs * row_b, &bars[s], pol);
+                bulk_g2s_hint(st + S.g_sz, rec + p.L.sz_gate + gr * grp_b, rs * grp_b, &bars[s], pol);
+                bulk_g2s_hint(st + S.u_sz, rec + p.L.sz_up + gr * grp_b, rs * grp_b, &bars[s], pol);
+            } else if (warp == kStages && r > 0) {
+                // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
+                const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
+                mbar_expect_tx(&bars[BAR_LORA], 2 * bgu + bd + r * ad_row);
+                const size_t bo = ((size_t)ad * p.I + n0_gu) * r * 2;
+                bulk_g2s(smem + S.b_gate, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA]);
+                bulk_g2s(smem + S.b_up, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA]);
+                bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd,
+                         &bars[BAR_LORA]);
+                for (int j = 0; j < r; ++j)
+                    bulk_g2s(smem + S.a_down + j * ad_row,
+                             static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0_gu) * 2, ad_row,
+                             &bars[BAR_LORA]);
             }
-            const int drow_b = p.I / 2, dgrp_b = (p.I / p.group) * 4;
-            mbar_expect_tx(&bars[kStages], (uint32_t)rows_d * (drow_b + dgrp_b));
-            bulk_g2s(smem + S.c_down, rec + p.L.codes_down + (size_t)n0_d * drow_b, rows_d * drow_b, &bars[kStages]);
-            bulk_g2s(smem + S.z_down, rec + p.L.sz_down + (size_t)n0_d * dgrp_b, rows_d * dgrp_b, &bars[kStages]);
+        }
+        trace_mark(p, 1);
+    }
+
+    // ---- head rows: per-warp partials, then the last warp publishes them (and finishes the routing
+    //      of the next step if they were the last to arrive).  Publishing comes after the flag wait
+    //      above, i.e. after the previous layer-step is done with the shared logits scratch.
+    if (n_pre > 0) {
+        for (int ri = 0; ri < n_pre; ++ri) {
+            const int e = (int)blockIdx.x + ri * (int)gridDim.x;
+            float v = e < p.E ? pre_row_partial(p, e, tid, pre_fast, lw[ri & 1], lx) : 0.f;
+            v = warp_sum(v);
+            if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
+        }
+        __syncthreads();
+        if (warp == kFW - 1) prerouter_finish(p, smem, S, s_red + kPreRed * kFW, n_pre, lane);
+    }
+    trace_mark(p, 12);
+
+    if (valid) {
+        const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
+        const int row_b = p.H / 2;
+        const int rs = rows_gu / kStages;                            // gate/up rows per stage
+        const int drow_b = sw / 2, gps = sw / p.group, dgrp_b = gps * 4;   // one row of the down block
+
+        // ---- LoRA: this CTA's share of the 2r rows of A_gate / A_up.  All threads take part: each
+        //      one covers 8 elements of a row per sweep, so a row costs one round trip to the L2.
+        const int per = (2 * r + kC - 1) / kC;
+        for (int q0 = 0; q0 < per; q0 += 4) {
+            float v[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int cc = tid * 8; cc < p.H; cc += kFW * 32 * 8) {
+                const uint4 ux = ld_keep16(p.x + cc);
+                uint4 ua[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int q = min(crank * per + min(q0 + u, per - 1), 2 * r - 1);
+                    const uint16_t* A = reinterpret_cast<const uint16_t*>((q / r) ? p.lora.A_up : p.lora.A_gate) + ((size_t)ad * r + q % r) * p.H;
+                    ua[u] = ld_keep16(A + cc);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    v[u] = fmaf(bf16_lo(ua[u].x), bf16_lo(ux.x), v[u]); v[u] = fmaf(bf16_hi(ua[u].x), bf16_hi(ux.x), v[u]);
+                    v[u] = fmaf(bf16_lo(ua[u].y), bf16_lo(ux.y), v[u]); v[u] = fmaf(bf16_hi(ua[u].y), bf16_hi(ux.y), v[u]);
+                    v[u] = fmaf(bf16_lo(ua[u].z), bf16_lo(ux.z), v[u]); v[u] = fmaf(bf16_hi(ua[u].z), bf16_hi(ux.z), v[u]);
+                    v[u] = fmaf(bf16_lo(ua[u].w), bf16_lo(ux.w), v[u]); v[u] = fmaf(bf16_hi(ua[u].w), bf16_hi(ux.w), v[u]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float t = warp_sum(v[u]);
+                if (lane == 0 && q0 + u < per) s_red[(q0 + u) * kFW + warp] = t;
+            }
         }
 
         // ---- hidden state -> pre-scaled registers (each lane owns NCH chunks of 32)
         float xs[NCH][32], xsum[NCH];
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
-            const uint4* xp = reinterpret_cast<const uint4*>(p.x + (lane + 32 * i) * 32);
             float xv[32];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const uint4 v = xp[q];
+                const uint4 v = xraw[i][q];
                 xv[q * 8 + 0] = bf16_lo(v.x); xv[q * 8 + 1] = bf16_hi(v.x);
                 xv[q * 8 + 2] = bf16_lo(v.y); xv[q * 8 + 3] = bf16_hi(v.y);
                 xv[q * 8 + 4] = bf16_lo(v.z); xv[q * 8 + 5] = bf16_hi(v.z);
@@ -268,34 +520,53 @@ __global__ void __launch_bounds__(kFW * 32, 1) fused_layer_kernel(FusedParams p)
             }
             xsum[i] = scale_chunk(xv, xs[i]);
         }
-
-        cluster_wait();                   // (#0)
-        // ---- LoRA: this CTA's share of the 2r rows of A_gate / A_up, broadcast to the cluster
-        if (r > 0) {
-            const int per = (2 * r + kC - 1) / kC;
-            for (int q = crank * per + warp; q < min(2 * r, (crank + 1) * per); q += kFW) {
-                const int proj = q / r, j = q % r;
-                const uint16_t* A = reinterpret_cast<const uint16_t*>(proj ? p.lora.A_up : p.lora.A_gate) + ((size_t)ad * r + j) * p.H;
-                const float v = warp_dot_bf16(A, p.x, p.H, lane);
-                if (lane < kC) cluster.map_shared_rank(s_u, lane)[proj * kMaxRank + j] = v;
+        if (p.trace != nullptr && tid == 0) { unsigned sm; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); p.trace[(size_t)blockIdx.x * kTraceMarks + 13] = sm; }
+        __syncthreads();                  // s_red complete
+        // every CTA of the cluster gets this CTA's adapter projections, counted on its BAR_U
+        for (int i = tid; i < per * kC; i += kFW * 32) {
+            const int qi = i / kC, dst = i % kC, q = crank * per + qi;
+            if (q < 2 * r) {
+                float v = 0.f;
+                for (int w = 0; w < kFW; ++w) v += s_red[qi * kFW + w];
+                st_async_f32(map_to_cta(&s_u[(q / r) * kMaxRank + (q % r)], dst), v, map_to_cta(&bars[BAR_U], dst));
             }
         }
-        __syncthreads();                  // barriers initialised before anyone polls them
-        cluster_arrive();                 // (#1) my A.x values are out; wait for the others later
+        trace_mark(p, 2);
 
-        // ---- gate/up GEMV over this CTA's rows, stage by stage as the copies land
+        // ---- gate/up GEMV over this CTA's rows, stage by stage as the copies land.  Once every
+        //      warp is past stages 0 and 1 their space is refilled with the CTA's block of down.
         {
             const int groups = p.H / p.group;
-            for (int lr = warp; lr < rows_gu; lr += kFW) {
-                mbar_wait(&bars[lr / rs], 0, p.status);
+            bool freed = false;
+            for (int lr = warp;; lr += kFW) {
+                const int s = lr < rows_gu ? lr / rs : kStages;
+                if (s >= 2 && !freed) {
+                    freed = true;
+                    if (lane == 0) mbar_arrive(&bars[BAR_FREE]);
+                    if (warp == 0) {
+                        mbar_wait(&bars[BAR_FREE], 0, p.status);
+                        if (lane == 0) {
+                            const uint64_t pol = policy_evict_first();
+                            const size_t row0 = (size_t)c * p.H + n0_d;      // first row of the block in the sliced layout
+                            mbar_expect_tx(&bars[BAR_DOWN], (uint32_t)rows_d * (drow_b + dgrp_b));
+                            bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + row0 * drow_b, rows_d * drow_b, &bars[BAR_DOWN], pol);
+                            bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + row0 * dgrp_b, rows_d * dgrp_b, &bars[BAR_DOWN], pol);
+                        }
+                    }
+                }
+                if (lr >= rows_gu) break;
+                mbar_wait(&bars[s], 0, p.status);
+                if (lr == warp) trace_mark(p, 3);
+                const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+                const int sr = lr - s * rs;                          // row inside the stage
                 float ag = 0.f, au = 0.f;
 #pragma unroll
                 for (int i = 0; i < NCH; ++i) {
-                    const int c = lane + 32 * i;
-                    const uint4 wg = *reinterpret_cast<const uint4*>(smem + S.c_gate + lr * row_b + c * 16);
-                    const uint4 wu = *reinterpret_cast<const uint4*>(smem + S.c_up + lr * row_b + c * 16);
-                    const uint32_t zg = *reinterpret_cast<const uint32_t*>(smem + S.z_gate + (lr * groups + (c * 32) / p.group) * 4);
-                    const uint32_t zu = *reinterpret_cast<const uint32_t*>(smem + S.z_up + (lr * groups + (c * 32) / p.group) * 4);
+                    const int ch = lane + 32 * i;
+                    const uint4 wg = *reinterpret_cast<const uint4*>(st + S.g_codes + sr * row_b + ch * 16);
+                    const uint4 wu = *reinterpret_cast<const uint4*>(st + S.u_codes + sr * row_b + ch * 16);
+                    const uint32_t zg = *reinterpret_cast<const uint32_t*>(st + S.g_sz + (sr * groups + (ch * 32) / p.group) * 4);
+                    const uint32_t zu = *reinterpret_cast<const uint32_t*>(st + S.u_sz + (sr * groups + (ch * 32) / p.group) * 4);
                     ag += chunk_affine(chunk_dot(wg, xs[i]), xsum[i], zg);
                     au += chunk_affine(chunk_dot(wu, xs[i]), xsum[i], zu);
                 }
@@ -305,46 +576,51 @@ __global__ void __launch_bounds__(kFW * 32, 1) fused_layer_kernel(FusedParams p)
             }
         }
         __syncthreads();
-        cluster_wait();                   // (#1) every CTA's A.x has landed in s_u
+        trace_mark(p, 4);
+        if (r > 0) mbar_wait(&bars[BAR_U], 0, p.status);            // every CTA's A.x has landed in s_u
+        trace_mark(p, 5);
 
-        // ---- finish gate/up: LoRA B, SiLU, product; all-gather h and the partial of A_down . h
-        if (warp == 0) {
-            float hval = 0.f;
-            if (lane < rows_gu) {
-                float g = s_gu[lane], u = s_gu[rows_gu + lane];
-                if (r > 0) {
-                    const size_t bo = ((size_t)ad * p.I + n0_gu + lane) * r;
-                    const uint16_t* Bg = reinterpret_cast<const uint16_t*>(p.lora.B_gate) + bo;
-                    const uint16_t* Bu = reinterpret_cast<const uint16_t*>(p.lora.B_up) + bo;
-                    float dg = 0.f, du = 0.f;
-                    for (int j = 0; j < r; ++j) {
-                        dg = fmaf(bf16_bits_to_float(Bg[j]), s_u[j], dg);
-                        du = fmaf(bf16_bits_to_float(Bu[j]), s_u[kMaxRank + j], du);
-                    }
-                    g = fmaf(p.sigma, dg, g);
-                    u = fmaf(p.sigma, du, u);
-                }
-                hval = silu_f(g) * u;
-                for (int c = 0; c < kC; ++c) cluster.map_shared_rank(s_h, c)[n0_gu + lane] = hval;
-            }
-            for (int j = 0; j < r; ++j) {
-                const uint16_t* Ad = reinterpret_cast<const uint16_t*>(p.lora.A_down) + ((size_t)ad * r + j) * p.I + n0_gu;
-                float v = lane < rows_gu ? bf16_bits_to_float(Ad[lane]) * hval : 0.f;
-                v = warp_sum(v);
-                if (lane < kC) cluster.map_shared_rank(s_ud_part, lane)[crank * kMaxRank + j] = v;
+        // ---- finish gate/up: LoRA B (one thread per (projection, row)), SiLU, product
+        if (r > 0 && tid < 2 * rows_gu) {
+            mbar_wait(&bars[BAR_LORA], 0, p.status);
+            const int proj = tid / rows_gu, row = tid % rows_gu;
+            const uint16_t* Bm = reinterpret_cast<const uint16_t*>(smem + (proj ? S.b_up : S.b_gate)) + row * r;
+            const float d = smem_b_dot(Bm, s_u + proj * kMaxRank, r);
+            s_gu[proj * rows_gu + row] = fmaf(p.sigma, d, s_gu[proj * rows_gu + row]);
+        }
+        __syncthreads();
+        if (tid < rows_gu) s_hloc[tid] = silu_f(s_gu[tid]) * s_gu[rows_gu + tid];
+        __syncthreads();
+        // all-gather h inside the cluster: this CTA's rows_gu values go to every CTA, 16 bytes at a time
+        {
+            const int vecs = rows_gu / 4;
+            for (int i = tid; i < vecs * kC; i += kFW * 32) {
+                const int v = i % vecs, dst = i / vecs;
+                st_async_f32x4(map_to_cta(&s_h[crank * rows_gu + 4 * v], dst), *reinterpret_cast<const float4*>(&s_hloc[4 * v]),
+                               map_to_cta(&bars[BAR_H], dst));
             }
         }
-        cluster_arrive();                 // (#2)
-        cluster_wait();                   // h and the A_down partials of the whole expert are here
+        // partial of A_down . h over this CTA's rows of h (kC lanes per rank index), sent to every CTA of the cluster
+        for (int j = tid / kC; j < r; j += kFW * 32 / kC) {
+            const int part = tid % kC;
+            const uint16_t* Ad = reinterpret_cast<const uint16_t*>(smem + S.a_down) + j * rows_gu;
+            float v = 0.f;
+            for (int n = part; n < rows_gu; n += kC) v = fmaf(bf16_bits_to_float(Ad[n]), s_hloc[n], v);
+            v = group_sum<kC>(v);
+            st_async_f32(map_to_cta(&s_ud_part[crank * kMaxRank + j], part), v, map_to_cta(&bars[BAR_H], part));
+        }
+        trace_mark(p, 6);
+        mbar_wait(&bars[BAR_H], 0, p.status);                       // the cluster's quarter of h and of A_down.h
+        trace_mark(p, 7);
 
-        // ---- down GEMV over this CTA's H/16 output rows
+        // ---- down: partial over this quarter of the columns, for this CTA's H/4 output rows
         if (tid < r) {
             float v = 0.f;
-            for (int c = 0; c < kC; ++c) v += s_ud_part[c * kMaxRank + tid];
+            for (int cc = 0; cc < kC; ++cc) v += s_ud_part[cc * kMaxRank + tid];
             s_ud[tid] = v;
         }
-        constexpr int RPW = 32 / LPR_I;
-        const int sub = lane % LPR_I, rsub = lane / LPR_I;
+        constexpr int RPW = 32 / LPR_D;
+        const int sub = lane % LPR_D, rsub = lane / LPR_D;
         float hs[32];
         float hsum;
         {
@@ -357,81 +633,93 @@ __global__ void __launch_bounds__(kFW * 32, 1) fused_layer_kernel(FusedParams p)
             }
             hsum = scale_chunk(hv, hs);
         }
-        __syncthreads();                  // s_ud ready
-        mbar_wait(&bars[kStages], 0, p.status);
-        const float gate_k = p.gates[k];
-        const int drow_b = p.I / 2, dgroups = p.I / p.group;
+        mbar_wait(&bars[BAR_DOWN], 0, p.status);
+#pragma unroll 2
         for (int lr = warp * RPW + rsub; lr < rows_d; lr += kFW * RPW) {
-            const uint4 wd = *reinterpret_cast<const uint4*>(smem + S.c_down + lr * drow_b + sub * 16);
-            const uint32_t zd = *reinterpret_cast<const uint32_t*>(smem + S.z_down + (lr * dgroups + (sub * 32) / p.group) * 4);
+            const uint4 wd = *reinterpret_cast<const uint4*>(smem + S.d_codes + lr * drow_b + sub * 16);
+            const uint32_t zd = *reinterpret_cast<const uint32_t*>(smem + S.d_sz + (lr * gps + (sub * 32) / p.group) * 4);
             float acc = chunk_affine(chunk_dot(wd, hs), hsum, zd);
-            acc = group_sum<LPR_I>(acc);
-            if (sub == 0) {
-                float o = acc * kUnscale;
-                if (r > 0) {
-                    const uint16_t* Bd = reinterpret_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d + lr) * r;
-                    float dd = 0.f;
-                    for (int j = 0; j < r; ++j) dd = fmaf(bf16_bits_to_float(Bd[j]), s_ud[j], dd);
-                    o = fmaf(p.sigma, dd, o);
-                }
-                s_o[lr] = gate_k * o;
-            }
+            acc = group_sum<LPR_D>(acc);
+            if (sub == 0) s_o[lr] = acc * kUnscale;
         }
-        __syncthreads();
+        __syncthreads();                  // s_o and s_ud complete
+        pdl_wait_prior_grid();            // the reduce scratch belongs to the previous layer-step until it ends
+        // LoRA B for down (on this quarter's share of A_down.h) and the gate weight: one thread per output row
+        for (int lr = tid; lr < rows_d; lr += kFW * 32) {
+            float o = s_o[lr];
+            if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
+            p.partial[((size_t)k * kDownSlices + c) * p.H + n0_d + lr] = gate_k * o;
+        }
+        trace_mark(p, 8);
     } else {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
-        for (int i = tid; i < rows_d; i += blockDim.x) s_o[i] = 0.f;     // a skipped expert contributes nothing
-        __syncthreads();
+        pdl_wait_prior_grid();
+        // a skipped expert contributes nothing
+        for (int i = tid; i < rows_d; i += blockDim.x) p.partial[((size_t)k * kDownSlices + c) * p.H + n0_d + i] = 0.f;
     }
 
-    // ---- a6: publish this expert's gate-weighted slice; the last arriver sums the K partials
-    for (int i = tid; i < rows_d; i += blockDim.x) p.partial[(size_t)k * p.H + n0_d + i] = s_o[i];
+    // ---- a6: this partial is published; the last arriver for the block of rows sums all 4K partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&p.counters[crank], 1) == p.K - 1) ? 1 : 0;
+    if (tid == 0) s_flag[0] = (atomicAdd(&p.counters[crank], 1) == p.K * kDownSlices - 1) ? 1 : 0;
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
-        for (int i = tid; i < rows_d; i += blockDim.x) {
-            float yv = 0.f;
-            for (int kk = 0; kk < p.K; ++kk) yv += __ldcg(&p.partial[(size_t)kk * p.H + n0_d + i]);
-            store_y(p.y, p.out_dtype, (size_t)n0_d + i, yv);
+        const int np = p.K * kDownSlices;
+        for (int i = tid; i < rows_d / 4; i += blockDim.x) {
+            float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int kk = 0; kk < np; ++kk) {
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(&p.partial[(size_t)kk * p.H + n0_d + 4 * i]));
+                yv.x += t.x; yv.y += t.y; yv.z += t.z; yv.w += t.w;
+            }
+            const size_t o = (size_t)n0_d + 4 * i;
+            store_y(p.y, p.out_dtype, o + 0, yv.x); store_y(p.y, p.out_dtype, o + 1, yv.y);
+            store_y(p.y, p.out_dtype, o + 2, yv.z); store_y(p.y, p.out_dtype, o + 3, yv.w);
         }
         if (tid == 0) p.counters[crank] = 0;
     }
+    trace_mark(p, 9);
 }
 
 // ---------------------------------------------------------------- host side
 
+static unsigned long long* g_trace = nullptr;     // set by edg_set_trace_buffer
+
+constexpr size_t kFusedSmemLimit = 112 * 1024;    // two CTAs per SM
+
 bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
-    if ((d.I / kC) % kStages != 0 || d.I / kC > 32) return false;
-    return fused_smem(d.H, d.I, d.group).total <= 200 * 1024;
+    if ((d.I / kE16) % kStages != 0 || d.I / kE16 > 32) return false;
+    if (d.rank % 8 != 0) return false;            // adapter slices are staged by 16-byte bulk copies
+    return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
 }
 
-template <int NCH, int LPR_I>
-static cudaError_t launch_fused(const FusedParams& p, bool with_pre, size_t smem, cudaStream_t st) {
-    auto kern = fused_layer_kernel<NCH, LPR_I>;
+template <int NCH, int LPR_D>
+static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cudaStream_t st) {
+    auto kern = fused_layer_kernel<NCH, LPR_D>;
     static bool configured = false;       // per-process, per-instantiation one-time attributes
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmemLimit);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        // two CTAs per SM: more clusters resident at once
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.K + (with_pre ? 1 : 0)) * kC, 1, 1);
+    cfg.gridDim = dim3(p.K * kE16, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = kC;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
@@ -439,7 +727,7 @@ static cudaError_t launch_fused(const FusedParams& p, bool with_pre, size_t smem
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, cudaStream_t st) {
+                        void* workspace, int flag_in, int flag_out, cudaStream_t st) {
     const bool has_lora = lora != nullptr && d->rank > 0;
     FusedParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);
@@ -451,7 +739,9 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     p.status = reinterpret_cast<int32_t*>(ws + W.ctrl);
     p.counters = reinterpret_cast<int32_t*>(ws + W.ctrl + 64);
+    p.pre_counter = reinterpret_cast<int32_t*>(ws + W.ctrl + 128);
     p.partial = reinterpret_cast<float*>(ws + W.partial);
+    p.logits_ws = reinterpret_cast<float*>(ws + W.logits);
     p.W_pre = W_pre; p.inds_next = inds_next; p.gates_next = gates_next; p.logits_next = logits_next;
     p.H = d->H; p.I = d->I; p.E = d->E; p.K = d->K; p.group = d->group;
     p.rank = has_lora ? d->rank : 0;
@@ -459,18 +749,31 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.pre_dtype = d->pre_dtype; p.out_dtype = d->out_dtype;
     p.sigma = d->lora_scale;
     p.L = record_layout(d->H, d->I, d->group);
-    size_t smem = fused_smem(d->H, d->I, d->group).total;
-    const size_t pre_smem = (size_t)(d->E + d->H) * sizeof(float);
-    if (W_pre != nullptr && pre_smem > smem) smem = pre_smem;
-    const bool with_pre = W_pre != nullptr;
+    p.trace = g_trace;
+    p.flags = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.flag_in = flag_in;
+    p.flag_out = W_pre != nullptr ? flag_out : -1;
+    const bool pdl = flag_in >= 0;
+    // a call that starts a chain clears flags a broken chain may have left raised
+    if (W_pre != nullptr && flag_in < 0) EDG_CUDA_TRY(cudaMemsetAsync(p.flags, 0, 4 * sizeof(int32_t), st));
+    const size_t smem = fused_smem(d->H, d->I, d->E, d->group, p.rank).total;
     cudaError_t e;
-    if (d->H == 2048 && d->I == 512) e = launch_fused<2, 16>(p, with_pre, smem, st);
-    else if (d->H == 2048 && d->I == 256) e = launch_fused<2, 8>(p, with_pre, smem, st);
-    else if (d->H == 1024 && d->I == 512) e = launch_fused<1, 16>(p, with_pre, smem, st);
-    else if (d->H == 1024 && d->I == 256) e = launch_fused<1, 8>(p, with_pre, smem, st);
+    if (d->H == 2048 && d->I == 512) e = launch_fused<2, 4>(p, smem, pdl, st);
+    else if (d->H == 2048 && d->I == 256) e = launch_fused<2, 2>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 512) e = launch_fused<1, 4>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 256) e = launch_fused<1, 2>(p, smem, pdl, st);
     else return EDG_E_SHAPE;
     EDG_CUDA_TRY(e);
     return EDG_OK;
 }
 
 }  // namespace edg
+
+// Tracing hook: with a device buffer of (CTAs in the grid) x 16 uint64, every CTA of the fused
+// layer kernel stamps %globaltimer (ns) at its phase boundaries: 0 start, 1 copies issued,
+// 2 adapter projections sent, 3 first weights landed, 4 gate/up done, 5 peers' projections in,
+// 6 h sent, 7 h of the whole expert in, 8 down done, 9 end.  NULL switches tracing off.
+extern "C" int32_t edg_set_trace_buffer(void* dev_buffer) {
+    edg::g_trace = static_cast<unsigned long long*>(dev_buffer);
+    return EDG_OK;
+}

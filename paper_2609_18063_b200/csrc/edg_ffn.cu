@@ -12,7 +12,7 @@ bool fused_supported(const edg_layer_desc& d);
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, cudaStream_t st);
+                        void* workspace, int flag_in, int flag_out, cudaStream_t st);
 
 struct FfnParams {
     const uint8_t* pool;        // slot records of one layer
@@ -95,10 +95,21 @@ __global__ void __launch_bounds__(256) lora_a_kernel(FfnParams p, int phase, int
     }
 }
 
-// sigma * sum_j B[row][j] * u[j]  (B bf16 [.][rank])
+// sum_j B[row][j] * u[j]  (B bf16 [.][rank]); 16-byte loads when the row allows it, so the
+// loads of a row are independent of one another
 __device__ __forceinline__ float lora_b_dot(const uint16_t* Brow, const float* u, int r) {
     float acc = 0.f;
-    for (int j = 0; j < r; ++j) acc = fmaf(bf16_bits_to_float(Brow[j]), u[j], acc);
+    if ((r & 7) == 0) {
+        for (int j = 0; j < r; j += 8) {
+            const uint4 b = *reinterpret_cast<const uint4*>(Brow + j);
+            acc = fmaf(bf16_lo(b.x), u[j + 0], acc); acc = fmaf(bf16_hi(b.x), u[j + 1], acc);
+            acc = fmaf(bf16_lo(b.y), u[j + 2], acc); acc = fmaf(bf16_hi(b.y), u[j + 3], acc);
+            acc = fmaf(bf16_lo(b.z), u[j + 4], acc); acc = fmaf(bf16_hi(b.z), u[j + 5], acc);
+            acc = fmaf(bf16_lo(b.w), u[j + 6], acc); acc = fmaf(bf16_hi(b.w), u[j + 7], acc);
+        }
+    } else {
+        for (int j = 0; j < r; ++j) acc = fmaf(bf16_bits_to_float(Brow[j]), u[j], acc);
+    }
     return acc;
 }
 
@@ -198,7 +209,6 @@ __global__ void __launch_bounds__(kWarps * 32) down_kernel(FfnParams p) {
     const int sub = lane % LPR, rsub = lane / LPR;
     const int t = blockIdx.z;
     const int n = blockIdx.x * (kWarps * RPW) + warp * RPW + rsub;
-    const int row_bytes = p.I / 2, groups = p.I / p.group;
     extern __shared__ float sud[];            // [K][rank]
 
     for (int i = threadIdx.x; i < p.K * p.rank; i += blockDim.x) sud[i] = p.u_d[(size_t)t * p.K * p.rank + i];
@@ -216,8 +226,8 @@ __global__ void __launch_bounds__(kWarps * 32) down_kernel(FfnParams p) {
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
             const int c = sub + LPR * i;
-            cd[i] = ld_stream16(rec + p.L.codes_down + (size_t)n * row_bytes + c * 16);
-            zd[i] = ld_stream4(rec + p.L.sz_down + ((size_t)n * groups + (c * 32) / p.group) * 4);
+            cd[i] = ld_stream16(rec + p.L.codes_down + down_code_off(p.H, p.I, n, c));
+            zd[i] = ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n, (c * 32) / p.group));
         }
         float acc = 0.f;
 #pragma unroll
@@ -294,7 +304,7 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
     // batch-1 decode on the shapes the fused kernel covers: one launch for the whole FFN
     if (T == 1 && fused_supported(*d))
         return run_fused_layer(d, slot_pool, slots, table, experts, gates, x, has_lora ? lora : nullptr, y,
-                               nullptr, nullptr, nullptr, nullptr, workspace, st);
+                               nullptr, nullptr, nullptr, nullptr, workspace, -1, -1, st);
 
     FfnParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);

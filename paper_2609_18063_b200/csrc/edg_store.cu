@@ -20,7 +20,7 @@ bool fused_supported(const edg_layer_desc& d);
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, cudaStream_t st);
+                        void* workspace, int flag_in, int flag_out, cudaStream_t st);
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
                       int32_t* inds, float* gates, float* logits_opt, cudaStream_t st);
 }  // namespace edg
@@ -58,6 +58,13 @@ struct edg_store {
     bool ring_used[kRing] = {};
     int ring_pos = 0;
     edg_store_stats stats{};
+    // chaining of consecutive batch-1 layer-steps: when a call consumes the routing that the
+    // previous call on the same stream and workspace produced, its kernel is launched as a
+    // programmatic dependent of that one and waits on a device flag instead of the kernel's end
+    const void* chain_inds = nullptr;
+    const void* chain_ws = nullptr;
+    void* chain_stream = nullptr;
+    int chain_flag = 0;
 };
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
@@ -256,10 +263,18 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         if (!workspace || !edg::aligned(workspace, 256) || workspace_bytes < edg::workspace_layout(s->d, 1).bytes)
             return EDG_E_WORKSPACE;
         if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
+        const bool chained = s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
+                             s->chain_stream == stream;
+        const int flag_in = chained ? s->chain_flag : -1;
+        const int flag_out = chained ? 1 - flag_in : 0;
         rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
-                                  logits_next_opt, workspace, st);
+                                  logits_next_opt, workspace, flag_in, flag_out, st);
         if (rc != EDG_OK) return rc;
+        s->chain_inds = W_pre_next != nullptr ? inds_next : nullptr;
+        s->chain_ws = workspace;
+        s->chain_stream = stream;
+        s->chain_flag = flag_out;
     } else {
         rc = edg::run_ffn(&s->d, pool, 1, inds_cur, table, nullptr, gates_cur, x, lora, y, workspace, workspace_bytes, st);
         if (rc != EDG_OK) return rc;
