@@ -72,6 +72,14 @@ struct WorkspaceLayout {
     size_t u_d;       // [T][K][rank] float         : A_down h
     size_t partial;   // [K*kDownSlices][H] float   : gate-weighted partial expert outputs of the fused batch-1 kernel
     size_t logits;    // [E] float                  : next-step head logits gathered across CTAs
+    // grouped path (T > 1) only:
+    size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
+    size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
+    size_t pair_ad;   // [T*K] int32                : adapter of every pair
+    size_t counts;    // [n_slots] int32            : pairs per slot
+    size_t n_tiles;   // int32
+    size_t tiles;     // [T*K/64 + n_slots][2] int32: (slot, first position) of every 64-pair tile
+    size_t lists;     // [n_slots][T] int32         : pairs of every slot, ascending
     size_t bytes;
 };
 
@@ -87,7 +95,19 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
     W.logits = round_up(W.partial + (size_t)d.K * 4 * d.H * sizeof(float), 256);
-    W.bytes = round_up(W.logits + (size_t)d.E * sizeof(float), 256);
+    size_t end = round_up(W.logits + (size_t)d.E * sizeof(float), 256);
+    W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
+    if (T > 1) {
+        const size_t P = (size_t)T * d.K;
+        W.o = end;                 end = round_up(W.o + P * d.H * sizeof(float), 256);
+        W.pair_slot = end;         end = round_up(W.pair_slot + P * 4, 256);
+        W.pair_ad = end;           end = round_up(W.pair_ad + P * 4, 256);
+        W.counts = end;            end = round_up(W.counts + (size_t)d.n_slots * 4, 256);
+        W.n_tiles = end;           end += 256;
+        W.tiles = end;             end = round_up(W.tiles + (P / 64 + 1 + d.n_slots) * 8, 256);
+        W.lists = end;             end = round_up(W.lists + (size_t)d.n_slots * T * 4, 256);
+    }
+    W.bytes = end;
     return W;
 }
 

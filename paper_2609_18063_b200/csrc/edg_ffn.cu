@@ -14,6 +14,10 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
                         void* workspace, int flag_in, int flag_out, cudaStream_t st);
 
+int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots, const int32_t* table,
+                    const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
+                    void* workspace, cudaStream_t st);
+
 struct FfnParams {
     const uint8_t* pool;        // slot records of one layer
     const int32_t* slots;       // [T][K] slot per routed expert, or expert ids when `table` is set
@@ -306,6 +310,9 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
         return run_fused_layer(d, slot_pool, slots, table, experts, gates, x, has_lora ? lora : nullptr, y,
                                nullptr, nullptr, nullptr, nullptr, workspace, -1, -1, st);
 
+    // several tokens: group the (token, choice) pairs per expert and run the tensor-core path
+    if (T > 1) return run_grouped(d, slot_pool, T, slots, table, experts, gates, x, has_lora ? lora : nullptr, y, workspace, st);
+
     FfnParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);
     p.slots = slots; p.table = table; p.experts = experts; p.gates = gates;
@@ -336,6 +343,22 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
     EDG_DISPATCH_CHUNKS(d->I / 32, launch_down, p, T, d->out_dtype, st);
     EDG_CUDA_TRY(cudaGetLastError());
     return EDG_OK;
+}
+
+// rank-r projections for the grouped path: phase 0 = A_gate/A_up . x, phase 1 = A_down . h
+void launch_lora_a(const edg_layer_desc* d, const void* slots, const void* table, const void* experts, const void* x,
+                   const edg_lora* lora, float* u_gu, float* h, float* u_d, int32_t* status, int T, int phase, cudaStream_t st) {
+    FfnParams p{};
+    p.slots = static_cast<const int32_t*>(slots); p.table = static_cast<const int32_t*>(table);
+    p.experts = static_cast<const int32_t*>(experts);
+    p.x = static_cast<const uint16_t*>(x);
+    p.lora = *lora;
+    p.status = status; p.u_gu = u_gu; p.h = h; p.u_d = u_d;
+    p.H = d->H; p.I = d->I; p.E = d->E; p.K = d->K; p.group = d->group; p.rank = d->rank;
+    p.n_adapters = d->n_adapters; p.n_slots = d->n_slots;
+    const int n_sets = d->n_adapters == 1 ? 1 : d->K;
+    const int warps = phase == 0 ? n_sets * 2 * p.rank : p.K * p.rank;
+    lora_a_kernel<<<dim3((warps + 7) / 8, T), 256, 0, st>>>(p, phase, n_sets);
 }
 
 }  // namespace edg

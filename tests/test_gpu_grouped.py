@@ -1,0 +1,114 @@
+"""Batched decode (config 4 shape) and prefill (config 5 shape, reduced token count): the grouped
+tensor-core path against the oracle applied token by token."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_18063_b200 as edg
+from oracle import moe_oracle as orc
+from paper_2609_18063_b200 import layer_io
+from workloads import synth
+
+from _gpu_util import TOL_MAX_ABS, TOL_REL_L2, device_layer, out_tensor, x_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _ffn_tokens(L, d, X_bits, inds, gates, T, use_table=True):
+    if L.ws.numel() < edg.ffn_workspace_bytes(d, T):
+        L.ws = layer_io.new_workspace(d, T)
+    L.ws[:256].zero_()
+    y = out_tensor(d, T)
+    table = torch.arange(d.E, dtype=torch.int32, device="cuda") if use_table else None
+    edg.moe_expert_ffn_int4_lora(d, L.pool, table, T, inds, inds, gates, x_dev(X_bits), L.lora, y, L.ws)
+    torch.cuda.synchronize()
+    assert edg.workspace_status(L.ws) == 0
+    return y.cpu().numpy()
+
+
+def _check_tokens(L, X_bits, inds_h, gates_h, Y, tokens):
+    cfg = L.cfg
+    worst_abs = worst_rel = 0.0
+    for t in tokens:
+        ref = orc.moe_ffn(X_bits[t], inds_h[t], gates_h[t].astype(np.float64), L.expert, L.get_lora, cfg.lora_scale, cfg.group)
+        worst_abs = max(worst_abs, orc.max_abs(Y[t], ref))
+        worst_rel = max(worst_rel, orc.rel_l2(Y[t], ref))
+    assert worst_abs <= TOL_MAX_ABS and worst_rel <= TOL_REL_L2, (worst_abs, worst_rel)
+    return worst_abs, worst_rel
+
+
+def test_batched_decode_cfg4_shape():
+    """64 concurrent tokens, independent top-8 routing from the head, union of experts resident."""
+    L = device_layer("cfg2")                      # same layer shape as cfg4; every expert resident
+    cfg = synth.CONFIGS["cfg4"]
+    T, K, E = cfg.T, cfg.K, cfg.E
+    X = synth.hidden_states(cfg, T, stream=31)
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    edg.prerouter_topk(L.desc, L.W.unsqueeze(0).expand(T, E, cfg.H).contiguous(), x_dev(X), T, inds, gates, None)
+    torch.cuda.synchronize()
+    inds_h, gates_h = inds.cpu().numpy(), gates.cpu().numpy()
+    for t in range(0, T, 7):                      # the routing is the oracle's (fp64 gap permitting)
+        l = orc.prerouter_logits(L.W_np, X[t])
+        srt = np.sort(l)[::-1]
+        if srt[K - 1] - srt[K] > 1e-4:
+            assert inds_h[t].tolist() == orc.softmax_topk(l, K)[0].tolist()
+    assert len(np.unique(inds_h)) > 150           # a wide union of experts, a few tokens each
+    Y = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    _check_tokens(L, X, inds_h, gates_h, Y, range(0, T, 3))
+    # the same call with slots given directly (no table) is bit-identical
+    Y2 = _ffn_tokens(L, L.desc, X, inds, gates, T, use_table=False)
+    assert np.array_equal(Y, Y2)
+
+
+def test_prefill_cfg5_shape_reduced_tokens():
+    """Zipf(1.1)-skewed routing from the router's own logits; ragged token count (not a tile multiple)."""
+    L = device_layer("cfg2")
+    cfg = synth.CONFIGS["cfg5"]
+    T, K, E = 300, cfg.K, cfg.E
+    X = synth.hidden_states(cfg, T, stream=32)
+    logits = synth.zipf_router_logits(cfg, T)
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    edg.softmax_topk_rows(L.desc, torch.from_numpy(logits).cuda(), T, inds, gates)
+    torch.cuda.synchronize()
+    inds_h, gates_h = inds.cpu().numpy(), gates.cpu().numpy()
+    for t in range(T):
+        i_ref, w_ref = orc.softmax_topk(logits[t], K)
+        assert inds_h[t].tolist() == i_ref.tolist() and np.abs(gates_h[t] - w_ref).max() <= 2e-6
+    counts = np.bincount(inds_h.ravel(), minlength=E)
+    assert counts.max() > 64 and counts.max() > 10 * max(1, np.median(counts))     # skewed: some groups span several tiles
+    Y = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    rng = np.random.default_rng(0)
+    sample = sorted(set(rng.choice(T, 14, replace=False).tolist()) | {0, T - 1})
+    _check_tokens(L, X, inds_h, gates_h, Y, sample)
+    assert np.isfinite(Y).all()
+
+
+def test_grouped_reduces_to_the_decode_path_and_handles_per_expert_adapters():
+    L = device_layer("cfg1", 16)                  # per-expert adapters
+    cfg = L.cfg
+    T = 7
+    X = synth.hidden_states(cfg, T, stream=33)
+    X[3] = X[0]                                   # two identical tokens with identical routing
+    rng = np.random.default_rng(1)
+    inds_h = np.stack([np.sort(rng.choice(cfg.E, cfg.K, replace=False)) for _ in range(T)]).astype(np.int32)
+    gates_h = rng.dirichlet(np.ones(cfg.K), size=T).astype(np.float32)
+    inds_h[3], gates_h[3] = inds_h[0], gates_h[0]
+    inds, gates = torch.from_numpy(inds_h).cuda(), torch.from_numpy(gates_h).cuda()
+    Y = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    _check_tokens(L, X, inds_h, gates_h, Y, range(T))
+    assert np.array_equal(Y[0], Y[3])
+    # T = 1 (fused decode kernel) on the same token agrees with the grouped result
+    y1 = _ffn_tokens(L, L.desc, X[:1], inds[:1].contiguous(), gates[:1].contiguous(), 1)
+    assert orc.max_abs(y1[0], Y[0]) <= TOL_MAX_ABS and orc.rel_l2(y1[0], Y[0]) <= TOL_REL_L2
+    # an out-of-range expert in one pair is skipped and flagged, the other tokens are untouched
+    bad = inds_h.copy(); bad[5, 1] = cfg.E
+    L.ws[:256].zero_()
+    y = out_tensor(L.desc, T)
+    edg.moe_expert_ffn_int4_lora(L.desc, L.pool, torch.arange(cfg.E, dtype=torch.int32, device="cuda"), T,
+                                 torch.from_numpy(bad).cuda(), None, gates, x_dev(X), L.lora, y, L.ws)
+    torch.cuda.synchronize()
+    assert edg.workspace_status(L.ws) == -4
+    yb = y.cpu().numpy()
+    assert np.array_equal(yb[0], Y[0]) and np.array_equal(yb[6], Y[6])
