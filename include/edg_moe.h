@@ -228,6 +228,26 @@ int32_t moe_expert_ffn_int4_lora(const edg_layer_desc* desc, const void* slot_po
                                  const void* x, const edg_lora* lora, void* y,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same batch-1 FFN (T = 1) for callers that cannot allocate device memory -- code running
+ * inside another engine's memory plan, a loop that must stay away from the allocator once it has
+ * started, a process whose GPU memory belongs to a pool it does not control.  (The paper has no
+ * counterpart: this is an addition for such hosts.)  Inputs and outputs are passed as for
+ * moe_expert_ffn_int4_lora; the kernel's scratch lives in a fixed 2 MiB array inside the library's
+ * device image (every GPU that loads the library holds it until the process exits).  The call
+ * makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Shapes whose scratch would not fit the array, or that the batch-1 kernel does not cover,
+ *     are rejected with EDG_E_WORKSPACE / EDG_E_SHAPE.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call before any stream capture.
+ *   - All calls on a device share the array.  Each call clears the control block it needs at zero
+ *     on `stream`; calls that overlap on the GPU (different streams without ordering) race.
+ *   - Out-of-range slot or expert indices are skipped as in the other entry points, but there is
+ *     no status word to read back. */
+int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* slot_pool,
+                                        const int32_t* slot_table, const int32_t* slots,
+                                        const int32_t* experts, const float* gates, const void* x,
+                                        const edg_lora* lora, void* y, void* stream);
+
 /* ---------------------------------------------------------------- the whole layer-step */
 
 /* One layer-step of batch-1 decode (Sec. 3.2 "Motivation": the double shift).  On `stream`:

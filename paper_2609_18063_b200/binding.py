@@ -16,7 +16,7 @@ __all__ = [
     "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
     "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "softmax_topk_rows",
-    "moe_expert_ffn_int4_lora", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
+    "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
 ]
 
 F32, F16, BF16 = 0, 1, 2
@@ -76,6 +76,7 @@ _SIG = {
     "edg_store_mark_computed": ([_P, C.c_int32, _P], C.c_int32),
     "stage_experts_to_slots": ([_P, C.c_int32, _P, C.c_int32, _P, C.POINTER(C.c_int32)], C.c_int32),
     "moe_expert_ffn_int4_lora": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P, C.POINTER(Lora), _P, _P, C.c_size_t, _P], C.c_int32),
+    "moe_expert_ffn_int4_lora_static": ([_D, _P, _P, _P, _P, _P, _P, C.POINTER(Lora), _P, _P], C.c_int32),
     "moe_layer_decode": ([_P, C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, C.c_size_t, _P], C.c_int32),
 }
 EXPORTS = tuple(_SIG)
@@ -229,6 +230,16 @@ def moe_expert_ffn_int4_lora(desc, slot_pool, slot_table, T, slots, experts, gat
                                          _ptr(experts), _ptr(gates), _ptr(x),
                                          None if lora is None else C.byref(lora), _ptr(y), _ptr(workspace),
                                          workspace_bytes, _stream(stream)), "moe_expert_ffn_int4_lora")
+
+
+def moe_expert_ffn_int4_lora_static(desc, slot_pool, slot_table, slots, experts, gates, x, lora, y, stream=None) -> None:
+    """Batch-1 FFN without a caller-provided workspace: for hosts that may not allocate device
+    memory.  The scratch is a fixed array inside the library; see the header for the rules
+    (first call per device before any stream capture; overlapping calls race)."""
+    _check(_lib.moe_expert_ffn_int4_lora_static(C.byref(desc), _ptr(slot_pool), _ptr(slot_table), _ptr(slots),
+                                                _ptr(experts), _ptr(gates), _ptr(x),
+                                                None if lora is None else C.byref(lora), _ptr(y), _stream(stream)),
+           "moe_expert_ffn_int4_lora_static")
 
 
 class Store:
