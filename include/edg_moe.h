@@ -154,6 +154,11 @@ int32_t edg_set_trace_buffer(void* dev_buffer);
 int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
                        int32_t* inds, float* gates, float* logits_opt, void* stream);
 
+/* The same for T hidden states that all use ONE head (batched decode of one layer):
+ * W_pre dev [E][H]; s dev bf16 [T][H]; outputs [T][K] / [T][E]. */
+int32_t prerouter_topk_tokens(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t T,
+                              int32_t* inds, float* gates, float* logits_opt, void* stream);
+
 /* a2 alone on given logits (a router's own gate at prefill): logits dev float [T][E] ->
  * inds dev int32 [T][K], gates dev float [T][K].  Same ordering and tie rule. */
 int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,

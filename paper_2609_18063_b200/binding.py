@@ -15,7 +15,7 @@ import numpy as np
 __all__ = [
     "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
-    "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "softmax_topk_rows",
+    "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows",
     "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
 ]
 
@@ -67,6 +67,7 @@ _SIG = {
     "edg_workspace_status": ([_P, _P, C.POINTER(C.c_int32)], C.c_int32),
     "edg_set_trace_buffer": ([_P], C.c_int32),
     "prerouter_topk": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
+    "prerouter_topk_tokens": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "softmax_topk_rows": ([_D, _P, C.c_int32, _P, _P, _P], C.c_int32),
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
@@ -215,6 +216,11 @@ def set_trace_buffer(dev_buffer) -> None:
 def prerouter_topk(desc, W_pre, s, n_heads, inds, gates, logits_opt=None, stream=None) -> None:
     _check(_lib.prerouter_topk(C.byref(desc), _ptr(W_pre), _ptr(s), n_heads, _ptr(inds), _ptr(gates),
                                _ptr(logits_opt), _stream(stream)), "prerouter_topk")
+
+
+def prerouter_topk_tokens(desc, W_pre, s, T, inds, gates, logits_opt=None, stream=None) -> None:
+    _check(_lib.prerouter_topk_tokens(C.byref(desc), _ptr(W_pre), _ptr(s), T, _ptr(inds), _ptr(gates),
+                                      _ptr(logits_opt), _stream(stream)), "prerouter_topk_tokens")
 
 
 def softmax_topk_rows(desc, logits, T, inds, gates, stream=None) -> None:

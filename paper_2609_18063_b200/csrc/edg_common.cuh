@@ -78,7 +78,7 @@ struct WorkspaceLayout {
     size_t pair_ad;   // [T*K] int32                : adapter of every pair
     size_t counts;    // [n_slots] int32            : pairs per slot
     size_t n_tiles;   // int32
-    size_t tiles;     // [T*K/64 + n_slots][2] int32: (slot, first position) of every 64-pair tile
+    size_t tiles;     // [T*K/8 + n_slots][2] int32 : (slot, first position) of every tile of 8 or 64 pairs
     size_t lists;     // [n_slots][T] int32         : pairs of every slot, ascending
     size_t bytes;
 };
@@ -104,7 +104,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
         W.pair_ad = end;           end = round_up(W.pair_ad + P * 4, 256);
         W.counts = end;            end = round_up(W.counts + (size_t)d.n_slots * 4, 256);
         W.n_tiles = end;           end += 256;
-        W.tiles = end;             end = round_up(W.tiles + (P / 64 + 1 + d.n_slots) * 8, 256);
+        W.tiles = end;             end = round_up(W.tiles + (P / 8 + 1 + d.n_slots) * 8, 256);
         W.lists = end;             end = round_up(W.lists + (size_t)d.n_slots * T * 4, 256);
     }
     W.bytes = end;

@@ -20,8 +20,7 @@
 
 namespace edg {
 
-constexpr int G_NTOK = 64;        // tokens per tile = 8 MMA column tiles
-constexpr int G_NT = G_NTOK / 8;
+constexpr int G_NTOK_MAX = 64;    // tokens per tile: 8 MMA column tiles for large groups, 1 (8 tokens) for small ones
 constexpr int G_KC = 256;         // gate/up: k per staged chunk (8 super-steps of 32)
 constexpr int G_KD = 128;         // down: k per staged chunk
 constexpr int G_WARPS = 8;
@@ -51,6 +50,7 @@ struct GroupedParams {
     int32_t* tiles;           // [max tiles][2] = (slot, first position in the slot's list)
     int32_t* n_tiles;
     int T, H, I, E, K, group, rank, n_adapters, n_slots, out_dtype;
+    int ntok;                 // tokens per tile of this call (8 or 64)
     float sigma;
     RecordLayout L;
 };
@@ -115,6 +115,7 @@ __device__ __forceinline__ uint4 permute8(const float (&v)[8]) {
 
 // The LoRA delta as one MMA k-step per 16 ranks: acc += Bl[rows][r] . (sigma * u[token][r]).
 // Bl: bf16 [..][rank], row pointers for rows g and g+8 of the tile; u row pointers per column tile.
+template <int G_NT>
 __device__ __forceinline__ void lora_mma(float (&acc)[G_NT][4], const uint16_t* b_row_g, const uint16_t* b_row_g8,
                                          const float* const (&u_tok)[G_NT], int rank, float sigma, int t4) {
     for (int kr = 0; kr < rank; kr += 16) {
@@ -173,7 +174,7 @@ __global__ void build_tiles_kernel(GroupedParams p) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     int n = 0;
     for (int s = 0; s < p.n_slots; ++s)
-        for (int first = 0; first < p.counts[s]; first += G_NTOK) { p.tiles[2 * n] = s; p.tiles[2 * n + 1] = first; ++n; }
+        for (int first = 0; first < p.counts[s]; first += p.ntok) { p.tiles[2 * n] = s; p.tiles[2 * n + 1] = first; ++n; }
     *p.n_tiles = n;
 }
 
@@ -181,7 +182,9 @@ __global__ void build_tiles_kernel(GroupedParams p) {
 // CTA = (tile of up to 64 pairs of one slot) x (128 rows of I).  Warp w owns rows 16w..16w+15 of
 // both gate and up, so silu(g) * u is formed in registers.
 
+template <int G_NT>
 __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(GroupedParams p) {
+    constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -210,8 +213,8 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(Groupe
     const int row_b = p.H / 2, groups = p.H / p.group;
     for (int kc = 0; kc < p.H / G_KC; ++kc) {
         __syncthreads();
-        {   // activations: token tid/4, 64 k starting at (tid%4)*64
-            const int i = tid >> 2, q = tid & 3;
+        for (int idx = tid; idx < G_NTOK * 4; idx += G_WARPS * 32) {   // activations: token idx/4, 64 k starting at (idx%4)*64
+            const int i = idx >> 2, q = idx & 3;
             const int pair = s_pair[i];
             const uint16_t* src = pair >= 0 ? p.x + (size_t)(pair / p.K) * p.H + kc * G_KC + q * 64 : nullptr;
 #pragma unroll
@@ -301,8 +304,8 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(Groupe
         }
         const uint16_t* Bg = reinterpret_cast<const uint16_t*>(p.lora.B_gate) + (size_t)ad * p.I * p.rank;
         const uint16_t* Bu = reinterpret_cast<const uint16_t*>(p.lora.B_up) + (size_t)ad * p.I * p.rank;
-        lora_mma(ag, Bg + (size_t)r_lo * p.rank, Bg + (size_t)r_hi * p.rank, ug, p.rank, p.sigma, t4);
-        lora_mma(au, Bu + (size_t)r_lo * p.rank, Bu + (size_t)r_hi * p.rank, uu, p.rank, p.sigma, t4);
+        lora_mma<G_NT>(ag, Bg + (size_t)r_lo * p.rank, Bg + (size_t)r_hi * p.rank, ug, p.rank, p.sigma, t4);
+        lora_mma<G_NT>(au, Bu + (size_t)r_lo * p.rank, Bu + (size_t)r_hi * p.rank, uu, p.rank, p.sigma, t4);
     }
 #pragma unroll
     for (int nt = 0; nt < G_NT; ++nt) {
@@ -321,7 +324,9 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(Groupe
 // ---------------------------------------------------------------- down
 // CTA = (tile of up to 64 pairs of one slot) x (256 rows of H).  Warp w owns rows 32w..32w+31.
 
+template <int G_NT>
 __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_down_kernel(GroupedParams p) {
+    constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
     extern __shared__ __align__(128) uint8_t smem[];
@@ -350,8 +355,8 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_down_kernel(GroupedPa
 
     for (int kc = 0; kc < p.I / G_KD; ++kc) {
         __syncthreads();
-        {   // h: token tid/4, 32 k starting at (tid%4)*32, fp32 -> fp16 (hi, lo)
-            const int i = tid >> 2, q = tid & 3;
+        for (int idx = tid; idx < G_NTOK * 4; idx += G_WARPS * 32) {   // h: token idx/4, 32 k starting at (idx%4)*32, fp32 -> fp16 (hi, lo)
+            const int i = idx >> 2, q = idx & 3;
             const int pair = s_pair[i];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -434,7 +439,7 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_down_kernel(GroupedPa
         const int r_lo = row0 + 32 * warp + 16 * m + g, r_hi = r_lo + 8;
         if (p.rank > 0) {
             const uint16_t* Bd = reinterpret_cast<const uint16_t*>(p.lora.B_down) + (size_t)ad * p.H * p.rank;
-            lora_mma(acc[m], Bd + (size_t)r_lo * p.rank, Bd + (size_t)r_hi * p.rank, ud, p.rank, p.sigma, t4);
+            lora_mma<G_NT>(acc[m], Bd + (size_t)r_lo * p.rank, Bd + (size_t)r_hi * p.rank, ud, p.rank, p.sigma, t4);
         }
 #pragma unroll
         for (int nt = 0; nt < G_NT; ++nt) {
@@ -504,25 +509,32 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     p.L = record_layout(d->H, d->I, d->group);
 
     const int P = T * d->K;
-    const int max_tiles = (P + G_NTOK - 1) / G_NTOK + d->n_slots;
+    // few tokens per expert (batched decode): tiles of 8 tokens, the kernels are then bound by streaming
+    // the weights; many (prefill): tiles of 64 so a dequantised weight tile is reused 8 times more
+    const bool small = P <= 8 * d->n_slots;
+    p.ntok = small ? 8 : 64;
+    const int max_tiles = (P + p.ntok - 1) / p.ntok + d->n_slots;
     resolve_pairs_kernel<<<(P + 255) / 256, 256, 0, st>>>(p);
     build_lists_kernel<<<(d->n_slots * 32 + 255) / 256, 256, 0, st>>>(p);
     build_tiles_kernel<<<1, 32, 0, st>>>(p);
     if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 0, st);
 
-    const int ng = G_KC / d->group;
-    const size_t sm_gu = (size_t)G_NTOK * G_XS + 2 * 128 * G_CS + 2 * 128 * ng * 4 + G_NTOK * 4;
-    const int ngd = G_KD / d->group;
-    const size_t sm_d = (size_t)2 * G_NTOK * G_XSD + 256 * G_CSD + 256 * ngd * 4 + G_NTOK * 4;
+    const int ng = G_KC / d->group, ngd = G_KD / d->group;
+    const size_t sm_gu = (size_t)p.ntok * G_XS + 2 * 128 * G_CS + 2 * 128 * ng * 4 + p.ntok * 4;
+    const size_t sm_d = (size_t)2 * p.ntok * G_XSD + 256 * G_CSD + 256 * ngd * 4 + p.ntok * 4;
     static bool configured = false;
     if (!configured) {
-        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
-        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_gate_up_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_gate_up_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_down_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
         configured = true;
     }
-    grouped_gate_up_kernel<<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
+    if (small) grouped_gate_up_kernel<1><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
+    else grouped_gate_up_kernel<8><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
     if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 1, st);
-    grouped_down_kernel<<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
+    if (small) grouped_down_kernel<1><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
+    else grouped_down_kernel<8><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
     const size_t n_out = (size_t)T * d->H;
     const int rb = (int)((n_out + 255) / 256);
     if (d->out_dtype == EDG_F32) reduce_pairs_kernel<float><<<rb, 256, 0, st>>>(p);

@@ -24,6 +24,7 @@ struct PreParams {
     float* gates;           // [n_heads][K]
     float* logits;          // [n_heads][E] or null
     int H, E, K;
+    int shared_head;        // 1: every state uses head 0 (batched tokens of one layer)
 };
 
 template <typename WT> struct RowDot;
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_kernel(PreParams p) 
     float* leader = cluster.map_shared_rank(s_logits, 0);
     const int per = (p.E + csize - 1) / csize;
     const int e0 = crank * per, e1 = min(p.E, e0 + per);
-    const size_t wbase = (size_t)head * p.E;
+    const size_t wbase = p.shared_head ? 0 : (size_t)head * p.E;
     for (int e = e0 + warp; e < e1; e += kPreWarps) {
         const float l = RowDot<WT>::run(p.W, wbase + e, s_x, p.H, lane);
         if (lane == 0) leader[e] = l;
@@ -113,12 +114,12 @@ __global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* log
 }
 
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
-                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st) {
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head = 0) {
     int32_t rc = check_desc(d);
     if (rc != EDG_OK) return rc;
     if (!W_pre || !s || !inds || !gates || n_heads < 1 || n_heads > 65535) return EDG_E_INVAL;
     if (!aligned(W_pre, 16) || !aligned(s, 16)) return EDG_E_INVAL;
-    PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K};
+    PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K, shared_head};
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kPreCluster, n_heads, 1);
@@ -142,6 +143,11 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
 extern "C" int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
                                   int32_t* inds, float* gates, float* logits_opt, void* stream) {
     return edg::run_prerouter(desc, W_pre, s, n_heads, inds, gates, logits_opt, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t prerouter_topk_tokens(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t T,
+                                         int32_t* inds, float* gates, float* logits_opt, void* stream) {
+    return edg::run_prerouter(desc, W_pre, s, T, inds, gates, logits_opt, static_cast<cudaStream_t>(stream), 1);
 }
 
 extern "C" int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,

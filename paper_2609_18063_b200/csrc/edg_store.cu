@@ -22,7 +22,7 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
                         void* workspace, int flag_in, int flag_out, cudaStream_t st);
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
-                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st);
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head);
 }  // namespace edg
 
 namespace {
@@ -279,7 +279,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         rc = edg::run_ffn(&s->d, pool, 1, inds_cur, table, nullptr, gates_cur, x, lora, y, workspace, workspace_bytes, st);
         if (rc != EDG_OK) return rc;
         if (W_pre_next != nullptr) {
-            rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st);
+            rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st, 0);
             if (rc != EDG_OK) return rc;
         }
     }

@@ -45,7 +45,7 @@ def test_batched_decode_cfg4_shape():
     X = synth.hidden_states(cfg, T, stream=31)
     inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
     gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
-    edg.prerouter_topk(L.desc, L.W.unsqueeze(0).expand(T, E, cfg.H).contiguous(), x_dev(X), T, inds, gates, None)
+    edg.prerouter_topk_tokens(L.desc, L.W, x_dev(X), T, inds, gates, None)
     torch.cuda.synchronize()
     inds_h, gates_h = inds.cpu().numpy(), gates.cpu().numpy()
     for t in range(0, T, 7):                      # the routing is the oracle's (fp64 gap permitting)
