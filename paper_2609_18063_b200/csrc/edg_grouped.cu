@@ -154,28 +154,56 @@ __global__ void resolve_pairs_kernel(GroupedParams p) {
     p.pair_ad[i] = ad;
 }
 
-// One warp per slot: the slot's pairs in ascending pair index (deterministic, no atomics).
-__global__ void __launch_bounds__(256) build_lists_kernel(GroupedParams p) {
-    const int s = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-    if (s >= p.n_slots) return;
+// One CTA per slot: the slot's pairs in ascending pair index (deterministic, no atomics).  Each
+// warp owns a contiguous range of pairs; a first pass counts, a second pass writes at the offsets.
+constexpr int kListWarps = 16;
+__global__ void __launch_bounds__(kListWarps * 32) build_lists_kernel(GroupedParams p) {
+    const int s = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __shared__ int s_cnt[kListWarps];
     const int P = p.T * p.K;
+    const int per = ((P + kListWarps - 1) / kListWarps + 31) / 32 * 32;      // pairs per warp, a multiple of 32
+    const int lo = warp * per, hi = min(P, lo + per);
     int cnt = 0;
-    for (int base = 0; base < P; base += 32) {
+    for (int base = lo; base < hi; base += 32) {
         const int i = base + lane;
-        const bool m = i < P && p.pair_slot[i] == s;
-        const unsigned bal = __ballot_sync(0xFFFFFFFFu, m);
-        if (m) p.lists[(size_t)s * p.T + cnt + __popc(bal & ((1u << lane) - 1))] = i;
-        cnt += __popc(bal);
+        cnt += __popc(__ballot_sync(0xFFFFFFFFu, i < hi && p.pair_slot[i] == s));
     }
-    if (lane == 0) p.counts[s] = cnt;
+    if (lane == 0) s_cnt[warp] = cnt;
+    __syncthreads();
+    int off = 0, total = 0;
+    for (int w = 0; w < kListWarps; ++w) { if (w < warp) off += s_cnt[w]; total += s_cnt[w]; }
+    for (int base = lo; base < hi; base += 32) {
+        const int i = base + lane;
+        const bool m = i < hi && p.pair_slot[i] == s;
+        const unsigned bal = __ballot_sync(0xFFFFFFFFu, m);
+        if (m) p.lists[(size_t)s * p.T + off + __popc(bal & ((1u << lane) - 1))] = i;
+        off += __popc(bal);
+    }
+    if (threadIdx.x == 0) p.counts[s] = total;
 }
 
-__global__ void build_tiles_kernel(GroupedParams p) {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    int n = 0;
-    for (int s = 0; s < p.n_slots; ++s)
+// Tile table: slot s contributes ceil(count / ntok) tiles; an exclusive scan over the slots gives
+// each its first tile.  One CTA, slots strided over the threads, scan through shared memory.
+__global__ void __launch_bounds__(1024) build_tiles_kernel(GroupedParams p) {
+    __shared__ int s_n[1024];
+    const int tid = threadIdx.x;
+    // n_slots can exceed the block: each thread owns a contiguous run of slots
+    const int per = (p.n_slots + 1023) / 1024;
+    const int s0 = tid * per, s1 = min(p.n_slots, s0 + per);
+    int mine = 0;
+    for (int s = s0; s < s1; ++s) mine += (p.counts[s] + p.ntok - 1) / p.ntok;
+    s_n[tid] = mine;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {          // inclusive scan
+        const int v = tid >= o ? s_n[tid - o] : 0;
+        __syncthreads();
+        s_n[tid] += v;
+        __syncthreads();
+    }
+    int n = s_n[tid] - mine;                       // exclusive prefix
+    for (int s = s0; s < s1; ++s)
         for (int first = 0; first < p.counts[s]; first += p.ntok) { p.tiles[2 * n] = s; p.tiles[2 * n + 1] = first; ++n; }
-    *p.n_tiles = n;
+    if (tid == 1023) *p.n_tiles = s_n[1023];
 }
 
 // ---------------------------------------------------------------- gate/up
@@ -183,7 +211,7 @@ __global__ void build_tiles_kernel(GroupedParams p) {
 // both gate and up, so silu(g) * u is formed in registers.
 
 template <int G_NT>
-__global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(GroupedParams p) {
+__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_gate_up_kernel(GroupedParams p) {
     constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
@@ -325,7 +353,7 @@ __global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_gate_up_kernel(Groupe
 // CTA = (tile of up to 64 pairs of one slot) x (256 rows of H).  Warp w owns rows 32w..32w+31.
 
 template <int G_NT>
-__global__ void __launch_bounds__(G_WARPS * 32, 2) grouped_down_kernel(GroupedParams p) {
+__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_down_kernel(GroupedParams p) {
     constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
@@ -515,8 +543,8 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     p.ntok = small ? 8 : 64;
     const int max_tiles = (P + p.ntok - 1) / p.ntok + d->n_slots;
     resolve_pairs_kernel<<<(P + 255) / 256, 256, 0, st>>>(p);
-    build_lists_kernel<<<(d->n_slots * 32 + 255) / 256, 256, 0, st>>>(p);
-    build_tiles_kernel<<<1, 32, 0, st>>>(p);
+    build_lists_kernel<<<d->n_slots, kListWarps * 32, 0, st>>>(p);
+    build_tiles_kernel<<<1, 1024, 0, st>>>(p);
     if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 0, st);
 
     const int ng = G_KC / d->group, ngd = G_KD / d->group;
