@@ -23,11 +23,16 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ---------------------------------------------------------------- record layout
 // One expert record: [gate codes][up codes][down codes][gate sz][up sz][down sz].
-// Codes are int4, low nibble first; sz is one (scale, zero) fp16 pair per group.  gate and up are
-// row-major [out][in].  down is stored as kDownSlices column slices, each row-major
-// [H][I/kDownSlices]: the batch-1 kernel splits the down projection over the intermediate
-// dimension, and a (slice, block of rows) is then one contiguous run of bytes.  All section
-// offsets are multiples of 256 bytes for the shapes edg_check_desc admits.
+// Codes are int4, low nibble first inside every 32-bit word (code k of a word in bits 4k..4k+3);
+// sz is one (scale, zero) fp16 pair per group.  Every [N][Kd] matrix is stored tile-major:
+//     codes: [N/16 row tiles][Kd/32 chunks][16 rows][16 bytes]     (a chunk = 32 consecutive codes of a row)
+//     sz:    [N/16 row tiles][Kd/group groups][16 rows][4 bytes]
+// so the 16 rows x 32 codes that one tensor-core k-step touches are 256 contiguous bytes (read
+// without shared-memory bank conflicts), and any block of whole row tiles is one contiguous run
+// for a bulk copy.  gate and up are [I][H].  down is stored as kDownSlices column slices, each a
+// tile-major [H][I/kDownSlices] matrix: the batch-1 kernel splits the down projection over the
+// intermediate dimension.  All section offsets are multiples of 256 bytes for the shapes
+// edg_check_desc admits.
 struct RecordLayout {
     uint32_t codes_gate, codes_up, codes_down;   // byte offsets
     uint32_t sz_gate, sz_up, sz_down;
@@ -36,15 +41,22 @@ struct RecordLayout {
 
 constexpr int kDownSlices = 4;
 
-// byte offset, inside the down code section, of the 16-byte chunk c (codes 32c .. 32c+31) of row n
+// byte offset, inside a tile-major code section of a [.][Kd] matrix, of chunk c (codes 32c..32c+31) of row n
+__host__ __device__ inline size_t code_off(int Kd, int n, int c) {
+    return ((((size_t)(n >> 4) * (Kd / 32) + c) * 16) + (n & 15)) * 16;
+}
+// byte offset, inside a tile-major sz section, of the (scale, zero) pair of group gi of row n
+__host__ __device__ inline size_t sz_off(int Kd, int group, int n, int gi) {
+    return ((((size_t)(n >> 4) * (Kd / group) + gi) * 16) + (n & 15)) * 4;
+}
+// the same for the sliced down matrix [H][I]
 __host__ __device__ inline size_t down_code_off(int H, int I, int n, int c) {
     const int sw = I / kDownSlices, cps = sw / 32;            // slice width in codes, chunks per row-slice
-    return ((size_t)(c / cps) * H + n) * (sw / 2) + (size_t)(c % cps) * 16;
+    return (size_t)(c / cps) * ((size_t)H * sw / 2) + code_off(sw, n, c % cps);
 }
-// byte offset, inside the down sz section, of the (scale, zero) pair of group gi of row n
 __host__ __device__ inline size_t down_sz_off(int H, int I, int group, int n, int gi) {
-    const int gps = (I / kDownSlices) / group;                // groups per row-slice
-    return (((size_t)(gi / gps) * H + n) * gps + (gi % gps)) * 4;
+    const int sw = I / kDownSlices, gps = sw / group;         // groups per row-slice
+    return (size_t)(gi / gps) * ((size_t)H * gps * 4) + sz_off(sw, group, n, gi % gps);
 }
 
 __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {

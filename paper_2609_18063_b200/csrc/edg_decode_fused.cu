@@ -26,7 +26,7 @@
 // step is still computing.
 #include <cooperative_groups.h>
 
-#include "edg_common.cuh"
+#include "edg_mma.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -177,26 +177,27 @@ __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, i
 }
 
 // ---------------------------------------------------------------- shared-memory carve-up
-// Byte offsets, identical on host and device.  The four gate/up stages come first; the down block
+// Byte offsets, identical on host and device.  The four gate/up stages (quarters of the K range)
+// come first; the down block
 // later reuses stages 0 and 1 (it is exactly half the size of the gate/up slice), which keeps a
 // CTA under half an SM's shared memory so two CTAs -- of this launch or of the next one -- can
 // share an SM.
 struct FusedSmem {
-    uint32_t stage0, stage_bytes;                      // stage s at stage0 + s * stage_bytes
-    uint32_t g_codes, u_codes, g_sz, u_sz;             // offsets inside a stage
+    uint32_t stage0, stage_bytes;                      // stage s (a quarter of the K range) at stage0 + s * stage_bytes
+    uint32_t mat_codes, mat_sz;                        // bytes of one (matrix, row tile) run of codes / sz inside a stage
+    uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
-    const uint32_t rows_gu = I / kE16, rows_d = H / kC, rs = rows_gu / kStages, sw = I / kDownSlices;
-    const uint32_t row_b = H / 2, grp_b = (H / group) * 4;
-    S.g_codes = 0;
-    S.u_codes = rs * row_b;
-    S.g_sz = 2 * rs * row_b;
-    S.u_sz = 2 * rs * row_b + rs * grp_b;
-    S.stage_bytes = 2 * rs * (row_b + grp_b);
+    const uint32_t rows_gu = I / kE16, rows_d = H / kC, sw = I / kDownSlices, tg = rows_gu / 16;
+    // a stage holds, for gate and up and each of their tg row tiles, H/128 chunks (H/4 codes per row)
+    S.mat_codes = (uint32_t)(H / 128) * 256;
+    S.mat_sz = (uint32_t)((H / 4) / group) * 64;
+    S.sz0 = 2 * tg * S.mat_codes;
+    S.stage_bytes = 2 * tg * (S.mat_codes + S.mat_sz);
     uint32_t o = 0;
     S.stage0 = o;     o += kStages * S.stage_bytes;
     S.d_codes = S.stage0;
@@ -217,6 +218,7 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
     S.s_hloc = o;     o += 32 * 4;
     S.s_topk = o;     o += (uint32_t)E * 4;           // logits gathered by the warp that finishes the routing
+    S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
     S.flag = o;       o += 16;
     S.total = (o + 15) / 16 * 16;
     return S;
@@ -312,11 +314,11 @@ __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* 
 }
 
 // ---------------------------------------------------------------- the fused kernel
-// NCH = H / 1024 (chunks of a gate/up row per lane), LPR_D = I / 128 (lanes per down row-slice).
+// NCW = H / 256 = chunks (of 32 codes) per warp in gate/up; DCH = I / 128 = chunks of a down row-slice.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
 
-template <int NCH, int LPR_D>
+template <int NCW, int DCH>
 __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b16 = blockIdx.x % kE16;             // CTA of the expert
@@ -324,6 +326,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     const int c = b16 / kC;                        // quarter of the intermediate dimension (cluster of the expert)
     const int crank = b16 % kC;                    // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    const int g8 = lane >> 2, t4 = lane & 3;       // fragment coordinates: row slot, quad lane
 
     const FusedSmem S = fused_smem(p.H, p.I, p.E, p.group, p.rank);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars);
@@ -335,9 +338,11 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     float* s_o = reinterpret_cast<float*>(smem + S.s_o);            // [rows_d]
     float* s_red = reinterpret_cast<float*>(smem + S.s_red);        // [40][kFW]
     float* s_hloc = reinterpret_cast<float*>(smem + S.s_hloc);      // [rows_gu]
+    float* s_part = reinterpret_cast<float*>(smem + S.s_part);      // [kFW][2 * rows_gu]
     int* s_flag = reinterpret_cast<int*>(smem + S.flag);
 
     const int rows_gu = p.I / kE16, rows_d = p.H / kC, sw = p.I / kDownSlices;
+    const int tg = rows_gu / 16;                   // row tiles per matrix in this CTA
     const int n0_gu = b16 * rows_gu;               // first gate/up row of this CTA (= c * sw + crank * rows_gu)
     const int n0_d = crank * rows_d;               // first down row of this CTA
     const int r = p.rank;
@@ -350,7 +355,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     //      SM, so none is used after this point.
     if (tid == 0) {
         for (int s = 0; s <= BAR_LORA; ++s) mbar_init(&bars[s], 1);
-        mbar_init(&bars[BAR_FREE], kFW);
+        mbar_init(&bars[BAR_FREE], kFW / 2);
         mbar_init(&bars[BAR_U], 1);
         mbar_init(&bars[BAR_H], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -362,13 +367,37 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     __syncthreads();
     cluster_arrive();
 
-    // ---- loads that do not depend on the routing: the hidden state chunks this lane multiplies with
-    uint4 xraw[NCH][4];
+    // ---- loads that do not depend on the routing.  The hidden state as the MMA's B operand: the
+    //      warp owns NCW chunks of 32 activations; the lanes of quad 0 hold them (column 0 of the
+    //      8-column tile), every other lane holds zeros.  xsum[j] = sum of the activations of
+    //      64-code block j (for the zero points).
+    uint32_t xb[NCW][4];
+    float xsum[(NCW + 1) / 2];
+    {
+        float part[(NCW + 1) / 2];
 #pragma unroll
-    for (int i = 0; i < NCH; ++i) {
-        const uint4* xp = reinterpret_cast<const uint4*>(p.x + (lane + 32 * i) * 32);
+        for (int j = 0; j < (NCW + 1) / 2; ++j) part[j] = 0.f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) xraw[i][q] = xp[q];
+        for (int i = 0; i < NCW; ++i) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (g8 == 0) v = *reinterpret_cast<const uint4*>(p.x + (warp * NCW + i) * 32 + t4 * 8);
+            const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
+                                bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
+            const uint4 q = permute8(f);
+            xb[i][0] = q.x; xb[i][1] = q.y; xb[i][2] = q.z; xb[i][3] = q.w;
+            // fp16 is exact for bf16 inputs in the normal range; sum what the MMA will see
+            float sum = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
+            part[i / 2] += sum;
+        }
+#pragma unroll
+        for (int j = 0; j < (NCW + 1) / 2; ++j) {
+            float v = part[j];
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+            xsum[j] = __shfl_sync(0xFFFFFFFFu, v, 0);
+        }
     }
 
     // ---- a1 for the next step: this CTA's rows of the head, every thread 8 elements of each.  They
@@ -419,24 +448,29 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     cluster_wait();                       // nothing is in flight yet: this returns at once
     trace_mark(p, 11);
 
+    const int cps = p.H / 128;            // chunks of a row per stage
+    const int gpst = (p.H / 4) / p.group; // groups of a row per stage
+    const int gps = sw / p.group;         // groups of a down row-slice
+
     if (valid) {
         const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-        const int row_b = p.H / 2, grp_b = (p.H / p.group) * 4;
-        const int rs = rows_gu / kStages;                            // gate/up rows per stage
-        const int drow_b = sw / 2, gps = sw / p.group, dgrp_b = gps * 4;   // one row of the down block
-
-        // ---- issue the copies of this CTA's gate/up slice and adapter rows, one warp per barrier
+        // ---- issue the copies of this CTA's gate/up slice (stage = a quarter of the K range, one run
+        //      per matrix and row tile) and of its adapter rows, one warp per barrier
         if (lane == 0) {
             const uint64_t pol = policy_evict_first();       // weights stream through L2 once
             if (warp < kStages) {
                 const int s = warp;
                 uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-                const size_t gr = (size_t)(n0_gu + s * rs);          // first row of the stage in the expert
                 mbar_expect_tx(&bars[s], S.stage_bytes);
-                bulk_g2s_hint(st + S.g_codes, rec + p.L.codes_gate + gr * row_b, rs * row_b, &bars[s], pol);
-                bulk_g2s_hint(st + S.u_codes, rec + p.L.codes_up + gr * row_b, rs * row_b, &bars[s], pol);
-                bulk_g2s_hint(st + S.g_sz, rec + p.L.sz_gate + gr * grp_b, rs * grp_b, &bars[s], pol);
-                bulk_g2s_hint(st + S.u_sz, rec + p.L.sz_up + gr * grp_b, rs * grp_b, &bars[s], pol);
+                for (int m = 0; m < 2; ++m) {
+                    const uint8_t* codes = rec + (m ? p.L.codes_up : p.L.codes_gate);
+                    const uint8_t* sz = rec + (m ? p.L.sz_up : p.L.sz_gate);
+                    for (int ti = 0; ti < tg; ++ti) {
+                        const int n = n0_gu + 16 * ti;
+                        bulk_g2s_hint(st + (m * tg + ti) * S.mat_codes, codes + code_off(p.H, n, s * cps), S.mat_codes, &bars[s], pol);
+                        bulk_g2s_hint(st + S.sz0 + (m * tg + ti) * S.mat_sz, sz + sz_off(p.H, p.group, n, s * gpst), S.mat_sz, &bars[s], pol);
+                    }
+                }
             } else if (warp == kStages && r > 0) {
                 // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
                 const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
@@ -472,9 +506,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
 
     if (valid) {
         const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-        const int row_b = p.H / 2;
-        const int rs = rows_gu / kStages;                            // gate/up rows per stage
-        const int drow_b = sw / 2, gps = sw / p.group, dgrp_b = gps * 4;   // one row of the down block
 
         // ---- LoRA: this CTA's share of the 2r rows of A_gate / A_up.  All threads take part: each
         //      one covers 8 elements of a row per sweep, so a row costs one round trip to the L2.
@@ -504,22 +535,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
                 if (lane == 0 && q0 + u < per) s_red[(q0 + u) * kFW + warp] = t;
             }
         }
-
-        // ---- hidden state -> pre-scaled registers (each lane owns NCH chunks of 32)
-        float xs[NCH][32], xsum[NCH];
-#pragma unroll
-        for (int i = 0; i < NCH; ++i) {
-            float xv[32];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const uint4 v = xraw[i][q];
-                xv[q * 8 + 0] = bf16_lo(v.x); xv[q * 8 + 1] = bf16_hi(v.x);
-                xv[q * 8 + 2] = bf16_lo(v.y); xv[q * 8 + 3] = bf16_hi(v.y);
-                xv[q * 8 + 4] = bf16_lo(v.z); xv[q * 8 + 5] = bf16_hi(v.z);
-                xv[q * 8 + 6] = bf16_lo(v.w); xv[q * 8 + 7] = bf16_hi(v.w);
-            }
-            xsum[i] = scale_chunk(xv, xs[i]);
-        }
         if (p.trace != nullptr && tid == 0) { unsigned sm; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); p.trace[(size_t)blockIdx.x * kTraceMarks + 13] = sm; }
         __syncthreads();                  // s_red complete
         // every CTA of the cluster gets this CTA's adapter projections, counted on its BAR_U
@@ -533,47 +548,88 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         }
         trace_mark(p, 2);
 
-        // ---- gate/up GEMV over this CTA's rows, stage by stage as the copies land.  Once every
-        //      warp is past stages 0 and 1 their space is refilled with the CTA's block of down.
+        // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside stage
+        //      w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile, chunk) are 256
+        //      contiguous bytes of shared memory, lane (g, t) reading word t of rows g and g+8.
+        //      Partial sums of a 64-code block are exact integer-code dot products in fp32;
+        //      scale and zero point are applied per block: acc += s * (c - z * sum(x)).
         {
-            const int groups = p.H / p.group;
-            bool freed = false;
-            for (int lr = warp;; lr += kFW) {
-                const int s = lr < rows_gu ? lr / rs : kStages;
-                if (s >= 2 && !freed) {
-                    freed = true;
-                    if (lane == 0) mbar_arrive(&bars[BAR_FREE]);
-                    if (warp == 0) {
-                        mbar_wait(&bars[BAR_FREE], 0, p.status);
-                        if (lane == 0) {
-                            const uint64_t pol = policy_evict_first();
-                            const size_t row0 = (size_t)c * p.H + n0_d;      // first row of the block in the sliced layout
-                            mbar_expect_tx(&bars[BAR_DOWN], (uint32_t)rows_d * (drow_b + dgrp_b));
-                            bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + row0 * drow_b, rows_d * drow_b, &bars[BAR_DOWN], pol);
-                            bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + row0 * dgrp_b, rows_d * dgrp_b, &bars[BAR_DOWN], pol);
+            const int s = warp / 2;
+            mbar_wait(&bars[s], 0, p.status);
+            if (warp == 0) trace_mark(p, 3);
+            const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+            const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
+            const int cpb = p.group >= 64 ? 2 : 1;                   // chunks per scaled block
+            for (int mt = 0; mt < 2 * tg; ++mt) {                    // (matrix, row tile)
+                const uint8_t* codes = st + mt * S.mat_codes;
+                const uint8_t* szs = st + S.sz0 + mt * S.mat_sz;
+                float acc_lo = 0.f, acc_hi = 0.f;                    // rows g and g+8, column 0
+#pragma unroll
+                for (int i0 = 0; i0 < NCW; i0 += 2) {
+#pragma unroll
+                    for (int b = 0; b < 2; b += 1) {
+                        // one scaled block = cpb chunks; with cpb == 1 the two chunks of this pair are two blocks
+                        if (cpb == 2 && b == 1) break;
+                        const int ia = i0 + b, nchunks = cpb;
+                        const int gi = ((ch0 + ia) * 32) / p.group;
+                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(szs + gi * 64 + g8 * 4));
+                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(szs + gi * 64 + 32 + g8 * 4));
+                        float cfr[4];
+                        float xs_blk = 0.f;
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            if (u < nchunks) {
+                                const int i = ia + u;
+                                uint32_t alo[4], ahi[4];
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(codes + (ch0 + i) * 256 + g8 * 16 + t4 * 4), alo);
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(codes + (ch0 + i) * 256 + 128 + g8 * 16 + t4 * 4), ahi);
+                                if (u == 0) mma16816_zero(cfr, alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
+                                else mma16816(cfr, alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
+                                mma16816(cfr, alo[2], ahi[2], alo[3], ahi[3], xb[i][2], xb[i][3]);
+                            }
                         }
+                        if (cpb == 2) xs_blk = xsum[ia / 2];
+                        else {   // 32-code blocks: the pair's sum was accumulated per 64; split it again
+                            xs_blk = 0.f;   // recomputed below for this single chunk
+                            const float v0 = __half2float(__low2half(u32_as_h2(xb[ia][0]))) + __half2float(__high2half(u32_as_h2(xb[ia][0])))
+                                           + __half2float(__low2half(u32_as_h2(xb[ia][1]))) + __half2float(__high2half(u32_as_h2(xb[ia][1])))
+                                           + __half2float(__low2half(u32_as_h2(xb[ia][2]))) + __half2float(__high2half(u32_as_h2(xb[ia][2])))
+                                           + __half2float(__low2half(u32_as_h2(xb[ia][3]))) + __half2float(__high2half(u32_as_h2(xb[ia][3])));
+                            float v = v0;
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                            xs_blk = __shfl_sync(0xFFFFFFFFu, v, 0);
+                        }
+                        acc_lo = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs_blk, cfr[0]), acc_lo);
+                        acc_hi = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs_blk, cfr[2]), acc_hi);
                     }
                 }
-                if (lr >= rows_gu) break;
-                mbar_wait(&bars[s], 0, p.status);
-                if (lr == warp) trace_mark(p, 3);
-                const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-                const int sr = lr - s * rs;                          // row inside the stage
-                float ag = 0.f, au = 0.f;
-#pragma unroll
-                for (int i = 0; i < NCH; ++i) {
-                    const int ch = lane + 32 * i;
-                    const uint4 wg = *reinterpret_cast<const uint4*>(st + S.g_codes + sr * row_b + ch * 16);
-                    const uint4 wu = *reinterpret_cast<const uint4*>(st + S.u_codes + sr * row_b + ch * 16);
-                    const uint32_t zg = *reinterpret_cast<const uint32_t*>(st + S.g_sz + (sr * groups + (ch * 32) / p.group) * 4);
-                    const uint32_t zu = *reinterpret_cast<const uint32_t*>(st + S.u_sz + (sr * groups + (ch * 32) / p.group) * 4);
-                    ag += chunk_affine(chunk_dot(wg, xs[i]), xsum[i], zg);
-                    au += chunk_affine(chunk_dot(wu, xs[i]), xsum[i], zu);
+                if (t4 == 0) {
+                    s_part[warp * 2 * rows_gu + mt * 16 + g8] = acc_lo;
+                    s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = acc_hi;
                 }
-                ag = warp_sum(ag);
-                au = warp_sum(au);
-                if (lane == 0) { s_gu[lr] = ag * kUnscale; s_gu[rows_gu + lr] = au * kUnscale; }
             }
+            // the down block goes into the space of stages 0 and 1 once their four warps are done
+            if (warp < kFW / 2) {
+                if (lane == 0) mbar_arrive(&bars[BAR_FREE]);
+                if (warp == 0) {
+                    mbar_wait(&bars[BAR_FREE], 0, p.status);
+                    if (lane == 0) {
+                        const uint64_t pol = policy_evict_first();
+                        const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
+                        mbar_expect_tx(&bars[BAR_DOWN], dcb + dzb);
+                        bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), dcb, &bars[BAR_DOWN], pol);
+                        bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
+        if (tid < 2 * rows_gu) {
+            float v = 0.f;
+            for (int w = 0; w < kFW; ++w) v += s_part[w * 2 * rows_gu + tid];
+            s_gu[tid] = v;
         }
         __syncthreads();
         trace_mark(p, 4);
@@ -613,34 +669,92 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         mbar_wait(&bars[BAR_H], 0, p.status);                       // the cluster's quarter of h and of A_down.h
         trace_mark(p, 7);
 
-        // ---- down: partial over this quarter of the columns, for this CTA's H/4 output rows
+        // ---- down on the tensor cores: partial over this quarter of the columns, for this CTA's H/4
+        //      output rows.  h is fp32: column 0 of the B tile carries its fp16 value, column 1 the
+        //      fp16 residual, and the two result columns are added.
         if (tid < r) {
             float v = 0.f;
             for (int cc = 0; cc < kC; ++cc) v += s_ud_part[cc * kMaxRank + tid];
             s_ud[tid] = v;
         }
-        constexpr int RPW = 32 / LPR_D;
-        const int sub = lane % LPR_D, rsub = lane / LPR_D;
-        float hs[32];
-        float hsum;
+        uint32_t hb[DCH][4];
+        float hsum[(DCH + 1) / 2];
         {
-            float hv[32];
-            const float4* hp = reinterpret_cast<const float4*>(s_h + sub * 32);
+            float part[(DCH + 1) / 2];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const float4 v = hp[q];
-                hv[q * 4 + 0] = v.x; hv[q * 4 + 1] = v.y; hv[q * 4 + 2] = v.z; hv[q * 4 + 3] = v.w;
+            for (int j = 0; j < (DCH + 1) / 2; ++j) part[j] = 0.f;
+#pragma unroll
+            for (int i = 0; i < DCH; ++i) {
+                float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (g8 < 2) {
+                    const float4 a = *reinterpret_cast<const float4*>(s_h + i * 32 + t4 * 8);
+                    const float4 b = *reinterpret_cast<const float4*>(s_h + i * 32 + t4 * 8 + 4);
+                    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+                }
+                const uint4 q = g8 == 0 ? permute8(f) : permute8_lo(f);       // lanes g >= 2 hold zeros either way
+                hb[i][0] = q.x; hb[i][1] = q.y; hb[i][2] = q.z; hb[i][3] = q.w;
+                float sum = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sum += f[e];             // hi + lo == h up to 2^-22: sum h itself
+                part[i / 2] += g8 == 0 ? sum : 0.f;
             }
-            hsum = scale_chunk(hv, hs);
+#pragma unroll
+            for (int j = 0; j < (DCH + 1) / 2; ++j) {
+                float v = part[j];
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                hsum[j] = __shfl_sync(0xFFFFFFFFu, v, 0);
+            }
         }
         mbar_wait(&bars[BAR_DOWN], 0, p.status);
-#pragma unroll 2
-        for (int lr = warp * RPW + rsub; lr < rows_d; lr += kFW * RPW) {
-            const uint4 wd = *reinterpret_cast<const uint4*>(smem + S.d_codes + lr * drow_b + sub * 16);
-            const uint32_t zd = *reinterpret_cast<const uint32_t*>(smem + S.d_sz + (lr * gps + (sub * 32) / p.group) * 4);
-            float acc = chunk_affine(chunk_dot(wd, hs), hsum, zd);
-            acc = group_sum<LPR_D>(acc);
-            if (sub == 0) s_o[lr] = acc * kUnscale;
+        {
+            const int cpb = p.group >= 64 ? 2 : 1;
+            const uint8_t* dcodes = smem + S.d_codes;
+            const uint8_t* dsz = smem + S.d_sz;
+            for (int ti = warp; ti < rows_d / 16; ti += kFW) {
+                float acc_lo = 0.f, acc_hi = 0.f;
+#pragma unroll
+                for (int i0 = 0; i0 < DCH; i0 += 2) {
+#pragma unroll
+                    for (int b = 0; b < 2; ++b) {
+                        if (cpb == 2 && b == 1) break;
+                        const int ia = i0 + b;
+                        if (ia >= DCH) break;
+                        const int gi = (ia * 32) / p.group;
+                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(dsz + (ti * gps + gi) * 64 + g8 * 4));
+                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(dsz + (ti * gps + gi) * 64 + 32 + g8 * 4));
+                        float cfr[4];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            if (u < cpb && ia + u < DCH) {
+                                const int i = ia + u;
+                                uint32_t alo[4], ahi[4];
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(dcodes + (ti * DCH + i) * 256 + g8 * 16 + t4 * 4), alo);
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(dcodes + (ti * DCH + i) * 256 + 128 + g8 * 16 + t4 * 4), ahi);
+                                if (u == 0) mma16816_zero(cfr, alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
+                                else mma16816(cfr, alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
+                                mma16816(cfr, alo[2], ahi[2], alo[3], ahi[3], hb[i][2], hb[i][3]);
+                            }
+                        }
+                        float hs_blk;
+                        if (cpb == 2) hs_blk = hsum[ia / 2];
+                        else {
+                            float v = 0.f;
+                            if (g8 == 0) {
+                                const float4 a = *reinterpret_cast<const float4*>(s_h + ia * 32 + t4 * 8);
+                                const float4 bb = *reinterpret_cast<const float4*>(s_h + ia * 32 + t4 * 8 + 4);
+                                v = a.x + a.y + a.z + a.w + bb.x + bb.y + bb.z + bb.w;
+                            }
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+                            hs_blk = __shfl_sync(0xFFFFFFFFu, v, 0);
+                        }
+                        acc_lo = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs_blk, cfr[0] + cfr[1]), acc_lo);
+                        acc_hi = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs_blk, cfr[2] + cfr[3]), acc_hi);
+                    }
+                }
+                if (t4 == 0) { s_o[ti * 16 + g8] = acc_lo; s_o[ti * 16 + 8 + g8] = acc_hi; }
+            }
         }
         __syncthreads();                  // s_o and s_ud complete
         pdl_wait_prior_grid();            // the reduce scratch belongs to the previous layer-step until it ends
@@ -689,14 +803,15 @@ constexpr size_t kFusedSmemLimit = 112 * 1024;    // two CTAs per SM
 
 bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
-    if ((d.I / kE16) % kStages != 0 || d.I / kE16 > 32) return false;
+    if ((d.I / kE16) % 16 != 0 || d.I / kE16 > 32) return false;   // whole 16-row tiles per CTA
+    if (d.group > 128) return false;
     if (d.rank % 8 != 0) return false;            // adapter slices are staged by 16-byte bulk copies
     return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
 }
 
-template <int NCH, int LPR_D>
+template <int NCW, int DCH>
 static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cudaStream_t st) {
-    auto kern = fused_layer_kernel<NCH, LPR_D>;
+    auto kern = fused_layer_kernel<NCW, DCH>;
     static bool configured = false;       // per-process, per-instantiation one-time attributes
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmemLimit);
@@ -758,10 +873,10 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     if (W_pre != nullptr && flag_in < 0) EDG_CUDA_TRY(cudaMemsetAsync(p.flags, 0, 4 * sizeof(int32_t), st));
     const size_t smem = fused_smem(d->H, d->I, d->E, d->group, p.rank).total;
     cudaError_t e;
-    if (d->H == 2048 && d->I == 512) e = launch_fused<2, 4>(p, smem, pdl, st);
-    else if (d->H == 2048 && d->I == 256) e = launch_fused<2, 2>(p, smem, pdl, st);
-    else if (d->H == 1024 && d->I == 512) e = launch_fused<1, 4>(p, smem, pdl, st);
-    else if (d->H == 1024 && d->I == 256) e = launch_fused<1, 2>(p, smem, pdl, st);
+    if (d->H == 2048 && d->I == 512) e = launch_fused<8, 4>(p, smem, pdl, st);
+    else if (d->H == 2048 && d->I == 256) e = launch_fused<8, 2>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 512) e = launch_fused<4, 4>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 256) e = launch_fused<4, 2>(p, smem, pdl, st);
     else return EDG_E_SHAPE;
     EDG_CUDA_TRY(e);
     return EDG_OK;

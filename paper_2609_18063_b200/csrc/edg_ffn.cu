@@ -162,7 +162,6 @@ __global__ void __launch_bounds__(kWarps * 32) gate_up_kernel(FfnParams p) {
     }
     __syncthreads();
 
-    const int row_bytes = p.H / 2, groups = p.H / p.group;
     const int row0 = blockIdx.x * (kWarps * RPW * kPasses);
     uint4 cg[kPasses][NCH], cu[kPasses][NCH];
     uint32_t zg[kPasses][NCH], zu[kPasses][NCH];
@@ -172,8 +171,8 @@ __global__ void __launch_bounds__(kWarps * 32) gate_up_kernel(FfnParams p) {
 #pragma unroll
         for (int i = 0; i < NCH; ++i) {
             const int c = sub + LPR * i;
-            const size_t co = (size_t)n * row_bytes + c * 16;
-            const size_t so = ((size_t)n * groups + (c * 32) / p.group) * 4;
+            const size_t co = code_off(p.H, n, c);
+            const size_t so = sz_off(p.H, p.group, n, (c * 32) / p.group);
             cg[ps][i] = ld_stream16(rec + p.L.codes_gate + co);
             cu[ps][i] = ld_stream16(rec + p.L.codes_up + co);
             zg[ps][i] = ld_stream4(rec + p.L.sz_gate + so);

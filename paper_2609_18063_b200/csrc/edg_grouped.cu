@@ -16,7 +16,7 @@
 // The LoRA delta is one more MMA k-step with A = B_lora rows and B = sigma * (A_lora . x).
 // Every pair's gate-weighted output goes to a [T*K][H] scratch and is reduced per token in the
 // order of its K choices, so y does not depend on how the groups were scheduled.
-#include "edg_common.cuh"
+#include "edg_mma.cuh"
 
 namespace edg {
 
@@ -54,64 +54,6 @@ struct GroupedParams {
     float sigma;
     RecordLayout L;
 };
-
-// ---------------------------------------------------------------- fragments
-
-__device__ __forceinline__ uint32_t lop3_and_or(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-__device__ __forceinline__ uint32_t h2_as_u32(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
-__device__ __forceinline__ __half2 u32_as_h2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
-
-// One 32-bit word = codes k0..k7 of one row.  Returns the four half2 (k0,k4) (k1,k5) (k2,k6) (k3,k7)
-// of q - z, exact for integer zero points.
-__device__ __forceinline__ void dequant_word(uint32_t w, __half2 z2, uint32_t (&out)[4]) {
-    const __half2 k1024 = __float2half2_rn(1024.f), k64 = __float2half2_rn(64.f), k16th = __float2half2_rn(0.0625f);
-    const uint32_t w2 = w >> 8;
-    const __half2 q04 = __hsub2(u32_as_h2(lop3_and_or(w, 0x000F000Fu, 0x64006400u)), k1024);
-    const __half2 q15 = __hfma2(u32_as_h2(lop3_and_or(w, 0x00F000F0u, 0x64006400u)), k16th, __hneg2(k64));
-    const __half2 q26 = __hsub2(u32_as_h2(lop3_and_or(w2, 0x000F000Fu, 0x64006400u)), k1024);
-    const __half2 q37 = __hfma2(u32_as_h2(lop3_and_or(w2, 0x00F000F0u, 0x64006400u)), k16th, __hneg2(k64));
-    out[0] = h2_as_u32(__hsub2(q04, z2));
-    out[1] = h2_as_u32(__hsub2(q15, z2));
-    out[2] = h2_as_u32(__hsub2(q26, z2));
-    out[3] = h2_as_u32(__hsub2(q37, z2));
-}
-
-// d = a . b  (fresh accumulator)
-__device__ __forceinline__ void mma16816_zero(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
-                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
-}
-__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// 8 consecutive fp32 activations -> the fp16 residuals v - fp16(v), same k-slot order
-__device__ __forceinline__ uint4 permute8_lo(const float (&v)[8]) {
-    float r[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) r[i] = v[i] - __half2float(__float2half_rn(v[i]));
-    uint4 o;
-    o.x = h2_as_u32(__floats2half2_rn(r[0], r[4]));
-    o.y = h2_as_u32(__floats2half2_rn(r[1], r[5]));
-    o.z = h2_as_u32(__floats2half2_rn(r[2], r[6]));
-    o.w = h2_as_u32(__floats2half2_rn(r[3], r[7]));
-    return o;
-}
-
-// 8 consecutive activations -> fp16 in the k-slot order of the fragments: (x0,x4,x1,x5,x2,x6,x3,x7)
-__device__ __forceinline__ uint4 permute8(const float (&v)[8]) {
-    uint4 r;
-    r.x = h2_as_u32(__floats2half2_rn(v[0], v[4]));
-    r.y = h2_as_u32(__floats2half2_rn(v[1], v[5]));
-    r.z = h2_as_u32(__floats2half2_rn(v[2], v[6]));
-    r.w = h2_as_u32(__floats2half2_rn(v[3], v[7]));
-    return r;
-}
 
 // The LoRA delta as one MMA k-step per 16 ranks: acc += Bl[rows][r] . (sigma * u[token][r]).
 // Bl: bf16 [..][rank], row pointers for rows g and g+8 of the tile; u row pointers per column tile.
@@ -238,7 +180,6 @@ __global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_gate_
 #pragma unroll
         for (int i = 0; i < 4; ++i) { ag[nt][i] = 0.f; au[nt][i] = 0.f; }
 
-    const int row_b = p.H / 2, groups = p.H / p.group;
     for (int kc = 0; kc < p.H / G_KC; ++kc) {
         __syncthreads();
         for (int idx = tid; idx < G_NTOK * 4; idx += G_WARPS * 32) {   // activations: token idx/4, 64 k starting at (idx%4)*64
@@ -260,13 +201,13 @@ __global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_gate_
 #pragma unroll
         for (int m = 0; m < 4; ++m) {   // codes: 128 rows x 128 bytes per matrix
             const int idx = tid + 256 * m, row = idx >> 3, seg = idx & 7;
-            const size_t off = (size_t)(row0 + row) * row_b + kc * (G_KC / 2) + seg * 16;
+            const size_t off = code_off(p.H, row0 + row, kc * (G_KC / 32) + seg);
             *reinterpret_cast<uint4*>(s_cg + row * G_CS + seg * 16) = ld_stream16(rec + p.L.codes_gate + off);
             *reinterpret_cast<uint4*>(s_cu + row * G_CS + seg * 16) = ld_stream16(rec + p.L.codes_up + off);
         }
         for (int idx = tid; idx < 128 * ng; idx += 256) {
             const int row = idx / ng, gi = idx % ng;
-            const size_t off = ((size_t)(row0 + row) * groups + kc * ng + gi) * 4;
+            const size_t off = sz_off(p.H, p.group, row0 + row, kc * ng + gi);
             s_zg[idx] = ld_stream4(rec + p.L.sz_gate + off);
             s_zu[idx] = ld_stream4(rec + p.L.sz_up + off);
         }

@@ -26,30 +26,21 @@ int32_t check_desc(const edg_layer_desc* d) {
     return EDG_OK;
 }
 
-// interleave (scale, zero) pairs: sz[i] = {scale[i], zero[i]}
-static void pack_sz(const uint16_t* s, const uint16_t* z, size_t n, uint8_t* dst) {
-    uint16_t* o = reinterpret_cast<uint16_t*>(dst);
-    for (size_t i = 0; i < n; ++i) { o[2 * i] = s[i]; o[2 * i + 1] = z[i]; }
-}
-static void unpack_sz(const uint8_t* src, size_t n, uint16_t* s, uint16_t* z) {
-    const uint16_t* o = reinterpret_cast<const uint16_t*>(src);
-    for (size_t i = 0; i < n; ++i) { s[i] = o[2 * i]; z[i] = o[2 * i + 1]; }
-}
-
-// down: canonical row-major [H][I] <-> kDownSlices column slices
-static void pack_down(const edg_layer_desc& d, const RecordLayout& L, const uint8_t* codes, const uint16_t* s,
-                      const uint16_t* z, uint8_t* r, bool to_record, uint8_t* codes_out, uint16_t* s_out, uint16_t* z_out) {
-    const int H = d.H, I = d.I, g = d.group;
-    for (int n = 0; n < H; ++n) {
-        for (int c = 0; c < I / 32; ++c) {
-            uint8_t* rec = r + L.codes_down + down_code_off(H, I, n, c);
-            const size_t can = (size_t)n * (I / 2) + (size_t)c * 16;
-            if (to_record) memcpy(rec, codes + can, 16); else memcpy(codes_out + can, rec, 16);
+// canonical row-major [N][Kd] (codes) / [N][Kd/group] (scales, zeros) <-> tile-major sections.
+// `down` selects the sliced variant.  to_record: canonical -> record, else record -> canonical.
+static void repack(const edg_layer_desc& d, int N, int Kd, bool down, uint8_t* rec_codes, uint8_t* rec_sz,
+                   uint8_t* codes, uint16_t* sc, uint16_t* ze, bool to_record) {
+    const int g = d.group;
+    for (int n = 0; n < N; ++n) {
+        for (int c = 0; c < Kd / 32; ++c) {
+            uint8_t* r = rec_codes + (down ? down_code_off(d.H, d.I, n, c) : code_off(Kd, n, c));
+            uint8_t* k = codes + (size_t)n * (Kd / 2) + (size_t)c * 16;
+            if (to_record) memcpy(r, k, 16); else memcpy(k, r, 16);
         }
-        for (int gi = 0; gi < I / g; ++gi) {
-            uint16_t* rec = reinterpret_cast<uint16_t*>(r + L.sz_down + down_sz_off(H, I, g, n, gi));
-            const size_t can = (size_t)n * (I / g) + gi;
-            if (to_record) { rec[0] = s[can]; rec[1] = z[can]; } else { s_out[can] = rec[0]; z_out[can] = rec[1]; }
+        for (int gi = 0; gi < Kd / g; ++gi) {
+            uint16_t* r = reinterpret_cast<uint16_t*>(rec_sz + (down ? down_sz_off(d.H, d.I, g, n, gi) : sz_off(Kd, g, n, gi)));
+            const size_t k = (size_t)n * (Kd / g) + gi;
+            if (to_record) { r[0] = sc[k]; r[1] = ze[k]; } else { sc[k] = r[0]; ze[k] = r[1]; }
         }
     }
 }
@@ -80,16 +71,15 @@ extern "C" int32_t edg_pack_expert(const edg_layer_desc* desc,
     if (rc != EDG_OK) return rc;
     if (!cg || !sg || !zg || !cu || !su || !zu || !cd || !sd || !zd || !record) return EDG_E_INVAL;
     const edg::RecordLayout L = edg::record_layout(desc->H, desc->I, desc->group);
-    const size_t cbytes = (size_t)desc->H * desc->I / 2, ngroups = (size_t)desc->H * desc->I / desc->group;
     uint8_t* r = static_cast<uint8_t*>(record);
-    // gate / up keep the canonical order (row-major, low nibble first): a 32-bit word then holds
-    // code k in bits 4k..4k+3, which is what the in-place nibble masks expect.  down keeps that
-    // order inside each of its column slices.
-    memcpy(r + L.codes_gate, cg, cbytes);
-    memcpy(r + L.codes_up, cu, cbytes);
-    edg::pack_sz(sg, zg, ngroups, r + L.sz_gate);
-    edg::pack_sz(su, zu, ngroups, r + L.sz_up);
-    edg::pack_down(*desc, L, cd, sd, zd, r, true, nullptr, nullptr, nullptr);
+    // Inside every 16-byte chunk the canonical nibble order is kept (a 32-bit word holds code k in
+    // bits 4k..4k+3); the chunks are re-arranged tile-major.
+    edg::repack(*desc, desc->I, desc->H, false, r + L.codes_gate, r + L.sz_gate, const_cast<uint8_t*>(cg),
+                const_cast<uint16_t*>(sg), const_cast<uint16_t*>(zg), true);
+    edg::repack(*desc, desc->I, desc->H, false, r + L.codes_up, r + L.sz_up, const_cast<uint8_t*>(cu),
+                const_cast<uint16_t*>(su), const_cast<uint16_t*>(zu), true);
+    edg::repack(*desc, desc->H, desc->I, true, r + L.codes_down, r + L.sz_down, const_cast<uint8_t*>(cd),
+                const_cast<uint16_t*>(sd), const_cast<uint16_t*>(zd), true);
     return EDG_OK;
 }
 
@@ -101,12 +91,10 @@ extern "C" int32_t edg_unpack_expert(const edg_layer_desc* desc, const void* rec
     if (rc != EDG_OK) return rc;
     if (!cg || !sg || !zg || !cu || !su || !zu || !cd || !sd || !zd || !record) return EDG_E_INVAL;
     const edg::RecordLayout L = edg::record_layout(desc->H, desc->I, desc->group);
-    const size_t cbytes = (size_t)desc->H * desc->I / 2, ngroups = (size_t)desc->H * desc->I / desc->group;
     const uint8_t* r = static_cast<const uint8_t*>(record);
-    memcpy(cg, r + L.codes_gate, cbytes);
-    memcpy(cu, r + L.codes_up, cbytes);
-    edg::unpack_sz(r + L.sz_gate, ngroups, sg, zg);
-    edg::unpack_sz(r + L.sz_up, ngroups, su, zu);
-    edg::pack_down(*desc, L, nullptr, nullptr, nullptr, const_cast<uint8_t*>(r), false, cd, sd, zd);
+    uint8_t* rr = const_cast<uint8_t*>(r);
+    edg::repack(*desc, desc->I, desc->H, false, rr + L.codes_gate, rr + L.sz_gate, cg, sg, zg, false);
+    edg::repack(*desc, desc->I, desc->H, false, rr + L.codes_up, rr + L.sz_up, cu, su, zu, false);
+    edg::repack(*desc, desc->H, desc->I, true, rr + L.codes_down, rr + L.sz_down, cd, sd, zd, false);
     return EDG_OK;
 }

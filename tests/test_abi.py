@@ -66,12 +66,24 @@ def test_pack_unpack_identity_and_layout(lib):
     for proj in ("gate", "up", "down"):
         for a, b in zip(ex[proj], back[proj]):
             assert np.array_equal(np.asarray(a).view(np.uint8), np.asarray(b).view(np.uint8))
-    # the record's code sections are the canonical nibble order the oracle unpacks
+    # tile-major sections: chunk c (codes 32c..32c+31) of row n sits at ((n//16 * Kd/32 + c) * 16 + n%16) * 16,
+    # with the canonical nibble order inside the chunk; (scale, zero) pairs at ((n//16 * Kd/g + gi) * 16 + n%16) * 4
     half = cfg.H * cfg.I // 2
-    assert np.array_equal(orc.unpack_codes(rec[:half].reshape(cfg.I, cfg.H // 2)), orc.unpack_codes(ex["gate"][0]))
-    # (scale, zero) pairs interleaved after the codes
-    sz = rec[3 * half:3 * half + 8].view(np.float16)
-    assert sz[0] == ex["gate"][1][0, 0] and sz[1] == ex["gate"][2][0, 0] and sz[2] == ex["gate"][1][0, 1]
+    def code_off(Kd, n, c):
+        return ((n // 16 * (Kd // 32) + c) * 16 + n % 16) * 16
+    for n, c in [(0, 0), (5, 3), (17, 31), (255, 7)]:
+        o = code_off(cfg.H, n, c)
+        assert np.array_equal(rec[o:o + 16], ex["gate"][0][n, 16 * c:16 * c + 16])
+        assert np.array_equal(rec[half + o:half + o + 16], ex["up"][0][n, 16 * c:16 * c + 16])
+    n, gi = 21, 9
+    o = 3 * half + ((n // 16 * (cfg.H // cfg.group) + gi) * 16 + n % 16) * 4
+    sz = rec[o:o + 4].view(np.float16)
+    assert sz[0] == ex["gate"][1][n, gi] and sz[1] == ex["gate"][2][n, gi]
+    # down: four column slices of I/4 codes, each tile-major
+    sw = cfg.I // 4
+    n, c = 700, 5                                              # chunk 5 = codes 160..191 -> slice 2, chunk 1 of the slice
+    o = 2 * half + (c // (sw // 32)) * (cfg.H * sw // 2) + code_off(sw, n, c % (sw // 32))
+    assert np.array_equal(rec[o:o + 16], ex["down"][0][n, 16 * c:16 * c + 16])
     with pytest.raises(ValueError):
         lib.pack_expert(lib.make_desc(synth.CONFIGS["cfg2"]), ex)
 
