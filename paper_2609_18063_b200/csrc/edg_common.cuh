@@ -75,15 +75,16 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 
 // Workspace layout for T tokens (floats unless noted).  The first 256 bytes are a control block
 // whose first int32 is the device-side status word; bytes 64..127 hold the per-slice arrival
-// counters of the fused kernel's reduce, byte 128 the count of head rows delivered (all zero
-// between launches) and bytes 160..175 the routing-ready flags of chained layer-steps.
+// counters of the fused kernel's reduce, bytes 128..143 the counts of head rows delivered (one per
+// ring slot of chained layer-steps) and bytes 160..175 the reader counts of the ring slots.
 struct WorkspaceLayout {
     size_t ctrl;      // 256 B control block
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
     size_t partial;   // [K*kDownSlices][H] float   : gate-weighted partial expert outputs of the fused batch-1 kernel
-    size_t logits;    // [E] float                  : next-step head logits gathered across CTAs
+    size_t logits;    // [4][E] float               : next-step head logits gathered across CTAs, one per ring slot
+    size_t route;     // 1 KB                       : routing handed between chained steps: [4][32] int32 + [4][32] float
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
     size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
@@ -107,7 +108,8 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
     W.logits = round_up(W.partial + (size_t)d.K * 4 * d.H * sizeof(float), 256);
-    size_t end = round_up(W.logits + (size_t)d.E * sizeof(float), 256);
+    W.route = round_up(W.logits + 4 * (size_t)d.E * sizeof(float), 256);
+    size_t end = W.route + 1024;
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;
@@ -221,40 +223,61 @@ __device__ __forceinline__ uint32_t ld_stream4(const void* p) {
     return v;
 }
 
+// Order-preserving map float -> uint32 (larger float <=> larger key; -0 < +0 is harmless here).
+__device__ __forceinline__ uint32_t float_key(float v) {
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// Best remaining candidate of a lane: entries lane, lane+32, ... of work[]; taken entries hold NaN.
+__device__ __forceinline__ void lane_best(const float* work, int E, int lane, uint32_t& key, int& idx) {
+    key = 0u;
+    idx = 0x7FFFFFFF;
+    for (int e = lane; e < E; e += 32) {
+        const float v = work[e];
+        if (v == v) {                                   // not taken (and not a NaN logit)
+            const uint32_t kk = float_key(v);
+            if (idx == 0x7FFFFFFF || kk > key) { key = kk; idx = e; }   // ascending e: the lowest index wins ties
+        }
+    }
+}
+
 // Top-k of work[0..E) by one warp, ties to the lower index; the K winners are written in
 // ascending index with gate weights exp(l - max) / sum over the winners (which equals
 // softmax(l)[inds] / sum softmax(l)[inds]: the full-softmax denominator cancels).
-// `work` is overwritten.
+// Every lane caches its best remaining candidate; a round is one warp-wide max on sortable keys
+// and one warp-wide min on the indices that hold it (redux.sync), and only the winning lane
+// rescans its candidates.  `work` is overwritten.
 __device__ __forceinline__ void warp_softmax_topk(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
     const unsigned full = 0xFFFFFFFFu;
     float myv = 0.f;
     int myi = 0x7FFFFFFF;
+    uint32_t key;
+    int idx;
+    lane_best(work, E, lane, key, idx);
     for (int j = 0; j < K; ++j) {
-        float bv = -__int_as_float(0x7f800000);
-        int bi = 0x7FFFFFFF;
-        for (int e = lane; e < E; e += 32) {
-            const float v = work[e];
-            if (v > bv || (v == bv && e < bi)) { bv = v; bi = e; }
+        const uint32_t best = __reduce_max_sync(full, idx == 0x7FFFFFFF ? 0u : key);
+        const int cand = (idx != 0x7FFFFFFF && key == best) ? idx : 0x7FFFFFFF;
+        const int win = (int)__reduce_min_sync(full, (unsigned)cand);
+        if (win == 0x7FFFFFFF) break;                   // fewer than K finite logits
+        const float wv = work[win];
+        if (lane == j) { myv = wv; myi = win; }
+        __syncwarp();
+        if (idx == win) {                               // the owner retires it and looks for its next best
+            work[win] = __int_as_float(0x7fffffff);
+            lane_best(work, E, lane, key, idx);
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(full, bv, o);
-            const int oi = __shfl_xor_sync(full, bi, o);
-            if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-        }
-        if (lane == j) { myv = bv; myi = bi; }
-        if (bi != 0x7FFFFFFF && (bi & 31) == lane) work[bi] = __int_as_float(0x7fffffff);   // taken: never compares true again
         __syncwarp();
     }
     const float m = __shfl_sync(full, myv, 0);
-    const float ex = lane < K ? expf(myv - m) : 0.f;
+    const float ex = (lane < K && myi != 0x7FFFFFFF) ? expf(myv - m) : 0.f;
     const float sum = warp_sum(ex);
     int rank = 0;
     for (int i = 0; i < K; ++i) {
         const int oi = __shfl_sync(full, myi, i);
         rank += (oi < myi) ? 1 : 0;
     }
-    if (lane < K) {
+    if (lane < K && myi != 0x7FFFFFFF) {
         inds[rank] = myi;
         gates[rank] = ex / sum;
     }

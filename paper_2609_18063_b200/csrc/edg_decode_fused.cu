@@ -38,6 +38,7 @@ constexpr int kFW = 8;            // warps per CTA
 constexpr int kStages = 4;        // gate/up copy stages per CTA
 constexpr int kMaxRank = 64;
 constexpr int kTraceMarks = 16;
+constexpr int kRing = 4;          // chained layer-steps in flight: hand-off slots for routing, logits scratch, counters
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
 
 struct FusedParams {
@@ -62,9 +63,11 @@ struct FusedParams {
     float sigma;
     RecordLayout L;
     unsigned long long* trace;    // optional [grid CTAs][kTraceMarks] globaltimer stamps, or null
-    int32_t* flags;               // [0..1] routing-ready flags, [2..3] CTAs that have consumed them
-    int flag_in;                  // -1: the routing is already in memory; 0/1: wait for flags[flag_in]
-    int flag_out;                 // -1 or the flag to raise once inds_next / gates_next are written
+    int32_t* seen;                // [kRing] CTAs that have consumed the routing in each ring slot
+    int32_t* route_inds;          // [kRing][32] routing handed from one chained step to the next (-1 = not yet written)
+    float* route_gates;           // [kRing][32] (negative / NaN = not yet written)
+    int flag_in;                  // -1: the routing is already in memory; else the ring slot to take it from
+    int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -143,6 +146,19 @@ __device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
 __device__ __forceinline__ void st_release_gpu(int32_t* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ int atom_add_acq_rel_gpu(int32_t* p, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+__device__ __forceinline__ int ld_relaxed_gpu(const int32_t* p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_gpu(int32_t* p, int v) {
+    asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 // programmatic dependent launch: let the next kernel in the stream start / wait for the previous one
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -188,7 +204,7 @@ struct FusedSmem {
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
@@ -217,8 +233,9 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_o = o;        o += rows_d * 4;
     S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
     S.s_hloc = o;     o += 32 * 4;
-    S.s_topk = o;     o += (uint32_t)E * 4;           // logits gathered by the warp that finishes the routing
+    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the routing, then its K winners
     S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
+    S.s_table = o;    o += (uint32_t)E * 4;           // this layer's slot table, fetched before the routing is known
     S.flag = o;       o += 16;
     S.total = (o + 15) / 16 * 16;
     return S;
@@ -265,32 +282,34 @@ __device__ __forceinline__ float pre_row_partial(const FusedParams& p, int e, in
 // One warp: publish this CTA's logits (summed from the per-warp partials in s_pre), and if they were
 // the last ones of the head, gather all E, do softmax + top-k and raise the routing-ready flag.
 __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const FusedSmem& S,
-                                                 const float* s_pre, int n_rows, int lane) {
-    const int ncta = gridDim.x;
+                                                 const float* s_pre, int n_rows, int ncta, int lane) {
     int mine = 0;
+    const int ring = p.flag_out >= 0 ? p.flag_out : 0;
+    float* logits_ws = p.logits_ws + (size_t)ring * p.E;
+    int32_t* pre_counter = p.pre_counter + ring;
     if (lane < n_rows) {
         const int e = blockIdx.x + lane * ncta;
         if (e < p.E) {
             float v = 0.f;
             for (int w = 0; w < kFW; ++w) v += s_pre[lane * kFW + w];
-            p.logits_ws[e] = v;
+            logits_ws[e] = v;
             mine = 1;
         }
     }
     const int n_mine = __popc(__ballot_sync(0xFFFFFFFFu, mine));
-    __threadfence();
+    __syncwarp();
     int last = 0;
-    if (lane == 0) last = (atomicAdd(p.pre_counter, n_mine) + n_mine == p.E) ? 1 : 0;
+    // the counting atomic releases this warp's logits and acquires everyone else's
+    if (lane == 0) last = (atom_add_acq_rel_gpu(pre_counter, n_mine) + n_mine == p.E) ? 1 : 0;
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
     if (last) {
-        __threadfence();
         float* work = reinterpret_cast<float*>(smem + S.s_topk);
         for (int i0 = 0; i0 < p.E; i0 += 256) {                 // 8 independent loads per lane and pass
             float v[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int i = i0 + u * 32 + lane;
-                v[u] = i < p.E ? __ldcg(&p.logits_ws[i]) : 0.f;
+                v[u] = i < p.E ? __ldcg(&logits_ws[i]) : 0.f;
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
@@ -302,23 +321,72 @@ __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* 
             }
         }
         __syncwarp();
-        warp_softmax_topk(work, p.E, p.K, lane, p.inds_next, p.gates_next);
+        int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_topk) + p.E;      // [K] winners, then [K] gates
+        float* s_g = reinterpret_cast<float*>(s_i + 32);
+        warp_softmax_topk(work, p.E, p.K, lane, s_i, s_g);
         __syncwarp();
+        if (lane < p.K) {
+            p.inds_next[lane] = s_i[lane];
+            p.gates_next[lane] = s_g[lane];
+            if (p.flag_out >= 0) {
+                // The chained next step polls exactly these two words per expert; each is valid by itself.
+                // The slot is reused every kRing steps: wait (bounded) until its last reader has
+                // invalidated it, so that a routing still being read is never overwritten.
+                int32_t* ri = &p.route_inds[p.flag_out * 32 + lane];
+                uint32_t it = 0;
+                while (ld_relaxed_gpu(ri) >= 0 && ++it < kSpinLimit) {}
+                if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
+                st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_out * 32 + lane]), __float_as_int(s_g[lane]));
+                st_relaxed_gpu(ri, s_i[lane]);
+            }
+        }
         if (lane == 0) {
-            *p.pre_counter = 0;
-            __threadfence();
-            if (p.flag_out >= 0) st_release_gpu(&p.flags[p.flag_out], 1);
+            *pre_counter = 0;
             if (p.trace != nullptr) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.trace[(size_t)blockIdx.x * kTraceMarks + 15] = t; }
         }
     }
 }
 
 // ---------------------------------------------------------------- the fused kernel
-// NCW = H / 256 = chunks (of 32 codes) per warp in gate/up; DCH = I / 128 = chunks of a down row-slice.
+// NCW = H / 256 = chunks (of 32 codes) per warp in gate/up; DCH = I / 128 = chunks of a down row-slice;
+// TG = I / 256 = row tiles per matrix and CTA in gate/up; TD = H / 512 = row tiles per warp in down;
+// CPB = chunks per scaled block (2 for groups of 64 or 128 codes, 1 for groups of 32).
+
+// This CTA's share of the 2r rows of A_gate / A_up: per-warp partial dot products into s_red.
+// All threads take part, each covering 8 elements of a row per sweep; the loads of up to 8 rows
+// are in flight together, so the whole share costs one round trip to memory.
+#define LORA_A_ROWS(AD)                                                                                          \
+    do {                                                                                                          \
+        const int per_ = (2 * r + kC - 1) / kC;                                                                   \
+        for (int q0 = 0; q0 < per_; q0 += 8) {                                                                    \
+            float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};                                                \
+            for (int cc = tid * 8; cc < p.H; cc += kFW * 32 * 8) {                                                \
+                const uint4 ux = ld_keep16(p.x + cc);                                                             \
+                uint4 ua[8];                                                                                      \
+                _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                   \
+                    const int q = min(crank * per_ + min(q0 + u, per_ - 1), 2 * r - 1);                           \
+                    const uint16_t* A = reinterpret_cast<const uint16_t*>((q / r) ? p.lora.A_up : p.lora.A_gate) + \
+                                        ((size_t)(AD) * r + q % r) * p.H;                                         \
+                    ua[u] = ld_keep16(A + cc);                                                                    \
+                }                                                                                                 \
+                _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                   \
+                    v[u] = fmaf(bf16_lo(ua[u].x), bf16_lo(ux.x), v[u]); v[u] = fmaf(bf16_hi(ua[u].x), bf16_hi(ux.x), v[u]); \
+                    v[u] = fmaf(bf16_lo(ua[u].y), bf16_lo(ux.y), v[u]); v[u] = fmaf(bf16_hi(ua[u].y), bf16_hi(ux.y), v[u]); \
+                    v[u] = fmaf(bf16_lo(ua[u].z), bf16_lo(ux.z), v[u]); v[u] = fmaf(bf16_hi(ua[u].z), bf16_hi(ux.z), v[u]); \
+                    v[u] = fmaf(bf16_lo(ua[u].w), bf16_lo(ux.w), v[u]); v[u] = fmaf(bf16_hi(ua[u].w), bf16_hi(ux.w), v[u]); \
+                }                                                                                                 \
+            }                                                                                                     \
+            _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                       \
+                const float t_ = warp_sum(v[u]);                                                                  \
+                if (lane == 0 && q0 + u < per_) s_red[(q0 + u) * kFW + warp] = t_;                                \
+            }                                                                                                     \
+        }                                                                                                         \
+    } while (0)
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
+constexpr int kMaxPre = 8;        // head rows per head CTA
 
-template <int NCW, int DCH>
+template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b16 = blockIdx.x % kE16;             // CTA of the expert
@@ -340,9 +408,10 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     float* s_hloc = reinterpret_cast<float*>(smem + S.s_hloc);      // [rows_gu]
     float* s_part = reinterpret_cast<float*>(smem + S.s_part);      // [kFW][2 * rows_gu]
     int* s_flag = reinterpret_cast<int*>(smem + S.flag);
+    int* s_table = reinterpret_cast<int*>(smem + S.s_table);       // [E]
 
     const int rows_gu = p.I / kE16, rows_d = p.H / kC, sw = p.I / kDownSlices;
-    const int tg = rows_gu / 16;                   // row tiles per matrix in this CTA
+    constexpr int tg = TG;                         // row tiles per matrix in this CTA
     const int n0_gu = b16 * rows_gu;               // first gate/up row of this CTA (= c * sw + crank * rows_gu)
     const int n0_d = crank * rows_d;               // first down row of this CTA
     const int r = p.rank;
@@ -366,17 +435,21 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     }
     __syncthreads();
     cluster_arrive();
+    // The next layer-step may start now: its head needs nothing from this one, and everything it
+    // shares with this step is either in its own ring slot or touched only after it has waited for
+    // this kernel to end.
+    pdl_launch_dependents();
 
     // ---- loads that do not depend on the routing.  The hidden state as the MMA's B operand: the
     //      warp owns NCW chunks of 32 activations; the lanes of quad 0 hold them (column 0 of the
     //      8-column tile), every other lane holds zeros.  xsum[j] = sum of the activations of
     //      64-code block j (for the zero points).
     uint32_t xb[NCW][4];
-    float xsum[(NCW + 1) / 2];
+    float xsum[NCW / CPB];
     {
-        float part[(NCW + 1) / 2];
+        float part[NCW / CPB];
 #pragma unroll
-        for (int j = 0; j < (NCW + 1) / 2; ++j) part[j] = 0.f;
+        for (int j = 0; j < NCW / CPB; ++j) part[j] = 0.f;
 #pragma unroll
         for (int i = 0; i < NCW; ++i) {
             uint4 v = make_uint4(0, 0, 0, 0);
@@ -389,10 +462,10 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
             float sum = 0.f;
 #pragma unroll
             for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
-            part[i / 2] += sum;
+            part[i / CPB] += sum;
         }
 #pragma unroll
-        for (int j = 0; j < (NCW + 1) / 2; ++j) {
+        for (int j = 0; j < NCW / CPB; ++j) {
             float v = part[j];
             v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
             v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
@@ -400,54 +473,109 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         }
     }
 
-    // ---- a1 for the next step: this CTA's rows of the head, every thread 8 elements of each.  They
-    //      depend on nothing but x, so their loads go out first of all.
-    const int n_pre = p.W_pre != nullptr ? (p.E + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-    const bool pre_fast = n_pre > 0 && n_pre <= 2 && p.pre_dtype == EDG_F16 && p.H == kFW * 32 * 8;
-    uint4 lw[2], lx = make_uint4(0, 0, 0, 0);
+    // ---- the slot table of this layer does not depend on the routing either: one coalesced read
+    //      now saves a dependent trip to memory once the routing is known
+    if (p.table != nullptr)
+        for (int i = tid; i < p.E; i += kFW * 32) s_table[i] = __ldcg(&p.table[i]);
+
+    // ---- a1 for the next step.  Only the first CTAs of the grid evaluate the head: they are
+    //      dispatched first, so the routing of the next step is ready a few microseconds after this
+    //      kernel starts, whatever the rest of the grid is still waiting for.  A row is split over
+    //      all threads of its CTA (8 elements each); the loads depend on nothing but x and go out
+    //      first of all.
+    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
+    const int n_pre = ((int)blockIdx.x < n_head_ctas) ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
+    const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H == kFW * 32 * 8;
+    uint4 lw[kMaxPre], lx = make_uint4(0, 0, 0, 0);
     if (pre_fast) {
         lx = ld_keep16(p.x + tid * 8);
 #pragma unroll
-        for (int ri = 0; ri < 2; ++ri) {
-            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * (int)gridDim.x, p.E - 1);
+        for (int ri = 0; ri < kMaxPre; ++ri) {
+            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * n_head_ctas, p.E - 1);
             lw[ri] = ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8);
         }
     }
 
+    // ---- everything that needs only x is finished before the routing is even looked at: the head
+    //      rows' partial sums, and the adapter projections when the layer has one shared adapter
+    if (n_pre > 0) {
+#pragma unroll
+        for (int ri = 0; ri < kMaxPre; ++ri) {
+            if (ri < n_pre) {
+                const int e = (int)blockIdx.x + ri * n_head_ctas;
+                float v = pre_row_partial(p, e, tid, pre_fast, lw[ri], lx);
+                v = warp_sum(v);
+                if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
+            }
+        }
+    }
+    if (n_pre > 0) {
+        __syncthreads();                  // the head CTAs publish at once: the routing of the next step is under way
+        if (warp == kFW - 1) {
+            prerouter_finish(p, smem, S, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane);
+            if (lane == 0 && p.trace != nullptr) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.trace[(size_t)blockIdx.x * kTraceMarks + 13] = t; }
+        }
+    }
+    const bool lora_early = r > 0 && p.n_adapters == 1;
+    if (lora_early) LORA_A_ROWS(0);
+    trace_mark(p, 11);
+
     // ---- the routing may still be on its way: the previous layer-step raises a flag when its top-k
     //      is written, long before that kernel ends (bounded wait; on a time-out fall back to
     //      waiting for the whole previous kernel, which is always sufficient)
+    int slot;
+    float gate_k;
     if (p.flag_in >= 0) {
+        // chained: thread 0 polls this expert's own entry (index and gate arrive independently and
+        // are each valid by themselves), everyone else waits at the barrier
         if (tid == 0) {
+            const int32_t* ri = &p.route_inds[p.flag_in * 32 + k];
+            const int32_t* rg = reinterpret_cast<const int32_t*>(&p.route_gates[p.flag_in * 32 + k]);
+            int vi = -1, vg = -1;
             uint32_t it = 0;
-            while (ld_acquire_gpu(&p.flags[p.flag_in]) == 0 && ++it < kSpinLimit) {}
-            if (it >= kSpinLimit) { atomicExch(p.status, EDG_E_TIMEOUT); pdl_wait_prior_grid(); }
+            do { vi = ld_relaxed_gpu(ri); vg = ld_relaxed_gpu(rg); } while ((vi < 0 || vg < 0) && ++it < kSpinLimit);
+            if (vi < 0 || vg < 0) {          // timed out: the whole previous kernel is always enough
+                atomicExch(p.status, EDG_E_TIMEOUT);
+                pdl_wait_prior_grid();
+                vi = __ldcg(&p.slots[k]);
+                vg = __float_as_int(__ldcg(&p.gates[k]));
+            }
+            s_flag[1] = vi; s_flag[2] = vg;
         }
         __syncthreads();
+        slot = s_flag[1];
+        gate_k = __int_as_float(s_flag[2]);
+    } else {
+        slot = __ldcg(&p.slots[k]);
+        gate_k = __ldcg(&p.gates[k]);
+        __syncthreads();                  // s_table and s_red complete (the chained path passed a barrier above)
     }
     trace_mark(p, 14);
 
     // ---- a3: take.  The decision is the same in every CTA of the expert.
-    int slot = __ldcg(&p.slots[k]);
     const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
-    if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? p.table[slot] : -1;
+    if (p.table != nullptr) {
+        slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
+    }
     int ad = 0;
     if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
     const bool valid = slot >= 0 && slot < p.n_slots && ad >= 0;
-    const float gate_k = __ldcg(&p.gates[k]);
     trace_mark(p, 10);
     if (p.flag_in >= 0) {
-        // the CTA that is last to have read the routing re-arms the flag for the step after next
-        if (tid == 0 && atomicAdd(&p.flags[2 + p.flag_in], 1) == (int)gridDim.x - 1) {
-            p.flags[2 + p.flag_in] = 0;
-            st_release_gpu(&p.flags[p.flag_in], 0);
+        // the CTA that is last to have read the routing frees its ring slot
+        if (tid == 0) s_flag[3] = (atomicAdd(&p.seen[p.flag_in], 1) == (int)gridDim.x - 1) ? 1 : 0;
+        __syncthreads();
+        if (s_flag[3]) {                  // every CTA has read its entry: invalidate them for the producer after next
+            if (tid < 32) {
+                st_relaxed_gpu(&p.route_inds[p.flag_in * 32 + tid], -1);
+                st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_in * 32 + tid]), -1);
+            }
+            if (tid == 0) p.seen[p.flag_in] = 0;
+            __threadfence();
         }
         __syncthreads();
     }
-    pdl_launch_dependents();              // the next layer-step may start its own prologue now
     cluster_wait();                       // nothing is in flight yet: this returns at once
-    trace_mark(p, 11);
-
     const int cps = p.H / 128;            // chunks of a row per stage
     const int gpst = (p.H / 4) / p.group; // groups of a row per stage
     const int gps = sw / p.group;         // groups of a down row-slice
@@ -456,22 +584,24 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
         // ---- issue the copies of this CTA's gate/up slice (stage = a quarter of the K range, one run
         //      per matrix and row tile) and of its adapter rows, one warp per barrier
+        if (warp < kStages) {
+            // lane 0 arms the barrier, then lanes 0 .. 4*tg-1 issue one run each (codes or sz of a (matrix, tile))
+            const int s = warp;
+            uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+            if (lane == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
+            __syncwarp();
+            if (lane < 4 * tg) {
+                const uint64_t pol = policy_evict_first();   // weights stream through L2 once
+                const int mt = lane >> 1, is_sz = lane & 1, m = mt / tg, ti = mt % tg;
+                const int n = n0_gu + 16 * ti;
+                if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
+                                          S.mat_codes, &bars[s], pol);
+                else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
+                                   S.mat_sz, &bars[s], pol);
+            }
+        }
         if (lane == 0) {
-            const uint64_t pol = policy_evict_first();       // weights stream through L2 once
-            if (warp < kStages) {
-                const int s = warp;
-                uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-                mbar_expect_tx(&bars[s], S.stage_bytes);
-                for (int m = 0; m < 2; ++m) {
-                    const uint8_t* codes = rec + (m ? p.L.codes_up : p.L.codes_gate);
-                    const uint8_t* sz = rec + (m ? p.L.sz_up : p.L.sz_gate);
-                    for (int ti = 0; ti < tg; ++ti) {
-                        const int n = n0_gu + 16 * ti;
-                        bulk_g2s_hint(st + (m * tg + ti) * S.mat_codes, codes + code_off(p.H, n, s * cps), S.mat_codes, &bars[s], pol);
-                        bulk_g2s_hint(st + S.sz0 + (m * tg + ti) * S.mat_sz, sz + sz_off(p.H, p.group, n, s * gpst), S.mat_sz, &bars[s], pol);
-                    }
-                }
-            } else if (warp == kStages && r > 0) {
+            if (warp == kStages && r > 0) {
                 // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
                 const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
                 mbar_expect_tx(&bars[BAR_LORA], 2 * bgu + bd + r * ad_row);
@@ -488,54 +618,13 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         }
         trace_mark(p, 1);
     }
-
-    // ---- head rows: per-warp partials, then the last warp publishes them (and finishes the routing
-    //      of the next step if they were the last to arrive).  Publishing comes after the flag wait
-    //      above, i.e. after the previous layer-step is done with the shared logits scratch.
-    if (n_pre > 0) {
-        for (int ri = 0; ri < n_pre; ++ri) {
-            const int e = (int)blockIdx.x + ri * (int)gridDim.x;
-            float v = e < p.E ? pre_row_partial(p, e, tid, pre_fast, lw[ri & 1], lx) : 0.f;
-            v = warp_sum(v);
-            if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
-        }
-        __syncthreads();
-        if (warp == kFW - 1) prerouter_finish(p, smem, S, s_red + kPreRed * kFW, n_pre, lane);
-    }
-    trace_mark(p, 12);
-
     if (valid) {
         const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
 
-        // ---- LoRA: this CTA's share of the 2r rows of A_gate / A_up.  All threads take part: each
-        //      one covers 8 elements of a row per sweep, so a row costs one round trip to the L2.
         const int per = (2 * r + kC - 1) / kC;
-        for (int q0 = 0; q0 < per; q0 += 4) {
-            float v[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int cc = tid * 8; cc < p.H; cc += kFW * 32 * 8) {
-                const uint4 ux = ld_keep16(p.x + cc);
-                uint4 ua[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int q = min(crank * per + min(q0 + u, per - 1), 2 * r - 1);
-                    const uint16_t* A = reinterpret_cast<const uint16_t*>((q / r) ? p.lora.A_up : p.lora.A_gate) + ((size_t)ad * r + q % r) * p.H;
-                    ua[u] = ld_keep16(A + cc);
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    v[u] = fmaf(bf16_lo(ua[u].x), bf16_lo(ux.x), v[u]); v[u] = fmaf(bf16_hi(ua[u].x), bf16_hi(ux.x), v[u]);
-                    v[u] = fmaf(bf16_lo(ua[u].y), bf16_lo(ux.y), v[u]); v[u] = fmaf(bf16_hi(ua[u].y), bf16_hi(ux.y), v[u]);
-                    v[u] = fmaf(bf16_lo(ua[u].z), bf16_lo(ux.z), v[u]); v[u] = fmaf(bf16_hi(ua[u].z), bf16_hi(ux.z), v[u]);
-                    v[u] = fmaf(bf16_lo(ua[u].w), bf16_lo(ux.w), v[u]); v[u] = fmaf(bf16_hi(ua[u].w), bf16_hi(ux.w), v[u]);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const float t = warp_sum(v[u]);
-                if (lane == 0 && q0 + u < per) s_red[(q0 + u) * kFW + warp] = t;
-            }
+        if (r > 0 && !lora_early) {
+            LORA_A_ROWS(ad);
         }
-        if (p.trace != nullptr && tid == 0) { unsigned sm; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); p.trace[(size_t)blockIdx.x * kTraceMarks + 13] = sm; }
         __syncthreads();                  // s_red complete
         // every CTA of the cluster gets this CTA's adapter projections, counted on its BAR_U
         for (int i = tid; i < per * kC; i += kFW * 32) {
@@ -559,54 +648,42 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
             if (warp == 0) trace_mark(p, 3);
             const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
             const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
-            const int cpb = p.group >= 64 ? 2 : 1;                   // chunks per scaled block
-            for (int mt = 0; mt < 2 * tg; ++mt) {                    // (matrix, row tile)
-                const uint8_t* codes = st + mt * S.mat_codes;
-                const uint8_t* szs = st + S.sz0 + mt * S.mat_sz;
-                float acc_lo = 0.f, acc_hi = 0.f;                    // rows g and g+8, column 0
+            constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
+            float acc_lo[NT], acc_hi[NT];                            // rows g and g+8, column 0
 #pragma unroll
-                for (int i0 = 0; i0 < NCW; i0 += 2) {
+            for (int mt = 0; mt < NT; ++mt) { acc_lo[mt] = 0.f; acc_hi[mt] = 0.f; }
 #pragma unroll
-                    for (int b = 0; b < 2; b += 1) {
-                        // one scaled block = cpb chunks; with cpb == 1 the two chunks of this pair are two blocks
-                        if (cpb == 2 && b == 1) break;
-                        const int ia = i0 + b, nchunks = cpb;
-                        const int gi = ((ch0 + ia) * 32) / p.group;
-                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(szs + gi * 64 + g8 * 4));
-                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(szs + gi * 64 + 32 + g8 * 4));
-                        float cfr[4];
-                        float xs_blk = 0.f;
+            for (int ib = 0; ib < NCW / CPB; ++ib) {                 // scaled blocks of this warp's K range
+                const int gi = ((ch0 + ib * CPB) * 32) / p.group;
+                float cfr[NT][4];
 #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            if (u < nchunks) {
-                                const int i = ia + u;
-                                uint32_t alo[4], ahi[4];
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(codes + (ch0 + i) * 256 + g8 * 16 + t4 * 4), alo);
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(codes + (ch0 + i) * 256 + 128 + g8 * 16 + t4 * 4), ahi);
-                                if (u == 0) mma16816_zero(cfr, alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
-                                else mma16816(cfr, alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
-                                mma16816(cfr, alo[2], ahi[2], alo[3], ahi[3], xb[i][2], xb[i][3]);
-                            }
-                        }
-                        if (cpb == 2) xs_blk = xsum[ia / 2];
-                        else {   // 32-code blocks: the pair's sum was accumulated per 64; split it again
-                            xs_blk = 0.f;   // recomputed below for this single chunk
-                            const float v0 = __half2float(__low2half(u32_as_h2(xb[ia][0]))) + __half2float(__high2half(u32_as_h2(xb[ia][0])))
-                                           + __half2float(__low2half(u32_as_h2(xb[ia][1]))) + __half2float(__high2half(u32_as_h2(xb[ia][1])))
-                                           + __half2float(__low2half(u32_as_h2(xb[ia][2]))) + __half2float(__high2half(u32_as_h2(xb[ia][2])))
-                                           + __half2float(__low2half(u32_as_h2(xb[ia][3]))) + __half2float(__high2half(u32_as_h2(xb[ia][3])));
-                            float v = v0;
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-                            xs_blk = __shfl_sync(0xFFFFFFFFu, v, 0);
-                        }
-                        acc_lo = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs_blk, cfr[0]), acc_lo);
-                        acc_hi = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs_blk, cfr[2]), acc_hi);
+                for (int u = 0; u < CPB; ++u) {
+                    const int i = ib * CPB + u;
+#pragma unroll
+                    for (int mt = 0; mt < NT; ++mt) {
+                        const uint8_t* cw = st + mt * S.mat_codes + (ch0 + i) * 256 + g8 * 16 + t4 * 4;
+                        uint32_t alo[4], ahi[4];
+                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                        if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
+                        else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
+                        mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb[i][2], xb[i][3]);
                     }
                 }
-                if (t4 == 0) {
-                    s_part[warp * 2 * rows_gu + mt * 16 + g8] = acc_lo;
-                    s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = acc_hi;
+#pragma unroll
+                for (int mt = 0; mt < NT; ++mt) {
+                    const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
+                    const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                    const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                    acc_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xsum[ib], cfr[mt][0]), acc_lo[mt]);
+                    acc_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xsum[ib], cfr[mt][2]), acc_hi[mt]);
+                }
+            }
+            if (t4 == 0) {
+#pragma unroll
+                for (int mt = 0; mt < NT; ++mt) {
+                    s_part[warp * 2 * rows_gu + mt * 16 + g8] = acc_lo[mt];
+                    s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = acc_hi[mt];
                 }
             }
             // the down block goes into the space of stages 0 and 1 once their four warps are done
@@ -678,11 +755,11 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
             s_ud[tid] = v;
         }
         uint32_t hb[DCH][4];
-        float hsum[(DCH + 1) / 2];
+        float hsum[DCH / CPB];
         {
-            float part[(DCH + 1) / 2];
+            float part[DCH / CPB];
 #pragma unroll
-            for (int j = 0; j < (DCH + 1) / 2; ++j) part[j] = 0.f;
+            for (int j = 0; j < DCH / CPB; ++j) part[j] = 0.f;
 #pragma unroll
             for (int i = 0; i < DCH; ++i) {
                 float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -696,10 +773,10 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
                 float sum = 0.f;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) sum += f[e];             // hi + lo == h up to 2^-22: sum h itself
-                part[i / 2] += g8 == 0 ? sum : 0.f;
+                part[i / CPB] += g8 == 0 ? sum : 0.f;
             }
 #pragma unroll
-            for (int j = 0; j < (DCH + 1) / 2; ++j) {
+            for (int j = 0; j < DCH / CPB; ++j) {
                 float v = part[j];
                 v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
                 v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
@@ -708,52 +785,47 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         }
         mbar_wait(&bars[BAR_DOWN], 0, p.status);
         {
-            const int cpb = p.group >= 64 ? 2 : 1;
             const uint8_t* dcodes = smem + S.d_codes;
             const uint8_t* dsz = smem + S.d_sz;
-            for (int ti = warp; ti < rows_d / 16; ti += kFW) {
-                float acc_lo = 0.f, acc_hi = 0.f;
+            float acc_lo[TD], acc_hi[TD];                            // TD independent row tiles per warp: interleaved
 #pragma unroll
-                for (int i0 = 0; i0 < DCH; i0 += 2) {
+            for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
 #pragma unroll
-                    for (int b = 0; b < 2; ++b) {
-                        if (cpb == 2 && b == 1) break;
-                        const int ia = i0 + b;
-                        if (ia >= DCH) break;
-                        const int gi = (ia * 32) / p.group;
-                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(dsz + (ti * gps + gi) * 64 + g8 * 4));
-                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(dsz + (ti * gps + gi) * 64 + 32 + g8 * 4));
-                        float cfr[4];
+            for (int ib = 0; ib < DCH / CPB; ++ib) {
+                const int gi = (ib * CPB * 32) / p.group;
+                float cfr[TD][4];
 #pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            if (u < cpb && ia + u < DCH) {
-                                const int i = ia + u;
-                                uint32_t alo[4], ahi[4];
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(dcodes + (ti * DCH + i) * 256 + g8 * 16 + t4 * 4), alo);
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(dcodes + (ti * DCH + i) * 256 + 128 + g8 * 16 + t4 * 4), ahi);
-                                if (u == 0) mma16816_zero(cfr, alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
-                                else mma16816(cfr, alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
-                                mma16816(cfr, alo[2], ahi[2], alo[3], ahi[3], hb[i][2], hb[i][3]);
-                            }
-                        }
-                        float hs_blk;
-                        if (cpb == 2) hs_blk = hsum[ia / 2];
-                        else {
-                            float v = 0.f;
-                            if (g8 == 0) {
-                                const float4 a = *reinterpret_cast<const float4*>(s_h + ia * 32 + t4 * 8);
-                                const float4 bb = *reinterpret_cast<const float4*>(s_h + ia * 32 + t4 * 8 + 4);
-                                v = a.x + a.y + a.z + a.w + bb.x + bb.y + bb.z + bb.w;
-                            }
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-                            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-                            hs_blk = __shfl_sync(0xFFFFFFFFu, v, 0);
-                        }
-                        acc_lo = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs_blk, cfr[0] + cfr[1]), acc_lo);
-                        acc_hi = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs_blk, cfr[2] + cfr[3]), acc_hi);
+                for (int u = 0; u < CPB; ++u) {
+                    const int i = ib * CPB + u;
+#pragma unroll
+                    for (int tt = 0; tt < TD; ++tt) {
+                        const int ti = warp + kFW * tt;
+                        const uint8_t* cw = dcodes + (ti * DCH + i) * 256 + g8 * 16 + t4 * 4;
+                        uint32_t alo[4], ahi[4];
+                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                        if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
+                        else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
+                        mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb[i][2], hb[i][3]);
                     }
                 }
-                if (t4 == 0) { s_o[ti * 16 + g8] = acc_lo; s_o[ti * 16 + 8 + g8] = acc_hi; }
+#pragma unroll
+                for (int tt = 0; tt < TD; ++tt) {
+                    const int ti = warp + kFW * tt;
+                    const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
+                    const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                    const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                    acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hsum[ib], cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
+                    acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hsum[ib], cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
+                }
+            }
+            if (t4 == 0) {
+#pragma unroll
+                for (int tt = 0; tt < TD; ++tt) {
+                    const int ti = warp + kFW * tt;
+                    s_o[ti * 16 + g8] = acc_lo[tt];
+                    s_o[ti * 16 + 8 + g8] = acc_hi[tt];
+                }
             }
         }
         __syncthreads();                  // s_o and s_ud complete
@@ -809,9 +881,9 @@ bool fused_supported(const edg_layer_desc& d) {
     return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
 }
 
-template <int NCW, int DCH>
+template <int NCW, int DCH, int TG, int TD, int CPB>
 static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cudaStream_t st) {
-    auto kern = fused_layer_kernel<NCW, DCH>;
+    auto kern = fused_layer_kernel<NCW, DCH, TG, TD, CPB>;
     static bool configured = false;       // per-process, per-instantiation one-time attributes
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmemLimit);
@@ -865,18 +937,24 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.sigma = d->lora_scale;
     p.L = record_layout(d->H, d->I, d->group);
     p.trace = g_trace;
-    p.flags = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.seen = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.route_inds = reinterpret_cast<int32_t*>(ws + W.route);
+    p.route_gates = reinterpret_cast<float*>(ws + W.route + kRing * 32 * 4);
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
     // a call that starts a chain clears flags a broken chain may have left raised
-    if (W_pre != nullptr && flag_in < 0) EDG_CUDA_TRY(cudaMemsetAsync(p.flags, 0, 4 * sizeof(int32_t), st));
+    if (W_pre != nullptr && flag_in < 0) {
+        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 64, st));           // head-row counters and reader counts of the ring
+        EDG_CUDA_TRY(cudaMemsetAsync(p.route_inds, 0xFF, 2 * kRing * 32 * 4, st));   // -1 / NaN: nothing handed over yet
+    }
     const size_t smem = fused_smem(d->H, d->I, d->E, d->group, p.rank).total;
     cudaError_t e;
-    if (d->H == 2048 && d->I == 512) e = launch_fused<8, 4>(p, smem, pdl, st);
-    else if (d->H == 2048 && d->I == 256) e = launch_fused<8, 2>(p, smem, pdl, st);
-    else if (d->H == 1024 && d->I == 512) e = launch_fused<4, 4>(p, smem, pdl, st);
-    else if (d->H == 1024 && d->I == 256) e = launch_fused<4, 2>(p, smem, pdl, st);
+    const bool wide = d->group >= 64;         // scaled blocks of 64 codes (groups of 64 or 128) or of 32
+    if (d->H == 2048 && d->I == 512) e = wide ? launch_fused<8, 4, 2, 4, 2>(p, smem, pdl, st) : launch_fused<8, 4, 2, 4, 1>(p, smem, pdl, st);
+    else if (d->H == 2048 && d->I == 256) e = wide ? launch_fused<8, 2, 1, 4, 2>(p, smem, pdl, st) : launch_fused<8, 2, 1, 4, 1>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 512) e = wide ? launch_fused<4, 4, 2, 2, 2>(p, smem, pdl, st) : launch_fused<4, 4, 2, 2, 1>(p, smem, pdl, st);
+    else if (d->H == 1024 && d->I == 256) e = wide ? launch_fused<4, 2, 1, 2, 2>(p, smem, pdl, st) : launch_fused<4, 2, 1, 2, 1>(p, smem, pdl, st);
     else return EDG_E_SHAPE;
     EDG_CUDA_TRY(e);
     return EDG_OK;
