@@ -82,7 +82,7 @@ struct WorkspaceLayout {
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
-    size_t partial;   // [K*kDownSlices][H] float   : gate-weighted partial expert outputs of the fused batch-1 kernel
+    size_t partial;   // [4][K*kDownSlices][H] float: gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
     size_t logits;    // [4][E] float               : next-step head logits gathered across CTAs, one per ring slot
     size_t route;     // 1 KB                       : routing handed between chained steps: [4][32] int32 + [4][32] float
     // grouped path (T > 1) only:
@@ -107,7 +107,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.logits = round_up(W.partial + (size_t)d.K * 4 * d.H * sizeof(float), 256);
+    W.logits = round_up(W.partial + 4 * (size_t)d.K * kDownSlices * d.H * sizeof(float), 256);
     W.route = round_up(W.logits + 4 * (size_t)d.E * sizeof(float), 256);
     size_t end = W.route + 1024;
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
@@ -242,13 +242,77 @@ __device__ __forceinline__ void lane_best(const float* work, int E, int lane, ui
     }
 }
 
+// Inverse of float_key.
+__device__ __forceinline__ float key_float(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+// Shared tail of the two top-k variants: lane j < K holds winner j (value myv, index myi, or
+// myi == INT_MAX when there were fewer than K finite logits), lane 0 the largest.  Writes the
+// winners in ascending index with gates exp(l - max) / sum over the winners.
+__device__ __forceinline__ void topk_emit(float myv, int myi, int K, int lane, int32_t* inds, float* gates) {
+    const unsigned full = 0xFFFFFFFFu;
+    const float m = __shfl_sync(full, myv, 0);
+    const float ex = (lane < K && myi != 0x7FFFFFFF) ? expf(myv - m) : 0.f;
+    const float sum = warp_sum(ex);
+    int rank = 0;
+#pragma unroll 1
+    for (int i = 0; i < K; ++i) {
+        const int oi = __shfl_sync(full, myi, i);
+        rank += (oi < myi) ? 1 : 0;
+    }
+    if (lane < K && myi != 0x7FFFFFFF) {
+        inds[rank] = myi;
+        gates[rank] = ex / sum;
+    }
+}
+
+// Top-k with the candidates in registers: lane l holds entries l, l+32, ... (V per lane, E <= 32 V)
+// as sortable keys, 0 meaning taken / absent / NaN.  A round is a warp-wide max on the keys and a
+// warp-wide min on the indices that hold it (redux.sync); only the winning lane updates its best.
+template <int V>
+__device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    const unsigned full = 0xFFFFFFFFu;
+    uint32_t key[V];
+#pragma unroll
+    for (int u = 0; u < V; ++u) {
+        const int e = u * 32 + lane;
+        const float v = e < E ? work[e] : __int_as_float(0x7fffffff);
+        key[u] = (v == v) ? float_key(v) : 0u;
+    }
+    float myv = 0.f;
+    int myi = 0x7FFFFFFF;
+#pragma unroll 1
+    for (int j = 0; j < K; ++j) {
+        uint32_t bk = 0u;
+        int bu = 0;
+#pragma unroll
+        for (int u = 0; u < V; ++u)
+            if (key[u] > bk) { bk = key[u]; bu = u; }             // ascending u: the lowest index wins ties
+        const uint32_t best = __reduce_max_sync(full, bk);
+        if (best == 0u) break;                                   // fewer than K finite logits
+        const int cand = (bk == best) ? bu * 32 + lane : 0x7FFFFFFF;
+        const int win = (int)__reduce_min_sync(full, (unsigned)cand);
+        if (lane == j) { myv = key_float(best); myi = win; }
+        if (cand == win) {
+#pragma unroll
+            for (int u = 0; u < V; ++u)
+                if (u == bu) key[u] = 0u;
+        }
+    }
+    topk_emit(myv, myi, K, lane, inds, gates);
+}
+
 // Top-k of work[0..E) by one warp, ties to the lower index; the K winners are written in
 // ascending index with gate weights exp(l - max) / sum over the winners (which equals
 // softmax(l)[inds] / sum softmax(l)[inds]: the full-softmax denominator cancels).
-// Every lane caches its best remaining candidate; a round is one warp-wide max on sortable keys
-// and one warp-wide min on the indices that hold it (redux.sync), and only the winning lane
-// rescans its candidates.  `work` is overwritten.
+// Up to 256 candidates are kept in registers; beyond that every lane caches its best remaining
+// candidate in `work` (which is then overwritten) and only the winning lane rescans its entries.
 __device__ __forceinline__ void warp_softmax_topk(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    if (E <= 256) {
+        warp_softmax_topk_reg<8>(work, E, K, lane, inds, gates);
+        return;
+    }
     const unsigned full = 0xFFFFFFFFu;
     float myv = 0.f;
     int myi = 0x7FFFFFFF;
@@ -269,18 +333,7 @@ __device__ __forceinline__ void warp_softmax_topk(float* work, int E, int K, int
         }
         __syncwarp();
     }
-    const float m = __shfl_sync(full, myv, 0);
-    const float ex = (lane < K && myi != 0x7FFFFFFF) ? expf(myv - m) : 0.f;
-    const float sum = warp_sum(ex);
-    int rank = 0;
-    for (int i = 0; i < K; ++i) {
-        const int oi = __shfl_sync(full, myi, i);
-        rank += (oi < myi) ? 1 : 0;
-    }
-    if (lane < K && myi != 0x7FFFFFFF) {
-        inds[rank] = myi;
-        gates[rank] = ex / sum;
-    }
+    topk_emit(myv, myi, K, lane, inds, gates);
 }
 
 template <typename T> __device__ __forceinline__ void store_out(T* y, size_t i, float v);

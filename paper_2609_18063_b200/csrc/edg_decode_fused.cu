@@ -24,6 +24,8 @@
 // Consecutive layer-steps are chained by programmatic dependent launch: the next step's kernel
 // starts early, waits for a flag raised by this step's top-k, and streams its weights while this
 // step is still computing.
+#include <stdio.h>
+#include <stdlib.h>
 #include <cooperative_groups.h>
 
 #include "edg_mma.cuh"
@@ -37,9 +39,63 @@ constexpr int kE16 = kC * kDownSlices;   // CTAs per expert
 constexpr int kFW = 8;            // warps per CTA
 constexpr int kStages = 4;        // gate/up copy stages per CTA
 constexpr int kMaxRank = 64;
-constexpr int kTraceMarks = 16;
+constexpr int kTraceMarks = 24;
 constexpr int kRing = 4;          // chained layer-steps in flight: hand-off slots for routing, logits scratch, counters
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
+
+// ---------------------------------------------------------------- shared-memory carve-up
+// Byte offsets, identical on host and device.  The four gate/up stages (quarters of the K range)
+// come first; the down block
+// later reuses stages 0 and 1 (it is exactly half the size of the gate/up slice), which keeps a
+// CTA under half an SM's shared memory so two CTAs -- of this launch or of the next one -- can
+// share an SM.
+struct FusedSmem {
+    uint32_t stage0, stage_bytes;                      // stage s (a quarter of the K range) at stage0 + s * stage_bytes
+    uint32_t mat_codes, mat_sz;                        // bytes of one (matrix, row tile) run of codes / sz inside a stage
+    uint32_t sz0;                                      // offset of the sz runs inside a stage
+    uint32_t d_codes, d_sz;                            // down block, from stage0
+    uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, flag, total;
+};
+__host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
+    FusedSmem S;
+    const uint32_t rows_gu = I / kE16, rows_d = H / kC, sw = I / kDownSlices, tg = rows_gu / 16;
+    // a stage holds, for gate and up and each of their tg row tiles, H/128 chunks (H/4 codes per row)
+    S.mat_codes = (uint32_t)(H / 128) * 256;
+    S.mat_sz = (uint32_t)((H / 4) / group) * 64;
+    S.sz0 = 2 * tg * S.mat_codes;
+    S.stage_bytes = 2 * tg * (S.mat_codes + S.mat_sz);
+    uint32_t o = 0;
+    S.stage0 = o;     o += kStages * S.stage_bytes;
+    S.d_codes = S.stage0;
+    S.d_sz = S.stage0 + rows_d * sw / 2;               // rows_d * (sw/2 + sw/group*4) == 2 * stage_bytes
+    S.b_gate = o;     o += rows_gu * (uint32_t)rank * 2;      // B_gate[n0 .. n0+rows_gu][rank]
+    S.b_up = o;       o += rows_gu * (uint32_t)rank * 2;
+    S.b_down = o;     o += rows_d * (uint32_t)rank * 2;       // B_down[n0 .. n0+rows_d][rank]
+    S.a_down = o;     o += (uint32_t)rank * rows_gu * 2;      // A_down[rank][my rows of h]
+    o = (o + 15) / 16 * 16;
+    S.bars = o;       o += 8 * (kStages + 5);
+    o = (o + 15) / 16 * 16;
+    S.s_u = o;        o += 2 * kMaxRank * 4;
+    S.s_h = o;        o += sw * 4;                    // the cluster's quarter of h
+    S.s_ud_part = o;  o += kC * kMaxRank * 4;
+    S.s_ud = o;       o += kMaxRank * 4;
+    S.s_gu = o;       o += 2 * rows_gu * 4;
+    S.s_o = o;        o += rows_d * 4;
+    S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
+    S.s_hloc = o;     o += 32 * 4;
+    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the routing, then its K winners
+    S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
+    S.s_table = o;    o += (uint32_t)E * 4;           // this layer's slot table, fetched before the routing is known
+    o = (o + 15) / 16 * 16;
+    S.s_xb = o;       o += (uint32_t)H * 2;           // x as fp16 B-fragment words, k-slot order
+    S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
+    S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the cluster's quarter of h as (hi, lo) B-fragment words
+    S.s_hsum = o;     o += (sw / 32) * 4;
+    S.flag = o;       o += 16;
+    S.total = (o + 15) / 16 * 16;
+    return S;
+}
 
 struct FusedParams {
     const uint8_t* pool;
@@ -51,9 +107,9 @@ struct FusedParams {
     edg_lora lora;
     void* y;                      // [H]
     int32_t* status;
-    int32_t* counters;            // [kC] one per block of output rows, zero between launches
+    int32_t* counters;            // [kRing][kC] one per ring slot and block of output rows, zero between uses
     int32_t* pre_counter;         // rows of the head delivered so far, zero between launches
-    float* partial;               // [K * kDownSlices][H]
+    float* partial;               // [kRing][K * kDownSlices][H]
     float* logits_ws;             // [E] logits of the next step's head, gathered across CTAs
     const void* W_pre;            // [E][H] or null
     int32_t* inds_next;
@@ -63,11 +119,14 @@ struct FusedParams {
     float sigma;
     RecordLayout L;
     unsigned long long* trace;    // optional [grid CTAs][kTraceMarks] globaltimer stamps, or null
-    int32_t* seen;                // [kRing] CTAs that have consumed the routing in each ring slot
+    int32_t* done;                // [kRing] reducers of the step that has read each routing slot and are finished
+    int ring;                     // ring slot of this step's reduce scratch
     int32_t* route_inds;          // [kRing][32] routing handed from one chained step to the next (-1 = not yet written)
     float* route_gates;           // [kRing][32] (negative / NaN = not yet written)
     int flag_in;                  // -1: the routing is already in memory; else the ring slot to take it from
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
+    int gshift;                   // log2(group)
+    FusedSmem S;                  // shared-memory carve-up
 };
 
 // ---------------------------------------------------------------- PTX wrappers
@@ -115,7 +174,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait: gives up after kSpinLimit polls, raises the status word and lets the caller go on
 // (the result is then wrong but flagged, and every barrier is still reached).
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
+__device__ __noinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status) {
     for (uint32_t i = 0; i < kSpinLimit; ++i)
         if (mbar_try_wait(bar, parity)) return;
     atomicExch(status, EDG_E_TIMEOUT);
@@ -173,6 +232,27 @@ __device__ __forceinline__ void trace_mark(const FusedParams& p, int m) {
     }
 }
 
+__device__ __forceinline__ void trace_stamp(const FusedParams& p, int m) {
+    if (p.trace != nullptr) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[(size_t)blockIdx.x * kTraceMarks + m] = t;
+    }
+}
+
+// four consecutive outputs (i a multiple of 4)
+__device__ __forceinline__ void store_y4(void* y, int out_dtype, size_t i, float4 v) {
+    if (out_dtype == EDG_F32) {
+        *reinterpret_cast<float4*>(static_cast<float*>(y) + i) = v;
+    } else if (out_dtype == EDG_F16) {
+        __half2 a = __floats2half2_rn(v.x, v.y), b = __floats2half2_rn(v.z, v.w);
+        *reinterpret_cast<uint2*>(static_cast<__half*>(y) + i) = make_uint2(h2_as_u32(a), h2_as_u32(b));
+    } else {
+        bf16_t* o = static_cast<bf16_t*>(y) + i;
+        store_out<bf16_t>(o, 0, v.x); store_out<bf16_t>(o, 1, v.y); store_out<bf16_t>(o, 2, v.z); store_out<bf16_t>(o, 3, v.w);
+    }
+}
+
 __device__ __forceinline__ void store_y(void* y, int out_dtype, size_t i, float v) {
     if (out_dtype == EDG_F32) store_out<float>(static_cast<float*>(y), i, v);
     else if (out_dtype == EDG_F16) store_out<__half>(static_cast<__half*>(y), i, v);
@@ -192,97 +272,48 @@ __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, i
     return d;
 }
 
-// ---------------------------------------------------------------- shared-memory carve-up
-// Byte offsets, identical on host and device.  The four gate/up stages (quarters of the K range)
-// come first; the down block
-// later reuses stages 0 and 1 (it is exactly half the size of the gate/up slice), which keeps a
-// CTA under half an SM's shared memory so two CTAs -- of this launch or of the next one -- can
-// share an SM.
-struct FusedSmem {
-    uint32_t stage0, stage_bytes;                      // stage s (a quarter of the K range) at stage0 + s * stage_bytes
-    uint32_t mat_codes, mat_sz;                        // bytes of one (matrix, row tile) run of codes / sz inside a stage
-    uint32_t sz0;                                      // offset of the sz runs inside a stage
-    uint32_t d_codes, d_sz;                            // down block, from stage0
-    uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, flag, total;
-};
-__host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
-    FusedSmem S;
-    const uint32_t rows_gu = I / kE16, rows_d = H / kC, sw = I / kDownSlices, tg = rows_gu / 16;
-    // a stage holds, for gate and up and each of their tg row tiles, H/128 chunks (H/4 codes per row)
-    S.mat_codes = (uint32_t)(H / 128) * 256;
-    S.mat_sz = (uint32_t)((H / 4) / group) * 64;
-    S.sz0 = 2 * tg * S.mat_codes;
-    S.stage_bytes = 2 * tg * (S.mat_codes + S.mat_sz);
-    uint32_t o = 0;
-    S.stage0 = o;     o += kStages * S.stage_bytes;
-    S.d_codes = S.stage0;
-    S.d_sz = S.stage0 + rows_d * sw / 2;               // rows_d * (sw/2 + sw/group*4) == 2 * stage_bytes
-    S.b_gate = o;     o += rows_gu * (uint32_t)rank * 2;      // B_gate[n0 .. n0+rows_gu][rank]
-    S.b_up = o;       o += rows_gu * (uint32_t)rank * 2;
-    S.b_down = o;     o += rows_d * (uint32_t)rank * 2;       // B_down[n0 .. n0+rows_d][rank]
-    S.a_down = o;     o += (uint32_t)rank * rows_gu * 2;      // A_down[rank][my rows of h]
-    o = (o + 15) / 16 * 16;
-    S.bars = o;       o += 8 * (kStages + 5);
-    o = (o + 15) / 16 * 16;
-    S.s_u = o;        o += 2 * kMaxRank * 4;
-    S.s_h = o;        o += sw * 4;                    // the cluster's quarter of h
-    S.s_ud_part = o;  o += kC * kMaxRank * 4;
-    S.s_ud = o;       o += kMaxRank * 4;
-    S.s_gu = o;       o += 2 * rows_gu * 4;
-    S.s_o = o;        o += rows_d * 4;
-    S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
-    S.s_hloc = o;     o += 32 * 4;
-    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the routing, then its K winners
-    S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
-    S.s_table = o;    o += (uint32_t)E * 4;           // this layer's slot table, fetched before the routing is known
-    S.flag = o;       o += 16;
-    S.total = (o + 15) / 16 * 16;
-    return S;
-}
-
 enum { BAR_DOWN = kStages, BAR_LORA = kStages + 1, BAR_FREE = kStages + 2, BAR_U = kStages + 3, BAR_H = kStages + 4 };
 
-// ---------------------------------------------------------------- prerouter rows (a1) and top-k (a2)
-// The E rows of the head are dealt round-robin to the CTAs of the grid; a row is split over all
-// threads of its CTA (one 16-byte read each), so it costs one trip to memory.  The warp that
-// delivers the last logits (an atomic counter) gathers all E and does softmax + top-k.
+// ---------------------------------------------------------------- head rows (a1) and top-k (a2)
+// The E rows of the head are dealt round-robin to the first CTAs of the grid; a row is split over
+// all threads of its CTA, so it costs one trip to memory.  The warp that delivers the last logits
+// (an atomic counter) gathers all E and does softmax + top-k.
 
-// Partial dot of one head row with the hidden state over this thread's elements (8 per sweep of
-// kFW*32*8).  `w0` / `x0` are the values of the first sweep when the caller loaded them early.
-__device__ __forceinline__ float pre_row_partial(const FusedParams& p, int e, int tid, bool preloaded, uint4 w0, uint4 x0) {
+// Partial dot of head row e with the hidden state over this thread's elements, any dtype and H.
+__device__ __noinline__ float head_row_partial(const void* W_pre, int pre_dtype, const uint16_t* x, int H, int e, int tid) {
     float acc = 0.f;
-    if (p.pre_dtype == EDG_F16) {
-        const __half* wr = static_cast<const __half*>(p.W_pre) + (size_t)e * p.H;
-        for (int c = tid * 8; c < p.H; c += kFW * 32 * 8) {
-            const bool first = preloaded && c == tid * 8;
-            const uint4 w = first ? w0 : ld_keep16(wr + c);
-            const uint4 x = first ? x0 : ld_keep16(p.x + c);
-            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
-            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
-            const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
-            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
-            acc = fmaf(a.x, bf16_lo(x.x), acc); acc = fmaf(a.y, bf16_hi(x.x), acc);
-            acc = fmaf(b.x, bf16_lo(x.y), acc); acc = fmaf(b.y, bf16_hi(x.y), acc);
-            acc = fmaf(d.x, bf16_lo(x.z), acc); acc = fmaf(d.y, bf16_hi(x.z), acc);
-            acc = fmaf(f.x, bf16_lo(x.w), acc); acc = fmaf(f.y, bf16_hi(x.w), acc);
+    if (pre_dtype == EDG_F16) {
+        const __half* wr = static_cast<const __half*>(W_pre) + (size_t)e * H;
+        for (int c = tid * 8; c < H; c += kFW * 32 * 8) {
+            const uint4 w = ld_keep16(wr + c);
+            const uint4 xv = ld_keep16(x + c);
+            const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+            const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
+            acc = fmaf(a.x, bf16_lo(xv.x), acc); acc = fmaf(a.y, bf16_hi(xv.x), acc);
+            acc = fmaf(b.x, bf16_lo(xv.y), acc); acc = fmaf(b.y, bf16_hi(xv.y), acc);
+            acc = fmaf(d.x, bf16_lo(xv.z), acc); acc = fmaf(d.y, bf16_hi(xv.z), acc);
+            acc = fmaf(f.x, bf16_lo(xv.w), acc); acc = fmaf(f.y, bf16_hi(xv.w), acc);
         }
     } else {
-        const float* wr = static_cast<const float*>(p.W_pre) + (size_t)e * p.H;
-        for (int c = tid * 4; c < p.H; c += kFW * 32 * 4) {
+        const float* wr = static_cast<const float*>(W_pre) + (size_t)e * H;
+        for (int c = tid * 4; c < H; c += kFW * 32 * 4) {
             const uint4 w = ld_keep16(wr + c);
-            const uint2 x = *reinterpret_cast<const uint2*>(p.x + c);
-            acc = fmaf(__uint_as_float(w.x), bf16_lo(x.x), acc); acc = fmaf(__uint_as_float(w.y), bf16_hi(x.x), acc);
-            acc = fmaf(__uint_as_float(w.z), bf16_lo(x.y), acc); acc = fmaf(__uint_as_float(w.w), bf16_hi(x.y), acc);
+            const uint2 xv = *reinterpret_cast<const uint2*>(x + c);
+            acc = fmaf(__uint_as_float(w.x), bf16_lo(xv.x), acc); acc = fmaf(__uint_as_float(w.y), bf16_hi(xv.x), acc);
+            acc = fmaf(__uint_as_float(w.z), bf16_lo(xv.y), acc); acc = fmaf(__uint_as_float(w.w), bf16_hi(xv.y), acc);
         }
     }
     return acc;
 }
 
+__device__ __noinline__ void topk_large(float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    warp_softmax_topk(work, E, K, lane, inds, gates);
+}
+
 // One warp: publish this CTA's logits (summed from the per-warp partials in s_pre), and if they were
-// the last ones of the head, gather all E, do softmax + top-k and raise the routing-ready flag.
-__device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const FusedSmem& S,
-                                                 const float* s_pre, int n_rows, int ncta, int lane) {
+// the last ones of the head, gather all E, do softmax + top-k and hand the routing on.
+__device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const float* s_pre, int n_rows,
+                                                 int ncta, int lane) {
     int mine = 0;
     const int ring = p.flag_out >= 0 ? p.flag_out : 0;
     float* logits_ws = p.logits_ws + (size_t)ring * p.E;
@@ -291,6 +322,7 @@ __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* 
         const int e = blockIdx.x + lane * ncta;
         if (e < p.E) {
             float v = 0.f;
+#pragma unroll
             for (int w = 0; w < kFW; ++w) v += s_pre[lane * kFW + w];
             logits_ws[e] = v;
             mine = 1;
@@ -302,48 +334,53 @@ __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* 
     // the counting atomic releases this warp's logits and acquires everyone else's
     if (lane == 0) last = (atom_add_acq_rel_gpu(pre_counter, n_mine) + n_mine == p.E) ? 1 : 0;
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (last) {
-        float* work = reinterpret_cast<float*>(smem + S.s_topk);
-        for (int i0 = 0; i0 < p.E; i0 += 256) {                 // 8 independent loads per lane and pass
-            float v[8];
+    if (!last) return;
+    if (lane == 0) trace_stamp(p, 16);
+    float* work = reinterpret_cast<float*>(smem + p.S.s_topk);
+#pragma unroll 1
+    for (int i0 = 0; i0 < p.E; i0 += 256) {                     // 8 independent loads per lane and pass
+        float v[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u * 32 + lane;
-                v[u] = i < p.E ? __ldcg(&logits_ws[i]) : 0.f;
-            }
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * 32 + lane;
+            v[u] = i < p.E ? __ldcg(&logits_ws[i]) : 0.f;
+        }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u * 32 + lane;
-                if (i < p.E) {
-                    work[i] = v[u];
-                    if (p.logits_next != nullptr) p.logits_next[i] = v[u];
-                }
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + u * 32 + lane;
+            if (i < p.E) {
+                work[i] = v[u];
+                if (p.logits_next != nullptr) p.logits_next[i] = v[u];
             }
         }
-        __syncwarp();
-        int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_topk) + p.E;      // [K] winners, then [K] gates
-        float* s_g = reinterpret_cast<float*>(s_i + 32);
-        warp_softmax_topk(work, p.E, p.K, lane, s_i, s_g);
-        __syncwarp();
-        if (lane < p.K) {
-            p.inds_next[lane] = s_i[lane];
-            p.gates_next[lane] = s_g[lane];
-            if (p.flag_out >= 0) {
-                // The chained next step polls exactly these two words per expert; each is valid by itself.
-                // The slot is reused every kRing steps: wait (bounded) until its last reader has
-                // invalidated it, so that a routing still being read is never overwritten.
-                int32_t* ri = &p.route_inds[p.flag_out * 32 + lane];
-                uint32_t it = 0;
-                while (ld_relaxed_gpu(ri) >= 0 && ++it < kSpinLimit) {}
-                if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
-                st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_out * 32 + lane]), __float_as_int(s_g[lane]));
-                st_relaxed_gpu(ri, s_i[lane]);
-            }
+    }
+    __syncwarp();
+    int32_t* s_i = reinterpret_cast<int32_t*>(smem + p.S.s_topk) + p.E;        // [K] winners, then [K] gates
+    float* s_g = reinterpret_cast<float*>(s_i + 32);
+    if (lane == 0) trace_stamp(p, 17);
+    if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
+    else topk_large(work, p.E, p.K, lane, s_i, s_g);
+    __syncwarp();
+    if (lane == 0) trace_stamp(p, 18);
+    if (lane < p.K) {
+        p.inds_next[lane] = s_i[lane];
+        p.gates_next[lane] = s_g[lane];
+        if (p.flag_out >= 0) {
+            // The chained next step polls exactly these two words per expert; each is valid by itself.
+            // The slot is reused every kRing steps: wait (bounded) until the step that read it last has
+            // handed it back, so that a routing still being read is never overwritten.
+            int32_t* ri = &p.route_inds[p.flag_out * 32 + lane];
+            uint32_t it = 0;
+            while (ld_relaxed_gpu(ri) >= 0 && ++it < kSpinLimit) {}
+            if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
+            asm volatile("fence.acq_rel.gpu;" ::: "memory");    // carries "that step is over" on to our reader
+            st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_out * 32 + lane]), __float_as_int(s_g[lane]));
+            st_relaxed_gpu(ri, s_i[lane]);
         }
-        if (lane == 0) {
-            *pre_counter = 0;
-            if (p.trace != nullptr) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.trace[(size_t)blockIdx.x * kTraceMarks + 15] = t; }
-        }
+    }
+    if (lane == 0) {
+        *pre_counter = 0;
+        trace_stamp(p, 15);
     }
 }
 
@@ -351,43 +388,15 @@ __device__ __forceinline__ void prerouter_finish(const FusedParams& p, uint8_t* 
 // NCW = H / 256 = chunks (of 32 codes) per warp in gate/up; DCH = I / 128 = chunks of a down row-slice;
 // TG = I / 256 = row tiles per matrix and CTA in gate/up; TD = H / 512 = row tiles per warp in down;
 // CPB = chunks per scaled block (2 for groups of 64 or 128 codes, 1 for groups of 32).
-
-// This CTA's share of the 2r rows of A_gate / A_up: per-warp partial dot products into s_red.
-// All threads take part, each covering 8 elements of a row per sweep; the loads of up to 8 rows
-// are in flight together, so the whole share costs one round trip to memory.
-#define LORA_A_ROWS(AD)                                                                                          \
-    do {                                                                                                          \
-        const int per_ = (2 * r + kC - 1) / kC;                                                                   \
-        for (int q0 = 0; q0 < per_; q0 += 8) {                                                                    \
-            float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};                                                \
-            for (int cc = tid * 8; cc < p.H; cc += kFW * 32 * 8) {                                                \
-                const uint4 ux = ld_keep16(p.x + cc);                                                             \
-                uint4 ua[8];                                                                                      \
-                _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                   \
-                    const int q = min(crank * per_ + min(q0 + u, per_ - 1), 2 * r - 1);                           \
-                    const uint16_t* A = reinterpret_cast<const uint16_t*>((q / r) ? p.lora.A_up : p.lora.A_gate) + \
-                                        ((size_t)(AD) * r + q % r) * p.H;                                         \
-                    ua[u] = ld_keep16(A + cc);                                                                    \
-                }                                                                                                 \
-                _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                   \
-                    v[u] = fmaf(bf16_lo(ua[u].x), bf16_lo(ux.x), v[u]); v[u] = fmaf(bf16_hi(ua[u].x), bf16_hi(ux.x), v[u]); \
-                    v[u] = fmaf(bf16_lo(ua[u].y), bf16_lo(ux.y), v[u]); v[u] = fmaf(bf16_hi(ua[u].y), bf16_hi(ux.y), v[u]); \
-                    v[u] = fmaf(bf16_lo(ua[u].z), bf16_lo(ux.z), v[u]); v[u] = fmaf(bf16_hi(ua[u].z), bf16_hi(ux.z), v[u]); \
-                    v[u] = fmaf(bf16_lo(ua[u].w), bf16_lo(ux.w), v[u]); v[u] = fmaf(bf16_hi(ua[u].w), bf16_hi(ux.w), v[u]); \
-                }                                                                                                 \
-            }                                                                                                     \
-            _Pragma("unroll") for (int u = 0; u < 8; ++u) {                                                       \
-                const float t_ = warp_sum(v[u]);                                                                  \
-                if (lane == 0 && q0 + u < per_) s_red[(q0 + u) * kFW + warp] = t_;                                \
-            }                                                                                                     \
-        }                                                                                                         \
-    } while (0)
+// The kernel is straight-line code that every CTA runs once, so its size is kept small on purpose
+// (loops over K blocks are not unrolled, operands come from shared memory): instruction fetches
+// compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
 constexpr int kMaxPre = 8;        // head rows per head CTA
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
-__global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p) {
+__global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_constant__ FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int b16 = blockIdx.x % kE16;             // CTA of the expert
     const int k = blockIdx.x / kE16;               // position of the expert in the routing
@@ -396,7 +405,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     const int g8 = lane >> 2, t4 = lane & 3;       // fragment coordinates: row slot, quad lane
 
-    const FusedSmem S = fused_smem(p.H, p.I, p.E, p.group, p.rank);
+    const FusedSmem& S = p.S;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars);
     float* s_u = reinterpret_cast<float*>(smem + S.s_u);            // [2][kMaxRank]
     float* s_h = reinterpret_cast<float*>(smem + S.s_h);            // [I/4]
@@ -408,20 +417,43 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
     float* s_hloc = reinterpret_cast<float*>(smem + S.s_hloc);      // [rows_gu]
     float* s_part = reinterpret_cast<float*>(smem + S.s_part);      // [kFW][2 * rows_gu]
     int* s_flag = reinterpret_cast<int*>(smem + S.flag);
-    int* s_table = reinterpret_cast<int*>(smem + S.s_table);       // [E]
+    int* s_table = reinterpret_cast<int*>(smem + S.s_table);        // [E]
+    uint4* s_xb = reinterpret_cast<uint4*>(smem + S.s_xb);          // [H/8]  x as B-fragment words
+    float* s_xsum = reinterpret_cast<float*>(smem + S.s_xsum);      // [H/(32 CPB)] block sums of x
+    uint4* s_hb = reinterpret_cast<uint4*>(smem + S.s_hb);          // [DCH][2][4] h (hi, lo) as B-fragment words
+    float* s_hsum = reinterpret_cast<float*>(smem + S.s_hsum);      // [DCH/CPB]
 
-    const int rows_gu = p.I / kE16, rows_d = p.H / kC, sw = p.I / kDownSlices;
-    constexpr int tg = TG;                         // row tiles per matrix in this CTA
+    constexpr int rows_gu = 16 * TG, rows_d = 128 * TD, sw = 32 * DCH;
     const int n0_gu = b16 * rows_gu;               // first gate/up row of this CTA (= c * sw + crank * rows_gu)
     const int n0_d = crank * rows_d;               // first down row of this CTA
     const int r = p.rank;
+    // reduce scratch of this step's ring slot: a chained step never waits for the previous kernel to
+    // end, so consecutive steps must not share it
+    float* partial = p.partial + (size_t)p.ring * p.K * kDownSlices * p.H;
+    int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
 
-    // ---- barriers first: peers will count bytes on BAR_U / BAR_H of this CTA, so they must exist
-    //      (and every CTA of the cluster must be running) before anyone sends.  The cluster
-    //      handshake completes while the routing loads below are in flight, and it happens before
-    //      any bulk copy is issued: a cluster-scope fence waits for every copy in flight into the
-    //      SM, so none is used after this point.
+    // ---- a1 for the next step, first of all: the loads of the head rows depend on nothing but x,
+    //      and the routing they lead to is what the next layer-step waits for.  Only the first CTAs
+    //      of the grid evaluate the head: they are dispatched first.  A row is split over all
+    //      threads of its CTA (8 elements each).
+    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
+    const bool head_cta = (int)blockIdx.x < n_head_ctas;
+    const int n_pre = head_cta ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
+    const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= kFW * 32 * 8;
+    const bool pre_lane = tid * 8 < p.H;
+    uint4 lw[kMaxPre], lx = make_uint4(0, 0, 0, 0);
+    if (pre_fast) {
+        if (pre_lane) lx = ld_keep16(p.x + tid * 8);
+#pragma unroll
+        for (int ri = 0; ri < kMaxPre; ++ri) {
+            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * n_head_ctas, p.E - 1);
+            lw[ri] = pre_lane ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8) : make_uint4(0, 0, 0, 0);
+        }
+    }
+
+    // ---- thread 0: the barriers (peers will count bytes on BAR_U / BAR_H of this CTA, so they must
+    //      exist, and every CTA of the cluster must be running, before anyone sends)
     if (tid == 0) {
         for (int s = 0; s <= BAR_LORA; ++s) mbar_init(&bars[s], 1);
         mbar_init(&bars[BAR_FREE], kFW / 2);
@@ -433,198 +465,196 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
     }
-    __syncthreads();
+    // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed just
+    // before the copies are issued: a cluster-scope barrier waits for every bulk copy in flight
+    // into the SM, those of a neighbouring CTA included, and that wait is hidden behind the loads
+    // below.
     cluster_arrive();
-    // The next layer-step may start now: its head needs nothing from this one, and everything it
-    // shares with this step is either in its own ring slot or touched only after it has waited for
-    // this kernel to end.
-    pdl_launch_dependents();
 
-    // ---- loads that do not depend on the routing.  The hidden state as the MMA's B operand: the
-    //      warp owns NCW chunks of 32 activations; the lanes of quad 0 hold them (column 0 of the
-    //      8-column tile), every other lane holds zeros.  xsum[j] = sum of the activations of
-    //      64-code block j (for the zero points).
-    uint32_t xb[NCW][4];
-    float xsum[NCW / CPB];
-    {
-        float part[NCW / CPB];
-#pragma unroll
-        for (int j = 0; j < NCW / CPB; ++j) part[j] = 0.f;
-#pragma unroll
-        for (int i = 0; i < NCW; ++i) {
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (g8 == 0) v = *reinterpret_cast<const uint4*>(p.x + (warp * NCW + i) * 32 + t4 * 8);
-            const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
-                                bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
-            const uint4 q = permute8(f);
-            xb[i][0] = q.x; xb[i][1] = q.y; xb[i][2] = q.z; xb[i][3] = q.w;
-            // fp16 is exact for bf16 inputs in the normal range; sum what the MMA will see
-            float sum = 0.f;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
-            part[i / CPB] += sum;
-        }
-#pragma unroll
-        for (int j = 0; j < NCW / CPB; ++j) {
-            float v = part[j];
-            v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-            v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-            xsum[j] = __shfl_sync(0xFFFFFFFFu, v, 0);
-        }
-    }
-
-    // ---- the slot table of this layer does not depend on the routing either: one coalesced read
-    //      now saves a dependent trip to memory once the routing is known
+    // ---- everyone: the slot table of this layer (one coalesced read now saves a dependent trip to
+    //      memory once the routing is known) and the hidden state as the MMA's B operand, kept in
+    //      shared memory.  Thread t converts activations 8t .. 8t+7 (word t%4 of chunk t/4) into
+    //      the k-slot order of the fragments; s_xsum[j] = sum of the activations of scaled block j
+    //      (for the zero points).
     if (p.table != nullptr)
         for (int i = tid; i < p.E; i += kFW * 32) s_table[i] = __ldcg(&p.table[i]);
-
-    // ---- a1 for the next step.  Only the first CTAs of the grid evaluate the head: they are
-    //      dispatched first, so the routing of the next step is ready a few microseconds after this
-    //      kernel starts, whatever the rest of the grid is still waiting for.  A row is split over
-    //      all threads of its CTA (8 elements each); the loads depend on nothing but x and go out
-    //      first of all.
-    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
-    const int n_pre = ((int)blockIdx.x < n_head_ctas) ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
-    const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H == kFW * 32 * 8;
-    uint4 lw[kMaxPre], lx = make_uint4(0, 0, 0, 0);
-    if (pre_fast) {
-        lx = ld_keep16(p.x + tid * 8);
+    {
+        float sum = 0.f;
+        if (pre_lane) {
+            const uint4 v = *reinterpret_cast<const uint4*>(p.x + tid * 8);
+            const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
+                                bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
+            s_xb[tid] = permute8(f);
+            // fp16 is exact for bf16 inputs in the normal range; sum what the MMA will see
 #pragma unroll
-        for (int ri = 0; ri < kMaxPre; ++ri) {
-            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * n_head_ctas, p.E - 1);
-            lw[ri] = ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8);
+            for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
         }
+        sum = group_sum<4 * CPB>(sum);
+        if (pre_lane && (tid % (4 * CPB)) == 0) s_xsum[tid / (4 * CPB)] = sum;
     }
 
-    // ---- everything that needs only x is finished before the routing is even looked at: the head
-    //      rows' partial sums, and the adapter projections when the layer has one shared adapter
+    // ---- the head rows' partial sums, published at once: the routing of the next step is under way
+    //      before this step's own routing is even looked at (one warp finishes the head while
+    //      thread 0 waits for the routing)
     if (n_pre > 0) {
+        if (pre_fast) {
 #pragma unroll
-        for (int ri = 0; ri < kMaxPre; ++ri) {
-            if (ri < n_pre) {
-                const int e = (int)blockIdx.x + ri * n_head_ctas;
-                float v = pre_row_partial(p, e, tid, pre_fast, lw[ri], lx);
+            for (int ri = 0; ri < kMaxPre; ++ri) {
+                const uint4 w = lw[ri];
+                const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+                const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
+                float v = a.x * bf16_lo(lx.x);
+                v = fmaf(a.y, bf16_hi(lx.x), v);
+                v = fmaf(b.x, bf16_lo(lx.y), v); v = fmaf(b.y, bf16_hi(lx.y), v);
+                v = fmaf(d.x, bf16_lo(lx.z), v); v = fmaf(d.y, bf16_hi(lx.z), v);
+                v = fmaf(f.x, bf16_lo(lx.w), v); v = fmaf(f.y, bf16_hi(lx.w), v);
+                v = warp_sum(v);
+                if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
+            }
+        } else {
+#pragma unroll 1
+            for (int ri = 0; ri < n_pre; ++ri) {
+                float v = head_row_partial(p.W_pre, p.pre_dtype, p.x, p.H, (int)blockIdx.x + ri * n_head_ctas, tid);
                 v = warp_sum(v);
                 if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
             }
         }
-    }
-    if (n_pre > 0) {
-        __syncthreads();                  // the head CTAs publish at once: the routing of the next step is under way
+        trace_mark(p, 12);
+        __syncthreads();
         if (warp == kFW - 1) {
-            prerouter_finish(p, smem, S, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane);
-            if (lane == 0 && p.trace != nullptr) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.trace[(size_t)blockIdx.x * kTraceMarks + 13] = t; }
+            prerouter_finish(p, smem, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane);
+            if (lane == 0) trace_stamp(p, 13);
         }
     }
-    const bool lora_early = r > 0 && p.n_adapters == 1;
-    if (lora_early) LORA_A_ROWS(0);
-    trace_mark(p, 11);
 
-    // ---- the routing may still be on its way: the previous layer-step raises a flag when its top-k
-    //      is written, long before that kernel ends (bounded wait; on a time-out fall back to
-    //      waiting for the whole previous kernel, which is always sufficient)
-    int slot;
-    float gate_k;
-    if (p.flag_in >= 0) {
-        // chained: thread 0 polls this expert's own entry (index and gate arrive independently and
-        // are each valid by themselves), everyone else waits at the barrier
-        if (tid == 0) {
+    // ---- thread 0: the routing.  A chained step takes it from the hand-off ring, where the previous
+    //      layer-step puts its top-k long before that kernel ends (bounded wait; on a time-out fall
+    //      back to waiting for the whole previous kernel, which is always sufficient).
+    if (tid == 0) {
+        // The next layer-step may start once every CTA of this one has said so.  The CTAs that
+        // evaluate the head say so only after their own routing has arrived, i.e. after the head
+        // of the step before this one has been finished: a step therefore never starts before the
+        // head two steps back is complete, which keeps the ring slots of the head scratch apart.
+        // Everything else two steps share is in a ring slot of its own, guarded by the hand-off.
+        if (!head_cta || p.flag_in < 0) pdl_launch_dependents();
+        int vi, vg;
+        if (p.flag_in >= 0) {
+            // this expert's own entry: index and gate arrive independently, each valid by itself
             const int32_t* ri = &p.route_inds[p.flag_in * 32 + k];
             const int32_t* rg = reinterpret_cast<const int32_t*>(&p.route_gates[p.flag_in * 32 + k]);
-            int vi = -1, vg = -1;
+            vi = -1; vg = -1;
             uint32_t it = 0;
             do { vi = ld_relaxed_gpu(ri); vg = ld_relaxed_gpu(rg); } while ((vi < 0 || vg < 0) && ++it < kSpinLimit);
-            if (vi < 0 || vg < 0) {          // timed out: the whole previous kernel is always enough
+            if (vi < 0 || vg < 0) {
                 atomicExch(p.status, EDG_E_TIMEOUT);
                 pdl_wait_prior_grid();
                 vi = __ldcg(&p.slots[k]);
                 vg = __float_as_int(__ldcg(&p.gates[k]));
             }
-            s_flag[1] = vi; s_flag[2] = vg;
+            trace_mark(p, 19);
+            // everything the producer of this routing had observed (the reduce scratch of this ring
+            // slot being free again, above all) is ordered before what this CTA does next
+            asm volatile("fence.acq_rel.gpu;" ::: "memory");
+            if (head_cta) pdl_launch_dependents();
+        } else {
+            vi = __ldcg(&p.slots[k]);
+            vg = __float_as_int(__ldcg(&p.gates[k]));
         }
-        __syncthreads();
-        slot = s_flag[1];
-        gate_k = __int_as_float(s_flag[2]);
-    } else {
-        slot = __ldcg(&p.slots[k]);
-        gate_k = __ldcg(&p.gates[k]);
-        __syncthreads();                  // s_table and s_red complete (the chained path passed a barrier above)
+        s_flag[1] = vi; s_flag[2] = vg;
+        trace_mark(p, 14);
     }
-    trace_mark(p, 14);
+    __syncthreads();                      // routing, slot table and x fragments are in shared memory
+    trace_mark(p, 20);
 
     // ---- a3: take.  The decision is the same in every CTA of the expert.
+    int slot = s_flag[1];
+    const float gate_k = __int_as_float(s_flag[2]);
     const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
-    if (p.table != nullptr) {
-        slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
-    }
+    if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
     int ad = 0;
     if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
     const bool valid = slot >= 0 && slot < p.n_slots && ad >= 0;
     trace_mark(p, 10);
-    if (p.flag_in >= 0) {
-        // the CTA that is last to have read the routing frees its ring slot
-        if (tid == 0) s_flag[3] = (atomicAdd(&p.seen[p.flag_in], 1) == (int)gridDim.x - 1) ? 1 : 0;
-        __syncthreads();
-        if (s_flag[3]) {                  // every CTA has read its entry: invalidate them for the producer after next
-            if (tid < 32) {
-                st_relaxed_gpu(&p.route_inds[p.flag_in * 32 + tid], -1);
-                st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_in * 32 + tid]), -1);
-            }
-            if (tid == 0) p.seen[p.flag_in] = 0;
-            __threadfence();
-        }
-        __syncthreads();
-    }
-    cluster_wait();                       // nothing is in flight yet: this returns at once
+    cluster_wait();
+    trace_mark(p, 21);
     const int cps = p.H / 128;            // chunks of a row per stage
-    const int gpst = (p.H / 4) / p.group; // groups of a row per stage
-    const int gps = sw / p.group;         // groups of a down row-slice
+    const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
+    const int gps = sw >> p.gshift;       // groups of a down row-slice
+    const uint8_t* rec = p.pool + (size_t)(valid ? slot : 0) * p.L.bytes;
 
     if (valid) {
-        const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
         // ---- issue the copies of this CTA's gate/up slice (stage = a quarter of the K range, one run
         //      per matrix and row tile) and of its adapter rows, one warp per barrier
         if (warp < kStages) {
-            // lane 0 arms the barrier, then lanes 0 .. 4*tg-1 issue one run each (codes or sz of a (matrix, tile))
+            // lane 0 arms the barrier, then lanes 0 .. 4*TG-1 issue one run each (codes or sz of a (matrix, tile))
             const int s = warp;
             uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
             if (lane == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
             __syncwarp();
-            if (lane < 4 * tg) {
+            if (lane < 4 * TG) {
                 const uint64_t pol = policy_evict_first();   // weights stream through L2 once
-                const int mt = lane >> 1, is_sz = lane & 1, m = mt / tg, ti = mt % tg;
+                const int mt = lane >> 1, is_sz = lane & 1, m = mt / TG, ti = mt % TG;
                 const int n = n0_gu + 16 * ti;
                 if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
                                           S.mat_codes, &bars[s], pol);
                 else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
                                    S.mat_sz, &bars[s], pol);
             }
-        }
-        if (lane == 0) {
-            if (warp == kStages && r > 0) {
-                // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
-                const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
-                mbar_expect_tx(&bars[BAR_LORA], 2 * bgu + bd + r * ad_row);
-                const size_t bo = ((size_t)ad * p.I + n0_gu) * r * 2;
-                bulk_g2s(smem + S.b_gate, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA]);
-                bulk_g2s(smem + S.b_up, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA]);
-                bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd,
+        } else if (warp == kStages && lane == 0 && r > 0) {
+            // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
+            const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
+            mbar_expect_tx(&bars[BAR_LORA], 2 * bgu + bd + r * ad_row);
+            const size_t bo = ((size_t)ad * p.I + n0_gu) * r * 2;
+            bulk_g2s(smem + S.b_gate, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA]);
+            bulk_g2s(smem + S.b_up, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA]);
+            bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd,
+                     &bars[BAR_LORA]);
+            for (int j = 0; j < r; ++j)
+                bulk_g2s(smem + S.a_down + j * ad_row,
+                         static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0_gu) * 2, ad_row,
                          &bars[BAR_LORA]);
-                for (int j = 0; j < r; ++j)
-                    bulk_g2s(smem + S.a_down + j * ad_row,
-                             static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0_gu) * 2, ad_row,
-                             &bars[BAR_LORA]);
-            }
         }
         trace_mark(p, 1);
     }
-    if (valid) {
-        const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
 
+    if (valid) {
+        // ---- with this CTA's weights on their way: its share of the 2r rows of A_gate / A_up, per-warp partial dot products
+        //      into s_red.  All threads take part, each covering 8 elements of a row per sweep; the
+        //      loads of up to 8 rows are in flight together, so the share costs one trip to memory.
         const int per = (2 * r + kC - 1) / kC;
-        if (r > 0 && !lora_early) {
-            LORA_A_ROWS(ad);
+        if (r > 0) {
+            const int adA = p.n_adapters == 1 ? 0 : ad;
+#pragma unroll 1
+            for (int q0 = 0; q0 < per; q0 += 8) {
+                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+                for (int cc = tid * 8; cc < p.H; cc += kFW * 32 * 8) {
+                    const uint4 ux = ld_keep16(p.x + cc);
+                    uint4 ua[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int q = min(crank * per + min(q0 + u, per - 1), 2 * r - 1);
+                        const int up = q >= r ? 1 : 0;
+                        const uint16_t* A = reinterpret_cast<const uint16_t*>(up ? p.lora.A_up : p.lora.A_gate) +
+                                            ((size_t)adA * r + (q - up * r)) * p.H;
+                        ua[u] = ld_keep16(A + cc);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v[u] = fmaf(bf16_lo(ua[u].x), bf16_lo(ux.x), v[u]); v[u] = fmaf(bf16_hi(ua[u].x), bf16_hi(ux.x), v[u]);
+                        v[u] = fmaf(bf16_lo(ua[u].y), bf16_lo(ux.y), v[u]); v[u] = fmaf(bf16_hi(ua[u].y), bf16_hi(ux.y), v[u]);
+                        v[u] = fmaf(bf16_lo(ua[u].z), bf16_lo(ux.z), v[u]); v[u] = fmaf(bf16_hi(ua[u].z), bf16_hi(ux.z), v[u]);
+                        v[u] = fmaf(bf16_lo(ua[u].w), bf16_lo(ux.w), v[u]); v[u] = fmaf(bf16_hi(ua[u].w), bf16_hi(ux.w), v[u]);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const float t_ = warp_sum(v[u]);
+                    if (lane == 0 && q0 + u < per) s_red[(q0 + u) * kFW + warp] = t_;
+                }
+            }
         }
+        trace_mark(p, 11);
         __syncthreads();                  // s_red complete
         // every CTA of the cluster gets this CTA's adapter projections, counted on its BAR_U
         for (int i = tid; i < per * kC; i += kFW * 32) {
@@ -632,16 +662,19 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
             if (q < 2 * r) {
                 float v = 0.f;
                 for (int w = 0; w < kFW; ++w) v += s_red[qi * kFW + w];
-                st_async_f32(map_to_cta(&s_u[(q / r) * kMaxRank + (q % r)], dst), v, map_to_cta(&bars[BAR_U], dst));
+                const int up = q >= r ? 1 : 0;
+                st_async_f32(map_to_cta(&s_u[up * kMaxRank + (q - up * r)], dst), v, map_to_cta(&bars[BAR_U], dst));
             }
         }
         trace_mark(p, 2);
 
         // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside stage
         //      w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile, chunk) are 256
-        //      contiguous bytes of shared memory, lane (g, t) reading word t of rows g and g+8.
-        //      Partial sums of a 64-code block are exact integer-code dot products in fp32;
-        //      scale and zero point are applied per block: acc += s * (c - z * sum(x)).
+        //      contiguous bytes of shared memory, lane (g, t) reading word t of rows g and g+8.  The
+        //      activations are column 0 of the 8-column B tile: the lanes of quad 0 read their words
+        //      from s_xb, every other lane holds zeros.  Partial sums of a scaled block are exact
+        //      integer-code dot products in fp32; scale and zero point are applied per block:
+        //      acc += s * (c - z * sum(x)).
         {
             const int s = warp / 2;
             mbar_wait(&bars[s], 0, p.status);
@@ -652,31 +685,36 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
             float acc_lo[NT], acc_hi[NT];                            // rows g and g+8, column 0
 #pragma unroll
             for (int mt = 0; mt < NT; ++mt) { acc_lo[mt] = 0.f; acc_hi[mt] = 0.f; }
-#pragma unroll
+            const uint8_t* cbase = st + ch0 * 256 + g8 * 16 + t4 * 4;
+            const uint4* xbp = s_xb + (warp * NCW) * 4 + t4;
+#pragma unroll 1
             for (int ib = 0; ib < NCW / CPB; ++ib) {                 // scaled blocks of this warp's K range
-                const int gi = ((ch0 + ib * CPB) * 32) / p.group;
                 float cfr[NT][4];
 #pragma unroll
                 for (int u = 0; u < CPB; ++u) {
                     const int i = ib * CPB + u;
+                    uint4 xb = make_uint4(0, 0, 0, 0);
+                    if (g8 == 0) xb = xbp[i * 4];
 #pragma unroll
                     for (int mt = 0; mt < NT; ++mt) {
-                        const uint8_t* cw = st + mt * S.mat_codes + (ch0 + i) * 256 + g8 * 16 + t4 * 4;
+                        const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
                         uint32_t alo[4], ahi[4];
                         dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
                         dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                        if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
-                        else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb[i][0], xb[i][1]);
-                        mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb[i][2], xb[i][3]);
+                        if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                        else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                        mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
                     }
                 }
+                const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
+                const float xs = s_xsum[(warp * NCW) / CPB + ib];
 #pragma unroll
                 for (int mt = 0; mt < NT; ++mt) {
                     const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
                     const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
                     const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                    acc_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xsum[ib], cfr[mt][0]), acc_lo[mt]);
-                    acc_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xsum[ib], cfr[mt][2]), acc_hi[mt]);
+                    acc_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), acc_lo[mt]);
+                    acc_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), acc_hi[mt]);
                 }
             }
             if (t4 == 0) {
@@ -726,7 +764,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
         __syncthreads();
         // all-gather h inside the cluster: this CTA's rows_gu values go to every CTA, 16 bytes at a time
         {
-            const int vecs = rows_gu / 4;
+            constexpr int vecs = rows_gu / 4;
             for (int i = tid; i < vecs * kC; i += kFW * 32) {
                 const int v = i % vecs, dst = i / vecs;
                 st_async_f32x4(map_to_cta(&s_h[crank * rows_gu + 4 * v], dst), *reinterpret_cast<const float4*>(&s_hloc[4 * v]),
@@ -748,75 +786,63 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
 
         // ---- down on the tensor cores: partial over this quarter of the columns, for this CTA's H/4
         //      output rows.  h is fp32: column 0 of the B tile carries its fp16 value, column 1 the
-        //      fp16 residual, and the two result columns are added.
+        //      fp16 residual (lanes of quads 0 and 1 read their words from s_hb), and the two result
+        //      columns are added.
         if (tid < r) {
             float v = 0.f;
             for (int cc = 0; cc < kC; ++cc) v += s_ud_part[cc * kMaxRank + tid];
             s_ud[tid] = v;
         }
-        uint32_t hb[DCH][4];
-        float hsum[DCH / CPB];
-        {
-            float part[DCH / CPB];
-#pragma unroll
-            for (int j = 0; j < DCH / CPB; ++j) part[j] = 0.f;
-#pragma unroll
-            for (int i = 0; i < DCH; ++i) {
-                float f[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                if (g8 < 2) {
-                    const float4 a = *reinterpret_cast<const float4*>(s_h + i * 32 + t4 * 8);
-                    const float4 b = *reinterpret_cast<const float4*>(s_h + i * 32 + t4 * 8 + 4);
-                    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
-                }
-                const uint4 q = g8 == 0 ? permute8(f) : permute8_lo(f);       // lanes g >= 2 hold zeros either way
-                hb[i][0] = q.x; hb[i][1] = q.y; hb[i][2] = q.z; hb[i][3] = q.w;
-                float sum = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) sum += f[e];             // hi + lo == h up to 2^-22: sum h itself
-                part[i / CPB] += g8 == 0 ? sum : 0.f;
-            }
-#pragma unroll
-            for (int j = 0; j < DCH / CPB; ++j) {
-                float v = part[j];
-                v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
-                v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
-                hsum[j] = __shfl_sync(0xFFFFFFFFu, v, 0);
-            }
+        if (tid < DCH * 8) {
+            const int i = tid >> 3, lo = (tid >> 2) & 1, q = tid & 3;
+            const float4 a = *reinterpret_cast<const float4*>(s_h + i * 32 + q * 8);
+            const float4 b = *reinterpret_cast<const float4*>(s_h + i * 32 + q * 8 + 4);
+            const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            s_hb[tid] = lo ? permute8_lo(f) : permute8(f);
+        } else if (tid >= 64 && tid < 64 + DCH / CPB) {
+            const int j = tid - 64;
+            float v = 0.f;
+            for (int e = 0; e < 32 * CPB; ++e) v += s_h[j * 32 * CPB + e];   // hi + lo == h up to 2^-22: sum h itself
+            s_hsum[j] = v;
         }
+        __syncthreads();
         mbar_wait(&bars[BAR_DOWN], 0, p.status);
         {
-            const uint8_t* dcodes = smem + S.d_codes;
+            const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
             const uint8_t* dsz = smem + S.d_sz;
             float acc_lo[TD], acc_hi[TD];                            // TD independent row tiles per warp: interleaved
 #pragma unroll
             for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
-#pragma unroll
+#pragma unroll 1
             for (int ib = 0; ib < DCH / CPB; ++ib) {
-                const int gi = (ib * CPB * 32) / p.group;
                 float cfr[TD][4];
 #pragma unroll
                 for (int u = 0; u < CPB; ++u) {
                     const int i = ib * CPB + u;
+                    uint4 hb = make_uint4(0, 0, 0, 0);
+                    if (g8 < 2) hb = s_hb[(i * 2 + g8) * 4 + t4];
 #pragma unroll
                     for (int tt = 0; tt < TD; ++tt) {
                         const int ti = warp + kFW * tt;
-                        const uint8_t* cw = dcodes + (ti * DCH + i) * 256 + g8 * 16 + t4 * 4;
+                        const uint8_t* cw = dbase + (ti * DCH + i) * 256;
                         uint32_t alo[4], ahi[4];
                         dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
                         dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                        if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
-                        else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb[i][0], hb[i][1]);
-                        mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb[i][2], hb[i][3]);
+                        if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                        else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                        mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
                     }
                 }
+                const int gi = (ib * CPB * 32) >> p.gshift;
+                const float hs = s_hsum[ib];
 #pragma unroll
                 for (int tt = 0; tt < TD; ++tt) {
                     const int ti = warp + kFW * tt;
                     const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
                     const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
                     const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                    acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hsum[ib], cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
-                    acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hsum[ib], cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
+                    acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
+                    acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
                 }
             }
             if (t4 == 0) {
@@ -828,42 +854,59 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(FusedParams p)
                 }
             }
         }
-        __syncthreads();                  // s_o and s_ud complete
-        pdl_wait_prior_grid();            // the reduce scratch belongs to the previous layer-step until it ends
+        __syncthreads();                  // s_o complete
         // LoRA B for down (on this quarter's share of A_down.h) and the gate weight: one thread per output row
         for (int lr = tid; lr < rows_d; lr += kFW * 32) {
             float o = s_o[lr];
             if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
-            p.partial[((size_t)k * kDownSlices + c) * p.H + n0_d + lr] = gate_k * o;
+            partial[((size_t)k * kDownSlices + c) * p.H + n0_d + lr] = gate_k * o;
         }
         trace_mark(p, 8);
     } else {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
-        pdl_wait_prior_grid();
         // a skipped expert contributes nothing
-        for (int i = tid; i < rows_d; i += blockDim.x) p.partial[((size_t)k * kDownSlices + c) * p.H + n0_d + i] = 0.f;
+        for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)k * kDownSlices + c) * p.H + n0_d + i] = 0.f;
     }
 
     // ---- a6: this partial is published; the last arriver for the block of rows sums all 4K partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&p.counters[crank], 1) == p.K * kDownSlices - 1) ? 1 : 0;
+    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == p.K * kDownSlices - 1) ? 1 : 0;
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
         const int np = p.K * kDownSlices;
-        for (int i = tid; i < rows_d / 4; i += blockDim.x) {
+        for (int i = tid; i < rows_d / 4; i += kFW * 32) {
             float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
             for (int kk = 0; kk < np; ++kk) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(&p.partial[(size_t)kk * p.H + n0_d + 4 * i]));
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)kk * p.H + n0_d + 4 * i]));
                 yv.x += t.x; yv.y += t.y; yv.z += t.z; yv.w += t.w;
             }
-            const size_t o = (size_t)n0_d + 4 * i;
-            store_y(p.y, p.out_dtype, o + 0, yv.x); store_y(p.y, p.out_dtype, o + 1, yv.y);
-            store_y(p.y, p.out_dtype, o + 2, yv.z); store_y(p.y, p.out_dtype, o + 3, yv.w);
+            store_y4(p.y, p.out_dtype, (size_t)n0_d + 4 * i, yv);
         }
-        if (tid == 0) p.counters[crank] = 0;
+        if (tid == 0) counters[crank] = 0;
+        if (p.flag_in >= 0) {
+            // The last of the kC reducers hands the routing slot this step has read back to its
+            // producer.  By then every CTA has read its entry and the reduce scratch of this ring
+            // slot is free again; the step that reuses either gets its own routing only after this.
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) s_flag[3] = (atomicAdd(&p.done[p.flag_in], 1) == kC - 1) ? 1 : 0;
+            __syncthreads();
+            if (s_flag[3]) {
+                if (tid == 0) p.done[p.flag_in] = 0;
+                __threadfence();
+                if (tid < 32) {
+                    st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_in * 32 + tid]), -1);
+                    st_relaxed_gpu(&p.route_inds[p.flag_in * 32 + tid], -1);
+                }
+            }
+        }
     }
+    // Kernels of a chain complete in order: one CTA of every grid waits for the grid before it, so
+    // work queued after the last kernel of a chain finds all of them finished.
+    if (p.flag_in >= 0 && blockIdx.x == 0) pdl_wait_prior_grid();
     trace_mark(p, 9);
 }
 
@@ -876,7 +919,7 @@ constexpr size_t kFusedSmemLimit = 112 * 1024;    // two CTAs per SM
 bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
     if ((d.I / kE16) % 16 != 0 || d.I / kE16 > 32) return false;   // whole 16-row tiles per CTA
-    if (d.group > 128) return false;
+    if (d.group > 128 || (d.group & (d.group - 1)) != 0) return false;
     if (d.rank % 8 != 0) return false;            // adapter slices are staged by 16-byte bulk copies
     return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
 }
@@ -891,6 +934,13 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         // two CTAs per SM: more clusters resident at once
         e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
+        if (const char* mb = getenv("EDG_L2_PERSIST_MB")) {
+            size_t want = (size_t)atoi(mb) << 20;
+            cudaError_t e2 = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want);
+            size_t got = 0;
+            cudaDeviceGetLimit(&got, cudaLimitPersistingL2CacheSize);
+            fprintf(stderr, "persisting L2: asked %zu, rc %d, now %zu\n", want, (int)e2, got);
+        }
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
@@ -936,8 +986,12 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.pre_dtype = d->pre_dtype; p.out_dtype = d->out_dtype;
     p.sigma = d->lora_scale;
     p.L = record_layout(d->H, d->I, d->group);
+    p.S = fused_smem(d->H, d->I, d->E, d->group, p.rank);
+    p.gshift = 0;
+    while ((1 << p.gshift) < d->group) ++p.gshift;
     p.trace = g_trace;
-    p.seen = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.ring = flag_in >= 0 ? (flag_in + 1) % kRing : 0;
     p.route_inds = reinterpret_cast<int32_t*>(ws + W.route);
     p.route_gates = reinterpret_cast<float*>(ws + W.route + kRing * 32 * 4);
     p.flag_in = flag_in;
@@ -948,7 +1002,7 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
         EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 64, st));           // head-row counters and reader counts of the ring
         EDG_CUDA_TRY(cudaMemsetAsync(p.route_inds, 0xFF, 2 * kRing * 32 * 4, st));   // -1 / NaN: nothing handed over yet
     }
-    const size_t smem = fused_smem(d->H, d->I, d->E, d->group, p.rank).total;
+    const size_t smem = p.S.total;
     cudaError_t e;
     const bool wide = d->group >= 64;         // scaled blocks of 64 codes (groups of 64 or 128) or of 32
     if (d->H == 2048 && d->I == 512) e = wide ? launch_fused<8, 4, 2, 4, 2>(p, smem, pdl, st) : launch_fused<8, 4, 2, 4, 1>(p, smem, pdl, st);
