@@ -83,8 +83,7 @@ struct WorkspaceLayout {
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
     size_t partial;   // [4][K*kDownSlices][H] float: gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
-    size_t logits;    // [4][E] float               : next-step head logits gathered across CTAs, one per ring slot
-    size_t route;     // 1 KB                       : routing handed between chained steps: [4][32] int32 + [4][32] float
+    size_t logits;    // [4][E] float               : next-step head logits handed to the chained next step, one set per ring slot
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
     size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
@@ -108,8 +107,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
     W.logits = round_up(W.partial + 4 * (size_t)d.K * kDownSlices * d.H * sizeof(float), 256);
-    W.route = round_up(W.logits + 4 * (size_t)d.E * sizeof(float), 256);
-    size_t end = W.route + 1024;
+    size_t end = round_up(W.logits + 4 * (size_t)d.E * sizeof(float), 256);
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;
@@ -267,37 +265,57 @@ __device__ __forceinline__ void topk_emit(float myv, int myi, int K, int lane, i
     }
 }
 
-// Top-k with the candidates in registers: lane l holds entries l, l+32, ... (V per lane, E <= 32 V)
-// as sortable keys, 0 meaning taken / absent / NaN.  A round is a warp-wide max on the keys and a
-// warp-wide min on the indices that hold it (redux.sync); only the winning lane updates its best.
+// Top-k with the candidates in registers: lane l holds entries l, l+32, ... (V = 8 per lane,
+// E <= 256) as sortable keys, 0 meaning absent / NaN.  Every lane first sorts its own candidates
+// (descending key, ascending index among equals) with a fixed network; a round is then one
+// warp-wide max on the lanes' best keys, the owner popping its list.  Only when several lanes hold
+// the same best key does a second reduction (min over their indices) decide.
+__device__ __forceinline__ void topk_cex(uint32_t& ka, int& ia, uint32_t& kb, int& ib) {
+    // (ka, ia) is the earlier position: swap when b must come first
+    const bool sw = kb > ka || (kb == ka && ib < ia);
+    const uint32_t tk = sw ? kb : ka, uk = sw ? ka : kb;
+    const int ti = sw ? ib : ia, ui = sw ? ia : ib;
+    ka = tk; kb = uk; ia = ti; ib = ui;
+}
+
 template <int V>
 __device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    static_assert(V == 8, "the sorting network below is for 8 candidates per lane");
     const unsigned full = 0xFFFFFFFFu;
     uint32_t key[V];
+    int idx[V];
 #pragma unroll
     for (int u = 0; u < V; ++u) {
         const int e = u * 32 + lane;
         const float v = e < E ? work[e] : __int_as_float(0x7fffffff);
         key[u] = (v == v) ? float_key(v) : 0u;
+        idx[u] = e;
     }
+    // 19-comparator network for 8 inputs
+#define EDG_CEX(a, b) topk_cex(key[a], idx[a], key[b], idx[b])
+    EDG_CEX(0, 1); EDG_CEX(2, 3); EDG_CEX(4, 5); EDG_CEX(6, 7);
+    EDG_CEX(0, 2); EDG_CEX(1, 3); EDG_CEX(4, 6); EDG_CEX(5, 7);
+    EDG_CEX(1, 2); EDG_CEX(5, 6); EDG_CEX(0, 4); EDG_CEX(3, 7);
+    EDG_CEX(1, 5); EDG_CEX(2, 6);
+    EDG_CEX(1, 4); EDG_CEX(3, 6);
+    EDG_CEX(2, 4); EDG_CEX(3, 5);
+    EDG_CEX(3, 4);
+#undef EDG_CEX
     float myv = 0.f;
     int myi = 0x7FFFFFFF;
 #pragma unroll 1
     for (int j = 0; j < K; ++j) {
-        uint32_t bk = 0u;
-        int bu = 0;
-#pragma unroll
-        for (int u = 0; u < V; ++u)
-            if (key[u] > bk) { bk = key[u]; bu = u; }             // ascending u: the lowest index wins ties
-        const uint32_t best = __reduce_max_sync(full, bk);
+        const uint32_t best = __reduce_max_sync(full, key[0]);
         if (best == 0u) break;                                   // fewer than K finite logits
-        const int cand = (bk == best) ? bu * 32 + lane : 0x7FFFFFFF;
-        const int win = (int)__reduce_min_sync(full, (unsigned)cand);
+        const unsigned who = __ballot_sync(full, key[0] == best);
+        int win;
+        if ((who & (who - 1)) == 0u) win = __shfl_sync(full, idx[0], __ffs(who) - 1);
+        else win = (int)__reduce_min_sync(full, key[0] == best ? (unsigned)idx[0] : 0x7FFFFFFFu);
         if (lane == j) { myv = key_float(best); myi = win; }
-        if (cand == win) {
+        if (key[0] == best && idx[0] == win) {                   // the owner pops its list
 #pragma unroll
-            for (int u = 0; u < V; ++u)
-                if (u == bu) key[u] = 0u;
+            for (int u = 0; u + 1 < V; ++u) { key[u] = key[u + 1]; idx[u] = idx[u + 1]; }
+            key[V - 1] = 0u;
         }
     }
     topk_emit(myv, myi, K, lane, inds, gates);

@@ -55,7 +55,7 @@ struct FusedSmem {
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, s_route, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
@@ -92,6 +92,7 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
     S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the cluster's quarter of h as (hi, lo) B-fragment words
     S.s_hsum = o;     o += (sw / 32) * 4;
+    S.s_route = o;    o += (uint32_t)E * 4 + 256;     // logits taken from the hand-off ring, then this step's K winners
     S.flag = o;       o += 16;
     S.total = (o + 15) / 16 * 16;
     return S;
@@ -108,9 +109,9 @@ struct FusedParams {
     void* y;                      // [H]
     int32_t* status;
     int32_t* counters;            // [kRing][kC] one per ring slot and block of output rows, zero between uses
-    int32_t* pre_counter;         // rows of the head delivered so far, zero between launches
+    int32_t* pre_counter;         // [kRing] rows of the head delivered so far, back to zero after every head
     float* partial;               // [kRing][K * kDownSlices][H]
-    float* logits_ws;             // [E] logits of the next step's head, gathered across CTAs
+    float* logits_ws;             // [kRing][E] logits of the next step's head; all-ones words = not yet written
     const void* W_pre;            // [E][H] or null
     int32_t* inds_next;
     float* gates_next;
@@ -121,8 +122,7 @@ struct FusedParams {
     unsigned long long* trace;    // optional [grid CTAs][kTraceMarks] globaltimer stamps, or null
     int32_t* done;                // [kRing] reducers of the step that has read each routing slot and are finished
     int ring;                     // ring slot of this step's reduce scratch
-    int32_t* route_inds;          // [kRing][32] routing handed from one chained step to the next (-1 = not yet written)
-    float* route_gates;           // [kRing][32] (negative / NaN = not yet written)
+    int32_t* fin;                 // [kRing] set once the head in that ring slot has been finished (its logits read)
     int flag_in;                  // -1: the routing is already in memory; else the ring slot to take it from
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
     int gshift;                   // log2(group)
@@ -218,6 +218,15 @@ __device__ __forceinline__ int ld_relaxed_gpu(const int32_t* p) {
 __device__ __forceinline__ void st_relaxed_gpu(int32_t* p, int v) {
     asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t ld_relaxed_gpu_u32(const void* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_gpu_u32(void* p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+constexpr uint32_t kNotYet = 0xFFFFFFFFu;      // a logit that has not been written (a NaN no arithmetic produces)
 // programmatic dependent launch: let the next kernel in the stream start / wait for the previous one
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -310,10 +319,14 @@ __device__ __noinline__ void topk_large(float* work, int E, int K, int lane, int
     warp_softmax_topk(work, E, K, lane, inds, gates);
 }
 
-// One warp: publish this CTA's logits (summed from the per-warp partials in s_pre), and if they were
-// the last ones of the head, gather all E, do softmax + top-k and hand the routing on.
+// One warp: publish this CTA's logits (summed from the per-warp partials in s_pre) into the ring slot
+// the next layer-step reads, and if they were the last ones of the head, compute the top-k for the
+// caller's inds_next / gates_next.  A chained next step does not wait for that: it takes the logits
+// from the ring and selects its experts itself.  `state` is this lane's entry of the ring slot as
+// it was when the kernel started: a slot is written again only after the step that read it has
+// ended and has reset it.
 __device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const float* s_pre, int n_rows,
-                                                 int ncta, int lane) {
+                                              int ncta, int lane, uint32_t state) {
     int mine = 0;
     const int ring = p.flag_out >= 0 ? p.flag_out : 0;
     float* logits_ws = p.logits_ws + (size_t)ring * p.E;
@@ -324,7 +337,14 @@ __device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* sme
             float v = 0.f;
 #pragma unroll
             for (int w = 0; w < kFW; ++w) v += s_pre[lane * kFW + w];
-            logits_ws[e] = v;
+            if (p.flag_out >= 0) {
+                uint32_t it = 0;
+                while (state != kNotYet && ++it < kSpinLimit) state = ld_relaxed_gpu_u32(&logits_ws[e]);
+                if (state != kNotYet) atomicExch(p.status, EDG_E_TIMEOUT);
+                // "the step that last read this slot is over" travels on to the reader of this logit
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");
+            }
+            st_relaxed_gpu_u32(&logits_ws[e], __float_as_uint(v));
             mine = 1;
         }
     }
@@ -335,7 +355,10 @@ __device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* sme
     if (lane == 0) last = (atom_add_acq_rel_gpu(pre_counter, n_mine) + n_mine == p.E) ? 1 : 0;
     last = __shfl_sync(0xFFFFFFFFu, last, 0);
     if (!last) return;
-    if (lane == 0) trace_stamp(p, 16);
+    if (lane == 0) {
+        atomicSub(pre_counter, p.E);      // commutes with the arrivals of the head that uses this slot next
+        trace_stamp(p, 16);
+    }
     float* work = reinterpret_cast<float*>(smem + p.S.s_topk);
 #pragma unroll 1
     for (int i0 = 0; i0 < p.E; i0 += 256) {                     // 8 independent loads per lane and pass
@@ -355,33 +378,19 @@ __device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* sme
         }
     }
     __syncwarp();
+    // the logits are in shared memory: the step that has read this ring slot may reset it
+    if (lane == 0 && p.flag_out >= 0) { __threadfence(); st_relaxed_gpu(&p.fin[ring], 1); }
     int32_t* s_i = reinterpret_cast<int32_t*>(smem + p.S.s_topk) + p.E;        // [K] winners, then [K] gates
     float* s_g = reinterpret_cast<float*>(s_i + 32);
     if (lane == 0) trace_stamp(p, 17);
     if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
     else topk_large(work, p.E, p.K, lane, s_i, s_g);
     __syncwarp();
-    if (lane == 0) trace_stamp(p, 18);
     if (lane < p.K) {
         p.inds_next[lane] = s_i[lane];
         p.gates_next[lane] = s_g[lane];
-        if (p.flag_out >= 0) {
-            // The chained next step polls exactly these two words per expert; each is valid by itself.
-            // The slot is reused every kRing steps: wait (bounded) until the step that read it last has
-            // handed it back, so that a routing still being read is never overwritten.
-            int32_t* ri = &p.route_inds[p.flag_out * 32 + lane];
-            uint32_t it = 0;
-            while (ld_relaxed_gpu(ri) >= 0 && ++it < kSpinLimit) {}
-            if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
-            asm volatile("fence.acq_rel.gpu;" ::: "memory");    // carries "that step is over" on to our reader
-            st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_out * 32 + lane]), __float_as_int(s_g[lane]));
-            st_relaxed_gpu(ri, s_i[lane]);
-        }
     }
-    if (lane == 0) {
-        *pre_counter = 0;
-        trace_stamp(p, 15);
-    }
+    if (lane == 0) trace_stamp(p, 15);
 }
 
 // ---------------------------------------------------------------- the fused kernel
@@ -450,6 +459,12 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * n_head_ctas, p.E - 1);
             lw[ri] = pre_lane ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8) : make_uint4(0, 0, 0, 0);
         }
+    }
+
+    uint32_t pre_state = kNotYet;         // this head row's entry of the ring slot, as the kernel finds it
+    if (n_pre > 0 && p.flag_out >= 0 && warp == kFW - 1 && lane < n_pre) {
+        const int e = (int)blockIdx.x + lane * n_head_ctas;
+        if (e < p.E) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + e]);
     }
 
     // ---- thread 0: the barriers (peers will count bytes on BAR_U / BAR_H of this CTA, so they must
@@ -522,45 +537,67 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         trace_mark(p, 12);
         __syncthreads();
         if (warp == kFW - 1) {
-            prerouter_finish(p, smem, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane);
+            prerouter_finish(p, smem, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane, pre_state);
             if (lane == 0) trace_stamp(p, 13);
         }
     }
 
-    // ---- thread 0: the routing.  A chained step takes it from the hand-off ring, where the previous
-    //      layer-step puts its top-k long before that kernel ends (bounded wait; on a time-out fall
-    //      back to waiting for the whole previous kernel, which is always sufficient).
-    if (tid == 0) {
+    // ---- warp 0: the routing.  A chained step reads the logits its predecessor's head has put into
+    //      the hand-off ring (long before that kernel ends) and selects its experts itself -- every
+    //      CTA the same way, which costs less than waiting for one warp to do it for all.  Bounded
+    //      wait; on a time-out fall back to waiting for the whole previous kernel and to the
+    //      routing it has written, which is always sufficient.
+    if (warp == 0) {
         // The next layer-step may start once every CTA of this one has said so.  The CTAs that
         // evaluate the head say so only after their own routing has arrived, i.e. after the head
-        // of the step before this one has been finished: a step therefore never starts before the
-        // head two steps back is complete, which keeps the ring slots of the head scratch apart.
+        // of the step before this one is complete: a step therefore never starts before the head
+        // two steps back is complete, which keeps the ring slots of the head scratch apart.
         // Everything else two steps share is in a ring slot of its own, guarded by the hand-off.
-        if (!head_cta || p.flag_in < 0) pdl_launch_dependents();
+        if (lane == 0 && (!head_cta || p.flag_in < 0)) pdl_launch_dependents();
         int vi, vg;
+        bool have = false;
         if (p.flag_in >= 0) {
-            // this expert's own entry: index and gate arrive independently, each valid by itself
-            const int32_t* ri = &p.route_inds[p.flag_in * 32 + k];
-            const int32_t* rg = reinterpret_cast<const int32_t*>(&p.route_gates[p.flag_in * 32 + k]);
-            vi = -1; vg = -1;
+            const float* lg = p.logits_ws + (size_t)p.flag_in * p.E;
+            float* work = reinterpret_cast<float*>(smem + S.s_route);
+            int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_route) + p.E;
+            float* s_g = reinterpret_cast<float*>(s_i + 32);
             uint32_t it = 0;
-            do { vi = ld_relaxed_gpu(ri); vg = ld_relaxed_gpu(rg); } while ((vi < 0 || vg < 0) && ++it < kSpinLimit);
-            if (vi < 0 || vg < 0) {
-                atomicExch(p.status, EDG_E_TIMEOUT);
-                pdl_wait_prior_grid();
-                vi = __ldcg(&p.slots[k]);
-                vg = __float_as_int(__ldcg(&p.gates[k]));
-            }
+            bool ok;
+            do {
+                ok = true;
+                for (int i = lane; i < p.E; i += 32) {
+                    const uint32_t w = ld_relaxed_gpu_u32(lg + i);
+                    ok = ok && (w != kNotYet);
+                    work[i] = __uint_as_float(w);
+                }
+                ok = __all_sync(0xFFFFFFFFu, ok);
+            } while (!ok && ++it < kSpinLimit);
             trace_mark(p, 19);
-            // everything the producer of this routing had observed (the reduce scratch of this ring
-            // slot being free again, above all) is ordered before what this CTA does next
-            asm volatile("fence.acq_rel.gpu;" ::: "memory");
-            if (head_cta) pdl_launch_dependents();
-        } else {
+            if (ok) {
+                // everything the writers of these logits had observed (the reduce scratch of this
+                // ring slot being free again, above all) is ordered before what this CTA does next
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");
+                if (lane == 0 && head_cta) pdl_launch_dependents();
+                __syncwarp();
+                trace_mark(p, 22);
+                if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
+                else topk_large(work, p.E, p.K, lane, s_i, s_g);
+                __syncwarp();
+                trace_mark(p, 23);
+                vi = s_i[k];
+                vg = __float_as_int(s_g[k]);
+                have = true;
+            } else if (lane == 0) {
+                atomicExch(p.status, EDG_E_TIMEOUT);
+                if (head_cta) pdl_launch_dependents();
+                pdl_wait_prior_grid();
+            }
+        }
+        if (!have) {
             vi = __ldcg(&p.slots[k]);
             vg = __float_as_int(__ldcg(&p.gates[k]));
         }
-        s_flag[1] = vi; s_flag[2] = vg;
+        if (lane == 0) { s_flag[1] = vi; s_flag[2] = vg; }
         trace_mark(p, 14);
     }
     __syncthreads();                      // routing, slot table and x fragments are in shared memory
@@ -887,20 +924,26 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         }
         if (tid == 0) counters[crank] = 0;
         if (p.flag_in >= 0) {
-            // The last of the kC reducers hands the routing slot this step has read back to its
-            // producer.  By then every CTA has read its entry and the reduce scratch of this ring
-            // slot is free again; the step that reuses either gets its own routing only after this.
+            // The last of the kC reducers resets the ring slot this step has taken its logits from.
+            // By then every CTA has read them and the reduce scratch of this ring slot is free
+            // again; the step that reuses either gets its own routing only after this.
             __threadfence();
             __syncthreads();
             if (tid == 0) s_flag[3] = (atomicAdd(&p.done[p.flag_in], 1) == kC - 1) ? 1 : 0;
             __syncthreads();
             if (s_flag[3]) {
-                if (tid == 0) p.done[p.flag_in] = 0;
-                __threadfence();
-                if (tid < 32) {
-                    st_relaxed_gpu(reinterpret_cast<int32_t*>(&p.route_gates[p.flag_in * 32 + tid]), -1);
-                    st_relaxed_gpu(&p.route_inds[p.flag_in * 32 + tid], -1);
+                if (tid == 0) {
+                    p.done[p.flag_in] = 0;
+                    // the head that filled the slot may still be copying the logits for its own top-k
+                    uint32_t it = 0;
+                    while (ld_relaxed_gpu(&p.fin[p.flag_in]) == 0 && ++it < kSpinLimit) {}
+                    if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
+                    st_relaxed_gpu(&p.fin[p.flag_in], 0);
+                    __threadfence();
                 }
+                __syncthreads();
+                for (int i = tid; i < p.E; i += kFW * 32)
+                    st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_in * p.E + i], kNotYet);
             }
         }
     }
@@ -992,15 +1035,14 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.trace = g_trace;
     p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
     p.ring = flag_in >= 0 ? (flag_in + 1) % kRing : 0;
-    p.route_inds = reinterpret_cast<int32_t*>(ws + W.route);
-    p.route_gates = reinterpret_cast<float*>(ws + W.route + kRing * 32 * 4);
+    p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + 176);
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
     // a call that starts a chain clears flags a broken chain may have left raised
     if (W_pre != nullptr && flag_in < 0) {
-        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 64, st));           // head-row counters and reader counts of the ring
-        EDG_CUDA_TRY(cudaMemsetAsync(p.route_inds, 0xFF, 2 * kRing * 32 * 4, st));   // -1 / NaN: nothing handed over yet
+        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 64, st));           // head-row counters, reader counts and "finished" marks of the ring
+        EDG_CUDA_TRY(cudaMemsetAsync(p.logits_ws, 0xFF, (size_t)kRing * d->E * sizeof(float), st));   // nothing handed over yet
     }
     const size_t smem = p.S.total;
     cudaError_t e;
