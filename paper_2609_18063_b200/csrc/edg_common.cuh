@@ -73,17 +73,25 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
     return L;
 }
 
-// Workspace layout for T tokens (floats unless noted).  The first 256 bytes are a control block
-// whose first int32 is the device-side status word; bytes 64..127 hold the per-slice arrival
-// counters of the fused kernel's reduce, bytes 128..143 the counts of head rows delivered (one per
-// ring slot of chained layer-steps) and bytes 160..175 the reader counts of the ring slots.
+// Workspace layout for T tokens (floats unless noted).  The first kCtrlBytes bytes are a control
+// block that must start out zero: its first int32 is the device-side status word, the rest are the
+// counters of the ring that chained batch-1 layer-steps share (arrivals of the reduce, head rows
+// delivered, reducers finished, head finished -- one set per ring slot).
+constexpr int kHandoffRing = 16;       // ring slots shared by chained batch-1 layer-steps in flight
+constexpr size_t kCtrlBytes = 512;     // control block: status word at 0, then the ring's counters
+constexpr size_t kCtrlCounters = 64;                               // [ring][4] arrivals per block of output rows
+constexpr size_t kCtrlHead = kCtrlCounters + kHandoffRing * 16;    // [ring] head rows delivered
+constexpr size_t kCtrlDone = kCtrlHead + kHandoffRing * 4;         // [ring] reducers finished
+constexpr size_t kCtrlFin = kCtrlDone + kHandoffRing * 4;          // [ring] head finished
+static_assert(kCtrlFin + kHandoffRing * 4 <= kCtrlBytes, "control block too small");
+
 struct WorkspaceLayout {
-    size_t ctrl;      // 256 B control block
+    size_t ctrl;      // kCtrlBytes control block
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
-    size_t partial;   // [4][K*kDownSlices][H] float: gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
-    size_t logits;    // [4][E] float               : next-step head logits handed to the chained next step, one set per ring slot
+    size_t partial;   // [ring][K][H] float       : gate-weighted expert outputs of the fused batch-1 kernel, one set per ring slot
+    size_t logits;    // [ring][E] float          : next-step head logits handed to the chained next step, one set per ring slot
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
     size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
@@ -102,12 +110,12 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     const size_t n_sets = d.n_adapters == 1 ? 1 : (size_t)d.K;
     const size_t r = d.rank > 0 ? (size_t)d.rank : 1;
     W.ctrl = 0;
-    W.u_gu = 256;
+    W.u_gu = kCtrlBytes;
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.logits = round_up(W.partial + 4 * (size_t)d.K * kDownSlices * d.H * sizeof(float), 256);
-    size_t end = round_up(W.logits + 4 * (size_t)d.E * sizeof(float), 256);
+    W.logits = round_up(W.partial + (size_t)kHandoffRing * d.K * d.H * sizeof(float), 256);
+    size_t end = round_up(W.logits + (size_t)kHandoffRing * d.E * sizeof(float), 256);
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;

@@ -39,8 +39,8 @@ constexpr int kE16 = kC * kDownSlices;   // CTAs per expert
 constexpr int kFW = 8;            // warps per CTA
 constexpr int kStages = 4;        // gate/up copy stages per CTA
 constexpr int kMaxRank = 64;
-constexpr int kTraceMarks = 24;
-constexpr int kRing = 4;          // chained layer-steps in flight: hand-off slots for routing, logits scratch, counters
+constexpr int kTraceMarks = 32;
+constexpr int kRing = kHandoffRing;   // chained layer-steps in flight: hand-off slots for logits, reduce scratch, counters
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
 
 // ---------------------------------------------------------------- shared-memory carve-up
@@ -54,7 +54,8 @@ struct FusedSmem {
     uint32_t mat_codes, mat_sz;                        // bytes of one (matrix, row tile) run of codes / sz inside a stage
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
-    uint32_t b_gate, b_up, b_down, a_down;             // LoRA slices (bf16)
+    uint32_t lora0, lora_bytes;                        // two buffers of per-quarter adapter slices: B_gate rows, B_up rows, A_down columns
+    uint32_t b_down;                                   // B_down rows of this CTA
     uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, s_route, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
@@ -69,28 +70,27 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.stage0 = o;     o += kStages * S.stage_bytes;
     S.d_codes = S.stage0;
     S.d_sz = S.stage0 + rows_d * sw / 2;               // rows_d * (sw/2 + sw/group*4) == 2 * stage_bytes
-    S.b_gate = o;     o += rows_gu * (uint32_t)rank * 2;      // B_gate[n0 .. n0+rows_gu][rank]
-    S.b_up = o;       o += rows_gu * (uint32_t)rank * 2;
+    S.lora_bytes = 3 * rows_gu * (uint32_t)rank * 2;   // B_gate[rows_gu][rank], B_up[rows_gu][rank], A_down[rank][rows_gu]
+    S.lora0 = o;      o += 2 * S.lora_bytes;
     S.b_down = o;     o += rows_d * (uint32_t)rank * 2;       // B_down[n0 .. n0+rows_d][rank]
-    S.a_down = o;     o += (uint32_t)rank * rows_gu * 2;      // A_down[rank][my rows of h]
     o = (o + 15) / 16 * 16;
-    S.bars = o;       o += 8 * (kStages + 5);
+    S.bars = o;       o += 8 * (kStages + 10);
     o = (o + 15) / 16 * 16;
     S.s_u = o;        o += 2 * kMaxRank * 4;
-    S.s_h = o;        o += sw * 4;                    // the cluster's quarter of h
-    S.s_ud_part = o;  o += kC * kMaxRank * 4;
+    S.s_h = o;        o += 2 * sw * 4;                // the quarter's h, double-buffered
+    S.s_ud_part = o;  o += 2 * kC * kMaxRank * 4;
     S.s_ud = o;       o += kMaxRank * 4;
     S.s_gu = o;       o += 2 * rows_gu * 4;
     S.s_o = o;        o += rows_d * 4;
     S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
     S.s_hloc = o;     o += 32 * 4;
-    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the routing, then its K winners
+    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the head, then its K winners
     S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
     S.s_table = o;    o += (uint32_t)E * 4;           // this layer's slot table, fetched before the routing is known
     o = (o + 15) / 16 * 16;
     S.s_xb = o;       o += (uint32_t)H * 2;           // x as fp16 B-fragment words, k-slot order
     S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
-    S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the cluster's quarter of h as (hi, lo) B-fragment words
+    S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the quarter's h as (hi, lo) B-fragment words
     S.s_hsum = o;     o += (sw / 32) * 4;
     S.s_route = o;    o += (uint32_t)E * 4 + 256;     // logits taken from the hand-off ring, then this step's K winners
     S.flag = o;       o += 16;
@@ -110,7 +110,7 @@ struct FusedParams {
     int32_t* status;
     int32_t* counters;            // [kRing][kC] one per ring slot and block of output rows, zero between uses
     int32_t* pre_counter;         // [kRing] rows of the head delivered so far, back to zero after every head
-    float* partial;               // [kRing][K * kDownSlices][H]
+    float* partial;               // [kRing][K][H]
     float* logits_ws;             // [kRing][E] logits of the next step's head; all-ones words = not yet written
     const void* W_pre;            // [E][H] or null
     int32_t* inds_next;
@@ -281,7 +281,10 @@ __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, i
     return d;
 }
 
-enum { BAR_DOWN = kStages, BAR_LORA = kStages + 1, BAR_FREE = kStages + 2, BAR_U = kStages + 3, BAR_H = kStages + 4 };
+// mbarriers: one per stage, then the down block, the adapter slices (two buffers), the B_down rows,
+// "stages 0-1 / 2-3 free after gate/up", "down block used", the adapter projections, h (two buffers)
+enum { BAR_DOWN = kStages, BAR_LORA = kStages + 1, BAR_BDOWN = kStages + 3, BAR_FREE01 = kStages + 4, BAR_FREE23 = kStages + 5,
+       BAR_DFREE = kStages + 6, BAR_U = kStages + 7, BAR_H = kStages + 8, kNumBars = kStages + 10 };
 
 // ---------------------------------------------------------------- head rows (a1) and top-k (a2)
 // The E rows of the head are dealt round-robin to the first CTAs of the grid; a row is split over
@@ -397,9 +400,9 @@ __device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* sme
 // NCW = H / 256 = chunks (of 32 codes) per warp in gate/up; DCH = I / 128 = chunks of a down row-slice;
 // TG = I / 256 = row tiles per matrix and CTA in gate/up; TD = H / 512 = row tiles per warp in down;
 // CPB = chunks per scaled block (2 for groups of 64 or 128 codes, 1 for groups of 32).
-// The kernel is straight-line code that every CTA runs once, so its size is kept small on purpose
-// (loops over K blocks are not unrolled, operands come from shared memory): instruction fetches
-// compete with the weight stream for the same memory system.
+// Most of the kernel is straight-line code that a CTA runs once or four times, so its size is kept
+// small on purpose (loops over K blocks are not unrolled, operands come from shared memory):
+// instruction fetches compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
 constexpr int kMaxPre = 8;        // head rows per head CTA
@@ -407,18 +410,16 @@ constexpr int kMaxPre = 8;        // head rows per head CTA
 template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_constant__ FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    const int b16 = blockIdx.x % kE16;             // CTA of the expert
-    const int k = blockIdx.x / kE16;               // position of the expert in the routing
-    const int c = b16 / kC;                        // quarter of the intermediate dimension (cluster of the expert)
-    const int crank = b16 % kC;                    // rank inside the cluster
+    const int k = blockIdx.x / kC;                 // position of the expert in the routing (= its cluster)
+    const int crank = blockIdx.x % kC;             // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     const int g8 = lane >> 2, t4 = lane & 3;       // fragment coordinates: row slot, quad lane
 
     const FusedSmem& S = p.S;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars);
     float* s_u = reinterpret_cast<float*>(smem + S.s_u);            // [2][kMaxRank]
-    float* s_h = reinterpret_cast<float*>(smem + S.s_h);            // [I/4]
-    float* s_ud_part = reinterpret_cast<float*>(smem + S.s_ud_part);// [kC][kMaxRank]
+    float* s_h = reinterpret_cast<float*>(smem + S.s_h);            // [2][I/4]   (double-buffered over quarters)
+    float* s_ud_part = reinterpret_cast<float*>(smem + S.s_ud_part);// [2][kC][kMaxRank]
     float* s_ud = reinterpret_cast<float*>(smem + S.s_ud);          // [kMaxRank]
     float* s_gu = reinterpret_cast<float*>(smem + S.s_gu);          // [2][rows_gu]
     float* s_o = reinterpret_cast<float*>(smem + S.s_o);            // [rows_d]
@@ -433,19 +434,18 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     float* s_hsum = reinterpret_cast<float*>(smem + S.s_hsum);      // [DCH/CPB]
 
     constexpr int rows_gu = 16 * TG, rows_d = 128 * TD, sw = 32 * DCH;
-    const int n0_gu = b16 * rows_gu;               // first gate/up row of this CTA (= c * sw + crank * rows_gu)
-    const int n0_d = crank * rows_d;               // first down row of this CTA
+    const int n0_d = crank * rows_d;               // first down (= output) row of this CTA
     const int r = p.rank;
     // reduce scratch of this step's ring slot: a chained step never waits for the previous kernel to
-    // end, so consecutive steps must not share it
-    float* partial = p.partial + (size_t)p.ring * p.K * kDownSlices * p.H;
+    // end, so steps in flight must not share it
+    float* partial = p.partial + (size_t)p.ring * p.K * p.H;
     int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
 
     // ---- a1 for the next step, first of all: the loads of the head rows depend on nothing but x,
-    //      and the routing they lead to is what the next layer-step waits for.  Only the first CTAs
-    //      of the grid evaluate the head: they are dispatched first.  A row is split over all
-    //      threads of its CTA (8 elements each).
+    //      and the routing they lead to is what the next layer-step waits for.  The rows are dealt
+    //      round-robin to the first CTAs of the grid; a row is split over all threads of its CTA
+    //      (8 elements each).
     const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
     const bool head_cta = (int)blockIdx.x < n_head_ctas;
     const int n_pre = head_cta ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
@@ -460,7 +460,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             lw[ri] = pre_lane ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8) : make_uint4(0, 0, 0, 0);
         }
     }
-
     uint32_t pre_state = kNotYet;         // this head row's entry of the ring slot, as the kernel finds it
     if (n_pre > 0 && p.flag_out >= 0 && warp == kFW - 1 && lane < n_pre) {
         const int e = (int)blockIdx.x + lane * n_head_ctas;
@@ -470,15 +469,15 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     // ---- thread 0: the barriers (peers will count bytes on BAR_U / BAR_H of this CTA, so they must
     //      exist, and every CTA of the cluster must be running, before anyone sends)
     if (tid == 0) {
-        for (int s = 0; s <= BAR_LORA; ++s) mbar_init(&bars[s], 1);
-        mbar_init(&bars[BAR_FREE], kFW / 2);
-        mbar_init(&bars[BAR_U], 1);
-        mbar_init(&bars[BAR_H], 1);
+        for (int s = 0; s < kNumBars; ++s)
+            mbar_init(&bars[s], (s == BAR_FREE01 || s == BAR_FREE23) ? kFW / 2 : (s == BAR_DFREE ? kFW : 1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        // bytes this CTA will receive: 2r adapter projections; then the cluster's quarter of h and kC partials of A_down.h
+        // bytes this CTA will receive: 2r adapter projections once; per quarter, that quarter of h
+        // and kC partials of A_down.h (the barriers of quarters 2 and 3 are re-armed below)
         if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
+        mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
     }
     // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed just
     // before the copies are issued: a cluster-scope barrier waits for every bulk copy in flight
@@ -507,10 +506,11 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         sum = group_sum<4 * CPB>(sum);
         if (pre_lane && (tid % (4 * CPB)) == 0) s_xsum[tid / (4 * CPB)] = sum;
     }
+    if (tid < kMaxRank) s_ud[tid] = 0.f;
 
     // ---- the head rows' partial sums, published at once: the routing of the next step is under way
     //      before this step's own routing is even looked at (one warp finishes the head while
-    //      thread 0 waits for the routing)
+    //      warp 0 waits for the routing)
     if (n_pre > 0) {
         if (pre_fast) {
 #pragma unroll
@@ -601,7 +601,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         trace_mark(p, 14);
     }
     __syncthreads();                      // routing, slot table and x fragments are in shared memory
-    trace_mark(p, 20);
 
     // ---- a3: take.  The decision is the same in every CTA of the expert.
     int slot = s_flag[1];
@@ -613,54 +612,69 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     const bool valid = slot >= 0 && slot < p.n_slots && ad >= 0;
     trace_mark(p, 10);
     cluster_wait();
-    trace_mark(p, 21);
     const int cps = p.H / 128;            // chunks of a row per stage
     const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
     const int gps = sw >> p.gshift;       // groups of a down row-slice
     const uint8_t* rec = p.pool + (size_t)(valid ? slot : 0) * p.L.bytes;
 
-    if (valid) {
-        // ---- issue the copies of this CTA's gate/up slice (stage = a quarter of the K range, one run
-        //      per matrix and row tile) and of its adapter rows, one warp per barrier
-        if (warp < kStages) {
-            // lane 0 arms the barrier, then lanes 0 .. 4*TG-1 issue one run each (codes or sz of a (matrix, tile))
-            const int s = warp;
+    // One warp issues two stages (K quarters 2 pair, 2 pair + 1) of the gate/up rows of quarter c:
+    // lanes 0 and 8 arm the barriers, then lanes 0..7 / 8..15 issue one run each (codes or sz of a
+    // (matrix, row tile)).
+    auto issue_gu = [&](int c, int pair) {
+        const int s = pair * 2 + (lane >> 3), run = lane & 7;
+        if (lane < 16 && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
+        __syncwarp();
+        if (lane < 16 && run < 4 * TG) {
             uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-            if (lane == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
-            __syncwarp();
-            if (lane < 4 * TG) {
-                const uint64_t pol = policy_evict_first();   // weights stream through L2 once
-                const int mt = lane >> 1, is_sz = lane & 1, m = mt / TG, ti = mt % TG;
-                const int n = n0_gu + 16 * ti;
-                if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
-                                          S.mat_codes, &bars[s], pol);
-                else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
-                                   S.mat_sz, &bars[s], pol);
-            }
-        } else if (warp == kStages && lane == 0 && r > 0) {
-            // the adapter rows this CTA needs in its two epilogues (kept in L2 across steps)
-            const uint32_t bgu = rows_gu * r * 2, bd = rows_d * r * 2, ad_row = rows_gu * 2;
-            mbar_expect_tx(&bars[BAR_LORA], 2 * bgu + bd + r * ad_row);
-            const size_t bo = ((size_t)ad * p.I + n0_gu) * r * 2;
-            bulk_g2s(smem + S.b_gate, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA]);
-            bulk_g2s(smem + S.b_up, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA]);
-            bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd,
-                     &bars[BAR_LORA]);
-            for (int j = 0; j < r; ++j)
-                bulk_g2s(smem + S.a_down + j * ad_row,
-                         static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0_gu) * 2, ad_row,
-                         &bars[BAR_LORA]);
+            const uint64_t pol = policy_evict_first();   // weights stream through L2 once
+            const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
+            const int n = c * sw + crank * rows_gu + 16 * ti;
+            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
+                                      S.mat_codes, &bars[s], pol);
+            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
+                               S.mat_sz, &bars[s], pol);
         }
-        trace_mark(p, 1);
-    }
+    };
+    // One warp issues the adapter slices of quarter c into buffer c & 1: this CTA's rows of B_gate
+    // and B_up, and its columns of A_down (one 16-byte-multiple run per rank index).
+    auto issue_lora = [&](int c) {
+        const uint32_t bgu = rows_gu * r * 2, ad_row = rows_gu * 2;
+        uint8_t* buf = smem + S.lora0 + (c & 1) * S.lora_bytes;
+        const int n0 = c * sw + crank * rows_gu;
+        if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (c & 1)], 2 * bgu + r * ad_row);
+        __syncwarp();
+        const size_t bo = ((size_t)ad * p.I + n0) * r * 2;
+        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (c & 1)]);
+        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (c & 1)]);
+        for (int j = lane; j < r; j += 32)
+            bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
+                     ad_row, &bars[BAR_LORA + (c & 1)]);
+    };
+
+    float acc_lo[TD], acc_hi[TD];         // down accumulators: rows g and g+8 of TD row tiles, over all quarters
+#pragma unroll
+    for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
 
     if (valid) {
-        // ---- with this CTA's weights on their way: its share of the 2r rows of A_gate / A_up, per-warp partial dot products
-        //      into s_red.  All threads take part, each covering 8 elements of a row per sweep; the
-        //      loads of up to 8 rows are in flight together, so the share costs one trip to memory.
+        // ---- issue the copies of the first quarter, and of the adapter rows every quarter needs
+        if (warp == 0) issue_gu(0, 0);
+        else if (warp == 1) issue_gu(0, 1);
+        else if (warp == 2 && r > 0) {
+            issue_lora(0);
+            if (lane == 0) {
+                const uint32_t bd = rows_d * r * 2;
+                mbar_expect_tx(&bars[BAR_BDOWN], bd);
+                bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd, &bars[BAR_BDOWN]);
+            }
+        }
+        trace_mark(p, 1);
+
+        // ---- with the weights on their way: this CTA's share of the 2r rows of A_gate / A_up, per-warp
+        //      partial dot products into s_red.  All threads take part, each covering 8 elements of a
+        //      row per sweep; the loads of up to 8 rows are in flight together, so the share costs one
+        //      trip to memory.
         const int per = (2 * r + kC - 1) / kC;
         if (r > 0) {
-            const int adA = p.n_adapters == 1 ? 0 : ad;
 #pragma unroll 1
             for (int q0 = 0; q0 < per; q0 += 8) {
                 float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -673,7 +687,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                         const int q = min(crank * per + min(q0 + u, per - 1), 2 * r - 1);
                         const int up = q >= r ? 1 : 0;
                         const uint16_t* A = reinterpret_cast<const uint16_t*>(up ? p.lora.A_up : p.lora.A_gate) +
-                                            ((size_t)adA * r + (q - up * r)) * p.H;
+                                            ((size_t)ad * r + (q - up * r)) * p.H;
                         ua[u] = ld_keep16(A + cc);
                     }
 #pragma unroll
@@ -691,7 +705,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 }
             }
         }
-        trace_mark(p, 11);
         __syncthreads();                  // s_red complete
         // every CTA of the cluster gets this CTA's adapter projections, counted on its BAR_U
         for (int i = tid; i < per * kC; i += kFW * 32) {
@@ -705,218 +718,253 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         }
         trace_mark(p, 2);
 
-        // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside stage
-        //      w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile, chunk) are 256
-        //      contiguous bytes of shared memory, lane (g, t) reading word t of rows g and g+8.  The
-        //      activations are column 0 of the 8-column B tile: the lanes of quad 0 read their words
-        //      from s_xb, every other lane holds zeros.  Partial sums of a scaled block are exact
-        //      integer-code dot products in fp32; scale and zero point are applied per block:
-        //      acc += s * (c - z * sum(x)).
-        {
-            const int s = warp / 2;
-            mbar_wait(&bars[s], 0, p.status);
-            if (warp == 0) trace_mark(p, 3);
-            const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-            const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
-            constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
-            float acc_lo[NT], acc_hi[NT];                            // rows g and g+8, column 0
-#pragma unroll
-            for (int mt = 0; mt < NT; ++mt) { acc_lo[mt] = 0.f; acc_hi[mt] = 0.f; }
-            const uint8_t* cbase = st + ch0 * 256 + g8 * 16 + t4 * 4;
-            const uint4* xbp = s_xb + (warp * NCW) * 4 + t4;
+        // ---- the four quarters of the intermediate dimension, one after the other.  For quarter c
+        //      this CTA computes its rows_gu gate/up rows (over all of K), the cluster exchanges
+        //      h = silu(gate) * up, and the CTA adds the quarter's columns to its rows_d output rows.
+        //      The weights stream through four stage buffers: gate/up of a quarter fills all four
+        //      (a K quarter each), its down block follows into stages 0-1 as soon as their warps
+        //      are done, the next quarter's K quarters 2-3 into stages 2-3 likewise, and its K
+        //      quarters 0-1 once the down block has been used.
 #pragma unroll 1
-            for (int ib = 0; ib < NCW / CPB; ++ib) {                 // scaled blocks of this warp's K range
-                float cfr[NT][4];
+        for (int c = 0; c < kDownSlices; ++c) {
+            const uint32_t par = c & 1, par2 = (c >> 1) & 1;
+            // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside
+            //      stage w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile,
+            //      chunk) are 256 contiguous bytes of shared memory, lane (g, t) reading word t of
+            //      rows g and g+8.  The activations are column 0 of the 8-column B tile: the lanes
+            //      of quad 0 read their words from s_xb, every other lane holds zeros.  Partial sums
+            //      of a scaled block are exact integer-code dot products in fp32; scale and zero
+            //      point are applied per block: acc += s * (c - z * sum(x)).
+            {
+                const int s = warp / 2;
+                mbar_wait(&bars[s], par, p.status);
+                if (c == 0) trace_mark(p, 3);
+                const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+                const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
+                constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
+                float a_lo[NT], a_hi[NT];                                // rows g and g+8, column 0
 #pragma unroll
-                for (int u = 0; u < CPB; ++u) {
-                    const int i = ib * CPB + u;
-                    uint4 xb = make_uint4(0, 0, 0, 0);
-                    if (g8 == 0) xb = xbp[i * 4];
+                for (int mt = 0; mt < NT; ++mt) { a_lo[mt] = 0.f; a_hi[mt] = 0.f; }
+                const uint8_t* cbase = st + ch0 * 256 + g8 * 16 + t4 * 4;
+                const uint4* xbp = s_xb + (warp * NCW) * 4 + t4;
+#pragma unroll 1
+                for (int ib = 0; ib < NCW / CPB; ++ib) {                 // scaled blocks of this warp's K range
+                    float cfr[NT][4];
+#pragma unroll
+                    for (int u = 0; u < CPB; ++u) {
+                        const int i = ib * CPB + u;
+                        uint4 xb = make_uint4(0, 0, 0, 0);
+                        if (g8 == 0) xb = xbp[i * 4];
+#pragma unroll
+                        for (int mt = 0; mt < NT; ++mt) {
+                            const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
+                            uint32_t alo[4], ahi[4];
+                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                            if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                            else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                            mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
+                        }
+                    }
+                    const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
+                    const float xs = s_xsum[(warp * NCW) / CPB + ib];
 #pragma unroll
                     for (int mt = 0; mt < NT; ++mt) {
-                        const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
-                        uint32_t alo[4], ahi[4];
-                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                        if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
-                        else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
-                        mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
+                        const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
+                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                        a_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), a_lo[mt]);
+                        a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), a_hi[mt]);
                     }
                 }
-                const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
-                const float xs = s_xsum[(warp * NCW) / CPB + ib];
+                if (t4 == 0) {
 #pragma unroll
-                for (int mt = 0; mt < NT; ++mt) {
-                    const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
-                    const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
-                    const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                    acc_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), acc_lo[mt]);
-                    acc_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), acc_hi[mt]);
+                    for (int mt = 0; mt < NT; ++mt) {
+                        s_part[warp * 2 * rows_gu + mt * 16 + g8] = a_lo[mt];
+                        s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = a_hi[mt];
+                    }
                 }
-            }
-            if (t4 == 0) {
-#pragma unroll
-                for (int mt = 0; mt < NT; ++mt) {
-                    s_part[warp * 2 * rows_gu + mt * 16 + g8] = acc_lo[mt];
-                    s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = acc_hi[mt];
-                }
-            }
-            // the down block goes into the space of stages 0 and 1 once their four warps are done
-            if (warp < kFW / 2) {
-                if (lane == 0) mbar_arrive(&bars[BAR_FREE]);
-                if (warp == 0) {
-                    mbar_wait(&bars[BAR_FREE], 0, p.status);
-                    if (lane == 0) {
-                        const uint64_t pol = policy_evict_first();
-                        const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
-                        mbar_expect_tx(&bars[BAR_DOWN], dcb + dzb);
-                        bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), dcb, &bars[BAR_DOWN], pol);
-                        bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
+                // stages 0-1: the quarter's down block follows; stages 2-3: the next quarter's K quarters 2-3
+                if (warp < kFW / 2) {
+                    if (lane == 0) mbar_arrive(&bars[BAR_FREE01]);
+                    if (warp == 0) {
+                        mbar_wait(&bars[BAR_FREE01], par, p.status);
+                        if (lane == 0) {
+                            const uint64_t pol = policy_evict_first();
+                            const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
+                            mbar_expect_tx(&bars[BAR_DOWN], dcb + dzb);
+                            bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), dcb, &bars[BAR_DOWN], pol);
+                            bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
+                        }
+                    }
+                } else {
+                    if (lane == 0) mbar_arrive(&bars[BAR_FREE23]);
+                    if (warp == kFW / 2 && c + 1 < kDownSlices) {
+                        mbar_wait(&bars[BAR_FREE23], par, p.status);
+                        issue_gu(c + 1, 1);
                     }
                 }
             }
-        }
-        __syncthreads();
-        // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
-        if (tid < 2 * rows_gu) {
-            float v = 0.f;
-            for (int w = 0; w < kFW; ++w) v += s_part[w * 2 * rows_gu + tid];
-            s_gu[tid] = v;
-        }
-        __syncthreads();
-        trace_mark(p, 4);
-        if (r > 0) mbar_wait(&bars[BAR_U], 0, p.status);            // every CTA's A.x has landed in s_u
-        trace_mark(p, 5);
-
-        // ---- finish gate/up: LoRA B (one thread per (projection, row)), SiLU, product
-        if (r > 0 && tid < 2 * rows_gu) {
-            mbar_wait(&bars[BAR_LORA], 0, p.status);
-            const int proj = tid / rows_gu, row = tid % rows_gu;
-            const uint16_t* Bm = reinterpret_cast<const uint16_t*>(smem + (proj ? S.b_up : S.b_gate)) + row * r;
-            const float d = smem_b_dot(Bm, s_u + proj * kMaxRank, r);
-            s_gu[proj * rows_gu + row] = fmaf(p.sigma, d, s_gu[proj * rows_gu + row]);
-        }
-        __syncthreads();
-        if (tid < rows_gu) s_hloc[tid] = silu_f(s_gu[tid]) * s_gu[rows_gu + tid];
-        __syncthreads();
-        // all-gather h inside the cluster: this CTA's rows_gu values go to every CTA, 16 bytes at a time
-        {
-            constexpr int vecs = rows_gu / 4;
-            for (int i = tid; i < vecs * kC; i += kFW * 32) {
-                const int v = i % vecs, dst = i / vecs;
-                st_async_f32x4(map_to_cta(&s_h[crank * rows_gu + 4 * v], dst), *reinterpret_cast<const float4*>(&s_hloc[4 * v]),
-                               map_to_cta(&bars[BAR_H], dst));
-            }
-        }
-        // partial of A_down . h over this CTA's rows of h (kC lanes per rank index), sent to every CTA of the cluster
-        for (int j = tid / kC; j < r; j += kFW * 32 / kC) {
-            const int part = tid % kC;
-            const uint16_t* Ad = reinterpret_cast<const uint16_t*>(smem + S.a_down) + j * rows_gu;
-            float v = 0.f;
-            for (int n = part; n < rows_gu; n += kC) v = fmaf(bf16_bits_to_float(Ad[n]), s_hloc[n], v);
-            v = group_sum<kC>(v);
-            st_async_f32(map_to_cta(&s_ud_part[crank * kMaxRank + j], part), v, map_to_cta(&bars[BAR_H], part));
-        }
-        trace_mark(p, 6);
-        mbar_wait(&bars[BAR_H], 0, p.status);                       // the cluster's quarter of h and of A_down.h
-        trace_mark(p, 7);
-
-        // ---- down on the tensor cores: partial over this quarter of the columns, for this CTA's H/4
-        //      output rows.  h is fp32: column 0 of the B tile carries its fp16 value, column 1 the
-        //      fp16 residual (lanes of quads 0 and 1 read their words from s_hb), and the two result
-        //      columns are added.
-        if (tid < r) {
-            float v = 0.f;
-            for (int cc = 0; cc < kC; ++cc) v += s_ud_part[cc * kMaxRank + tid];
-            s_ud[tid] = v;
-        }
-        if (tid < DCH * 8) {
-            const int i = tid >> 3, lo = (tid >> 2) & 1, q = tid & 3;
-            const float4 a = *reinterpret_cast<const float4*>(s_h + i * 32 + q * 8);
-            const float4 b = *reinterpret_cast<const float4*>(s_h + i * 32 + q * 8 + 4);
-            const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-            s_hb[tid] = lo ? permute8_lo(f) : permute8(f);
-        } else if (tid >= 64 && tid < 64 + DCH / CPB) {
-            const int j = tid - 64;
-            float v = 0.f;
-            for (int e = 0; e < 32 * CPB; ++e) v += s_h[j * 32 * CPB + e];   // hi + lo == h up to 2^-22: sum h itself
-            s_hsum[j] = v;
-        }
-        __syncthreads();
-        mbar_wait(&bars[BAR_DOWN], 0, p.status);
-        {
-            const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
-            const uint8_t* dsz = smem + S.d_sz;
-            float acc_lo[TD], acc_hi[TD];                            // TD independent row tiles per warp: interleaved
+            __syncthreads();
+            // the adapter slices of the next quarter go into the buffer the previous quarter used
+            if (warp == kFW - 1 && r > 0 && c + 1 < kDownSlices) issue_lora(c + 1);
+            // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
+            if (tid < 2 * rows_gu) {
+                float v = 0.f;
 #pragma unroll
-            for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
+                for (int w = 0; w < kFW; ++w) v += s_part[w * 2 * rows_gu + tid];
+                s_gu[tid] = v;
+            }
+            __syncthreads();
+            if (c == 0) {
+                trace_mark(p, 4);
+                if (r > 0) mbar_wait(&bars[BAR_U], 0, p.status);        // every CTA's A.x has landed in s_u
+                trace_mark(p, 5);
+            }
+
+            // ---- finish gate/up: LoRA B (one thread per (projection, row)), SiLU, product
+            const uint8_t* lbuf = smem + S.lora0 + par * S.lora_bytes;
+            if (r > 0 && tid < 2 * rows_gu) {
+                mbar_wait(&bars[BAR_LORA + par], par2, p.status);
+                const int proj = tid / rows_gu, row = tid % rows_gu;
+                const uint16_t* Bm = reinterpret_cast<const uint16_t*>(lbuf) + (proj * rows_gu + row) * r;
+                const float d = smem_b_dot(Bm, s_u + proj * kMaxRank, r);
+                s_gu[proj * rows_gu + row] = fmaf(p.sigma, d, s_gu[proj * rows_gu + row]);
+            }
+            __syncthreads();
+            if (tid < rows_gu) s_hloc[tid] = silu_f(s_gu[tid]) * s_gu[rows_gu + tid];
+            __syncthreads();
+            // all-gather h inside the cluster: this CTA's rows_gu values go to every CTA, 16 bytes at a time
+            float* hq = s_h + par * sw;
+            {
+                constexpr int vecs = rows_gu / 4;
+                for (int i = tid; i < vecs * kC; i += kFW * 32) {
+                    const int v = i % vecs, dst = i / vecs;
+                    st_async_f32x4(map_to_cta(&hq[crank * rows_gu + 4 * v], dst), *reinterpret_cast<const float4*>(&s_hloc[4 * v]),
+                                   map_to_cta(&bars[BAR_H + par], dst));
+                }
+            }
+            // partial of A_down . h over this CTA's rows of h (kC lanes per rank index), sent to every CTA of the cluster
+            float* udp = s_ud_part + par * kC * kMaxRank;
+            for (int j = tid / kC; j < r; j += kFW * 32 / kC) {
+                const int part = tid % kC;
+                const uint16_t* Ad = reinterpret_cast<const uint16_t*>(lbuf + 2 * rows_gu * r * 2) + j * rows_gu;
+                float v = 0.f;
+                for (int n = part; n < rows_gu; n += kC) v = fmaf(bf16_bits_to_float(Ad[n]), s_hloc[n], v);
+                v = group_sum<kC>(v);
+                st_async_f32(map_to_cta(&udp[crank * kMaxRank + j], part), v, map_to_cta(&bars[BAR_H + par], part));
+            }
+            if (c == 0) trace_mark(p, 6);
+            mbar_wait(&bars[BAR_H + par], par2, p.status);              // the quarter's h and A_down.h partials
+            if (c == 0) trace_mark(p, 7);
+
+            // ---- down on the tensor cores: this quarter's columns for this CTA's H/4 output rows.  h is
+            //      fp32: column 0 of the B tile carries its fp16 value, column 1 the fp16 residual
+            //      (lanes of quads 0 and 1 read their words from s_hb), and the two result columns
+            //      are added.
+            if (tid < r) {
+                float v = s_ud[tid];
+                for (int cc = 0; cc < kC; ++cc) v += udp[cc * kMaxRank + tid];
+                s_ud[tid] = v;
+            }
+            if (tid < DCH * 8) {
+                const int i = tid >> 3, lo = (tid >> 2) & 1, q = tid & 3;
+                const float4 a = *reinterpret_cast<const float4*>(hq + i * 32 + q * 8);
+                const float4 b = *reinterpret_cast<const float4*>(hq + i * 32 + q * 8 + 4);
+                const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                s_hb[tid] = lo ? permute8_lo(f) : permute8(f);
+            } else if (tid >= 64 && tid < 64 + DCH / CPB) {
+                const int j = tid - 64;
+                float v = 0.f;
+                for (int e = 0; e < 32 * CPB; ++e) v += hq[j * 32 * CPB + e];   // hi + lo == h up to 2^-22: sum h itself
+                s_hsum[j] = v;
+            }
+            __syncthreads();
+            // this buffer's barrier is used again two quarters on: arm it before anyone can send
+            if (tid == 0 && c + 2 < kDownSlices) mbar_expect_tx(&bars[BAR_H + par], (uint32_t)(sw + kC * r) * 4u);
+            mbar_wait(&bars[BAR_DOWN], par, p.status);
+            {
+                const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
+                const uint8_t* dsz = smem + S.d_sz;
 #pragma unroll 1
-            for (int ib = 0; ib < DCH / CPB; ++ib) {
-                float cfr[TD][4];
+                for (int ib = 0; ib < DCH / CPB; ++ib) {
+                    float cfr[TD][4];
 #pragma unroll
-                for (int u = 0; u < CPB; ++u) {
-                    const int i = ib * CPB + u;
-                    uint4 hb = make_uint4(0, 0, 0, 0);
-                    if (g8 < 2) hb = s_hb[(i * 2 + g8) * 4 + t4];
+                    for (int u = 0; u < CPB; ++u) {
+                        const int i = ib * CPB + u;
+                        uint4 hb = make_uint4(0, 0, 0, 0);
+                        if (g8 < 2) hb = s_hb[(i * 2 + g8) * 4 + t4];
+#pragma unroll
+                        for (int tt = 0; tt < TD; ++tt) {
+                            const int ti = warp + kFW * tt;
+                            const uint8_t* cw = dbase + (ti * DCH + i) * 256;
+                            uint32_t alo[4], ahi[4];
+                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                            if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                            else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                            mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
+                        }
+                    }
+                    const int gi = (ib * CPB * 32) >> p.gshift;
+                    const float hs = s_hsum[ib];
 #pragma unroll
                     for (int tt = 0; tt < TD; ++tt) {
                         const int ti = warp + kFW * tt;
-                        const uint8_t* cw = dbase + (ti * DCH + i) * 256;
-                        uint32_t alo[4], ahi[4];
-                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                        dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                        if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
-                        else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
-                        mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
+                        const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
+                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                        acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
+                        acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
                     }
                 }
-                const int gi = (ib * CPB * 32) >> p.gshift;
-                const float hs = s_hsum[ib];
-#pragma unroll
-                for (int tt = 0; tt < TD; ++tt) {
-                    const int ti = warp + kFW * tt;
-                    const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
-                    const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
-                    const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                    acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
-                    acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
+            }
+            // the next quarter's K quarters 0-1 go into stages 0-1 once every warp is done with the down block
+            if (c + 1 < kDownSlices) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars[BAR_DFREE]);
+                if (warp == 0) {
+                    mbar_wait(&bars[BAR_DFREE], par, p.status);
+                    issue_gu(c + 1, 0);
                 }
             }
-            if (t4 == 0) {
+            if (c == 0) trace_mark(p, 24);
+        }
+
+        if (t4 == 0) {
 #pragma unroll
-                for (int tt = 0; tt < TD; ++tt) {
-                    const int ti = warp + kFW * tt;
-                    s_o[ti * 16 + g8] = acc_lo[tt];
-                    s_o[ti * 16 + 8 + g8] = acc_hi[tt];
-                }
+            for (int tt = 0; tt < TD; ++tt) {
+                const int ti = warp + kFW * tt;
+                s_o[ti * 16 + g8] = acc_lo[tt];
+                s_o[ti * 16 + 8 + g8] = acc_hi[tt];
             }
         }
-        __syncthreads();                  // s_o complete
-        // LoRA B for down (on this quarter's share of A_down.h) and the gate weight: one thread per output row
+        if (r > 0) mbar_wait(&bars[BAR_BDOWN], 0, p.status);
+        __syncthreads();                  // s_o, s_ud and the B_down rows complete
+        // LoRA B for down (A_down.h summed over the quarters) and the gate weight: one thread per output row
         for (int lr = tid; lr < rows_d; lr += kFW * 32) {
             float o = s_o[lr];
             if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
-            partial[((size_t)k * kDownSlices + c) * p.H + n0_d + lr] = gate_k * o;
+            partial[(size_t)k * p.H + n0_d + lr] = gate_k * o;
         }
         trace_mark(p, 8);
     } else {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
         // a skipped expert contributes nothing
-        for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)k * kDownSlices + c) * p.H + n0_d + i] = 0.f;
+        for (int i = tid; i < rows_d; i += kFW * 32) partial[(size_t)k * p.H + n0_d + i] = 0.f;
     }
 
-    // ---- a6: this partial is published; the last arriver for the block of rows sums all 4K partials
+    // ---- a6: this partial is published; the last arriver for the block of rows sums the K partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == p.K * kDownSlices - 1) ? 1 : 0;
+    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == p.K - 1) ? 1 : 0;
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
-        const int np = p.K * kDownSlices;
         for (int i = tid; i < rows_d / 4; i += kFW * 32) {
             float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-            for (int kk = 0; kk < np; ++kk) {
+            for (int kk = 0; kk < p.K; ++kk) {
                 const float4 t = __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)kk * p.H + n0_d + 4 * i]));
                 yv.x += t.x; yv.y += t.y; yv.z += t.z; yv.w += t.w;
             }
@@ -962,6 +1010,9 @@ constexpr size_t kFusedSmemLimit = 112 * 1024;    // two CTAs per SM
 bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
     if ((d.I / kE16) % 16 != 0 || d.I / kE16 > 32) return false;   // whole 16-row tiles per CTA
+    // the head rows are dealt to the first CTAs of the grid, at most kMaxPre each
+    const int grid = d.K * kC, head_ctas = grid < 32 ? grid : (grid < (d.E + kMaxPre - 1) / kMaxPre ? grid : ((d.E + kMaxPre - 1) / kMaxPre > 32 ? (d.E + kMaxPre - 1) / kMaxPre : 32));
+    if (head_ctas * kMaxPre < d.E) return false;
     if (d.group > 128 || (d.group & (d.group - 1)) != 0) return false;
     if (d.rank % 8 != 0) return false;            // adapter slices are staged by 16-byte bulk copies
     return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
@@ -987,7 +1038,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.K * kE16, 1, 1);
+    cfg.gridDim = dim3(p.K * kC, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -1018,8 +1069,8 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     const WorkspaceLayout W = workspace_layout(*d, 1);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     p.status = reinterpret_cast<int32_t*>(ws + W.ctrl);
-    p.counters = reinterpret_cast<int32_t*>(ws + W.ctrl + 64);
-    p.pre_counter = reinterpret_cast<int32_t*>(ws + W.ctrl + 128);
+    p.counters = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlCounters);
+    p.pre_counter = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlHead);
     p.partial = reinterpret_cast<float*>(ws + W.partial);
     p.logits_ws = reinterpret_cast<float*>(ws + W.logits);
     p.W_pre = W_pre; p.inds_next = inds_next; p.gates_next = gates_next; p.logits_next = logits_next;
@@ -1033,15 +1084,15 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.gshift = 0;
     while ((1 << p.gshift) < d->group) ++p.gshift;
     p.trace = g_trace;
-    p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + 160);
+    p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlDone);
     p.ring = flag_in >= 0 ? (flag_in + 1) % kRing : 0;
-    p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + 176);
+    p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlFin);
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
     // a call that starts a chain clears flags a broken chain may have left raised
     if (W_pre != nullptr && flag_in < 0) {
-        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 64, st));           // head-row counters, reader counts and "finished" marks of the ring
+        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 3 * kHandoffRing * 4, st));           // head-row counters, reader counts and "finished" marks of the ring
         EDG_CUDA_TRY(cudaMemsetAsync(p.logits_ws, 0xFF, (size_t)kRing * d->E * sizeof(float), st));   // nothing handed over yet
     }
     const size_t smem = p.S.total;

@@ -59,7 +59,7 @@ extern "C" int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, c
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // The array keeps whatever the last call left.  Only the control block (status word, arrival
     // counters) has to start at zero; everything else is written before it is read.
-    EDG_CUDA_TRY(cudaMemsetAsync(scratch, 0, 256, st));
+    EDG_CUDA_TRY(cudaMemsetAsync(scratch, 0, edg::kCtrlBytes, st));
     return edg::run_fused_layer(desc, slot_pool, slots, slot_table, experts, gates, x, has_lora ? lora : nullptr, y,
                                 nullptr, nullptr, nullptr, nullptr, scratch, -1, -1, st);
 }

@@ -266,7 +266,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         const bool chained = s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
                              s->chain_stream == stream;
         const int flag_in = chained ? s->chain_flag : -1;            // ring slot this step's routing arrives in
-        const int flag_out = chained ? (flag_in + 1) % 4 : 0;        // ring slot for the routing it produces
+        const int flag_out = chained ? (flag_in + 1) % edg::kHandoffRing : 0;        // ring slot for the routing it produces
         rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
                                   logits_next_opt, workspace, flag_in, flag_out, st);
