@@ -322,34 +322,27 @@ __device__ __noinline__ void topk_large(float* work, int E, int K, int lane, int
     warp_softmax_topk(work, E, K, lane, inds, gates);
 }
 
-// One warp: publish this CTA's logits (summed from the per-warp partials in s_pre) into the ring slot
-// the next layer-step reads, and if they were the last ones of the head, compute the top-k for the
-// caller's inds_next / gates_next.  A chained next step does not wait for that: it takes the logits
-// from the ring and selects its experts itself.  `state` is this lane's entry of the ring slot as
-// it was when the kernel started: a slot is written again only after the step that read it has
-// ended and has reset it.
-__device__ __noinline__ void prerouter_finish(const FusedParams& p, uint8_t* smem, const float* s_pre, int n_rows,
-                                              int ncta, int lane, uint32_t state) {
+// One warp publishes head logits -- lane l owns logit `e` with value `v` when `own` is set -- into the
+// ring slot the next layer-step reads, and if they were the last ones of the head, computes the
+// top-k for the caller's inds_next / gates_next.  A chained next step does not wait for that: it
+// takes the logits from the ring and selects its experts itself.  `state` is the lane's entry of
+// the ring slot as it was when the kernel started: a slot is written again only after the step
+// that read it has ended and has reset it.
+__device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, float v, int e, bool own, int lane, uint32_t state) {
     int mine = 0;
     const int ring = p.flag_out >= 0 ? p.flag_out : 0;
     float* logits_ws = p.logits_ws + (size_t)ring * p.E;
     int32_t* pre_counter = p.pre_counter + ring;
-    if (lane < n_rows) {
-        const int e = blockIdx.x + lane * ncta;
-        if (e < p.E) {
-            float v = 0.f;
-#pragma unroll
-            for (int w = 0; w < kFW; ++w) v += s_pre[lane * kFW + w];
-            if (p.flag_out >= 0) {
-                uint32_t it = 0;
-                while (state != kNotYet && ++it < kSpinLimit) state = ld_relaxed_gpu_u32(&logits_ws[e]);
-                if (state != kNotYet) atomicExch(p.status, EDG_E_TIMEOUT);
-                // "the step that last read this slot is over" travels on to the reader of this logit
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");
-            }
-            st_relaxed_gpu_u32(&logits_ws[e], __float_as_uint(v));
-            mine = 1;
+    if (own) {
+        if (p.flag_out >= 0) {
+            uint32_t it = 0;
+            while (state != kNotYet && ++it < kSpinLimit) state = ld_relaxed_gpu_u32(&logits_ws[e]);
+            if (state != kNotYet) atomicExch(p.status, EDG_E_TIMEOUT);
+            // "the step that last read this slot is over" travels on to the reader of this logit
+            asm volatile("fence.acq_rel.gpu;" ::: "memory");
         }
+        st_relaxed_gpu_u32(&logits_ws[e], __float_as_uint(v));
+        mine = 1;
     }
     const int n_mine = __popc(__ballot_sync(0xFFFFFFFFu, mine));
     __syncwarp();
@@ -449,21 +442,27 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
     const bool head_cta = (int)blockIdx.x < n_head_ctas;
     const int n_pre = head_cta ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
-    const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= kFW * 32 * 8;
-    const bool pre_lane = tid * 8 < p.H;
-    uint4 lw[kMaxPre], lx = make_uint4(0, 0, 0, 0);
-    if (pre_fast) {
-        if (pre_lane) lx = ld_keep16(p.x + tid * 8);
+    // Usual case (fp16 head, H <= 2048): warp w evaluates row w of this CTA's rows by itself, each
+    // lane covering 8 runs of 8 elements, and publishes it without waiting for any other warp.
+    const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= 2048;
+    const int my_e = (int)blockIdx.x + warp * n_head_ctas;       // fast path: this warp's row
+    const bool my_row = pre_fast && warp < n_pre && my_e < p.E;
+    uint4 lw[8];
+    if (my_row) {
 #pragma unroll
-        for (int ri = 0; ri < kMaxPre; ++ri) {
-            const int e = min((int)blockIdx.x + min(ri, n_pre - 1) * n_head_ctas, p.E - 1);
-            lw[ri] = pre_lane ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)e * p.H + tid * 8) : make_uint4(0, 0, 0, 0);
+        for (int j = 0; j < 8; ++j) {
+            const int i = (j * 32 + lane) * 8;
+            lw[j] = i < p.H ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)my_e * p.H + i) : make_uint4(0, 0, 0, 0);
         }
     }
-    uint32_t pre_state = kNotYet;         // this head row's entry of the ring slot, as the kernel finds it
-    if (n_pre > 0 && p.flag_out >= 0 && warp == kFW - 1 && lane < n_pre) {
-        const int e = (int)blockIdx.x + lane * n_head_ctas;
-        if (e < p.E) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + e]);
+    const bool pre_lane = tid * 8 < p.H;
+    uint32_t pre_state = kNotYet;         // the ring-slot entry this lane will publish into, as the kernel finds it
+    if (p.flag_out >= 0) {
+        if (my_row && lane == 0) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + my_e]);
+        if (n_pre > 0 && !pre_fast && warp == kFW - 1 && lane < n_pre) {
+            const int e = (int)blockIdx.x + lane * n_head_ctas;
+            if (e < p.E) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + e]);
+        }
     }
 
     // ---- thread 0: the barriers (peers will count bytes on BAR_U / BAR_H of this CTA, so they must
@@ -508,45 +507,13 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     }
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
-    // ---- the head rows' partial sums, published at once: the routing of the next step is under way
-    //      before this step's own routing is even looked at (one warp finishes the head while
-    //      warp 0 waits for the routing)
-    if (n_pre > 0) {
-        if (pre_fast) {
-#pragma unroll
-            for (int ri = 0; ri < kMaxPre; ++ri) {
-                const uint4 w = lw[ri];
-                const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
-                const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
-                float v = a.x * bf16_lo(lx.x);
-                v = fmaf(a.y, bf16_hi(lx.x), v);
-                v = fmaf(b.x, bf16_lo(lx.y), v); v = fmaf(b.y, bf16_hi(lx.y), v);
-                v = fmaf(d.x, bf16_lo(lx.z), v); v = fmaf(d.y, bf16_hi(lx.z), v);
-                v = fmaf(f.x, bf16_lo(lx.w), v); v = fmaf(f.y, bf16_hi(lx.w), v);
-                v = warp_sum(v);
-                if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
-            }
-        } else {
-#pragma unroll 1
-            for (int ri = 0; ri < n_pre; ++ri) {
-                float v = head_row_partial(p.W_pre, p.pre_dtype, p.x, p.H, (int)blockIdx.x + ri * n_head_ctas, tid);
-                v = warp_sum(v);
-                if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
-            }
-        }
-        trace_mark(p, 12);
-        __syncthreads();
-        if (warp == kFW - 1) {
-            prerouter_finish(p, smem, s_red + kPreRed * kFW, n_pre, n_head_ctas, lane, pre_state);
-            if (lane == 0) trace_stamp(p, 13);
-        }
-    }
-
-    // ---- warp 0: the routing.  A chained step reads the logits its predecessor's head has put into
+    // ---- warp 0: the routing, before anything that has to wait for memory: the next layer-step is
+    //      released as soon as this one has its routing.  A chained step reads the logits its predecessor's head has put into
     //      the hand-off ring (long before that kernel ends) and selects its experts itself -- every
     //      CTA the same way, which costs less than waiting for one warp to do it for all.  Bounded
     //      wait; on a time-out fall back to waiting for the whole previous kernel and to the
     //      routing it has written, which is always sufficient.
+    bool have = false;                    // warp 0: the logits of this step's routing are in shared memory
     if (warp == 0) {
         // The next layer-step may start once every CTA of this one has said so.  The CTAs that
         // evaluate the head say so only after their own routing has arrived, i.e. after the head
@@ -554,8 +521,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         // two steps back is complete, which keeps the ring slots of the head scratch apart.
         // Everything else two steps share is in a ring slot of its own, guarded by the hand-off.
         if (lane == 0 && (!head_cta || p.flag_in < 0)) pdl_launch_dependents();
-        int vi, vg;
-        bool have = false;
         if (p.flag_in >= 0) {
             const float* lg = p.logits_ws + (size_t)p.flag_in * p.E;
             float* work = reinterpret_cast<float*>(smem + S.s_route);
@@ -580,12 +545,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 if (lane == 0 && head_cta) pdl_launch_dependents();
                 __syncwarp();
                 trace_mark(p, 22);
-                if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
-                else topk_large(work, p.E, p.K, lane, s_i, s_g);
-                __syncwarp();
-                trace_mark(p, 23);
-                vi = s_i[k];
-                vg = __float_as_int(s_g[k]);
                 have = true;
             } else if (lane == 0) {
                 atomicExch(p.status, EDG_E_TIMEOUT);
@@ -593,14 +552,71 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 pdl_wait_prior_grid();
             }
         }
-        if (!have) {
+    }
+
+    // ---- the head rows (their loads have been in flight since the kernel started), each published
+    //      by its warp as soon as it is summed
+    if (my_row) {
+        float v = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = (j * 32 + lane) * 8;
+            if (i < p.H) {
+                const uint4 xv = *reinterpret_cast<const uint4*>(p.x + i);
+                const uint4 w = lw[j];
+                const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+                const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
+                v = fmaf(a.x, bf16_lo(xv.x), v); v = fmaf(a.y, bf16_hi(xv.x), v);
+                v = fmaf(b.x, bf16_lo(xv.y), v); v = fmaf(b.y, bf16_hi(xv.y), v);
+                v = fmaf(d.x, bf16_lo(xv.z), v); v = fmaf(d.y, bf16_hi(xv.z), v);
+                v = fmaf(f.x, bf16_lo(xv.w), v); v = fmaf(f.y, bf16_hi(xv.w), v);
+            }
+        }
+        v = warp_sum(v);
+        if (warp == 0) trace_mark(p, 12);
+        head_publish(p, smem, v, my_e, lane == 0, lane, pre_state);
+        if (warp == 0) trace_mark(p, 13);
+    }
+
+    // ---- warp 0 again: this step's experts from the logits it has read
+    if (warp == 0) {
+        int vi, vg;
+        if (have) {
+            float* work = reinterpret_cast<float*>(smem + S.s_route);
+            int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_route) + p.E;
+            float* s_g = reinterpret_cast<float*>(s_i + 32);
+            if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
+            else topk_large(work, p.E, p.K, lane, s_i, s_g);
+            __syncwarp();
+            trace_mark(p, 23);
+            vi = s_i[k];
+            vg = __float_as_int(s_g[k]);
+        } else {
             vi = __ldcg(&p.slots[k]);
             vg = __float_as_int(__ldcg(&p.gates[k]));
         }
         if (lane == 0) { s_flag[1] = vi; s_flag[2] = vg; }
         trace_mark(p, 14);
     }
+    // ---- any other head (fp32 weights, wider rows): every row is split over all threads of the CTA
+    //      and published by one warp after the barrier below
+    if (n_pre > 0 && !pre_fast) {
+#pragma unroll 1
+        for (int ri = 0; ri < n_pre; ++ri) {
+            float v = head_row_partial(p.W_pre, p.pre_dtype, p.x, p.H, (int)blockIdx.x + ri * n_head_ctas, tid);
+            v = warp_sum(v);
+            if (lane == 0) s_red[(kPreRed + ri) * kFW + warp] = v;
+        }
+    }
     __syncthreads();                      // routing, slot table and x fragments are in shared memory
+    if (n_pre > 0 && !pre_fast && warp == kFW - 1) {
+        const int e = (int)blockIdx.x + lane * n_head_ctas;
+        const bool own = lane < n_pre && e < p.E;
+        float v = 0.f;
+        if (own)
+            for (int w = 0; w < kFW; ++w) v += s_red[(kPreRed + lane) * kFW + w];
+        head_publish(p, smem, v, e, own, lane, pre_state);
+    }
 
     // ---- a3: take.  The decision is the same in every CTA of the expert.
     int slot = s_flag[1];
