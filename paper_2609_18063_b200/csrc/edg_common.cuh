@@ -90,8 +90,9 @@ struct WorkspaceLayout {
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
-    size_t partial;   // [ring][K][H] float       : gate-weighted expert outputs of the fused batch-1 kernel, one set per ring slot
     size_t logits;    // [ring][E] float          : next-step head logits handed to the chained next step, one set per ring slot
+    size_t partial;   // [ring][4K][H] float      : gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
+    size_t lone_bytes;// what a batch-1 call that never chains needs: everything up to the first set of partials
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
     size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
@@ -113,9 +114,11 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_gu = kCtrlBytes;
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
-    W.partial = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.logits = round_up(W.partial + (size_t)kHandoffRing * d.K * d.H * sizeof(float), 256);
-    size_t end = round_up(W.logits + (size_t)kHandoffRing * d.E * sizeof(float), 256);
+    W.logits = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
+    W.partial = round_up(W.logits + (size_t)kHandoffRing * d.E * sizeof(float), 256);
+    const size_t one_set = (size_t)kDownSlices * d.K * d.H * sizeof(float);
+    W.lone_bytes = W.partial + one_set;
+    size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;

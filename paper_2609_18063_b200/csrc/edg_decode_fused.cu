@@ -126,6 +126,8 @@ struct FusedParams {
     int flag_in;                  // -1: the routing is already in memory; else the ring slot to take it from
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
     int gshift;                   // log2(group)
+    int qpc;                      // quarters of the intermediate dimension per cluster: 4 (one cluster per expert), 2 or 1
+    int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     FusedSmem S;                  // shared-memory carve-up
 };
 
@@ -403,7 +405,10 @@ constexpr int kMaxPre = 8;        // head rows per head CTA
 template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_constant__ FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
-    const int k = blockIdx.x / kC;                 // position of the expert in the routing (= its cluster)
+    const int cl = blockIdx.x / kC;                // cluster: an expert, or some quarters of it
+    const int nq = kDownSlices / p.qpc;            // clusters per expert
+    const int k = cl / nq;                         // position of the expert in the routing
+    const int c0 = (cl - k * nq) * p.qpc;          // first quarter of the intermediate dimension of this cluster
     const int crank = blockIdx.x % kC;             // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     const int g8 = lane >> 2, t4 = lane & 3;       // fragment coordinates: row slot, quad lane
@@ -431,9 +436,16 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     const int r = p.rank;
     // reduce scratch of this step's ring slot: a chained step never waits for the previous kernel to
     // end, so steps in flight must not share it
-    float* partial = p.partial + (size_t)p.ring * p.K * p.H;
+    const int np = p.K * nq;                       // partial outputs per output row
+    float* partial = p.partial + (size_t)p.ring * kDownSlices * p.K * p.H;
     int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
+    // A call that does not continue a chain runs alone on its workspace: it clears what the last
+    // head left unread in the ring.
+    if (p.stale >= 0 && blockIdx.x == 0) {
+        for (int i = tid; i < p.E; i += kFW * 32) st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.stale * p.E + i], kNotYet);
+        if (tid == 0) st_relaxed_gpu(&p.fin[p.stale], 0);
+    }
 
     // ---- a1 for the next step, first of all: the loads of the head rows depend on nothing but x,
     //      and the routing they lead to is what the next layer-step waits for.  The rows are dealt
@@ -476,7 +488,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         // and kC partials of A_down.h (the barriers of quarters 2 and 3 are re-armed below)
         if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
-        mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
+        if (p.qpc > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
     }
     // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed just
     // before the copies are issued: a cluster-scope barrier waits for every bulk copy in flight
@@ -651,20 +663,20 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                                S.mat_sz, &bars[s], pol);
         }
     };
-    // One warp issues the adapter slices of quarter c into buffer c & 1: this CTA's rows of B_gate
+    // One warp issues the adapter slices of quarter c (the it-th of this cluster) into buffer it & 1: this CTA's rows of B_gate
     // and B_up, and its columns of A_down (one 16-byte-multiple run per rank index).
-    auto issue_lora = [&](int c) {
+    auto issue_lora = [&](int c, int it) {
         const uint32_t bgu = rows_gu * r * 2, ad_row = rows_gu * 2;
-        uint8_t* buf = smem + S.lora0 + (c & 1) * S.lora_bytes;
+        uint8_t* buf = smem + S.lora0 + (it & 1) * S.lora_bytes;
         const int n0 = c * sw + crank * rows_gu;
-        if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (c & 1)], 2 * bgu + r * ad_row);
+        if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (it & 1)], 2 * bgu + r * ad_row);
         __syncwarp();
         const size_t bo = ((size_t)ad * p.I + n0) * r * 2;
-        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (c & 1)]);
-        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (c & 1)]);
+        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
+        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
         for (int j = lane; j < r; j += 32)
             bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
-                     ad_row, &bars[BAR_LORA + (c & 1)]);
+                     ad_row, &bars[BAR_LORA + (it & 1)]);
     };
 
     float acc_lo[TD], acc_hi[TD];         // down accumulators: rows g and g+8 of TD row tiles, over all quarters
@@ -673,10 +685,10 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
 
     if (valid) {
         // ---- issue the copies of the first quarter, and of the adapter rows every quarter needs
-        if (warp == 0) issue_gu(0, 0);
-        else if (warp == 1) issue_gu(0, 1);
+        if (warp == 0) issue_gu(c0, 0);
+        else if (warp == 1) issue_gu(c0, 1);
         else if (warp == 2 && r > 0) {
-            issue_lora(0);
+            issue_lora(c0, 0);
             if (lane == 0) {
                 const uint32_t bd = rows_d * r * 2;
                 mbar_expect_tx(&bars[BAR_BDOWN], bd);
@@ -742,8 +754,9 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         //      are done, the next quarter's K quarters 2-3 into stages 2-3 likewise, and its K
         //      quarters 0-1 once the down block has been used.
 #pragma unroll 1
-        for (int c = 0; c < kDownSlices; ++c) {
-            const uint32_t par = c & 1, par2 = (c >> 1) & 1;
+        for (int it = 0; it < p.qpc; ++it) {
+            const int c = c0 + it;
+            const uint32_t par = it & 1, par2 = (it >> 1) & 1;
             // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside
             //      stage w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile,
             //      chunk) are 256 contiguous bytes of shared memory, lane (g, t) reading word t of
@@ -754,7 +767,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             {
                 const int s = warp / 2;
                 mbar_wait(&bars[s], par, p.status);
-                if (c == 0) trace_mark(p, 3);
+                if (it == 0) trace_mark(p, 3);
                 const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
                 const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
                 constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
@@ -815,7 +828,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                     }
                 } else {
                     if (lane == 0) mbar_arrive(&bars[BAR_FREE23]);
-                    if (warp == kFW / 2 && c + 1 < kDownSlices) {
+                    if (warp == kFW / 2 && it + 1 < p.qpc) {
                         mbar_wait(&bars[BAR_FREE23], par, p.status);
                         issue_gu(c + 1, 1);
                     }
@@ -823,7 +836,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             }
             __syncthreads();
             // the adapter slices of the next quarter go into the buffer the previous quarter used
-            if (warp == kFW - 1 && r > 0 && c + 1 < kDownSlices) issue_lora(c + 1);
+            if (warp == kFW - 1 && r > 0 && it + 1 < p.qpc) issue_lora(c + 1, it + 1);
             // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
             if (tid < 2 * rows_gu) {
                 float v = 0.f;
@@ -832,7 +845,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 s_gu[tid] = v;
             }
             __syncthreads();
-            if (c == 0) {
+            if (it == 0) {
                 trace_mark(p, 4);
                 if (r > 0) mbar_wait(&bars[BAR_U], 0, p.status);        // every CTA's A.x has landed in s_u
                 trace_mark(p, 5);
@@ -870,9 +883,9 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 v = group_sum<kC>(v);
                 st_async_f32(map_to_cta(&udp[crank * kMaxRank + j], part), v, map_to_cta(&bars[BAR_H + par], part));
             }
-            if (c == 0) trace_mark(p, 6);
+            if (it == 0) trace_mark(p, 6);
             mbar_wait(&bars[BAR_H + par], par2, p.status);              // the quarter's h and A_down.h partials
-            if (c == 0) trace_mark(p, 7);
+            if (it == 0) trace_mark(p, 7);
 
             // ---- down on the tensor cores: this quarter's columns for this CTA's H/4 output rows.  h is
             //      fp32: column 0 of the B tile carries its fp16 value, column 1 the fp16 residual
@@ -897,7 +910,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             }
             __syncthreads();
             // this buffer's barrier is used again two quarters on: arm it before anyone can send
-            if (tid == 0 && c + 2 < kDownSlices) mbar_expect_tx(&bars[BAR_H + par], (uint32_t)(sw + kC * r) * 4u);
+            if (tid == 0 && it + 2 < p.qpc) mbar_expect_tx(&bars[BAR_H + par], (uint32_t)(sw + kC * r) * 4u);
             mbar_wait(&bars[BAR_DOWN], par, p.status);
             {
                 const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
@@ -936,7 +949,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 }
             }
             // the next quarter's K quarters 0-1 go into stages 0-1 once every warp is done with the down block
-            if (c + 1 < kDownSlices) {
+            if (it + 1 < p.qpc) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[BAR_DFREE]);
                 if (warp == 0) {
@@ -944,7 +957,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                     issue_gu(c + 1, 0);
                 }
             }
-            if (c == 0) trace_mark(p, 24);
+            if (it == 0) trace_mark(p, 24);
         }
 
         if (t4 == 0) {
@@ -961,26 +974,26 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         for (int lr = tid; lr < rows_d; lr += kFW * 32) {
             float o = s_o[lr];
             if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
-            partial[(size_t)k * p.H + n0_d + lr] = gate_k * o;
+            partial[(size_t)cl * p.H + n0_d + lr] = gate_k * o;
         }
         trace_mark(p, 8);
     } else {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
         // a skipped expert contributes nothing
-        for (int i = tid; i < rows_d; i += kFW * 32) partial[(size_t)k * p.H + n0_d + i] = 0.f;
+        for (int i = tid; i < rows_d; i += kFW * 32) partial[(size_t)cl * p.H + n0_d + i] = 0.f;
     }
 
-    // ---- a6: this partial is published; the last arriver for the block of rows sums the K partials
+    // ---- a6: this partial is published; the last arriver for the block of rows sums all partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == p.K - 1) ? 1 : 0;
+    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == np - 1) ? 1 : 0;
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
         for (int i = tid; i < rows_d / 4; i += kFW * 32) {
             float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
-            for (int kk = 0; kk < p.K; ++kk) {
+            for (int kk = 0; kk < np; ++kk) {
                 const float4 t = __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)kk * p.H + n0_d + 4 * i]));
                 yv.x += t.x; yv.y += t.y; yv.z += t.z; yv.w += t.w;
             }
@@ -1054,7 +1067,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.K * kC, 1, 1);
+    cfg.gridDim = dim3(p.K * (kDownSlices / p.qpc) * kC, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -1074,7 +1087,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, cudaStream_t st) {
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st) {
     const bool has_lora = lora != nullptr && d->rank > 0;
     FusedParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);
@@ -1101,16 +1114,14 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     while ((1 << p.gshift) < d->group) ++p.gshift;
     p.trace = g_trace;
     p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlDone);
-    p.ring = flag_in >= 0 ? (flag_in + 1) % kRing : 0;
+    p.ring = ring;
+    p.stale = stale;
+    // a chained step shares the GPU with its neighbours: few, long-lived CTAs; a lone step wants all SMs at once
+    p.qpc = flag_in >= 0 ? kDownSlices : 1;
     p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlFin);
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
-    // a call that starts a chain clears flags a broken chain may have left raised
-    if (W_pre != nullptr && flag_in < 0) {
-        EDG_CUDA_TRY(cudaMemsetAsync(p.pre_counter, 0, 3 * kHandoffRing * 4, st));           // head-row counters, reader counts and "finished" marks of the ring
-        EDG_CUDA_TRY(cudaMemsetAsync(p.logits_ws, 0xFF, (size_t)kRing * d->E * sizeof(float), st));   // nothing handed over yet
-    }
     const size_t smem = p.S.total;
     cudaError_t e;
     const bool wide = d->group >= 64;         // scaled blocks of 64 codes (groups of 64 or 128) or of 32

@@ -12,7 +12,7 @@ bool fused_supported(const edg_layer_desc& d);
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, cudaStream_t st);
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st);
 
 int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots, const int32_t* table,
                     const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
@@ -307,7 +307,7 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
     // batch-1 decode on the shapes the fused kernel covers: one launch for the whole FFN
     if (T == 1 && fused_supported(*d))
         return run_fused_layer(d, slot_pool, slots, table, experts, gates, x, has_lora ? lora : nullptr, y,
-                               nullptr, nullptr, nullptr, nullptr, workspace, -1, -1, st);
+                               nullptr, nullptr, nullptr, nullptr, workspace, -1, -1, 0, -1, st);
 
     // several tokens: group the (token, choice) pairs per expert and run the tensor-core path
     if (T > 1) return run_grouped(d, slot_pool, T, slots, table, experts, gates, x, has_lora ? lora : nullptr, y, workspace, st);

@@ -12,7 +12,7 @@ bool fused_supported(const edg_layer_desc& d);
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, cudaStream_t st);
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st);
 }  // namespace edg
 
 namespace {
@@ -37,7 +37,7 @@ extern "C" int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, c
     if (!slot_pool || !slots || !gates || !x || !y) return EDG_E_INVAL;
     if (!edg::aligned(slot_pool, 256) || !edg::aligned(x, 16) || !edg::aligned(y, 16)) return EDG_E_INVAL;
     if (!edg::fused_supported(*desc)) return EDG_E_SHAPE;
-    if (edg::workspace_layout(*desc, 1).bytes > kStaticScratchBytes) return EDG_E_WORKSPACE;   // beyond the fixed array
+    if (edg::workspace_layout(*desc, 1).lone_bytes > kStaticScratchBytes) return EDG_E_WORKSPACE;   // beyond the fixed array
     const bool has_lora = lora != nullptr && desc->rank > 0;
     if (has_lora) {
         if (!lora->A_gate || !lora->B_gate || !lora->A_up || !lora->B_up || !lora->A_down || !lora->B_down) return EDG_E_INVAL;
@@ -61,5 +61,5 @@ extern "C" int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, c
     // counters) has to start at zero; everything else is written before it is read.
     EDG_CUDA_TRY(cudaMemsetAsync(scratch, 0, edg::kCtrlBytes, st));
     return edg::run_fused_layer(desc, slot_pool, slots, slot_table, experts, gates, x, has_lora ? lora : nullptr, y,
-                                nullptr, nullptr, nullptr, nullptr, scratch, -1, -1, st);
+                                nullptr, nullptr, nullptr, nullptr, scratch, -1, -1, 0, -1, st);
 }

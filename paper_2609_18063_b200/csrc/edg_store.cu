@@ -20,7 +20,7 @@ bool fused_supported(const edg_layer_desc& d);
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, cudaStream_t st);
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st);
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
                       int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head);
 }  // namespace edg
@@ -65,6 +65,9 @@ struct edg_store {
     const void* chain_ws = nullptr;
     void* chain_stream = nullptr;
     int chain_flag = 0;
+    const void* ring_ws = nullptr;         // workspace whose hand-off ring this store has initialised
+    int ring_next = 0;                     // ring slot of the next batch-1 layer-step
+    int pub_slot = -1;                     // ring slot holding logits no step has read yet, or -1
 };
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
@@ -265,11 +268,31 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
         const bool chained = s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
                              s->chain_stream == stream;
-        const int flag_in = chained ? s->chain_flag : -1;            // ring slot this step's routing arrives in
-        const int flag_out = chained ? (flag_in + 1) % edg::kHandoffRing : 0;        // ring slot for the routing it produces
+        // A workspace seen for the first time gets its ring cleared: counters to zero, logits to
+        // "not yet written".  After that the ring looks after itself: a chained step resets the
+        // slot it has read, and a step that starts over clears the slot the last head left unread.
+        bool fresh = s->ring_ws != workspace;
+        if (fresh) {
+            uint8_t* w8 = static_cast<uint8_t*>(workspace);
+            const edg::WorkspaceLayout W = edg::workspace_layout(s->d, 1);
+            EDG_CUDA_TRY(cudaMemsetAsync(w8 + edg::kCtrlCounters, 0, edg::kCtrlBytes - edg::kCtrlCounters, st));
+            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.logits, 0xFF, (size_t)edg::kHandoffRing * s->d.E * sizeof(float), st));
+            s->ring_ws = workspace;
+            s->ring_next = 0;
+            s->pub_slot = -1;
+        }
+        const bool chain = chained && !fresh;
+        const int flag_in = chain ? s->chain_flag : -1;              // ring slot this step's logits arrive in
+        int stale = -1;
+        if (!chain && s->pub_slot >= 0) stale = s->pub_slot;         // nobody will read that head's logits
+        s->pub_slot = -1;
+        const int ring = s->ring_next;                               // ring slot of this step's scratch and of the head it evaluates
+        const int flag_out = W_pre_next != nullptr ? ring : -1;
+        s->ring_next = (ring + 1) % edg::kHandoffRing;
         rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
-                                  logits_next_opt, workspace, flag_in, flag_out, st);
+                                  logits_next_opt, workspace, flag_in, flag_out, ring, stale, st);
+        if (W_pre_next != nullptr) s->pub_slot = flag_out;
         if (rc != EDG_OK) return rc;
         s->chain_inds = W_pre_next != nullptr ? inds_next : nullptr;
         s->chain_ws = workspace;
