@@ -52,7 +52,7 @@ extern "C" {
 #define EDG_E_SLOTS    -3   /* more experts to stage than slots in the pool                     */
 #define EDG_E_RANGE    -4   /* expert / layer / slot index out of range, or duplicate expert    */
 #define EDG_E_CUDA     -5   /* a CUDA runtime call failed; see edg_last_cuda_error              */
-#define EDG_E_TIMEOUT  -6   /* a bounded host wait ran out                                      */
+#define EDG_E_TIMEOUT  -6   /* a bounded wait (host or device side) ran out                     */
 #define EDG_E_WORKSPACE -7  /* workspace too small or misaligned                                */
 
 /* dtypes */
@@ -129,16 +129,22 @@ int32_t edg_unpack_expert(const edg_layer_desc* desc, const void* record,
 /* Bytes of device scratch the FFN calls need for T tokens (T = 1 for batch-1 decode). */
 int32_t edg_ffn_workspace_bytes(const edg_layer_desc* desc, int32_t T, size_t* bytes);
 
-/* Reads the device-side status word that the kernels keep at the start of a workspace: 0, or an
+/* Reads the device-side status word that the kernels keep at the start of a workspace: 0, an
  * EDG_E_RANGE raised by a slot or expert index outside its range (the kernel skips that access
- * instead of faulting).  Synchronises `stream`. */
+ * instead of faulting), or an EDG_E_TIMEOUT raised by a bounded device-side wait that gave up (the
+ * kernel then falls back to waiting for the previous kernel, or goes on with a flagged result).
+ * Synchronises `stream`. */
 int32_t edg_workspace_status(const void* workspace, void* stream, int32_t* status);
 
-/* Tracing: with a dev buffer of (CTAs in the grid) x 16 uint64 (the batch-1 layer kernel launches
- * (K + 1) x 16 CTAs), every CTA stamps the GPU's nanosecond timer at its phase boundaries, in slot
- * 0 start, 1 copies issued, 2 adapter projections sent, 3 first weights landed, 4 gate/up done,
- * 5 peers' projections in, 6 h sent, 7 whole h in, 8 down done, 9 end.  NULL switches it off
- * (the default).  Process-wide; set it while no launch is in flight. */
+/* Tracing: with a dev buffer of (CTAs in the grid) x 32 uint64 (the batch-1 layer kernel launches
+ * 4K CTAs for a chained step and 16K for a lone one), every CTA stamps the GPU's nanosecond timer
+ * at its phase boundaries, in slot 0 start, 1 first copies issued, 2 adapter projections sent,
+ * 3 first weights landed, 4 gate/up of the first quarter done, 5 peers' projections in, 6 h sent,
+ * 7 h of the quarter in, 8 partial output written, 9 end, 10 slot taken, 12 head row summed,
+ * 13 head row published, 14 routing known, 19 logits read from the hand-off ring, 22 fence passed,
+ * 23 experts selected, 24 first quarter finished; 15-18 are stamped by the warp that computes the
+ * caller's top-k.  NULL switches it off (the default).  Process-wide; set it while no launch is
+ * in flight. */
 int32_t edg_set_trace_buffer(void* dev_buffer);
 
 /* ---------------------------------------------------------------- a1 + a2: prerouter */
@@ -221,10 +227,10 @@ int32_t edg_store_mark_computed(edg_store* store, int32_t layer, void* stream);
  *   lora        host struct of dev pointers, or NULL for no adapter
  *   y           dev [T][H] of out_dtype
  *   workspace   dev, edg_ffn_workspace_bytes(desc, T) bytes, 256-byte aligned; holds the
- *               intermediate h and the rank-r projections.  Its first 256 bytes are a control
- *               block (sticky status word, see edg_workspace_status) that the caller zeroes once
- *               before first use; the rest needs no initialisation.  Calls that share a
- *               workspace must be ordered on the device.
+ *               intermediate h and the rank-r projections.  Its first 512 bytes are a control
+ *               block (sticky status word, see edg_workspace_status, and arrival counters) that
+ *               the caller zeroes once before first use; the rest needs no initialisation.
+ *               Calls that share a workspace must be ordered on the device.
  * An index outside its range makes the kernels skip that expert and raise the status word; no
  * out-of-range address is ever formed.
  * T = 1 is batch-1 decode (fused dequant GEMV kernels).  T > 1 is batched decode / prefill. */
@@ -263,12 +269,29 @@ int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* 
  *   x dev bf16 [H]; inds_cur dev int32 [K]; gates_cur dev float [K];
  *   W_pre_next dev [E][H] (NULL skips the prediction); inds_next dev int32 [K];
  *   gates_next dev float [K]; logits_next_opt dev float [E] or NULL; y dev [H] of out_dtype;
- *   workspace as for moe_expert_ffn_int4_lora with T = 1. */
+ *   workspace as for moe_expert_ffn_int4_lora with T = 1.
+ *
+ * Chained calls.  When a call's inds_cur / gates_cur are the very buffers the previous call on this
+ * store wrote as inds_next / gates_next, with the same workspace and stream, the two layer-steps
+ * are chained: the later kernel is launched as a programmatic dependent of the earlier one, starts
+ * while that one is still running, takes the head's logits from a ring inside the workspace as
+ * soon as they are written, and selects its experts itself (same top-k, same result).  Up to 16
+ * chained steps share the GPU.  The results are those of unchained calls; what changes is the
+ * contract on the inputs: a chained call reads x, W_pre_next and the slot pool as soon as it
+ * starts, so they must already be valid when the call is made -- not produced by work queued
+ * on the stream between the two calls.  Callers that cannot promise this switch chaining off
+ * with edg_store_set_chaining.  A chain captured in a CUDA graph that is replayed back to back
+ * must hold a multiple of 16 layer-steps, so that every replay finds the ring where the
+ * previous one left it. */
 int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          const int32_t* inds_cur, const float* gates_cur,
                          const void* W_pre_next, int32_t* inds_next, float* gates_next,
                          float* logits_next_opt, void* y,
                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* Switches the chaining of consecutive moe_layer_decode calls on (default) or off.  With chaining
+ * off every layer-step is an ordinary stream-ordered launch. */
+int32_t edg_store_set_chaining(edg_store* store, int32_t enable);
 
 #ifdef __cplusplus
 }

@@ -72,6 +72,7 @@ _SIG = {
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
     "edg_store_get_stats": ([_P, C.POINTER(StoreStats)], C.c_int32),
+    "edg_store_set_chaining": ([_P, C.c_int32], C.c_int32),
     "edg_store_snapshot": ([_P, C.c_int32, _P, _P], C.c_int32),
     "edg_store_wait_staged": ([_P, C.c_int32, _P], C.c_int32),
     "edg_store_mark_computed": ([_P, C.c_int32, _P], C.c_int32),
@@ -275,6 +276,9 @@ class Store:
             self.close()
         except Exception:
             pass
+
+    def set_chaining(self, enable: bool) -> None:
+        _check(_lib.edg_store_set_chaining(self.handle, 1 if enable else 0), "edg_store_set_chaining")
 
     def stats(self) -> dict:
         s = StoreStats()

@@ -1136,10 +1136,9 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
 
 }  // namespace edg
 
-// Tracing hook: with a device buffer of (CTAs in the grid) x 16 uint64, every CTA of the fused
-// layer kernel stamps %globaltimer (ns) at its phase boundaries: 0 start, 1 copies issued,
-// 2 adapter projections sent, 3 first weights landed, 4 gate/up done, 5 peers' projections in,
-// 6 h sent, 7 h of the whole expert in, 8 down done, 9 end.  NULL switches tracing off.
+// Tracing hook: with a device buffer of (CTAs in the grid) x kTraceMarks uint64, every CTA of the
+// fused layer kernel stamps %globaltimer (ns) at its phase boundaries (the header lists the slots).
+// NULL switches tracing off.
 extern "C" int32_t edg_set_trace_buffer(void* dev_buffer) {
     edg::g_trace = static_cast<unsigned long long*>(dev_buffer);
     return EDG_OK;

@@ -68,6 +68,7 @@ struct edg_store {
     const void* ring_ws = nullptr;         // workspace whose hand-off ring this store has initialised
     int ring_next = 0;                     // ring slot of the next batch-1 layer-step
     int pub_slot = -1;                     // ring slot holding logits no step has read yet, or -1
+    bool chaining = true;
 };
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
@@ -266,7 +267,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         if (!workspace || !edg::aligned(workspace, 256) || workspace_bytes < edg::workspace_layout(s->d, 1).bytes)
             return EDG_E_WORKSPACE;
         if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
-        const bool chained = s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
+        const bool chained = s->chaining && s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
                              s->chain_stream == stream;
         // A workspace seen for the first time gets its ring cleared: counters to zero, logits to
         // "not yet written".  After that the ring looks after itself: a chained step resets the
@@ -307,4 +308,10 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         }
     }
     return edg_store_mark_computed(s, layer, stream);
+}
+
+extern "C" int32_t edg_store_set_chaining(edg_store* s, int32_t enable) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    s->chaining = enable != 0;
+    return EDG_OK;
 }

@@ -1,0 +1,60 @@
+"""Chained layer-steps (Sec. 3.2: step t+1 consumes the routing predicted during step t) launched
+back to back without host synchronisation, so that several steps are in flight at once and the
+hand-off ring inside the workspace wraps around several times.  Every checked step must match the
+oracle on the routing the GPU itself produced, the routing must be the exact top-k of the GPU's own
+logits, and switching the chaining off must give the same indices and the same outputs."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2609_18063_b200 as edg
+from paper_2609_18063_b200 import layer_io
+from oracle import moe_oracle as orc
+from workloads import synth
+from tests._gpu_util import x_dev, out_tensor
+from tests.test_gpu_parity import _make_store, _check_routing, _assert_close
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, store, d, W, xd, steps, ws, chaining):
+    store.set_chaining(chaining)
+    inds = torch.zeros((steps + 1, cfg.K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((steps + 1, cfg.K), dtype=torch.float32, device="cuda")
+    logits = torch.zeros((steps + 1, cfg.E), dtype=torch.float32, device="cuda")
+    edg.prerouter_topk(d, W, xd[steps], 1, inds[0], gates[0], logits[0])
+    y = out_tensor(d, steps)
+    for t in range(steps):                      # no host synchronisation inside the loop
+        edg.moe_layer_decode(store, 0, xd[t], inds[t], gates[t], W, inds[t + 1], gates[t + 1], logits[t + 1], y[t], ws)
+    torch.cuda.synchronize()
+    assert edg.workspace_status(ws) == 0
+    return inds.cpu().numpy(), gates.cpu().numpy(), logits.cpu().numpy(), y.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("name,steps,stride", [("cfg1", 50, 1), ("cfg2", 50, 7)])
+def test_chained_steps_in_flight_match_oracle_and_unchained(name, steps, stride):
+    cfg = synth.CONFIGS[name]
+    store, d, hosts, slots, tables, cs, _ = _make_store(cfg, n_slots=cfg.E)
+    for e0 in range(0, cfg.E, 64):              # everything resident: no staging between the steps
+        edg.stage_experts_to_slots(store, 0, np.arange(e0, min(cfg.E, e0 + 64), dtype=np.int32))
+    torch.cuda.synchronize()
+    W_np = synth.prerouter_weights(cfg)
+    W = torch.from_numpy(W_np).cuda()
+    X = synth.hidden_states(cfg, steps + 1, stream=23)
+    xd = x_dev(X)
+    ws = layer_io.new_workspace(d)
+    inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, xd, steps, ws, True)
+    inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, xd, steps, ws, False)
+    # integer work is bit-exact between the two launch modes, floats agree far inside the tolerance
+    assert np.array_equal(inds_c, inds_u)
+    assert np.array_equal(logits_c, logits_u)
+    assert np.array_equal(gates_c, gates_u)
+    assert np.abs(y_c - y_u).max() <= 1e-4
+    experts = {}
+    get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
+    lora = synth.lora_tensors(cfg, 0, 0)
+    for t in list(range(0, steps, stride)) + [steps - 1]:
+        ref = orc.moe_ffn(X[t], inds_c[t], gates_c[t].astype(np.float64), get, lambda e: lora, cfg.lora_scale, cfg.group)
+        _assert_close(y_c[t], ref)
+        _check_routing(logits_c[t + 1], inds_c[t + 1], gates_c[t + 1], W_np, X[t], cfg.K)
+    store.close()
