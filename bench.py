@@ -145,7 +145,8 @@ def run_b200(args):
 
     cfg = synth.CONFIGS["cfg2"]
     n_inst = args.instances
-    first_layer = rank * n_inst            # replicas: every rank serves its own layer instances
+    from paper_2609_18063_b200 import replicas
+    first_layer = replicas.first_instance(rank, n_inst)   # replicas: every rank serves its own layer instances
     desc = edg.make_desc(cfg, n_slots=cfg.E, out_dtype="f32")
     R = edg.record_bytes(desc)
     K, E, H = cfg.K, cfg.E, cfg.H
@@ -240,11 +241,8 @@ def run_b200(args):
     if status != 0 or not bool(torch.isfinite(y).all()):
         raise SystemExit(f"bench: bad device status {status} or non-finite output")
 
-    t_ms = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_max = float(t_ms.item())
-    value = world * steps / (ms_max * 1e-3)
+    ms_max = replicas.max_over_ranks(ms, "cuda")
+    value = replicas.whole_job_rate(world, steps, ms_max)
     ms_per_step = ms_max / steps
 
     # ---- e2e arm: pinned-host store, 8 slots, copies inside the timed region
@@ -336,13 +334,12 @@ def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1)
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    from paper_2609_18063_b200 import replicas
+    ms_max = replicas.max_over_ranks(ms, "cuda")
     after = store.stats()
     miss_bytes = (after["bytes_copied"] - base["bytes_copied"]) / n
     table_bytes = (after["table_updates"] - base["table_updates"]) * E * 4 / n
-    out = {"value": round(world * n / (float(t.item()) * 1e-3), 1), "unit": UNIT,
+    out = {"value": round(replicas.whole_job_rate(world, n, ms_max), 1), "unit": UNIT,
            "h2d_bytes_per_step": int(H * 2 + miss_bytes + table_bytes), "d2h_bytes_per_step": H * 4 + K * 4,
            "steps": n, "slots": cfg.n_slots,
            "misses_per_step": round((after["misses"] - base["misses"]) / n, 3),
