@@ -16,7 +16,7 @@
 // The LoRA delta is one more MMA k-step with A = B_lora rows and B = sigma * (A_lora . x).
 // Every pair's gate-weighted output goes to a [T*K][H] scratch and is reduced per token in the
 // order of its K choices, so y does not depend on how the groups were scheduled.
-#include "edg_mma.cuh"
+#include "edg_grouped.cuh"
 
 namespace edg {
 
@@ -28,32 +28,6 @@ constexpr int G_XS = G_KC * 2 + 64;   // bytes per token row of the staged activ
 constexpr int G_CS = G_KC / 2 + 16;   // bytes per weight row of the staged codes (padded: conflict-free 4-byte reads)
 constexpr int G_XSD = G_KD * 2 + 64;
 constexpr int G_CSD = G_KD / 2 + 16;
-
-struct GroupedParams {
-    const uint8_t* pool;
-    const int32_t* slots;     // [T][K] slots, or expert ids when table != null
-    const int32_t* table;
-    const int32_t* experts;
-    const float* gates;       // [T][K]
-    const uint16_t* x;        // [T][H] bf16
-    edg_lora lora;
-    void* y;
-    int32_t* status;
-    float* u_gu;              // [T][n_sets][2][rank]
-    float* h;                 // [T*K][I]
-    float* u_d;               // [T*K][rank]
-    float* o;                 // [T*K][H]
-    int32_t* pair_slot;       // [T*K]
-    int32_t* pair_ad;         // [T*K]
-    int32_t* counts;          // [n_slots]
-    int32_t* lists;           // [n_slots][T]
-    int32_t* tiles;           // [max tiles][2] = (slot, first position in the slot's list)
-    int32_t* n_tiles;
-    int T, H, I, E, K, group, rank, n_adapters, n_slots, out_dtype;
-    int ntok;                 // tokens per tile of this call (8 or 64)
-    float sigma;
-    RecordLayout L;
-};
 
 // The LoRA delta as one MMA k-step per 16 ranks: acc += Bl[rows][r] . (sigma * u[token][r]).
 // Bl: bf16 [..][rank], row pointers for rows g and g+8 of the tile; u row pointers per column tile.
@@ -481,7 +455,9 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     // few tokens per expert (batched decode): tiles of 8 tokens, the kernels are then bound by streaming
     // the weights; many (prefill): tiles of 64 so a dequantised weight tile is reused 8 times more
     const bool small = P <= 8 * d->n_slots;
-    p.ntok = small ? 8 : 64;
+    // large groups: tiles of 128 tokens on the tcgen05 path
+    const bool umma = !small && umma_grouped_supported(*d);
+    p.ntok = small ? 8 : (umma ? kUmmaTokens : 64);
     const int max_tiles = (P + p.ntok - 1) / p.ntok + d->n_slots;
     resolve_pairs_kernel<<<(P + 255) / 256, 256, 0, st>>>(p);
     build_lists_kernel<<<d->n_slots, kListWarps * 32, 0, st>>>(p);
@@ -499,10 +475,12 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
         EDG_CUDA_TRY(cudaFuncSetAttribute(grouped_down_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
         configured = true;
     }
-    if (small) grouped_gate_up_kernel<1><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
+    if (umma) EDG_CUDA_TRY(launch_umma_gate_up(p, max_tiles, st));
+    else if (small) grouped_gate_up_kernel<1><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
     else grouped_gate_up_kernel<8><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
     if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 1, st);
-    if (small) grouped_down_kernel<1><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
+    if (umma) EDG_CUDA_TRY(launch_umma_down(p, max_tiles, st));
+    else if (small) grouped_down_kernel<1><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
     else grouped_down_kernel<8><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
     const size_t n_out = (size_t)T * d->H;
     const int rb = (int)((n_out + 255) / 256);
