@@ -18,8 +18,10 @@
 // The 8 k values of a core row are kept in the order (k0,k4,k1,k5,k2,k6,k3,k7) in which the int4 codes
 // come out of a 32-bit word -- for A and B alike, so the dot product is unchanged.
 //
-// Warps 0-3 (128 threads, one weight row and one token each) dequantise / convert into a two-stage
-// ring and later run the epilogue; warp 4 allocates the tensor memory and its lane 0 issues the MMAs.
+// Warps 0-7 (two threads per weight row and per token, each covering half of a stage's k) dequantise /
+// convert into a two-stage ring, with the loads of the next chunk in flight while the current one is
+// processed, and later run the epilogue (each warp its 32 lanes of tensor memory, half of the token
+// columns); warp 8 allocates the tensor memory and its lane 0 issues the MMAs.
 // Every wait is bounded: a wait that gives up raises the status word and the kernel still frees its
 // tensor memory and returns.
 #include "edg_grouped.cuh"
@@ -34,7 +36,8 @@ constexpr uint32_t U_TILE = 128 * U_KC * 2;  // bytes of a [128 x 32] fp16 opera
 constexpr uint32_t U_LBO = 16 * 128;         // between k cores
 constexpr uint32_t U_SBO = 128;              // between row groups
 constexpr uint32_t U_SPIN = 1u << 22;
-constexpr int U_THREADS = 160;
+constexpr int U_PROD_WARPS = 8;
+constexpr int U_THREADS = (U_PROD_WARPS + 1) * 32;
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void bar_init(uint64_t* b, uint32_t count) {
@@ -140,15 +143,15 @@ __device__ __forceinline__ UmmaSmem carve(uint8_t* smem, int tiles_per_stage) {
 constexpr size_t umma_smem_bytes(int tiles_per_stage) { return (size_t)U_STAGES * tiles_per_stage * U_TILE + 64 + U_TN * 4; }
 
 // common prologue: pair list, barriers, tensor memory
-__device__ __forceinline__ uint32_t umma_begin(const GroupedParams& p, const UmmaSmem& S, int slot, int first, int cnt, int cols) {
+__device__ __forceinline__ uint32_t umma_begin(const GroupedParams& p, const UmmaSmem& S, int slot, int first, int cnt, int cols, int full_count) {
     const int tid = threadIdx.x, warp = tid >> 5;
     if (tid < U_TN) S.pair[tid] = tid < cnt ? p.lists[(size_t)slot * p.T + first + tid] : -1;
     if (tid == 0) {
-        for (int s = 0; s < U_STAGES; ++s) { bar_init(&S.full[s], 4); bar_init(&S.empty[s], 1); }
+        for (int s = 0; s < U_STAGES; ++s) { bar_init(&S.full[s], full_count); bar_init(&S.empty[s], 1); }
         bar_init(S.done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == U_PROD_WARPS) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(S.tptr)), "r"(cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -160,7 +163,7 @@ __device__ __forceinline__ uint32_t umma_begin(const GroupedParams& p, const Umm
 __device__ __forceinline__ void umma_end(uint32_t tmem, int cols) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if ((threadIdx.x >> 5) == 4)
+    if ((threadIdx.x >> 5) == U_PROD_WARPS)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(cols) : "memory");
 }
 // a producer warp has written its part of a stage
@@ -182,25 +185,33 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
     const int cnt = min(U_TN, p.counts[slot] - first);
     const int row0 = blockIdx.y * 128;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN);
+    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN, U_PROD_WARPS);
     const int n_chunks = p.H / U_KC;
     const int r_chunks = p.rank > 0 ? (p.rank + 31) / 32 : 0;          // adapter: chunks of up to 32 ranks
     const int gshift = 31 - __clz(p.group);
 
-    if (warp < 4) {
-        const int r = tid;                                           // weight row and token of this thread
+    if (warp < U_PROD_WARPS) {
+        const int r = tid & 127, half = tid >> 7;                    // weight row and token of this thread; its k cores 2 half, 2 half + 1
         const int pair = S.pair[r];
-        const uint16_t* xrow = pair >= 0 ? p.x + (size_t)(pair / p.K) * p.H : nullptr;
-        const uint8_t* cgp = rec + p.L.codes_gate, *cup = rec + p.L.codes_up;
-        uint4 cg = ld_stream16(cgp + code_off(p.H, row0 + r, 0)), cu = ld_stream16(cup + code_off(p.H, row0 + r, 0));
+        const uint16_t* xrow = pair >= 0 ? p.x + (size_t)(pair / p.K) * p.H + half * 16 : nullptr;
+        const uint8_t* cgp = rec + p.L.codes_gate + half * 8, *cup = rec + p.L.codes_up + half * 8;
+        auto ld8 = [](const uint8_t* q) { return *reinterpret_cast<const uint2*>(q); };
+        uint2 cg = ld8(cgp + code_off(p.H, row0 + r, 0)), cu = ld8(cup + code_off(p.H, row0 + r, 0));
+        uint4 xv[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) xv[j] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + j * 8) : make_uint4(0, 0, 0, 0);
         __half2 sg = __float2half2_rn(0.f), zg = sg, su = sg, zu = sg;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES;
             const uint32_t use = (uint32_t)(c / U_STAGES);
-            uint4 ng = cg, nu = cu;
-            if (c + 1 < n_chunks) {                                  // next chunk's codes: in flight during this one
-                ng = ld_stream16(cgp + code_off(p.H, row0 + r, c + 1));
-                nu = ld_stream16(cup + code_off(p.H, row0 + r, c + 1));
+            uint2 ng = cg, nu = cu;
+            uint4 nx[2] = {xv[0], xv[1]};
+            if (c + 1 < n_chunks) {                                  // next chunk's codes and activations: in flight during this one
+                ng = ld8(cgp + code_off(p.H, row0 + r, c + 1));
+                nu = ld8(cup + code_off(p.H, row0 + r, c + 1));
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    nx[j] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + (c + 1) * U_KC + j * 8) : make_uint4(0, 0, 0, 0);
             }
             if (((c * U_KC) & (p.group - 1)) == 0) {                 // a new group: its (scale, zero)
                 const int gi = (c * U_KC) >> gshift;
@@ -208,29 +219,26 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
                 const __half2 b = u32_as_h2(ld_stream4(rec + p.L.sz_up + sz_off(p.H, p.group, row0 + r, gi)));
                 sg = __low2half2(a); zg = __high2half2(a); su = __low2half2(b); zu = __high2half2(b);
             }
-            uint4 xv[4];
-#pragma unroll
-            for (int kc = 0; kc < 4; ++kc)
-                xv[kc] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + c * U_KC + kc * 8) : make_uint4(0, 0, 0, 0);
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);          // the MMAs that read this stage are done
             uint8_t* sb = S.stage[st];
-            const uint32_t wg[4] = {cg.x, cg.y, cg.z, cg.w}, wu[4] = {cu.x, cu.y, cu.z, cu.w};
+            const uint32_t wg[2] = {cg.x, cg.y}, wu[2] = {cu.x, cu.y};
 #pragma unroll
-            for (int kc = 0; kc < 4; ++kc) {
+            for (int j = 0; j < 2; ++j) {
+                const int kc = 2 * half + j;
                 uint4 hi, lo;
-                dequant_hi_lo(wg[kc], sg, zg, hi, lo);
+                dequant_hi_lo(wg[j], sg, zg, hi, lo);
                 *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = hi;
                 *reinterpret_cast<uint4*>(sb + 1 * U_TILE + core_off(r, kc)) = lo;
-                dequant_hi_lo(wu[kc], su, zu, hi, lo);
+                dequant_hi_lo(wu[j], su, zu, hi, lo);
                 *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = hi;
                 *reinterpret_cast<uint4*>(sb + 3 * U_TILE + core_off(r, kc)) = lo;
-                const uint4 v = xv[kc];
+                const uint4 v = xv[j];
                 const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
                                     bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
                 *reinterpret_cast<uint4*>(sb + 4 * U_TILE + core_off(r, kc)) = permute8(f);
             }
             stage_written(&S.full[st]);
-            cg = ng; cu = nu;
+            cg = ng; cu = nu; xv[0] = nx[0]; xv[1] = nx[1];
         }
         // the adapter as extra k: A = B_gate / B_up rows (fp16 of bf16), B = sigma * (A_gate x), sigma * (A_up x)
         if (r_chunks > 0) {
@@ -247,7 +255,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
-                for (int kc = 0; kc < 4; ++kc) {
+                for (int j = 0; j < 2; ++j) {
+                    const int kc = 2 * half + j;
                     const int j0 = rc * 32 + kc * 8, n = p.rank - j0;          // rank is a multiple of 8
                     uint4 ag = make_uint4(0, 0, 0, 0), au = ag;
                     if (n > 0) {
@@ -265,42 +274,63 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
         // ---- epilogue: h = silu(gate) * up, thread = weight row, 32 token columns at a time
         bar_wait(S.done, 0, p.status);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        for (int c0 = 0; c0 < cnt; c0 += 32) {
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        for (int c0 = half * (U_TN / 2); c0 < min(cnt, (half + 1) * (U_TN / 2)); c0 += 32) {
             uint32_t g[32], u[32];
             tmem_ld32(lane_addr + c0, g);
             tmem_ld32(lane_addr + U_TN + c0, u);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            // h goes out twice: fp32 per pair (for the down adapter's projection), and as the down
+            // kernel's B operand: fp16 value and fp16 residual in operand-tile order, this row being k
+            // index i = row0 + r of the tile's chunk i / 32 (k core (i % 32) / 8, slot of i % 8 in the
+            // (k0,k4,k1,k5,k2,k6,k3,k7) order)
+            const int i = row0 + r, e = i & 7;
+            uint8_t* hq = p.hq + ((size_t)tile * (p.I / 32) + (i >> 5)) * 2 * U_TILE + (size_t)((e < 4 ? 2 * e : 2 * (e - 4) + 1) * 2);
+            const int kc = (i & 31) >> 3;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const int pr = (c0 + j) < cnt ? S.pair[c0 + j] : -1;
-                if (pr >= 0) p.h[(size_t)pr * p.I + row0 + r] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+                if (pr >= 0) {
+                    const float hv = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+                    p.h[(size_t)pr * p.I + i] = hv;
+                    const __half hh = __float2half_rn(hv);
+                    const __half hl = __float2half_rn(hv - __half2float(hh));
+                    *reinterpret_cast<__half*>(hq + core_off(c0 + j, kc)) = hh;
+                    *reinterpret_cast<__half*>(hq + U_TILE + core_off(c0 + j, kc)) = hl;
+                }
             }
         }
     } else if (lane == 0) {
-        // ---- the MMA issuer
+        // ---- the MMA issuer.  Descriptors differ only in their address field: base + offset >> 4.
         const uint32_t idesc = umma_idesc((cnt + 15) & ~15);
-        for (int c = 0; c < n_chunks + r_chunks; ++c) {
+        const uint64_t d0 = umma_desc(s32(S.stage[0]));
+        constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (5 * U_TILE) >> 4;
+        const uint32_t tg = tmem, tu = tmem + U_TN;
+        for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES;
             bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t sb = s32(S.stage[st]);
-            const bool adapter = c >= n_chunks;
-            int ksteps = U_KC / 16;
-            if (adapter) ksteps = min(2, (p.rank - (c - n_chunks) * 32 + 15) / 16);
+            const uint64_t ds = d0 + st * kStage;
+#pragma unroll
+            for (int ks = 0; ks < U_KC / 16; ++ks) {
+                const uint64_t dk = ds + ks * kStep, db = dk + 4 * kTile;
+                umma(tg, dk, db, idesc, c > 0 || ks > 0);
+                umma(tg, dk + kTile, db, idesc, true);
+                umma(tu, dk + 2 * kTile, db, idesc, c > 0 || ks > 0);
+                umma(tu, dk + 3 * kTile, db, idesc, true);
+            }
+            umma_commit(&S.empty[st]);
+        }
+        for (int rc = 0; rc < r_chunks; ++rc) {
+            const int c = n_chunks + rc, st = c % U_STAGES;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t ds = d0 + st * kStage;
+            const int ksteps = min(2, (p.rank - rc * 32 + 15) / 16);
             for (int ks = 0; ks < ksteps; ++ks) {
-                const uint32_t ko = ks * 2 * U_LBO;
-                const bool fresh = c == 0 && ks == 0;
-                if (!adapter) {
-                    const uint64_t db = umma_desc(sb + 4 * U_TILE + ko);
-                    umma(tmem, umma_desc(sb + 0 * U_TILE + ko), db, idesc, !fresh);
-                    umma(tmem, umma_desc(sb + 1 * U_TILE + ko), db, idesc, true);
-                    umma(tmem + U_TN, umma_desc(sb + 2 * U_TILE + ko), db, idesc, !fresh);
-                    umma(tmem + U_TN, umma_desc(sb + 3 * U_TILE + ko), db, idesc, true);
-                } else {
-                    umma(tmem, umma_desc(sb + 0 * U_TILE + ko), umma_desc(sb + 4 * U_TILE + ko), idesc, true);
-                    umma(tmem + U_TN, umma_desc(sb + 2 * U_TILE + ko), umma_desc(sb + 1 * U_TILE + ko), idesc, true);
-                }
+                const uint64_t dk = ds + ks * kStep;
+                umma(tg, dk, dk + 4 * kTile, idesc, true);
+                umma(tu, dk + 2 * kTile, dk + kTile, idesc, true);
             }
             umma_commit(&S.empty[st]);
         }
@@ -310,7 +340,7 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
 }
 
 // ---------------------------------------------------------------- down
-// stage = [W hi][W lo][h hi][h lo]; tensor memory: 128 columns.  o = gate weight * (W h + sigma B (A h))
+// stage = [W hi][W lo][h hi][h lo] (h by bulk copy); tensor memory: 128 columns.  o = gate weight * (W h + sigma B (A h))
 __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p) {
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
@@ -321,44 +351,45 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
     const int cnt = min(U_TN, p.counts[slot] - first);
     const int row0 = blockIdx.y * 128;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, U_TN);
+    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, U_TN, U_PROD_WARPS + 1);
     const int n_chunks = p.I / U_KC;
     const int r_chunks = p.rank > 0 ? (p.rank + 31) / 32 : 0;
     const int gshift = 31 - __clz(p.group);
 
-    if (warp < 4) {
-        const int r = tid;
+    if (warp < U_PROD_WARPS) {
+        const int r = tid & 127, half = tid >> 7;
         const int pair = S.pair[r];
-        const float* hrow = pair >= 0 ? p.h + (size_t)pair * p.I : nullptr;
-        const uint8_t* cdp = rec + p.L.codes_down;
-        uint4 cd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + r, 0));
+        // the B operand (h as fp16 value and residual) was written in operand-tile order by the gate/up
+        // kernel: one bulk copy of 16 KB per chunk, counted on the stage's barrier
+        const uint8_t* hq = p.hq + (size_t)tile * (p.I / 32) * 2 * U_TILE;
+        const uint8_t* cdp = rec + p.L.codes_down + half * 8;
+        auto ld8 = [](const uint8_t* q) { return *reinterpret_cast<const uint2*>(q); };
+        uint2 cd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, 0));
         __half2 sd = __float2half2_rn(0.f), zd = sd;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES;
             const uint32_t use = (uint32_t)(c / U_STAGES);
-            uint4 nd = cd;
-            if (c + 1 < n_chunks) nd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + r, c + 1));
+            uint2 nd = cd;
+            if (c + 1 < n_chunks) nd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, c + 1));
             if (((c * U_KC) & (p.group - 1)) == 0) {
                 const __half2 a = u32_as_h2(ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + r, (c * U_KC) >> gshift)));
                 sd = __low2half2(a); zd = __high2half2(a);
             }
-            float4 hv[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                hv[q] = hrow != nullptr ? *reinterpret_cast<const float4*>(hrow + c * U_KC + q * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
             uint8_t* sb = S.stage[st];
-            const uint32_t wd[4] = {cd.x, cd.y, cd.z, cd.w};
+            if (tid == 0) {
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&S.full[st])), "r"(2 * U_TILE) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(s32(sb + 2 * U_TILE)), "l"(hq + (size_t)c * 2 * U_TILE), "r"(2 * U_TILE), "r"(s32(&S.full[st])) : "memory");
+            }
+            const uint32_t wd[2] = {cd.x, cd.y};
 #pragma unroll
-            for (int kc = 0; kc < 4; ++kc) {
+            for (int j = 0; j < 2; ++j) {
+                const int kc = 2 * half + j;
                 uint4 hi, lo;
-                dequant_hi_lo(wd[kc], sd, zd, hi, lo);
+                dequant_hi_lo(wd[j], sd, zd, hi, lo);
                 *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = hi;
                 *reinterpret_cast<uint4*>(sb + 1 * U_TILE + core_off(r, kc)) = lo;
-                const float4 a = hv[2 * kc], b = hv[2 * kc + 1];
-                const float f[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-                *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = permute8(f);
-                *reinterpret_cast<uint4*>(sb + 3 * U_TILE + core_off(r, kc)) = permute8_lo(f);
             }
             stage_written(&S.full[st]);
             cd = nd;
@@ -374,21 +405,23 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
-                for (int kc = 0; kc < 4; ++kc) {
+                for (int j = 0; j < 2; ++j) {
+                    const int kc = 2 * half + j;
                     const int j0 = rc * 32 + kc * 8, n = p.rank - j0;
                     uint4 a = make_uint4(0, 0, 0, 0);
                     if (n > 0) a = bf16x8_to_f16(*reinterpret_cast<const uint4*>(Bd + j0));
                     *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = a;
                     *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = f32x8_to_f16(ud != nullptr ? ud + j0 : nullptr, n, p.sigma);
                 }
+                if (tid == 0) bar_arrive(&S.full[st]);               // stands in for the bulk copy's arrival
                 stage_written(&S.full[st]);
             }
         }
         // ---- epilogue: o[pair][row] = gate weight * acc
         bar_wait(S.done, 0, p.status);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        for (int c0 = 0; c0 < cnt; c0 += 32) {
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        for (int c0 = half * (U_TN / 2); c0 < min(cnt, (half + 1) * (U_TN / 2)); c0 += 32) {
             uint32_t v[32];
             tmem_ld32(lane_addr + c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -400,25 +433,29 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
         }
     } else if (lane == 0) {
         const uint32_t idesc = umma_idesc((cnt + 15) & ~15);
-        for (int c = 0; c < n_chunks + r_chunks; ++c) {
+        const uint64_t d0 = umma_desc(s32(S.stage[0]));
+        constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (4 * U_TILE) >> 4;
+        for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES;
             bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t sb = s32(S.stage[st]);
-            const bool adapter = c >= n_chunks;
-            int ksteps = U_KC / 16;
-            if (adapter) ksteps = min(2, (p.rank - (c - n_chunks) * 32 + 15) / 16);
-            for (int ks = 0; ks < ksteps; ++ks) {
-                const uint32_t ko = ks * 2 * U_LBO;
-                const uint64_t whi = umma_desc(sb + 0 * U_TILE + ko), hhi = umma_desc(sb + 2 * U_TILE + ko);
-                if (!adapter) {
-                    umma(tmem, whi, hhi, idesc, !(c == 0 && ks == 0));
-                    umma(tmem, umma_desc(sb + 1 * U_TILE + ko), hhi, idesc, true);
-                    umma(tmem, whi, umma_desc(sb + 3 * U_TILE + ko), idesc, true);
-                } else {
-                    umma(tmem, whi, hhi, idesc, true);
-                }
+            const uint64_t ds = d0 + st * kStage;
+#pragma unroll
+            for (int ks = 0; ks < U_KC / 16; ++ks) {
+                const uint64_t whi = ds + ks * kStep, hhi = whi + 2 * kTile;
+                umma(tmem, whi, hhi, idesc, c > 0 || ks > 0);
+                umma(tmem, whi + kTile, hhi, idesc, true);
+                umma(tmem, whi, hhi + kTile, idesc, true);
             }
+            umma_commit(&S.empty[st]);
+        }
+        for (int rc = 0; rc < r_chunks; ++rc) {
+            const int c = n_chunks + rc, st = c % U_STAGES;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t ds = d0 + st * kStage;
+            const int ksteps = min(2, (p.rank - rc * 32 + 15) / 16);
+            for (int ks = 0; ks < ksteps; ++ks) umma(tmem, ds + ks * kStep, ds + ks * kStep + 2 * kTile, idesc, true);
             umma_commit(&S.empty[st]);
         }
         umma_commit(S.done);
