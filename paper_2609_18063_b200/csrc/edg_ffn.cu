@@ -52,50 +52,71 @@ __device__ __forceinline__ int resolve_adapter(const FfnParams& p, int tk) {
 }
 
 // ---------------------------------------------------------------- rank-r projections u = A . v
-// One warp per output.  phase 0: v = x (bf16), outputs u_gu[t][set][proj][j];
-//                       phase 1: v = h[t][k] (float), outputs u_d[t][k][j].
+// One warp per 8 outputs of one token (or pair): the vector is loaded once per sweep and used for the
+// 8 rows of A, whose loads are in flight together.
+//   phase 0: v = x (bf16), outputs u_gu[t][set][proj][j];  phase 1: v = h[t][k] (float), outputs u_d[t][k][j].
 __global__ void __launch_bounds__(256) lora_a_kernel(FfnParams p, int phase, int n_sets) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.y;
     const int r = p.rank;
+    const int g8 = (r + 7) / 8;                                  // groups of 8 outputs per (set, proj) or per pair
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     if (phase == 0) {
-        if (warp >= n_sets * 2 * r) return;
-        const int j = warp % r, proj = (warp / r) & 1, set = warp / (2 * r);
+        if (warp >= n_sets * 2 * g8) return;
+        const int jg = warp % g8, proj = (warp / g8) & 1, set = warp / (2 * g8);
         const int ad = p.n_adapters == 1 ? 0 : resolve_adapter(p, t * p.K + set);
         if (ad < 0) { if (lane == 0) atomicExch(p.status, EDG_E_RANGE); return; }
-        const uint16_t* A = reinterpret_cast<const uint16_t*>(proj ? p.lora.A_up : p.lora.A_gate) + ((size_t)ad * r + j) * p.H;
+        const uint16_t* A = reinterpret_cast<const uint16_t*>(proj ? p.lora.A_up : p.lora.A_gate) + ((size_t)ad * r + jg * 8) * p.H;
+        const int nj = min(8, r - jg * 8);
         const uint16_t* xv = p.x + (size_t)t * p.H;
-        float acc = 0.f;
         for (int c = lane * 8; c < p.H; c += 256) {
-            const uint4 a = *reinterpret_cast<const uint4*>(A + c);
             const uint4 b = *reinterpret_cast<const uint4*>(xv + c);
-            acc = fmaf(bf16_lo(a.x), bf16_lo(b.x), acc); acc = fmaf(bf16_hi(a.x), bf16_hi(b.x), acc);
-            acc = fmaf(bf16_lo(a.y), bf16_lo(b.y), acc); acc = fmaf(bf16_hi(a.y), bf16_hi(b.y), acc);
-            acc = fmaf(bf16_lo(a.z), bf16_lo(b.z), acc); acc = fmaf(bf16_hi(a.z), bf16_hi(b.z), acc);
-            acc = fmaf(bf16_lo(a.w), bf16_lo(b.w), acc); acc = fmaf(bf16_hi(a.w), bf16_hi(b.w), acc);
+            uint4 a[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] = *reinterpret_cast<const uint4*>(A + (size_t)min(u, nj - 1) * p.H + c);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                acc[u] = fmaf(bf16_lo(a[u].x), bf16_lo(b.x), acc[u]); acc[u] = fmaf(bf16_hi(a[u].x), bf16_hi(b.x), acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].y), bf16_lo(b.y), acc[u]); acc[u] = fmaf(bf16_hi(a[u].y), bf16_hi(b.y), acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].z), bf16_lo(b.z), acc[u]); acc[u] = fmaf(bf16_hi(a[u].z), bf16_hi(b.z), acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].w), bf16_lo(b.w), acc[u]); acc[u] = fmaf(bf16_hi(a[u].w), bf16_hi(b.w), acc[u]);
+            }
         }
-        acc = warp_sum(acc);
-        if (lane == 0) p.u_gu[(((size_t)t * n_sets + set) * 2 + proj) * r + j] = acc;
+        float* out = p.u_gu + (((size_t)t * n_sets + set) * 2 + proj) * r + jg * 8;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float v = warp_sum(acc[u]);
+            if (lane == 0 && u < nj) out[u] = v;
+        }
     } else {
-        if (warp >= p.K * r) return;
-        const int j = warp % r, k = warp / r;
+        if (warp >= p.K * g8) return;
+        const int jg = warp % g8, k = warp / g8;
         const int ad = resolve_adapter(p, t * p.K + k);
         if (ad < 0) { if (lane == 0) atomicExch(p.status, EDG_E_RANGE); return; }
-        const uint16_t* A = reinterpret_cast<const uint16_t*>(p.lora.A_down) + ((size_t)ad * r + j) * p.I;
+        const uint16_t* A = reinterpret_cast<const uint16_t*>(p.lora.A_down) + ((size_t)ad * r + jg * 8) * p.I;
+        const int nj = min(8, r - jg * 8);
         const float* hv = p.h + ((size_t)t * p.K + k) * p.I;
-        float acc = 0.f;
         for (int c = lane * 8; c < p.I; c += 256) {
-            const uint4 a = *reinterpret_cast<const uint4*>(A + c);
             const float4 h0 = *reinterpret_cast<const float4*>(hv + c);
             const float4 h1 = *reinterpret_cast<const float4*>(hv + c + 4);
-            acc = fmaf(bf16_lo(a.x), h0.x, acc); acc = fmaf(bf16_hi(a.x), h0.y, acc);
-            acc = fmaf(bf16_lo(a.y), h0.z, acc); acc = fmaf(bf16_hi(a.y), h0.w, acc);
-            acc = fmaf(bf16_lo(a.z), h1.x, acc); acc = fmaf(bf16_hi(a.z), h1.y, acc);
-            acc = fmaf(bf16_lo(a.w), h1.z, acc); acc = fmaf(bf16_hi(a.w), h1.w, acc);
+            uint4 a[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) a[u] = *reinterpret_cast<const uint4*>(A + (size_t)min(u, nj - 1) * p.I + c);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                acc[u] = fmaf(bf16_lo(a[u].x), h0.x, acc[u]); acc[u] = fmaf(bf16_hi(a[u].x), h0.y, acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].y), h0.z, acc[u]); acc[u] = fmaf(bf16_hi(a[u].y), h0.w, acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].z), h1.x, acc[u]); acc[u] = fmaf(bf16_hi(a[u].z), h1.y, acc[u]);
+                acc[u] = fmaf(bf16_lo(a[u].w), h1.z, acc[u]); acc[u] = fmaf(bf16_hi(a[u].w), h1.w, acc[u]);
+            }
         }
-        acc = warp_sum(acc);
-        if (lane == 0) p.u_d[((size_t)t * p.K + k) * r + j] = acc;
+        float* out = p.u_d + ((size_t)t * p.K + k) * r + jg * 8;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float v = warp_sum(acc[u]);
+            if (lane == 0 && u < nj) out[u] = v;
+        }
     }
 }
 
@@ -356,7 +377,8 @@ void launch_lora_a(const edg_layer_desc* d, const void* slots, const void* table
     p.H = d->H; p.I = d->I; p.E = d->E; p.K = d->K; p.group = d->group; p.rank = d->rank;
     p.n_adapters = d->n_adapters; p.n_slots = d->n_slots;
     const int n_sets = d->n_adapters == 1 ? 1 : d->K;
-    const int warps = phase == 0 ? n_sets * 2 * p.rank : p.K * p.rank;
+    const int g8 = (p.rank + 7) / 8;
+    const int warps = phase == 0 ? n_sets * 2 * g8 : p.K * g8;
     lora_a_kernel<<<dim3((warps + 7) / 8, T), 256, 0, st>>>(p, phase, n_sets);
 }
 

@@ -19,7 +19,7 @@
 // come out of a 32-bit word -- for A and B alike, so the dot product is unchanged.
 //
 // Warps 0-7 (two threads per weight row and per token, each covering half of a stage's k) dequantise /
-// convert into a two-stage ring, with the loads of the next chunk in flight while the current one is
+// convert into a ring of two (gate/up) or three (down) stages, with the loads of the next chunk in flight while the current one is
 // processed, and later run the epilogue (each warp its 32 lanes of tensor memory, half of the token
 // columns); warp 8 allocates the tensor memory and its lane 0 issues the MMAs.
 // Every wait is bounded: a wait that gives up raises the status word and the kernel still frees its
@@ -31,7 +31,7 @@ namespace {
 
 constexpr int U_TN = kUmmaTokens;            // token columns per tile
 constexpr int U_KC = 32;                     // k per stage
-constexpr int U_STAGES = 2;
+constexpr int U_STAGES_MAX = 3;
 constexpr uint32_t U_TILE = 128 * U_KC * 2;  // bytes of a [128 x 32] fp16 operand tile
 constexpr uint32_t U_LBO = 16 * 128;         // between k cores
 constexpr uint32_t U_SBO = 128;              // between row groups
@@ -122,32 +122,33 @@ __device__ __forceinline__ uint4 f32x8_to_f16(const float* src, int n, float sig
 }
 
 struct UmmaSmem {
-    uint8_t* stage[U_STAGES];
-    uint64_t* full;     // [U_STAGES] operands written (one arrival per producer warp)
-    uint64_t* empty;    // [U_STAGES] MMAs that read the stage have completed
+    uint8_t* stage[U_STAGES_MAX];
+    uint64_t* full;     // [stages] operands written (one arrival per producer warp)
+    uint64_t* empty;    // [stages] MMAs that read the stage have completed
     uint64_t* done;     // all MMAs of the tile have completed
     uint32_t* tptr;
     int* pair;          // [U_TN]
 };
-__device__ __forceinline__ UmmaSmem carve(uint8_t* smem, int tiles_per_stage) {
+__device__ __forceinline__ UmmaSmem carve(uint8_t* smem, int tiles_per_stage, int stages) {
     UmmaSmem S;
-    for (int s = 0; s < U_STAGES; ++s) S.stage[s] = smem + (size_t)s * tiles_per_stage * U_TILE;
-    uint8_t* o = smem + (size_t)U_STAGES * tiles_per_stage * U_TILE;
+    for (int s = 0; s < U_STAGES_MAX; ++s) S.stage[s] = smem + (size_t)(s < stages ? s : 0) * tiles_per_stage * U_TILE;
+    uint8_t* o = smem + (size_t)stages * tiles_per_stage * U_TILE;
     S.full = reinterpret_cast<uint64_t*>(o);
-    S.empty = S.full + U_STAGES;
-    S.done = S.empty + U_STAGES;
+    S.empty = S.full + U_STAGES_MAX;
+    S.done = S.empty + U_STAGES_MAX;
     S.tptr = reinterpret_cast<uint32_t*>(S.done + 1);
     S.pair = reinterpret_cast<int*>(S.tptr + 2);
     return S;
 }
-constexpr size_t umma_smem_bytes(int tiles_per_stage) { return (size_t)U_STAGES * tiles_per_stage * U_TILE + 64 + U_TN * 4; }
+constexpr size_t umma_smem_bytes(int tiles_per_stage, int stages) { return (size_t)stages * tiles_per_stage * U_TILE + 128 + U_TN * 4; }
+constexpr int U_STAGES_GU = 2, U_STAGES_D = 2;
 
 // common prologue: pair list, barriers, tensor memory
 __device__ __forceinline__ uint32_t umma_begin(const GroupedParams& p, const UmmaSmem& S, int slot, int first, int cnt, int cols, int full_count) {
     const int tid = threadIdx.x, warp = tid >> 5;
     if (tid < U_TN) S.pair[tid] = tid < cnt ? p.lists[(size_t)slot * p.T + first + tid] : -1;
     if (tid == 0) {
-        for (int s = 0; s < U_STAGES; ++s) { bar_init(&S.full[s], full_count); bar_init(&S.empty[s], 1); }
+        for (int s = 0; s < U_STAGES_MAX; ++s) { bar_init(&S.full[s], full_count); bar_init(&S.empty[s], 1); }
         bar_init(S.done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -176,14 +177,14 @@ __device__ __forceinline__ void stage_written(uint64_t* full) {
 // ---------------------------------------------------------------- gate/up
 // stage = [gate hi][gate lo][up hi][up lo][x]; tensor memory: gate in columns 0..127, up in 128..255
 __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParams p) {
-    const int tile = blockIdx.x;
+    const int tile = blockIdx.y;             // row blocks of a tile are neighbours in the grid: they share its activations in L2
     if (tile >= *p.n_tiles) return;
     extern __shared__ __align__(128) uint8_t smem[];
-    const UmmaSmem S = carve(smem, 5);
+    const UmmaSmem S = carve(smem, 5, U_STAGES_GU);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = p.tiles[2 * tile], first = p.tiles[2 * tile + 1];
     const int cnt = min(U_TN, p.counts[slot] - first);
-    const int row0 = blockIdx.y * 128;
+    const int row0 = blockIdx.x * 128;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
     const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN, U_PROD_WARPS);
     const int n_chunks = p.H / U_KC;
@@ -202,8 +203,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
         for (int j = 0; j < 2; ++j) xv[j] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + j * 8) : make_uint4(0, 0, 0, 0);
         __half2 sg = __float2half2_rn(0.f), zg = sg, su = sg, zu = sg;
         for (int c = 0; c < n_chunks; ++c) {
-            const int st = c % U_STAGES;
-            const uint32_t use = (uint32_t)(c / U_STAGES);
+            const int st = c % U_STAGES_GU;
+            const uint32_t use = (uint32_t)(c / U_STAGES_GU);
             uint2 ng = cg, nu = cu;
             uint4 nx[2] = {xv[0], xv[1]};
             if (c + 1 < n_chunks) {                                  // next chunk's codes and activations: in flight during this one
@@ -250,8 +251,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
             const uint16_t* Bg = reinterpret_cast<const uint16_t*>(p.lora.B_gate) + ((size_t)ad * p.I + row0 + r) * p.rank;
             const uint16_t* Bu = reinterpret_cast<const uint16_t*>(p.lora.B_up) + ((size_t)ad * p.I + row0 + r) * p.rank;
             for (int rc = 0; rc < r_chunks; ++rc) {
-                const int c = n_chunks + rc, st = c % U_STAGES;
-                const uint32_t use = (uint32_t)(c / U_STAGES);
+                const int c = n_chunks + rc, st = c % U_STAGES_GU;
+                const uint32_t use = (uint32_t)(c / U_STAGES_GU);
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
@@ -307,8 +308,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
         constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (5 * U_TILE) >> 4;
         const uint32_t tg = tmem, tu = tmem + U_TN;
         for (int c = 0; c < n_chunks; ++c) {
-            const int st = c % U_STAGES;
-            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            const int st = c % U_STAGES_GU;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES_GU) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ds = d0 + st * kStage;
 #pragma unroll
@@ -322,8 +323,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
             umma_commit(&S.empty[st]);
         }
         for (int rc = 0; rc < r_chunks; ++rc) {
-            const int c = n_chunks + rc, st = c % U_STAGES;
-            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            const int c = n_chunks + rc, st = c % U_STAGES_GU;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES_GU) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ds = d0 + st * kStage;
             const int ksteps = min(2, (p.rank - rc * 32 + 15) / 16);
@@ -342,14 +343,14 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
 // ---------------------------------------------------------------- down
 // stage = [W hi][W lo][h hi][h lo] (h by bulk copy); tensor memory: 128 columns.  o = gate weight * (W h + sigma B (A h))
 __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p) {
-    const int tile = blockIdx.x;
+    const int tile = blockIdx.y;             // row blocks of a tile are neighbours in the grid: they share its activations in L2
     if (tile >= *p.n_tiles) return;
     extern __shared__ __align__(128) uint8_t smem[];
-    const UmmaSmem S = carve(smem, 4);
+    const UmmaSmem S = carve(smem, 4, U_STAGES_D);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = p.tiles[2 * tile], first = p.tiles[2 * tile + 1];
     const int cnt = min(U_TN, p.counts[slot] - first);
-    const int row0 = blockIdx.y * 128;
+    const int row0 = blockIdx.x * 128;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
     const uint32_t tmem = umma_begin(p, S, slot, first, cnt, U_TN, U_PROD_WARPS + 1);
     const int n_chunks = p.I / U_KC;
@@ -367,8 +368,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
         uint2 cd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, 0));
         __half2 sd = __float2half2_rn(0.f), zd = sd;
         for (int c = 0; c < n_chunks; ++c) {
-            const int st = c % U_STAGES;
-            const uint32_t use = (uint32_t)(c / U_STAGES);
+            const int st = c % U_STAGES_D;
+            const uint32_t use = (uint32_t)(c / U_STAGES_D);
             uint2 nd = cd;
             if (c + 1 < n_chunks) nd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, c + 1));
             if (((c * U_KC) & (p.group - 1)) == 0) {
@@ -400,8 +401,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             const float* ud = pair >= 0 ? p.u_d + (size_t)pair * p.rank : nullptr;
             const uint16_t* Bd = reinterpret_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + row0 + r) * p.rank;
             for (int rc = 0; rc < r_chunks; ++rc) {
-                const int c = n_chunks + rc, st = c % U_STAGES;
-                const uint32_t use = (uint32_t)(c / U_STAGES);
+                const int c = n_chunks + rc, st = c % U_STAGES_D;
+                const uint32_t use = (uint32_t)(c / U_STAGES_D);
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
@@ -436,8 +437,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
         const uint64_t d0 = umma_desc(s32(S.stage[0]));
         constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (4 * U_TILE) >> 4;
         for (int c = 0; c < n_chunks; ++c) {
-            const int st = c % U_STAGES;
-            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            const int st = c % U_STAGES_D;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES_D) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ds = d0 + st * kStage;
 #pragma unroll
@@ -450,8 +451,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             umma_commit(&S.empty[st]);
         }
         for (int rc = 0; rc < r_chunks; ++rc) {
-            const int c = n_chunks + rc, st = c % U_STAGES;
-            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES) & 1, p.status);
+            const int c = n_chunks + rc, st = c % U_STAGES_D;
+            bar_wait(&S.full[st], (uint32_t)(c / U_STAGES_D) & 1, p.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ds = d0 + st * kStage;
             const int ksteps = min(2, (p.rank - rc * 32 + 15) / 16);
@@ -472,22 +473,22 @@ bool umma_grouped_supported(const edg_layer_desc& d) {
 cudaError_t launch_umma_gate_up(const GroupedParams& p, int max_tiles, cudaStream_t st) {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(umma_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(5));
+        cudaError_t e = cudaFuncSetAttribute(umma_gate_up_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(5, U_STAGES_GU));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    umma_gate_up_kernel<<<dim3(max_tiles, p.I / 128), U_THREADS, umma_smem_bytes(5), st>>>(p);
+    umma_gate_up_kernel<<<dim3(p.I / 128, max_tiles), U_THREADS, umma_smem_bytes(5, U_STAGES_GU), st>>>(p);
     return cudaGetLastError();
 }
 
 cudaError_t launch_umma_down(const GroupedParams& p, int max_tiles, cudaStream_t st) {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(4));
+        cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(4, U_STAGES_D));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    umma_down_kernel<<<dim3(max_tiles, p.H / 128), U_THREADS, umma_smem_bytes(4), st>>>(p);
+    umma_down_kernel<<<dim3(p.H / 128, max_tiles), U_THREADS, umma_smem_bytes(4, U_STAGES_D), st>>>(p);
     return cudaGetLastError();
 }
 
