@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def _ffn_tokens(L, d, X_bits, inds, gates, T, use_table=True):
     if L.ws.numel() < edg.ffn_workspace_bytes(d, T):
         L.ws = layer_io.new_workspace(d, T)
-    L.ws[:256].zero_()
+    L.ws[:512].zero_()
     y = out_tensor(d, T)
     table = torch.arange(d.E, dtype=torch.int32, device="cuda") if use_table else None
     edg.moe_expert_ffn_int4_lora(d, L.pool, table, T, inds, inds, gates, x_dev(X_bits), L.lora, y, L.ws)
@@ -85,6 +85,36 @@ def test_prefill_cfg5_shape_reduced_tokens():
     assert np.isfinite(Y).all()
 
 
+def test_prefill_cfg5_full_size_sampled_tokens():
+    """The full 4096-token prefill in the launch configuration the benchmark times (tiles of 128
+    tokens on the tcgen05 path; the popular experts span many tiles, the unpopular ones a ragged
+    fraction of one).  The oracle computes sampled tokens one by one; every output must be finite."""
+    L = device_layer("cfg2")
+    cfg = synth.CONFIGS["cfg5"]
+    T, K, E = cfg.T, cfg.K, cfg.E
+    assert T == 4096
+    X = synth.hidden_states(cfg, T, stream=34)
+    logits = synth.zipf_router_logits(cfg, T)
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    edg.softmax_topk_rows(L.desc, torch.from_numpy(logits).cuda(), T, inds, gates)
+    torch.cuda.synchronize()
+    inds_h, gates_h = inds.cpu().numpy(), gates.cpu().numpy()
+    counts = np.bincount(inds_h.ravel(), minlength=E)
+    assert counts.max() > 8 * 128 and counts.min() < 128          # many tiles for some experts, a partial tile for others
+    Y = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    assert np.isfinite(Y).all()
+    rng = np.random.default_rng(3)
+    # tokens routed to the most and to the least popular expert, plus a random sample and both ends
+    hot, cold = int(np.argmax(counts)), int(np.argmin(np.where(counts > 0, counts, 1 << 30)))
+    pick = {0, T - 1, int(np.nonzero((inds_h == hot).any(axis=1))[0][-1]), int(np.nonzero((inds_h == cold).any(axis=1))[0][0])}
+    pick |= set(rng.choice(T, 12, replace=False).tolist())
+    _check_tokens(L, X, inds_h, gates_h, Y, sorted(pick))
+    # a second run is bit-identical (fixed reduction order, no atomics on the data path)
+    Y2 = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    assert np.array_equal(Y, Y2)
+
+
 def test_grouped_reduces_to_the_decode_path_and_handles_per_expert_adapters():
     L = device_layer("cfg1", 16)                  # per-expert adapters
     cfg = L.cfg
@@ -104,7 +134,7 @@ def test_grouped_reduces_to_the_decode_path_and_handles_per_expert_adapters():
     assert orc.max_abs(y1[0], Y[0]) <= TOL_MAX_ABS and orc.rel_l2(y1[0], Y[0]) <= TOL_REL_L2
     # an out-of-range expert in one pair is skipped and flagged, the other tokens are untouched
     bad = inds_h.copy(); bad[5, 1] = cfg.E
-    L.ws[:256].zero_()
+    L.ws[:512].zero_()
     y = out_tensor(L.desc, T)
     edg.moe_expert_ffn_int4_lora(L.desc, L.pool, torch.arange(cfg.E, dtype=torch.int32, device="cuda"), T,
                                  torch.from_numpy(bad).cuda(), None, gates, x_dev(X), L.lora, y, L.ws)
