@@ -341,39 +341,38 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
 }
 
 // ---------------------------------------------------------------- down
-// stage = [W hi][W lo][h hi][h lo] (h by bulk copy); tensor memory: 128 columns.  o = gate weight * (W h + sigma B (A h))
+// A CTA covers 256 output rows (two accumulators of 128 columns in tensor memory) for the tile's tokens:
+// stage = [W0 hi][W0 lo][W1 hi][W1 lo][h hi][h lo], the h tiles arriving by one bulk copy per chunk
+// (written in operand order by the gate/up kernel), thread t dequantising row t of the 256.
+// o = gate weight * (W h + sigma B (A h))
 __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p) {
     const int tile = blockIdx.y;             // row blocks of a tile are neighbours in the grid: they share its activations in L2
     if (tile >= *p.n_tiles) return;
     extern __shared__ __align__(128) uint8_t smem[];
-    const UmmaSmem S = carve(smem, 4, U_STAGES_D);
+    const UmmaSmem S = carve(smem, 6, U_STAGES_D);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int slot = p.tiles[2 * tile], first = p.tiles[2 * tile + 1];
     const int cnt = min(U_TN, p.counts[slot] - first);
-    const int row0 = blockIdx.x * 128;
+    const int row0 = blockIdx.x * 256;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, U_TN, U_PROD_WARPS + 1);
+    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN, U_PROD_WARPS + 1);
     const int n_chunks = p.I / U_KC;
     const int r_chunks = p.rank > 0 ? (p.rank + 31) / 32 : 0;
     const int gshift = 31 - __clz(p.group);
 
     if (warp < U_PROD_WARPS) {
-        const int r = tid & 127, half = tid >> 7;
-        const int pair = S.pair[r];
-        // the B operand (h as fp16 value and residual) was written in operand-tile order by the gate/up
-        // kernel: one bulk copy of 16 KB per chunk, counted on the stage's barrier
+        const int r = tid & 127, m = tid >> 7;                       // row r of half m: output row row0 + tid
         const uint8_t* hq = p.hq + (size_t)tile * (p.I / 32) * 2 * U_TILE;
-        const uint8_t* cdp = rec + p.L.codes_down + half * 8;
-        auto ld8 = [](const uint8_t* q) { return *reinterpret_cast<const uint2*>(q); };
-        uint2 cd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, 0));
+        const uint8_t* cdp = rec + p.L.codes_down;
+        uint4 cd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + tid, 0));
         __half2 sd = __float2half2_rn(0.f), zd = sd;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES_D;
             const uint32_t use = (uint32_t)(c / U_STAGES_D);
-            uint2 nd = cd;
-            if (c + 1 < n_chunks) nd = ld8(cdp + down_code_off(p.H, p.I, row0 + r, c + 1));
+            uint4 nd = cd;
+            if (c + 1 < n_chunks) nd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + tid, c + 1));
             if (((c * U_KC) & (p.group - 1)) == 0) {
-                const __half2 a = u32_as_h2(ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + r, (c * U_KC) >> gshift)));
+                const __half2 a = u32_as_h2(ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + tid, (c * U_KC) >> gshift)));
                 sd = __low2half2(a); zd = __high2half2(a);
             }
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
@@ -381,16 +380,15 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             if (tid == 0) {
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&S.full[st])), "r"(2 * U_TILE) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(s32(sb + 2 * U_TILE)), "l"(hq + (size_t)c * 2 * U_TILE), "r"(2 * U_TILE), "r"(s32(&S.full[st])) : "memory");
+                             ::"r"(s32(sb + 4 * U_TILE)), "l"(hq + (size_t)c * 2 * U_TILE), "r"(2 * U_TILE), "r"(s32(&S.full[st])) : "memory");
             }
-            const uint32_t wd[2] = {cd.x, cd.y};
+            const uint32_t wd[4] = {cd.x, cd.y, cd.z, cd.w};
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int kc = 2 * half + j;
+            for (int kc = 0; kc < 4; ++kc) {
                 uint4 hi, lo;
-                dequant_hi_lo(wd[j], sd, zd, hi, lo);
-                *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = hi;
-                *reinterpret_cast<uint4*>(sb + 1 * U_TILE + core_off(r, kc)) = lo;
+                dequant_hi_lo(wd[kc], sd, zd, hi, lo);
+                *reinterpret_cast<uint4*>(sb + (2 * m) * U_TILE + core_off(r, kc)) = hi;
+                *reinterpret_cast<uint4*>(sb + (2 * m + 1) * U_TILE + core_off(r, kc)) = lo;
             }
             stage_written(&S.full[st]);
             cd = nd;
@@ -398,44 +396,44 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
         if (r_chunks > 0) {
             const int first_pair = S.pair[0];
             const int ad = first_pair >= 0 ? p.pair_ad[first_pair] : 0;
-            const float* ud = pair >= 0 ? p.u_d + (size_t)pair * p.rank : nullptr;
-            const uint16_t* Bd = reinterpret_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + row0 + r) * p.rank;
+            const int pair = S.pair[r];
+            const float* ud = (m == 0 && pair >= 0) ? p.u_d + (size_t)pair * p.rank : nullptr;
+            const uint16_t* Bd = reinterpret_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + row0 + tid) * p.rank;
             for (int rc = 0; rc < r_chunks; ++rc) {
                 const int c = n_chunks + rc, st = c % U_STAGES_D;
                 const uint32_t use = (uint32_t)(c / U_STAGES_D);
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int kc = 2 * half + j;
+                for (int kc = 0; kc < 4; ++kc) {
                     const int j0 = rc * 32 + kc * 8, n = p.rank - j0;
                     uint4 a = make_uint4(0, 0, 0, 0);
                     if (n > 0) a = bf16x8_to_f16(*reinterpret_cast<const uint4*>(Bd + j0));
-                    *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = a;
-                    *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = f32x8_to_f16(ud != nullptr ? ud + j0 : nullptr, n, p.sigma);
+                    *reinterpret_cast<uint4*>(sb + (2 * m) * U_TILE + core_off(r, kc)) = a;
+                    if (m == 0) *reinterpret_cast<uint4*>(sb + 4 * U_TILE + core_off(r, kc)) = f32x8_to_f16(ud != nullptr ? ud + j0 : nullptr, n, p.sigma);
                 }
                 if (tid == 0) bar_arrive(&S.full[st]);               // stands in for the bulk copy's arrival
                 stage_written(&S.full[st]);
             }
         }
-        // ---- epilogue: o[pair][row] = gate weight * acc
+        // ---- epilogue: o[pair][row] = gate weight * acc; thread t = row t, accumulator t / 128
         bar_wait(S.done, 0, p.status);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        for (int c0 = half * (U_TN / 2); c0 < min(cnt, (half + 1) * (U_TN / 2)); c0 += 32) {
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + m * U_TN;
+        for (int c0 = 0; c0 < cnt; c0 += 32) {
             uint32_t v[32];
             tmem_ld32(lane_addr + c0, v);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 const int pr = (c0 + j) < cnt ? S.pair[c0 + j] : -1;
-                if (pr >= 0) p.o[(size_t)pr * p.H + row0 + r] = p.gates[pr] * __uint_as_float(v[j]);
+                if (pr >= 0) p.o[(size_t)pr * p.H + row0 + tid] = p.gates[pr] * __uint_as_float(v[j]);
             }
         }
     } else if (lane == 0) {
         const uint32_t idesc = umma_idesc((cnt + 15) & ~15);
         const uint64_t d0 = umma_desc(s32(S.stage[0]));
-        constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (4 * U_TILE) >> 4;
+        constexpr uint64_t kTile = U_TILE >> 4, kStep = (2 * U_LBO) >> 4, kStage = (6 * U_TILE) >> 4;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES_D;
             bar_wait(&S.full[st], (uint32_t)(c / U_STAGES_D) & 1, p.status);
@@ -443,10 +441,14 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             const uint64_t ds = d0 + st * kStage;
 #pragma unroll
             for (int ks = 0; ks < U_KC / 16; ++ks) {
-                const uint64_t whi = ds + ks * kStep, hhi = whi + 2 * kTile;
-                umma(tmem, whi, hhi, idesc, c > 0 || ks > 0);
-                umma(tmem, whi + kTile, hhi, idesc, true);
-                umma(tmem, whi, hhi + kTile, idesc, true);
+                const uint64_t w0 = ds + ks * kStep, hhi = w0 + 4 * kTile;
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {
+                    const uint64_t whi = w0 + 2 * m * kTile;
+                    umma(tmem + m * U_TN, whi, hhi, idesc, c > 0 || ks > 0);
+                    umma(tmem + m * U_TN, whi + kTile, hhi, idesc, true);
+                    umma(tmem + m * U_TN, whi, hhi + kTile, idesc, true);
+                }
             }
             umma_commit(&S.empty[st]);
         }
@@ -456,18 +458,22 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint64_t ds = d0 + st * kStage;
             const int ksteps = min(2, (p.rank - rc * 32 + 15) / 16);
-            for (int ks = 0; ks < ksteps; ++ks) umma(tmem, ds + ks * kStep, ds + ks * kStep + 2 * kTile, idesc, true);
+            for (int ks = 0; ks < ksteps; ++ks) {
+                const uint64_t w0 = ds + ks * kStep;
+                umma(tmem, w0, w0 + 4 * kTile, idesc, true);
+                umma(tmem + U_TN, w0 + 2 * kTile, w0 + 4 * kTile, idesc, true);
+            }
             umma_commit(&S.empty[st]);
         }
         umma_commit(S.done);
     }
-    umma_end(tmem, U_TN);
+    umma_end(tmem, 2 * U_TN);
 }
 
 }  // namespace
 
 bool umma_grouped_supported(const edg_layer_desc& d) {
-    return d.H % 128 == 0 && d.I % 128 == 0 && (d.group & (d.group - 1)) == 0 && d.group >= 32 && d.rank % 8 == 0;
+    return d.H % 256 == 0 && d.I % 128 == 0 && (d.group & (d.group - 1)) == 0 && d.group >= 32 && d.rank % 8 == 0;
 }
 
 cudaError_t launch_umma_gate_up(const GroupedParams& p, int max_tiles, cudaStream_t st) {
@@ -484,11 +490,11 @@ cudaError_t launch_umma_gate_up(const GroupedParams& p, int max_tiles, cudaStrea
 cudaError_t launch_umma_down(const GroupedParams& p, int max_tiles, cudaStream_t st) {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(4, U_STAGES_D));
+        cudaError_t e = cudaFuncSetAttribute(umma_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)umma_smem_bytes(6, U_STAGES_D));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    umma_down_kernel<<<dim3(p.H / 128, max_tiles), U_THREADS, umma_smem_bytes(4, U_STAGES_D), st>>>(p);
+    umma_down_kernel<<<dim3(p.H / 256, max_tiles), U_THREADS, umma_smem_bytes(6, U_STAGES_D), st>>>(p);
     return cudaGetLastError();
 }
 
