@@ -102,6 +102,7 @@ struct WorkspaceLayout {
     size_t tiles;     // [T*K/8 + n_slots][2] int32 : (slot, first position) of every tile of 8 or 64 pairs
     size_t lists;     // [n_slots][T] int32         : pairs of every slot, ascending
     size_t hq;        // [T*K/128 + n_slots][I/32][2][128 x 32] fp16: h of every 128-token tile as tensor-core operand tiles (value, residual)
+    size_t xq;        // [T*K/128 + n_slots][H/32][128 x 32] fp16: the gathered token states of every tile as operand tiles
     size_t bytes;
 };
 
@@ -120,7 +121,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     const size_t one_set = (size_t)kDownSlices * d.K * d.H * sizeof(float);
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);
-    W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = W.hq = end;
+    W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = W.hq = W.xq = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;
         W.o = end;                 end = round_up(W.o + P * d.H * sizeof(float), 256);
@@ -131,6 +132,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
         W.tiles = end;             end = round_up(W.tiles + (P / 8 + 1 + d.n_slots) * 8, 256);
         W.lists = end;             end = round_up(W.lists + (size_t)d.n_slots * T * 4, 256);
         W.hq = end;                end = round_up(W.hq + ((P + 127) / 128 + d.n_slots) * (size_t)(d.I / 32) * 2 * 8192, 256);
+        W.xq = end;                end = round_up(W.xq + ((P + 127) / 128 + d.n_slots) * (size_t)(d.H / 32) * 8192, 256);
     }
     W.bytes = end;
     return W;

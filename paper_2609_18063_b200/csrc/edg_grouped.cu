@@ -446,6 +446,7 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     p.tiles = reinterpret_cast<int32_t*>(ws + W.tiles);
     p.lists = reinterpret_cast<int32_t*>(ws + W.lists);
     p.hq = ws + W.hq;
+    p.xq = ws + W.xq;
     p.T = T; p.H = d->H; p.I = d->I; p.E = d->E; p.K = d->K; p.group = d->group;
     p.rank = has_lora ? d->rank : 0;
     p.n_adapters = d->n_adapters; p.n_slots = d->n_slots; p.out_dtype = d->out_dtype;

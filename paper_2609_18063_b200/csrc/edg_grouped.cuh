@@ -27,6 +27,7 @@ struct GroupedParams {
     int32_t* tiles;           // [max tiles][2] = (slot, first position in the slot's list)
     int32_t* n_tiles;
     uint8_t* hq;              // h of every 128-token tile as fp16 operand tiles (tcgen05 path)
+    uint8_t* xq;              // the gathered token states of every tile as fp16 operand tiles (tcgen05 path)
     int T, H, I, E, K, group, rank, n_adapters, n_slots, out_dtype;
     int ntok;                 // tokens per tile of this call (8, 64 or 128)
     float sigma;

@@ -174,8 +174,35 @@ __device__ __forceinline__ void stage_written(uint64_t* full) {
     if ((threadIdx.x & 31) == 0) bar_arrive(full);
 }
 
+// ---------------------------------------------------------------- token states as operand tiles
+// xq[tile][chunk of 32 k][128 tokens x 32 k]: thread = (token of the tile, k core); the four row blocks
+// of a tile then fetch every chunk with one bulk copy instead of gathering it again.
+__global__ void __launch_bounds__(256) umma_gather_x_kernel(GroupedParams p) {
+    const int tile = blockIdx.y;
+    if (tile >= *p.n_tiles) return;
+    const int slot = p.tiles[2 * tile], first = p.tiles[2 * tile + 1];
+    const int cnt = min(U_TN, p.counts[slot] - first);
+    const int cores = p.H / 8;                                   // 16-byte pieces per token
+    uint8_t* out = p.xq + (size_t)tile * (p.H / 32) * U_TILE;
+    // consecutive threads take consecutive tokens of one k core: their 16-byte pieces are adjacent
+    // in the operand tile (coalesced writes); the reads are 16 bytes from 128 different rows
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < U_TN * cores; i += gridDim.x * blockDim.x) {
+        const int tok = i % U_TN, kcg = i / U_TN;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (tok < cnt) {
+            const int pair = p.lists[(size_t)slot * p.T + first + tok];
+            const uint4 raw = *reinterpret_cast<const uint4*>(p.x + (size_t)(pair / p.K) * p.H + kcg * 8);
+            const float f[8] = {bf16_lo(raw.x), bf16_hi(raw.x), bf16_lo(raw.y), bf16_hi(raw.y),
+                                bf16_lo(raw.z), bf16_hi(raw.z), bf16_lo(raw.w), bf16_hi(raw.w)};
+            v = permute8(f);
+        }
+        *reinterpret_cast<uint4*>(out + (size_t)(kcg >> 2) * U_TILE + core_off(tok, kcg & 3)) = v;
+    }
+}
+
 // ---------------------------------------------------------------- gate/up
-// stage = [gate hi][gate lo][up hi][up lo][x]; tensor memory: gate in columns 0..127, up in 128..255
+// stage = [gate hi][gate lo][up hi][up lo][x] (x by one bulk copy per chunk); tensor memory: gate in
+// columns 0..127, up in 128..255.  Thread t dequantises row t % 128 of gate (t < 128) or up.
 __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParams p) {
     const int tile = blockIdx.y;             // row blocks of a tile are neighbours in the grid: they share its activations in L2
     if (tile >= *p.n_tiles) return;
@@ -186,89 +213,69 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
     const int cnt = min(U_TN, p.counts[slot] - first);
     const int row0 = blockIdx.x * 128;
     const uint8_t* rec = p.pool + (size_t)slot * p.L.bytes;
-    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN, U_PROD_WARPS);
+    const uint32_t tmem = umma_begin(p, S, slot, first, cnt, 2 * U_TN, U_PROD_WARPS + 1);
     const int n_chunks = p.H / U_KC;
     const int r_chunks = p.rank > 0 ? (p.rank + 31) / 32 : 0;          // adapter: chunks of up to 32 ranks
     const int gshift = 31 - __clz(p.group);
 
     if (warp < U_PROD_WARPS) {
-        const int r = tid & 127, half = tid >> 7;                    // weight row and token of this thread; its k cores 2 half, 2 half + 1
+        const int r = tid & 127, half = tid >> 7;                    // weight row; matrix (0 gate, 1 up) and, in the epilogue, half of the columns
         const int pair = S.pair[r];
-        const uint16_t* xrow = pair >= 0 ? p.x + (size_t)(pair / p.K) * p.H + half * 16 : nullptr;
-        const uint8_t* cgp = rec + p.L.codes_gate + half * 8, *cup = rec + p.L.codes_up + half * 8;
-        auto ld8 = [](const uint8_t* q) { return *reinterpret_cast<const uint2*>(q); };
-        uint2 cg = ld8(cgp + code_off(p.H, row0 + r, 0)), cu = ld8(cup + code_off(p.H, row0 + r, 0));
-        uint4 xv[2];
-#pragma unroll
-        for (int j = 0; j < 2; ++j) xv[j] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + j * 8) : make_uint4(0, 0, 0, 0);
-        __half2 sg = __float2half2_rn(0.f), zg = sg, su = sg, zu = sg;
+        const uint8_t* xq = p.xq + (size_t)tile * (p.H / 32) * U_TILE;
+        const uint8_t* cp = rec + (half ? p.L.codes_up : p.L.codes_gate);
+        const uint8_t* zp = rec + (half ? p.L.sz_up : p.L.sz_gate);
+        uint4 cw = ld_stream16(cp + code_off(p.H, row0 + r, 0));
+        __half2 sc = __float2half2_rn(0.f), zr = sc;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES_GU;
             const uint32_t use = (uint32_t)(c / U_STAGES_GU);
-            uint2 ng = cg, nu = cu;
-            uint4 nx[2] = {xv[0], xv[1]};
-            if (c + 1 < n_chunks) {                                  // next chunk's codes and activations: in flight during this one
-                ng = ld8(cgp + code_off(p.H, row0 + r, c + 1));
-                nu = ld8(cup + code_off(p.H, row0 + r, c + 1));
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-                    nx[j] = xrow != nullptr ? *reinterpret_cast<const uint4*>(xrow + (c + 1) * U_KC + j * 8) : make_uint4(0, 0, 0, 0);
-            }
+            uint4 nw = cw;
+            if (c + 1 < n_chunks) nw = ld_stream16(cp + code_off(p.H, row0 + r, c + 1));   // in flight during this chunk
             if (((c * U_KC) & (p.group - 1)) == 0) {                 // a new group: its (scale, zero)
-                const int gi = (c * U_KC) >> gshift;
-                const __half2 a = u32_as_h2(ld_stream4(rec + p.L.sz_gate + sz_off(p.H, p.group, row0 + r, gi)));
-                const __half2 b = u32_as_h2(ld_stream4(rec + p.L.sz_up + sz_off(p.H, p.group, row0 + r, gi)));
-                sg = __low2half2(a); zg = __high2half2(a); su = __low2half2(b); zu = __high2half2(b);
+                const __half2 a = u32_as_h2(ld_stream4(zp + sz_off(p.H, p.group, row0 + r, (c * U_KC) >> gshift)));
+                sc = __low2half2(a); zr = __high2half2(a);
             }
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);          // the MMAs that read this stage are done
             uint8_t* sb = S.stage[st];
-            const uint32_t wg[2] = {cg.x, cg.y}, wu[2] = {cu.x, cu.y};
+            if (tid == 0) {
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(&S.full[st])), "r"(U_TILE) : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(s32(sb + 4 * U_TILE)), "l"(xq + (size_t)c * U_TILE), "r"(U_TILE), "r"(s32(&S.full[st])) : "memory");
+            }
+            const uint32_t w[4] = {cw.x, cw.y, cw.z, cw.w};
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                const int kc = 2 * half + j;
+            for (int kc = 0; kc < 4; ++kc) {
                 uint4 hi, lo;
-                dequant_hi_lo(wg[j], sg, zg, hi, lo);
-                *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = hi;
-                *reinterpret_cast<uint4*>(sb + 1 * U_TILE + core_off(r, kc)) = lo;
-                dequant_hi_lo(wu[j], su, zu, hi, lo);
-                *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = hi;
-                *reinterpret_cast<uint4*>(sb + 3 * U_TILE + core_off(r, kc)) = lo;
-                const uint4 v = xv[j];
-                const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
-                                    bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
-                *reinterpret_cast<uint4*>(sb + 4 * U_TILE + core_off(r, kc)) = permute8(f);
+                dequant_hi_lo(w[kc], sc, zr, hi, lo);
+                *reinterpret_cast<uint4*>(sb + (2 * half) * U_TILE + core_off(r, kc)) = hi;
+                *reinterpret_cast<uint4*>(sb + (2 * half + 1) * U_TILE + core_off(r, kc)) = lo;
             }
             stage_written(&S.full[st]);
-            cg = ng; cu = nu; xv[0] = nx[0]; xv[1] = nx[1];
+            cw = nw;
         }
-        // the adapter as extra k: A = B_gate / B_up rows (fp16 of bf16), B = sigma * (A_gate x), sigma * (A_up x)
+        // the adapter as extra k: A = B_gate / B_up rows (fp16 of bf16), B = sigma * (A_gate x) / sigma * (A_up x);
+        // the threads of matrix m write its A rows and its B rows (gate's B in slot 4, up's in slot 1)
         if (r_chunks > 0) {
             const int first_pair = S.pair[0];
             const int ad = first_pair >= 0 ? p.pair_ad[first_pair] : 0;
             const int n_sets = p.n_adapters == 1 ? 1 : p.K;
-            const float* ug = nullptr;
-            if (pair >= 0) ug = p.u_gu + (((size_t)(pair / p.K) * n_sets + (p.n_adapters == 1 ? 0 : pair % p.K)) * 2) * p.rank;
-            const uint16_t* Bg = reinterpret_cast<const uint16_t*>(p.lora.B_gate) + ((size_t)ad * p.I + row0 + r) * p.rank;
-            const uint16_t* Bu = reinterpret_cast<const uint16_t*>(p.lora.B_up) + ((size_t)ad * p.I + row0 + r) * p.rank;
+            const float* um = nullptr;
+            if (pair >= 0) um = p.u_gu + (((size_t)(pair / p.K) * n_sets + (p.n_adapters == 1 ? 0 : pair % p.K)) * 2 + half) * p.rank;
+            const uint16_t* Bm = reinterpret_cast<const uint16_t*>(half ? p.lora.B_up : p.lora.B_gate) + ((size_t)ad * p.I + row0 + r) * p.rank;
             for (int rc = 0; rc < r_chunks; ++rc) {
                 const int c = n_chunks + rc, st = c % U_STAGES_GU;
                 const uint32_t use = (uint32_t)(c / U_STAGES_GU);
                 bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
                 uint8_t* sb = S.stage[st];
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int kc = 2 * half + j;
+                for (int kc = 0; kc < 4; ++kc) {
                     const int j0 = rc * 32 + kc * 8, n = p.rank - j0;          // rank is a multiple of 8
-                    uint4 ag = make_uint4(0, 0, 0, 0), au = ag;
-                    if (n > 0) {
-                        ag = bf16x8_to_f16(*reinterpret_cast<const uint4*>(Bg + j0));
-                        au = bf16x8_to_f16(*reinterpret_cast<const uint4*>(Bu + j0));
-                    }
-                    *reinterpret_cast<uint4*>(sb + 0 * U_TILE + core_off(r, kc)) = ag;
-                    *reinterpret_cast<uint4*>(sb + 2 * U_TILE + core_off(r, kc)) = au;
-                    *reinterpret_cast<uint4*>(sb + 4 * U_TILE + core_off(r, kc)) = f32x8_to_f16(ug != nullptr ? ug + j0 : nullptr, n, p.sigma);
-                    *reinterpret_cast<uint4*>(sb + 1 * U_TILE + core_off(r, kc)) = f32x8_to_f16(ug != nullptr ? ug + p.rank + j0 : nullptr, n, p.sigma);
+                    uint4 a = make_uint4(0, 0, 0, 0);
+                    if (n > 0) a = bf16x8_to_f16(*reinterpret_cast<const uint4*>(Bm + j0));
+                    *reinterpret_cast<uint4*>(sb + (2 * half) * U_TILE + core_off(r, kc)) = a;
+                    *reinterpret_cast<uint4*>(sb + (half ? 1 : 4) * U_TILE + core_off(r, kc)) = f32x8_to_f16(um != nullptr ? um + j0 : nullptr, n, p.sigma);
                 }
+                if (tid == 0) bar_arrive(&S.full[st]);               // stands in for the bulk copy's arrival
                 stage_written(&S.full[st]);
             }
         }
@@ -483,6 +490,7 @@ cudaError_t launch_umma_gate_up(const GroupedParams& p, int max_tiles, cudaStrea
         if (e != cudaSuccess) return e;
         configured = true;
     }
+    umma_gather_x_kernel<<<dim3(8, max_tiles), 256, 0, st>>>(p);
     umma_gate_up_kernel<<<dim3(p.I / 128, max_tiles), U_THREADS, umma_smem_bytes(5, U_STAGES_GU), st>>>(p);
     return cudaGetLastError();
 }
