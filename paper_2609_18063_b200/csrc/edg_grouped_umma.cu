@@ -225,15 +225,18 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_gate_up_kernel(GroupedParam
         const uint8_t* cp = rec + (half ? p.L.codes_up : p.L.codes_gate);
         const uint8_t* zp = rec + (half ? p.L.sz_up : p.L.sz_gate);
         uint4 cw = ld_stream16(cp + code_off(p.H, row0 + r, 0));
+        const int n_groups = p.H >> gshift;
+        uint32_t nsz = ld_stream4(zp + sz_off(p.H, p.group, row0 + r, 0));      // (scale, zero) one group ahead
         __half2 sc = __float2half2_rn(0.f), zr = sc;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES_GU;
             const uint32_t use = (uint32_t)(c / U_STAGES_GU);
             uint4 nw = cw;
             if (c + 1 < n_chunks) nw = ld_stream16(cp + code_off(p.H, row0 + r, c + 1));   // in flight during this chunk
-            if (((c * U_KC) & (p.group - 1)) == 0) {                 // a new group: its (scale, zero)
-                const __half2 a = u32_as_h2(ld_stream4(zp + sz_off(p.H, p.group, row0 + r, (c * U_KC) >> gshift)));
+            if (((c * U_KC) & (p.group - 1)) == 0) {                 // a new group: its (scale, zero), and the load of the next
+                const __half2 a = u32_as_h2(nsz);
                 sc = __low2half2(a); zr = __high2half2(a);
+                nsz = ld_stream4(zp + sz_off(p.H, p.group, row0 + r, min(((c * U_KC) >> gshift) + 1, n_groups - 1)));
             }
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);          // the MMAs that read this stage are done
             uint8_t* sb = S.stage[st];
@@ -372,6 +375,8 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
         const uint8_t* hq = p.hq + (size_t)tile * (p.I / 32) * 2 * U_TILE;
         const uint8_t* cdp = rec + p.L.codes_down;
         uint4 cd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + tid, 0));
+        const int n_groups = p.I >> gshift;
+        uint32_t nsz = ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + tid, 0));
         __half2 sd = __float2half2_rn(0.f), zd = sd;
         for (int c = 0; c < n_chunks; ++c) {
             const int st = c % U_STAGES_D;
@@ -379,8 +384,9 @@ __global__ void __launch_bounds__(U_THREADS, 2) umma_down_kernel(GroupedParams p
             uint4 nd = cd;
             if (c + 1 < n_chunks) nd = ld_stream16(cdp + down_code_off(p.H, p.I, row0 + tid, c + 1));
             if (((c * U_KC) & (p.group - 1)) == 0) {
-                const __half2 a = u32_as_h2(ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + tid, (c * U_KC) >> gshift)));
+                const __half2 a = u32_as_h2(nsz);
                 sd = __low2half2(a); zd = __high2half2(a);
+                nsz = ld_stream4(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, row0 + tid, min(((c * U_KC) >> gshift) + 1, n_groups - 1)));
             }
             bar_wait(&S.empty[st], (use & 1) ^ 1, p.status);
             uint8_t* sb = S.stage[st];
