@@ -1,31 +1,39 @@
 // The batch-1 layer-step as ONE kernel (a1-a2 for the next step, a3 take, a4-a6 for this step).
 //
-// Work split.  Every routed expert is handled by 16 CTAs, arranged as four thread-block clusters
-// of kC = 4 CTAs (clusters of 4 can all be placed one CTA per SM on a B200; eight clusters of 16
-// cannot, and a cluster that shares SMs finishes last).  Cluster c of an expert owns a quarter of
-// the intermediate dimension: its CTAs compute the gate/up rows of that quarter, exchange
-// h = silu(gate) * up inside the cluster, and then compute a partial of the down projection over
-// that quarter of the columns for all H rows (a K-split) -- so no exchange ever crosses a cluster.
-//   * At kernel start every CTA issues bulk asynchronous copies (cp.async.bulk, completion on
-//     mbarriers) that bring its gate/up slice of the record into shared memory in four stages; its
-//     block of the down matrix follows into the space of the first two stages as soon as every
-//     warp is done with them, and lands while the rest of gate/up is being computed.
+// Work split.  CTAs of 256 threads in thread-block clusters of kC = 4 (clusters of 4 can all be placed
+// one CTA per SM on a B200; eight clusters of 16 cannot, and a cluster that shares SMs finishes last).
+// A cluster owns `qpc` quarters of the intermediate dimension of one routed expert and walks them one
+// after the other: for a quarter its CTAs compute their gate/up rows (over all of K), exchange
+// h = silu(gate) * up inside the cluster, and add the quarter's columns to the H/4 output rows each
+// CTA owns (accumulators stay in registers), so no exchange ever crosses a cluster.  A step chained
+// to its predecessor uses one cluster per expert (qpc = 4: few, long-lived CTAs, several steps share
+// the GPU); a step launched alone uses four (qpc = 1: all SMs at once).
+//   * Weights stream through four stage buffers by bulk asynchronous copies (cp.async.bulk, completion
+//     on mbarriers): the gate/up rows of a quarter fill all four (a K quarter each), the quarter's down
+//     block follows into stages 0-1 as soon as their warps are done, the next quarter's K quarters 2-3
+//     into stages 2-3 likewise, and its K quarters 0-1 once the down block has been used.
+//   * Both projections run on mma.sync.m16n8k16 fragments: exact integer codes in fp16 (one lop3 per
+//     pair of codes), the activations as column 0 of the B tile, scale and zero point applied in
+//     fp32 per 64-code block.  The loops over K blocks are rolled and the operands live in shared
+//     memory on purpose: a CTA runs most of this code once, and instruction fetch competes with the
+//     weight stream.
 //   * The rank-r LoRA projections A.x are split over the CTAs of a cluster and exchanged through
-//     distributed shared memory, as is h and the partial of A_down.h; the down adapter is applied
-//     per quarter (B (A h) is linear in h).  The exchanges are remote stores that count their bytes
-//     on an mbarrier of the receiving CTA (st.async); the only cluster barrier is a handshake at
-//     start-up, before any copy is issued, because a cluster-scope fence also waits for every bulk
-//     copy in flight into the SM.
-//   * The rows of the prerouter head are dealt over all CTAs of the grid and finished by whichever
-//     warp delivers the last logits.
-// The reduce y = sum_k w_k o_k goes through a [4K][H] fp32 scratch: each CTA writes its
-// gate-weighted partial, and the last CTA to arrive for a block of rows (one atomic counter per
-// block) sums the 4K partials in a fixed order, so the result does not depend on arrival order.
+//     distributed shared memory, as are h and the partials of A_down.h (summed over the quarters,
+//     B_down applied once at the end).  The exchanges are remote stores that count their bytes on an
+//     mbarrier of the receiving CTA (st.async); the only cluster barrier is a handshake at start-up,
+//     before any copy is issued, because a cluster-scope barrier also waits for every bulk copy in
+//     flight into the SM.
+//   * The rows of the prerouter head are dealt to the first CTAs of the grid, one row per warp; every
+//     warp publishes its logit into a ring slot of the workspace by itself, and the warp that
+//     delivers the last one also computes the caller's inds_next / gates_next.
+// The reduce y = sum_k w_k o_k goes through an fp32 scratch (one set per ring slot): each CTA writes
+// its gate-weighted partial, and the last CTA to arrive for a block of rows (one atomic counter per
+// block) sums the partials in a fixed order, so the result does not depend on arrival order.
 // Consecutive layer-steps are chained by programmatic dependent launch: the next step's kernel
-// starts early, waits for a flag raised by this step's top-k, and streams its weights while this
-// step is still computing.
-#include <stdio.h>
-#include <stdlib.h>
+// starts early, takes the head's logits from the ring as soon as they are written, selects its
+// experts itself and streams its weights while earlier steps are still computing; it never waits
+// for the previous kernel to end.  Every wait on another CTA or kernel is bounded and falls back to
+// a safe path (or flags the result) when it gives up.
 #include <cooperative_groups.h>
 
 #include "edg_mma.cuh"
@@ -1057,13 +1065,6 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         // two CTAs per SM: more clusters resident at once
         e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
-        if (const char* mb = getenv("EDG_L2_PERSIST_MB")) {
-            size_t want = (size_t)atoi(mb) << 20;
-            cudaError_t e2 = cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want);
-            size_t got = 0;
-            cudaDeviceGetLimit(&got, cudaLimitPersistingL2CacheSize);
-            fprintf(stderr, "persisting L2: asked %zu, rc %d, now %zu\n", want, (int)e2, got);
-        }
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
