@@ -100,6 +100,96 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_kernel(PreParams p) 
         warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds + (size_t)head * p.K, p.gates + (size_t)head * p.K);
 }
 
+// One head, T hidden states (batched decode of one layer): a cluster handles kTokBlock tokens, so
+// a row of the head is read once per token block instead of once per token.  CTA c of the cluster
+// computes its share of the E rows for all tokens of the block (one warp per row, the tokens' states
+// in shared memory as fp32), writes the logits into the leader's shared memory, and after the cluster
+// barrier warp w of the leader does softmax + top-k for token w of the block.
+constexpr int kTokBlock = 8;
+
+template <typename WT>
+__global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_kernel(PreParams p, int T) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
+    const int csize = (int)cluster.num_blocks();
+    const int t0 = blockIdx.y * kTokBlock;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    extern __shared__ float smem[];
+    float* s_logits = smem;                         // [kTokBlock][E]  (the leader's copy collects every CTA's rows)
+    float* s_x = smem + kTokBlock * p.E;            // [kTokBlock][H]  hidden states widened to fp32
+    for (int tt = 0; tt < kTokBlock; ++tt) {
+        const int t = t0 + tt;
+        for (int i = threadIdx.x; i < p.H; i += blockDim.x)
+            s_x[tt * p.H + i] = t < T ? bf16_bits_to_float(p.s[(size_t)t * p.H + i]) : 0.f;
+    }
+    __syncthreads();
+
+    float* leader = cluster.map_shared_rank(s_logits, 0);
+    const int per = (p.E + csize - 1) / csize;
+    const int e0 = crank * per, e1 = min(p.E, e0 + per);
+    constexpr int VPL = 16 / (int)sizeof(WT);       // weights per 16-byte load
+    const int n16 = p.H / VPL;                      // 16-byte pieces of a row
+    for (int e = e0 + warp; e < e1; e += kPreWarps) {
+        const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const WT*>(p.W) + (size_t)e * p.H);
+        float acc[kTokBlock];
+#pragma unroll
+        for (int t = 0; t < kTokBlock; ++t) acc[t] = 0.f;
+        for (int c0 = 0; c0 < n16; c0 += 8 * 32) {   // 8 independent loads per lane in flight, then the arithmetic
+            uint4 wr[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int c = c0 + j * 32 + lane;
+                wr[j] = c < n16 ? ld_stream16(wp + c) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int c = c0 + j * 32 + lane;
+                if (c >= n16) continue;
+                const uint4 w = wr[j];
+                float wf[8];
+                if (VPL == 8) {
+                    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+                    const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+                    const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
+                    wf[0] = a.x; wf[1] = a.y; wf[2] = b.x; wf[3] = b.y; wf[4] = d.x; wf[5] = d.y; wf[6] = f.x; wf[7] = f.y;
+                } else {
+                    wf[0] = __uint_as_float(w.x); wf[1] = __uint_as_float(w.y); wf[2] = __uint_as_float(w.z); wf[3] = __uint_as_float(w.w);
+                    wf[4] = wf[5] = wf[6] = wf[7] = 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < kTokBlock; ++t) {
+                    const float* x = s_x + t * p.H + c * VPL;
+                    const float4 x0 = *reinterpret_cast<const float4*>(x);
+                    float a = acc[t];
+                    a = fmaf(wf[0], x0.x, a); a = fmaf(wf[1], x0.y, a); a = fmaf(wf[2], x0.z, a); a = fmaf(wf[3], x0.w, a);
+                    if (VPL == 8) {
+                        const float4 x1 = *reinterpret_cast<const float4*>(x + 4);
+                        a = fmaf(wf[4], x1.x, a); a = fmaf(wf[5], x1.y, a); a = fmaf(wf[6], x1.z, a); a = fmaf(wf[7], x1.w, a);
+                    }
+                    acc[t] = a;
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < kTokBlock; ++t) {
+            const float l = warp_sum(acc[t]);
+            if (lane == 0) leader[t * p.E + e] = l;
+        }
+    }
+    cluster.sync();                     // every CTA's logits have landed in the leader
+    if (crank != 0) return;
+
+    const int t = t0 + warp;            // kPreWarps == kTokBlock: warp w finishes token w of the block
+    if (warp < kTokBlock && t < T) {
+        float* row = s_logits + warp * p.E;
+        if (p.logits != nullptr)
+            for (int e = lane; e < p.E; e += 32) p.logits[(size_t)t * p.E + e] = row[e];
+        __syncwarp();
+        warp_softmax_topk(row, p.E, p.K, lane, p.inds + (size_t)t * p.K, p.gates + (size_t)t * p.K);
+    }
+}
+
 // a2 alone: one warp per row of given logits.
 __global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* logits, int T, int E, int K,
                                                                 int32_t* inds, float* gates) {
@@ -121,10 +211,11 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
     if (!aligned(W_pre, 16) || !aligned(s, 16)) return EDG_E_INVAL;
     PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K, shared_head};
 
+    const bool batched = shared_head != 0 && n_heads > 1;     // one head, several tokens: a cluster per block of tokens
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kPreCluster, n_heads, 1);
+    cfg.gridDim = dim3(kPreCluster, batched ? (n_heads + kTokBlock - 1) / kTokBlock : n_heads, 1);
     cfg.blockDim = dim3(kPreWarps * 32, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)(d->E + d->H) * sizeof(float);
+    cfg.dynamicSmemBytes = (size_t)(d->E + d->H) * sizeof(float) * (batched ? kTokBlock : 1);
     cfg.stream = st;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
@@ -133,6 +224,18 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
     at[0].val.clusterDim.z = 1;
     cfg.attrs = at;
     cfg.numAttrs = 1;
+    if (batched) {
+        static bool configured = false;
+        if (!configured) {
+            EDG_CUDA_TRY(cudaFuncSetAttribute(prerouter_tokens_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            EDG_CUDA_TRY(cudaFuncSetAttribute(prerouter_tokens_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            configured = true;
+        }
+        if (cfg.dynamicSmemBytes > 200 * 1024) return EDG_E_SHAPE;
+        if (d->pre_dtype == EDG_F16) EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_kernel<__half>, p, (int)n_heads));
+        else EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_kernel<float>, p, (int)n_heads));
+        return EDG_OK;
+    }
     if (d->pre_dtype == EDG_F16) EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_kernel<__half>, p));
     else EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_kernel<float>, p));
     return EDG_OK;
