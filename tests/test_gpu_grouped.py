@@ -115,6 +115,26 @@ def test_prefill_cfg5_full_size_sampled_tokens():
     assert np.array_equal(Y, Y2)
 
 
+@pytest.mark.parametrize("n_adapters", [1, 16])
+def test_large_groups_on_the_small_layer_shape(n_adapters):
+    """The tensor-memory path on the other supported shape: H 1024, I 256, groups of 32 (a new scale
+    every chunk), rank 8 (half an MMA k-step, zero-padded), shared and per-expert adapters, ragged
+    tiles (token counts that are no multiple of 16) and experts that span several tiles."""
+    L = device_layer("cfg1", n_adapters)
+    cfg = L.cfg
+    T = 333
+    X = synth.hidden_states(cfg, T, stream=35)
+    rng = np.random.default_rng(7)
+    pop = np.array([8.0] * 2 + [1.0] * (cfg.E - 2)); pop /= pop.sum()            # two hot experts
+    inds_h = np.stack([np.sort(rng.choice(cfg.E, cfg.K, replace=False, p=pop)) for _ in range(T)]).astype(np.int32)
+    gates_h = rng.dirichlet(np.ones(cfg.K), size=T).astype(np.float32)
+    counts = np.bincount(inds_h.ravel(), minlength=cfg.E)
+    assert T * cfg.K > 8 * cfg.E and counts.max() > 128 and (counts % 16 != 0).any()
+    inds, gates = torch.from_numpy(inds_h).cuda(), torch.from_numpy(gates_h).cuda()
+    Y = _ffn_tokens(L, L.desc, X, inds, gates, T)
+    _check_tokens(L, X, inds_h, gates_h, Y, range(T))
+
+
 def test_grouped_reduces_to_the_decode_path_and_handles_per_expert_adapters():
     L = device_layer("cfg1", 16)                  # per-expert adapters
     cfg = L.cfg
