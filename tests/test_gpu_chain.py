@@ -58,3 +58,47 @@ def test_chained_steps_in_flight_match_oracle_and_unchained(name, steps, stride)
         _assert_close(y_c[t], ref)
         _check_routing(logits_c[t + 1], inds_c[t + 1], gates_c[t + 1], W_np, X[t], cfg.K)
     store.close()
+
+
+def test_a_hand_off_that_never_arrives_times_out_and_falls_back():
+    """Failure path of the chained hand-off, provoked from the host: after a step has published its
+    head's logits in the workspace ring, the test wipes that ring slot (back to "not yet written"), so
+    the chained next step polls for logits that never come.  Its bounded wait must run out, raise
+    EDG_E_TIMEOUT in the status word, fall back to waiting for the previous kernel and to the routing
+    that kernel wrote -- and still produce the right output.  Nothing faults or hangs."""
+    cfg = synth.CONFIGS["cfg1"]
+    store, d, hosts, slots, tables, cs, _ = _make_store(cfg, n_slots=cfg.E)
+    edg.stage_experts_to_slots(store, 0, np.arange(cfg.E, dtype=np.int32))
+    torch.cuda.synchronize()
+    W_np = synth.prerouter_weights(cfg)
+    W = torch.from_numpy(W_np).cuda()
+    X = synth.hidden_states(cfg, 3, stream=29)
+    xd = x_dev(X)
+    ws = layer_io.new_workspace(d)
+    inds = torch.zeros((3, cfg.K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((3, cfg.K), dtype=torch.float32, device="cuda")
+    logits = torch.zeros((3, cfg.E), dtype=torch.float32, device="cuda")
+    y = out_tensor(d, 2)
+    edg.prerouter_topk(d, W, xd[2], 1, inds[0], gates[0], logits[0])
+    edg.moe_layer_decode(store, 0, xd[0], inds[0], gates[0], W, inds[1], gates[1], logits[1], y[0], ws)
+    torch.cuda.synchronize()
+    assert edg.workspace_status(ws) == 0
+    # find the ring slot that holds the published logits and wipe it
+    wsf = ws.view(torch.float32)
+    first = (wsf == logits[1][0]).nonzero().flatten().tolist()
+    hits = [i for i in first if i + cfg.E <= wsf.numel() and torch.equal(wsf[i:i + cfg.E], logits[1])]
+    assert len(hits) == 1
+    ws.view(torch.int32)[hits[0]:hits[0] + cfg.E] = -1
+    torch.cuda.synchronize()
+    edg.moe_layer_decode(store, 0, xd[1], inds[1], gates[1], W, inds[2], gates[2], logits[2], y[1], ws)   # chained
+    torch.cuda.synchronize()
+    assert edg.workspace_status(ws) == -6                      # EDG_E_TIMEOUT, sticky
+    inds_h, gates_h, y_h = inds.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy()
+    experts = {}
+    get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
+    lora = synth.lora_tensors(cfg, 0, 0)
+    for t in range(2):
+        ref = orc.moe_ffn(X[t], inds_h[t], gates_h[t].astype(np.float64), get, lambda e: lora, cfg.lora_scale, cfg.group)
+        _assert_close(y_h[t], ref)
+    _check_routing(logits[2].cpu().numpy(), inds_h[2], gates_h[2], W_np, X[1], cfg.K)
+    store.close()
