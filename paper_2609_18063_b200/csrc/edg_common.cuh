@@ -77,8 +77,9 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 // block that must start out zero: its first int32 is the device-side status word, the rest are the
 // counters of the ring that chained batch-1 layer-steps share (arrivals of the reduce, head rows
 // delivered, reducers finished, head finished -- one set per ring slot).
-constexpr int kHandoffRing = 16;       // ring slots shared by chained batch-1 layer-steps in flight
-constexpr size_t kCtrlBytes = 512;     // control block: status word at 0, then the ring's counters
+constexpr int kPairWords = 64;         // words behind the logits of a ring slot: 32 (expert, gate) pairs, the routing itself
+constexpr int kHandoffRing = 32;       // ring slots shared by chained batch-1 layer-steps in flight
+constexpr size_t kCtrlBytes = 1024;    // control block: status word at 0, then the ring's counters
 constexpr size_t kCtrlCounters = 64;                               // [ring][4] arrivals per block of output rows
 constexpr size_t kCtrlHead = kCtrlCounters + kHandoffRing * 16;    // [ring] head rows delivered
 constexpr size_t kCtrlDone = kCtrlHead + kHandoffRing * 4;         // [ring] reducers finished
@@ -90,7 +91,7 @@ struct WorkspaceLayout {
     size_t u_gu;      // [T][n_sets][2][rank] float : A_gate x and A_up x
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
-    size_t logits;    // [ring][E] float          : next-step head logits handed to the chained next step, one set per ring slot
+    size_t logits;    // [ring][E + 64] float     : next-step head logits, then the (expert, gate) pairs chosen from them, handed to the chained next step; one set per ring slot
     size_t partial;   // [ring][4K][H] float      : gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
     size_t lone_bytes;// what a batch-1 call that never chains needs: everything up to the first set of partials
     // grouped path (T > 1) only:
@@ -117,7 +118,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.logits = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.partial = round_up(W.logits + (size_t)kHandoffRing * d.E * sizeof(float), 256);
+    W.partial = round_up(W.logits + (size_t)kHandoffRing * (d.E + kPairWords) * sizeof(float), 256);
     const size_t one_set = (size_t)kDownSlices * d.K * d.H * sizeof(float);
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);

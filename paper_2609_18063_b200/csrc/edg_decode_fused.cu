@@ -64,7 +64,7 @@ struct FusedSmem {
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t lora0, lora_bytes;                        // two buffers of per-quarter adapter slices: B_gate rows, B_up rows, A_down columns
     uint32_t b_down;                                   // B_down rows of this CTA
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, s_route, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
@@ -100,7 +100,6 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
     S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the quarter's h as (hi, lo) B-fragment words
     S.s_hsum = o;     o += (sw / 32) * 4;
-    S.s_route = o;    o += (uint32_t)E * 4 + 256;     // logits taken from the hand-off ring, then this step's K winners
     S.flag = o;       o += 16;
     S.total = (o + 15) / 16 * 16;
     return S;
@@ -135,6 +134,7 @@ struct FusedParams {
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
     int gshift;                   // log2(group)
     int qpc;                      // quarters of the intermediate dimension per cluster: 4 (one cluster per expert), 2 or 1
+    int epc;                      // experts per cluster, one after the other: 1, or 2 (only with qpc = 4)
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     FusedSmem S;                  // shared-memory carve-up
 };
@@ -235,6 +235,14 @@ __device__ __forceinline__ uint32_t ld_relaxed_gpu_u32(const void* p) {
 }
 __device__ __forceinline__ void st_relaxed_gpu_u32(void* p, uint32_t v) {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed_gpu_u64(const void* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed_gpu_u64(void* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 constexpr uint32_t kNotYet = 0xFFFFFFFFu;      // a logit that has not been written (a NaN no arithmetic produces)
 // programmatic dependent launch: let the next kernel in the stream start / wait for the previous one
@@ -341,7 +349,7 @@ __device__ __noinline__ void topk_large(float* work, int E, int K, int lane, int
 __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, float v, int e, bool own, int lane, uint32_t state) {
     int mine = 0;
     const int ring = p.flag_out >= 0 ? p.flag_out : 0;
-    float* logits_ws = p.logits_ws + (size_t)ring * p.E;
+    float* logits_ws = p.logits_ws + (size_t)ring * (p.E + kPairWords);
     int32_t* pre_counter = p.pre_counter + ring;
     if (own) {
         if (p.flag_out >= 0) {
@@ -395,6 +403,13 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
     if (lane < p.K) {
         p.inds_next[lane] = s_i[lane];
         p.gates_next[lane] = s_g[lane];
+        // the hand-off proper: (expert, gate) as one word per choice behind the logits of the ring
+        // slot, released after everything the publishers of the logits had observed
+        if (p.flag_out >= 0) {
+            __threadfence();
+            st_relaxed_gpu_u64(reinterpret_cast<unsigned long long*>(logits_ws + p.E) + lane,
+                               ((unsigned long long)__float_as_uint(s_g[lane]) << 32) | (uint32_t)s_i[lane]);
+        }
     }
     if (lane == 0) trace_stamp(p, 15);
 }
@@ -408,15 +423,16 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
 // instruction fetches compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
-constexpr int kMaxPre = 8;        // head rows per head CTA
+constexpr int kMaxPre = 16;       // head rows per head CTA (two per warp)
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_constant__ FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int cl = blockIdx.x / kC;                // cluster: an expert, or some quarters of it
     const int nq = kDownSlices / p.qpc;            // clusters per expert
-    const int k = cl / nq;                         // position of the expert in the routing
-    const int c0 = (cl - k * nq) * p.qpc;          // first quarter of the intermediate dimension of this cluster
+    const int k = (cl / nq) * p.epc;               // position of the cluster's (first) expert in the routing
+    const int cq = cl % nq;                        // which of the expert's clusters this is
+    const int c0 = cq * p.qpc;                     // first quarter of the intermediate dimension of this cluster
     const int crank = blockIdx.x % kC;             // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     const int g8 = lane >> 2, t4 = lane & 3;       // fragment coordinates: row slot, quad lane
@@ -448,10 +464,11 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     float* partial = p.partial + (size_t)p.ring * kDownSlices * p.K * p.H;
     int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
+    if (tid == 0) pdl_launch_dependents();
     // A call that does not continue a chain runs alone on its workspace: it clears what the last
     // head left unread in the ring.
     if (p.stale >= 0 && blockIdx.x == 0) {
-        for (int i = tid; i < p.E; i += kFW * 32) st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.stale * p.E + i], kNotYet);
+        for (int i = tid; i < p.E + kPairWords; i += kFW * 32) st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.stale * (p.E + kPairWords) + i], kNotYet);
         if (tid == 0) st_relaxed_gpu(&p.fin[p.stale], 0);
     }
 
@@ -459,15 +476,18 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     //      and the routing they lead to is what the next layer-step waits for.  The rows are dealt
     //      round-robin to the first CTAs of the grid; a row is split over all threads of its CTA
     //      (8 elements each).
-    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + kMaxPre - 1) / kMaxPre)) : 0;
+    const int max_pre = (p.pre_dtype == EDG_F16 && p.H <= 2048) ? kMaxPre : kFW;     // two rows per warp only on the fast path below
+    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + max_pre - 1) / max_pre)) : 0;
     const bool head_cta = (int)blockIdx.x < n_head_ctas;
-    const int n_pre = head_cta ? min(kMaxPre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
+    const int n_pre = head_cta ? min(max_pre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
     // Usual case (fp16 head, H <= 2048): warp w evaluates row w of this CTA's rows by itself, each
     // lane covering 8 runs of 8 elements, and publishes it without waiting for any other warp.
     const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= 2048;
-    const int my_e = (int)blockIdx.x + warp * n_head_ctas;       // fast path: this warp's row
+    const int my_e = (int)blockIdx.x + warp * n_head_ctas;       // fast path: this warp's row, and its second row
+    const int my_e2 = (int)blockIdx.x + (warp + kFW) * n_head_ctas;
     const bool my_row = pre_fast && warp < n_pre && my_e < p.E;
-    uint4 lw[8];
+    const bool my_row2 = pre_fast && warp + kFW < n_pre && my_e2 < p.E;
+    uint4 lw[8], lw2[8];
     if (my_row) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -475,13 +495,21 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             lw[j] = i < p.H ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)my_e * p.H + i) : make_uint4(0, 0, 0, 0);
         }
     }
+    if (my_row2) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = (j * 32 + lane) * 8;
+            lw2[j] = i < p.H ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)my_e2 * p.H + i) : make_uint4(0, 0, 0, 0);
+        }
+    }
     const bool pre_lane = tid * 8 < p.H;
-    uint32_t pre_state = kNotYet;         // the ring-slot entry this lane will publish into, as the kernel finds it
+    uint32_t pre_state = kNotYet, pre_state2 = kNotYet;   // the ring-slot entries this lane will publish into, as the kernel finds them
     if (p.flag_out >= 0) {
-        if (my_row && lane == 0) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + my_e]);
+        if (my_row && lane == 0) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e]);
+        if (my_row2 && lane == 0) pre_state2 = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e2]);
         if (n_pre > 0 && !pre_fast && warp == kFW - 1 && lane < n_pre) {
             const int e = (int)blockIdx.x + lane * n_head_ctas;
-            if (e < p.E) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * p.E + e]);
+            if (e < p.E) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + e]);
         }
     }
 
@@ -496,7 +524,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         // and kC partials of A_down.h (the barriers of quarters 2 and 3 are re-armed below)
         if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
-        if (p.qpc > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
+        if (p.qpc * p.epc > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
     }
     // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed just
     // before the copies are issued: a cluster-scope barrier waits for every bulk copy in flight
@@ -509,8 +537,8 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     //      shared memory.  Thread t converts activations 8t .. 8t+7 (word t%4 of chunk t/4) into
     //      the k-slot order of the fragments; s_xsum[j] = sum of the activations of scaled block j
     //      (for the zero points).
-    if (p.table != nullptr)
-        for (int i = tid; i < p.E; i += kFW * 32) s_table[i] = __ldcg(&p.table[i]);
+    if (p.table != nullptr && warp == 0)      // (warp 0 alone: it resolves the routing before the CTA's first barrier)
+        for (int i = lane; i < p.E; i += 32) s_table[i] = __ldcg(&p.table[i]);
     {
         float sum = 0.f;
         if (pre_lane) {
@@ -527,97 +555,189 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     }
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
-    // ---- warp 0: the routing, before anything that has to wait for memory: the next layer-step is
-    //      released as soon as this one has its routing.  A chained step reads the logits its predecessor's head has put into
-    //      the hand-off ring (long before that kernel ends) and selects its experts itself -- every
-    //      CTA the same way, which costs less than waiting for one warp to do it for all.  Bounded
-    //      wait; on a time-out fall back to waiting for the whole previous kernel and to the
-    //      routing it has written, which is always sufficient.
-    bool have = false;                    // warp 0: the logits of this step's routing are in shared memory
-    if (warp == 0) {
-        // The next layer-step may start once every CTA of this one has said so.  The CTAs that
-        // evaluate the head say so only after their own routing has arrived, i.e. after the head
-        // of the step before this one is complete: a step therefore never starts before the head
-        // two steps back is complete, which keeps the ring slots of the head scratch apart.
-        // Everything else two steps share is in a ring slot of its own, guarded by the hand-off.
-        if (lane == 0 && (!head_cta || p.flag_in < 0)) pdl_launch_dependents();
-        if (p.flag_in >= 0) {
-            const float* lg = p.logits_ws + (size_t)p.flag_in * p.E;
-            float* work = reinterpret_cast<float*>(smem + S.s_route);
-            int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_route) + p.E;
-            float* s_g = reinterpret_cast<float*>(s_i + 32);
-            uint32_t it = 0;
-            bool ok;
-            do {
-                ok = true;
-                for (int i = lane; i < p.E; i += 32) {
-                    const uint32_t w = ld_relaxed_gpu_u32(lg + i);
-                    ok = ok && (w != kNotYet);
-                    work[i] = __uint_as_float(w);
-                }
-                ok = __all_sync(0xFFFFFFFFu, ok);
-            } while (!ok && ++it < kSpinLimit);
-            trace_mark(p, 19);
-            if (ok) {
-                // everything the writers of these logits had observed (the reduce scratch of this
-                // ring slot being free again, above all) is ordered before what this CTA does next
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");
-                if (lane == 0 && head_cta) pdl_launch_dependents();
-                __syncwarp();
-                trace_mark(p, 22);
-                have = true;
-            } else if (lane == 0) {
-                atomicExch(p.status, EDG_E_TIMEOUT);
-                if (head_cta) pdl_launch_dependents();
-                pdl_wait_prior_grid();
-            }
+    // ---- a3: take, for the one or two experts of this cluster, as a function of the routing in
+    //      s_flag.  The decision is the same in every CTA of the cluster.  An expert that is out of
+    //      range is skipped (and flagged).  Warp 0 takes early, for the copies it issues; everyone
+    //      takes after the barrier.
+    int ad = 0;                               // two experts per cluster only with one shared adapter: ad = 0 for both
+    float gate0 = 0.f, gate1 = 0.f;
+    const uint8_t* rec0 = p.pool, *rec1 = p.pool;
+    bool ok0 = false, ok1 = false, valid = false;
+    int e_first = 0, n_items = 0;             // the items of this cluster's stream: the quarters of its valid experts, one expert after the other
+    auto take = [&]() {
+        {
+            int slot = s_flag[1];
+            gate0 = __int_as_float(s_flag[2]);
+            const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
+            if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
+            ad = 0;
+            if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
+            ok0 = slot >= 0 && slot < p.n_slots && ad >= 0;
+            if (ok0) rec0 = p.pool + (size_t)slot * p.L.bytes;
+            if (ad < 0) ad = 0;
         }
-    }
+        if (p.epc == 2) {
+            int slot = s_flag[0];
+            gate1 = __int_as_float(s_flag[3]);
+            if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
+            ok1 = slot >= 0 && slot < p.n_slots;
+            if (ok1) rec1 = p.pool + (size_t)slot * p.L.bytes;
+        }
+        valid = ok0 || ok1;
+        e_first = ok0 ? 0 : 1;
+        n_items = ((ok0 ? 1 : 0) + (ok1 ? 1 : 0)) * p.qpc;
+    };
+    auto item_expert = [&](int w) { return (ok0 && ok1) ? w / p.qpc : e_first; };
+    const int cps = p.H / 128;            // chunks of a row per stage
+    const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
+    const int gps = sw >> p.gshift;       // groups of a down row-slice
 
-    // ---- the head rows (their loads have been in flight since the kernel started), each published
-    //      by its warp as soon as it is summed
-    if (my_row) {
-        float v = 0.f;
+    // One warp issues two stages (K quarters 2 pair, 2 pair + 1) of the gate/up rows of item w (a
+    // quarter of one of the cluster's experts): lanes 0 and 8 arm the barriers, then lanes 0..7 /
+    // 8..15 issue one run each (codes or sz of a (matrix, row tile)).
+    auto issue_gu = [&](int w, int pair) {
+        const int c = c0 + w % p.qpc;
+        const uint8_t* rec = item_expert(w) ? rec1 : rec0;
+        const int s = pair * 2 + (lane >> 3), run = lane & 7;
+        if (lane < 16 && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
+        __syncwarp();
+        if (lane < 16 && run < 4 * TG) {
+            uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+            const uint64_t pol = policy_evict_first();   // weights stream through L2 once
+            const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
+            const int n = c * sw + crank * rows_gu + 16 * ti;
+            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
+                                      S.mat_codes, &bars[s], pol);
+            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
+                               S.mat_sz, &bars[s], pol);
+        }
+    };
+    // One warp issues the adapter slices of item w into buffer w & 1: this CTA's rows of B_gate and
+    // B_up for the item's quarter, and its columns of A_down (one 16-byte-multiple run per rank index).
+    auto issue_lora = [&](int w) {
+        const int c = c0 + w % p.qpc, it = w;
+        const uint32_t bgu = rows_gu * r * 2, ad_row = rows_gu * 2;
+        uint8_t* buf = smem + S.lora0 + (it & 1) * S.lora_bytes;
+        const int n0 = c * sw + crank * rows_gu;
+        if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (it & 1)], 2 * bgu + r * ad_row);
+        __syncwarp();
+        const size_t bo = ((size_t)ad * p.I + n0) * r * 2;
+        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
+        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
+        for (int j = lane; j < r; j += 32)
+            bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
+                     ad_row, &bars[BAR_LORA + (it & 1)]);
+    };
+
+    // ---- the routing and the first copies (warp 0), around the head rows (every warp).  A chained
+    //      step takes its routing from the hand-off ring: the (expert, gate) pairs that the head of
+    //      the step before it has left behind its logits, long before that kernel ends.  Its own
+    //      head rows come first (pass 0) -- nothing this kernel owes to a later step is ever held
+    //      back by a wait -- then warp 0 waits for the pairs (pass 1), takes, and issues the copies
+    //      of the first quarter by itself, ahead of the CTA's first barrier.  A step that is not
+    //      chained has its routing in memory and issues before its head rows.  Bounded wait; on a
+    //      time-out fall back to waiting for the whole previous kernel and to the routing it has
+    //      written, which is always sufficient.
+    bool routed = false;                  // warp 0: routing taken, first copies issued
+#pragma unroll 1
+    for (int pass = 0; pass < 2; ++pass) {
+        if (warp == 0 && !routed && (pass || p.flag_in < 0)) {
+            int vi[2] = {-1, -1}, vg[2] = {0, 0};
+            bool got = false;
+            if (p.flag_in >= 0) {
+                const unsigned long long* pr = reinterpret_cast<const unsigned long long*>(p.logits_ws + (size_t)p.flag_in * (p.E + kPairWords) + p.E);
+                uint32_t it = 0;
+                unsigned long long w = 0;
+                do {
+                    if (lane < p.K) w = ld_relaxed_gpu_u64(pr + lane);
+                    got = __all_sync(0xFFFFFFFFu, (uint32_t)w != kNotYet);
+                } while (!got && ++it < kSpinLimit);
+                if (got) {
+                    // everything the writers of this routing had observed (the reduce scratch of this
+                    // ring slot being free again, above all) is ordered before what this CTA does next
+                    asm volatile("fence.acq_rel.gpu;" ::: "memory");
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int i = (j * 32 + lane) * 8;
-            if (i < p.H) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(p.x + i);
-                const uint4 w = lw[j];
-                const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
-                const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
-                v = fmaf(a.x, bf16_lo(xv.x), v); v = fmaf(a.y, bf16_hi(xv.x), v);
-                v = fmaf(b.x, bf16_lo(xv.y), v); v = fmaf(b.y, bf16_hi(xv.y), v);
-                v = fmaf(d.x, bf16_lo(xv.z), v); v = fmaf(d.y, bf16_hi(xv.z), v);
-                v = fmaf(f.x, bf16_lo(xv.w), v); v = fmaf(f.y, bf16_hi(xv.w), v);
+                    for (int e = 0; e < 2; ++e) {
+                        const unsigned long long we = __shfl_sync(0xFFFFFFFFu, w, (k + e) & 31);
+                        if (e < p.epc) { vi[e] = (int)(uint32_t)we; vg[e] = (int)(uint32_t)(we >> 32); }
+                    }
+                    trace_mark(p, 19);
+                } else if (pass) {
+                    if (lane == 0) {
+                        atomicExch(p.status, EDG_E_TIMEOUT);
+                        pdl_wait_prior_grid();
+                    }
+                    __syncwarp();
+                }
+            }
+            if (p.flag_in < 0 || (!got && pass)) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                    if (e < p.epc) { vi[e] = __ldcg(&p.slots[k + e]); vg[e] = __float_as_int(__ldcg(&p.gates[k + e])); }
+                got = true;
+            }
+            if (got) {
+                // (the second expert's pair sits in words 0 and 3, which the end of the kernel uses for its flags)
+                if (lane == 0) { s_flag[1] = vi[0]; s_flag[2] = vg[0]; s_flag[0] = vi[1]; s_flag[3] = vg[1]; }
+                __syncwarp();
+                trace_mark(p, 14);
+                take();
+                if (valid) {
+                    // the copies of the first quarter, and of the adapter rows every quarter needs
+                    issue_gu(0, 0);
+                    issue_gu(0, 1);
+                    if (r > 0) {
+                        issue_lora(0);
+                        if (lane == 0) {
+                            const uint32_t bd = rows_d * r * 2;
+                            mbar_expect_tx(&bars[BAR_BDOWN], bd);
+                            bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd, &bars[BAR_BDOWN]);
+                        }
+                    }
+                }
+                trace_mark(p, 1);
+                routed = true;
             }
         }
-        v = warp_sum(v);
-        if (warp == 0) trace_mark(p, 12);
-        head_publish(p, smem, v, my_e, lane == 0, lane, pre_state);
-        if (warp == 0) trace_mark(p, 13);
+        if (pass) break;
+        // ---- the head rows (their loads have been in flight since the kernel started), each published
+        //      by its warp as soon as it is summed
+        if (my_row) {
+            float v = 0.f, v2 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int i = (j * 32 + lane) * 8;
+                if (i < p.H) {
+                    const uint4 xv = *reinterpret_cast<const uint4*>(p.x + i);
+                    const float x0 = bf16_lo(xv.x), x1 = bf16_hi(xv.x), x2 = bf16_lo(xv.y), x3 = bf16_hi(xv.y);
+                    const float x4 = bf16_lo(xv.z), x5 = bf16_hi(xv.z), x6 = bf16_lo(xv.w), x7 = bf16_hi(xv.w);
+                    {
+                        const uint4 w = lw[j];
+                        const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+                        const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
+                        v = fmaf(a.x, x0, v); v = fmaf(a.y, x1, v); v = fmaf(b.x, x2, v); v = fmaf(b.y, x3, v);
+                        v = fmaf(d.x, x4, v); v = fmaf(d.y, x5, v); v = fmaf(f.x, x6, v); v = fmaf(f.y, x7, v);
+                    }
+                    if (my_row2) {
+                        const uint4 w = lw2[j];
+                        const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+                        const float2 d = __half22float2(u32_as_h2(w.z)), f = __half22float2(u32_as_h2(w.w));
+                        v2 = fmaf(a.x, x0, v2); v2 = fmaf(a.y, x1, v2); v2 = fmaf(b.x, x2, v2); v2 = fmaf(b.y, x3, v2);
+                        v2 = fmaf(d.x, x4, v2); v2 = fmaf(d.y, x5, v2); v2 = fmaf(f.x, x6, v2); v2 = fmaf(f.y, x7, v2);
+                    }
+                }
+            }
+            v = warp_sum(v);
+            v2 = warp_sum(v2);
+            if (warp == 0) trace_mark(p, 12);
+            // both rows in one go: lane 0 publishes the first, lane 1 the second
+            const uint32_t st2 = __shfl_sync(0xFFFFFFFFu, pre_state2, 0);
+            head_publish(p, smem, lane == 1 ? v2 : v, lane == 1 ? my_e2 : my_e, lane == 0 || (lane == 1 && my_row2), lane,
+                         lane == 1 ? st2 : pre_state);
+            if (warp == 0) trace_mark(p, 13);
+        }
     }
 
-    // ---- warp 0 again: this step's experts from the logits it has read
-    if (warp == 0) {
-        int vi, vg;
-        if (have) {
-            float* work = reinterpret_cast<float*>(smem + S.s_route);
-            int32_t* s_i = reinterpret_cast<int32_t*>(smem + S.s_route) + p.E;
-            float* s_g = reinterpret_cast<float*>(s_i + 32);
-            if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
-            else topk_large(work, p.E, p.K, lane, s_i, s_g);
-            __syncwarp();
-            trace_mark(p, 23);
-            vi = s_i[k];
-            vg = __float_as_int(s_g[k]);
-        } else {
-            vi = __ldcg(&p.slots[k]);
-            vg = __float_as_int(__ldcg(&p.gates[k]));
-        }
-        if (lane == 0) { s_flag[1] = vi; s_flag[2] = vg; }
-        trace_mark(p, 14);
-    }
     // ---- any other head (fp32 weights, wider rows): every row is split over all threads of the CTA
     //      and published by one warp after the barrier below
     if (n_pre > 0 && !pre_fast) {
@@ -638,73 +758,15 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         head_publish(p, smem, v, e, own, lane, pre_state);
     }
 
-    // ---- a3: take.  The decision is the same in every CTA of the expert.
-    int slot = s_flag[1];
-    const float gate_k = __int_as_float(s_flag[2]);
-    const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
-    if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
-    int ad = 0;
-    if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
-    const bool valid = slot >= 0 && slot < p.n_slots && ad >= 0;
+    take();
     trace_mark(p, 10);
     cluster_wait();
-    const int cps = p.H / 128;            // chunks of a row per stage
-    const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
-    const int gps = sw >> p.gshift;       // groups of a down row-slice
-    const uint8_t* rec = p.pool + (size_t)(valid ? slot : 0) * p.L.bytes;
-
-    // One warp issues two stages (K quarters 2 pair, 2 pair + 1) of the gate/up rows of quarter c:
-    // lanes 0 and 8 arm the barriers, then lanes 0..7 / 8..15 issue one run each (codes or sz of a
-    // (matrix, row tile)).
-    auto issue_gu = [&](int c, int pair) {
-        const int s = pair * 2 + (lane >> 3), run = lane & 7;
-        if (lane < 16 && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
-        __syncwarp();
-        if (lane < 16 && run < 4 * TG) {
-            uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-            const uint64_t pol = policy_evict_first();   // weights stream through L2 once
-            const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
-            const int n = c * sw + crank * rows_gu + 16 * ti;
-            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
-                                      S.mat_codes, &bars[s], pol);
-            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
-                               S.mat_sz, &bars[s], pol);
-        }
-    };
-    // One warp issues the adapter slices of quarter c (the it-th of this cluster) into buffer it & 1: this CTA's rows of B_gate
-    // and B_up, and its columns of A_down (one 16-byte-multiple run per rank index).
-    auto issue_lora = [&](int c, int it) {
-        const uint32_t bgu = rows_gu * r * 2, ad_row = rows_gu * 2;
-        uint8_t* buf = smem + S.lora0 + (it & 1) * S.lora_bytes;
-        const int n0 = c * sw + crank * rows_gu;
-        if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (it & 1)], 2 * bgu + r * ad_row);
-        __syncwarp();
-        const size_t bo = ((size_t)ad * p.I + n0) * r * 2;
-        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
-        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
-        for (int j = lane; j < r; j += 32)
-            bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
-                     ad_row, &bars[BAR_LORA + (it & 1)]);
-    };
 
     float acc_lo[TD], acc_hi[TD];         // down accumulators: rows g and g+8 of TD row tiles, over all quarters
 #pragma unroll
     for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
 
     if (valid) {
-        // ---- issue the copies of the first quarter, and of the adapter rows every quarter needs
-        if (warp == 0) issue_gu(c0, 0);
-        else if (warp == 1) issue_gu(c0, 1);
-        else if (warp == 2 && r > 0) {
-            issue_lora(c0, 0);
-            if (lane == 0) {
-                const uint32_t bd = rows_d * r * 2;
-                mbar_expect_tx(&bars[BAR_BDOWN], bd);
-                bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd, &bars[BAR_BDOWN]);
-            }
-        }
-        trace_mark(p, 1);
-
         // ---- with the weights on their way: this CTA's share of the 2r rows of A_gate / A_up, per-warp
         //      partial dot products into s_red.  All threads take part, each covering 8 elements of a
         //      row per sweep; the loads of up to 8 rows are in flight together, so the share costs one
@@ -762,9 +824,10 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
         //      are done, the next quarter's K quarters 2-3 into stages 2-3 likewise, and its K
         //      quarters 0-1 once the down block has been used.
 #pragma unroll 1
-        for (int it = 0; it < p.qpc; ++it) {
-            const int c = c0 + it;
-            const uint32_t par = it & 1, par2 = (it >> 1) & 1;
+        for (int w = 0; w < n_items; ++w) {
+            const int it = w % p.qpc, c = c0 + it, e = item_expert(w);
+            const uint8_t* rec = e ? rec1 : rec0;
+            const uint32_t par = w & 1, par2 = (w >> 1) & 1;
             // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside
             //      stage w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile,
             //      chunk) are 256 contiguous bytes of shared memory, lane (g, t) reading word t of
@@ -775,7 +838,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             {
                 const int s = warp / 2;
                 mbar_wait(&bars[s], par, p.status);
-                if (it == 0) trace_mark(p, 3);
+                if (w == 0) trace_mark(p, 3);
                 const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
                 const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
                 constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
@@ -836,15 +899,15 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                     }
                 } else {
                     if (lane == 0) mbar_arrive(&bars[BAR_FREE23]);
-                    if (warp == kFW / 2 && it + 1 < p.qpc) {
+                    if (warp == kFW / 2 && w + 1 < n_items) {
                         mbar_wait(&bars[BAR_FREE23], par, p.status);
-                        issue_gu(c + 1, 1);
+                        issue_gu(w + 1, 1);
                     }
                 }
             }
             __syncthreads();
             // the adapter slices of the next quarter go into the buffer the previous quarter used
-            if (warp == kFW - 1 && r > 0 && it + 1 < p.qpc) issue_lora(c + 1, it + 1);
+            if (warp == kFW - 1 && r > 0 && w + 1 < n_items) issue_lora(w + 1);
             // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
             if (tid < 2 * rows_gu) {
                 float v = 0.f;
@@ -853,7 +916,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 s_gu[tid] = v;
             }
             __syncthreads();
-            if (it == 0) {
+            if (w == 0) {
                 trace_mark(p, 4);
                 if (r > 0) mbar_wait(&bars[BAR_U], 0, p.status);        // every CTA's A.x has landed in s_u
                 trace_mark(p, 5);
@@ -891,9 +954,9 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 v = group_sum<kC>(v);
                 st_async_f32(map_to_cta(&udp[crank * kMaxRank + j], part), v, map_to_cta(&bars[BAR_H + par], part));
             }
-            if (it == 0) trace_mark(p, 6);
+            if (w == 0) trace_mark(p, 6);
             mbar_wait(&bars[BAR_H + par], par2, p.status);              // the quarter's h and A_down.h partials
-            if (it == 0) trace_mark(p, 7);
+            if (w == 0) trace_mark(p, 7);
 
             // ---- down on the tensor cores: this quarter's columns for this CTA's H/4 output rows.  h is
             //      fp32: column 0 of the B tile carries its fp16 value, column 1 the fp16 residual
@@ -918,7 +981,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             }
             __syncthreads();
             // this buffer's barrier is used again two quarters on: arm it before anyone can send
-            if (tid == 0 && it + 2 < p.qpc) mbar_expect_tx(&bars[BAR_H + par], (uint32_t)(sw + kC * r) * 4u);
+            if (tid == 0 && w + 2 < n_items) mbar_expect_tx(&bars[BAR_H + par], (uint32_t)(sw + kC * r) * 4u);
             mbar_wait(&bars[BAR_DOWN], par, p.status);
             {
                 const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
@@ -957,44 +1020,59 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 }
             }
             // the next quarter's K quarters 0-1 go into stages 0-1 once every warp is done with the down block
-            if (it + 1 < p.qpc) {
+            if (w + 1 < n_items) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bars[BAR_DFREE]);
                 if (warp == 0) {
                     mbar_wait(&bars[BAR_DFREE], par, p.status);
-                    issue_gu(c + 1, 0);
+                    issue_gu(w + 1, 0);
                 }
             }
-            if (it == 0) trace_mark(p, 24);
-        }
+            if (w == 0) trace_mark(p, 24);
 
-        if (t4 == 0) {
+            // ---- the last quarter of an expert: its gate-weighted output rows go to the reduce scratch
+            if (it == p.qpc - 1) {
+                if (t4 == 0) {
 #pragma unroll
-            for (int tt = 0; tt < TD; ++tt) {
-                const int ti = warp + kFW * tt;
-                s_o[ti * 16 + g8] = acc_lo[tt];
-                s_o[ti * 16 + 8 + g8] = acc_hi[tt];
+                    for (int tt = 0; tt < TD; ++tt) {
+                        const int ti = warp + kFW * tt;
+                        s_o[ti * 16 + g8] = acc_lo[tt];
+                        s_o[ti * 16 + 8 + g8] = acc_hi[tt];
+                    }
+                }
+#pragma unroll
+                for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
+                if (r > 0) mbar_wait(&bars[BAR_BDOWN], 0, p.status);
+                __syncthreads();          // s_o, s_ud and the B_down rows complete
+                // LoRA B for down (A_down.h summed over the quarters) and the gate weight: one thread per output row
+                const float gate_k = e ? gate1 : gate0;
+                float* prow = partial + ((size_t)(k + e) * nq + cq) * p.H + n0_d;
+                for (int lr = tid; lr < rows_d; lr += kFW * 32) {
+                    float o = s_o[lr];
+                    if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
+                    prow[lr] = gate_k * o;
+                }
+                if (w + 1 < n_items) {   // another expert follows: its A_down.h starts from zero
+                    __syncthreads();
+                    if (tid < kMaxRank) s_ud[tid] = 0.f;
+                }
             }
         }
-        if (r > 0) mbar_wait(&bars[BAR_BDOWN], 0, p.status);
-        __syncthreads();                  // s_o, s_ud and the B_down rows complete
-        // LoRA B for down (A_down.h summed over the quarters) and the gate weight: one thread per output row
-        for (int lr = tid; lr < rows_d; lr += kFW * 32) {
-            float o = s_o[lr];
-            if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
-            partial[(size_t)cl * p.H + n0_d + lr] = gate_k * o;
-        }
         trace_mark(p, 8);
-    } else {
+    }
+    // a skipped expert contributes nothing
+    if (!ok0 || (p.epc == 2 && !ok1)) {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
-        // a skipped expert contributes nothing
-        for (int i = tid; i < rows_d; i += kFW * 32) partial[(size_t)cl * p.H + n0_d + i] = 0.f;
+        if (!ok0)
+            for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)k * nq + cq) * p.H + n0_d + i] = 0.f;
+        if (p.epc == 2 && !ok1)
+            for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)(k + 1) * nq + cq) * p.H + n0_d + i] = 0.f;
     }
 
     // ---- a6: this partial is published; the last arriver for the block of rows sums all partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == np - 1) ? 1 : 0;
+    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == (int)gridDim.x / kC - 1) ? 1 : 0;   // one arrival per cluster
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
@@ -1027,8 +1105,13 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                     __threadfence();
                 }
                 __syncthreads();
+                // (the routing pairs behind the logits first: whoever finds a logit reset finds them reset too)
+                for (int i = tid; i < kPairWords; i += kFW * 32)
+                    st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_in * (p.E + kPairWords) + p.E + i], kNotYet);
+                __threadfence();
+                __syncthreads();
                 for (int i = tid; i < p.E; i += kFW * 32)
-                    st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_in * p.E + i], kNotYet);
+                    st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_in * (p.E + kPairWords) + i], kNotYet);
             }
         }
     }
@@ -1048,8 +1131,10 @@ bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
     if ((d.I / kE16) % 16 != 0 || d.I / kE16 > 32) return false;   // whole 16-row tiles per CTA
     // the head rows are dealt to the first CTAs of the grid, at most kMaxPre each
-    const int grid = d.K * kC, head_ctas = grid < 32 ? grid : (grid < (d.E + kMaxPre - 1) / kMaxPre ? grid : ((d.E + kMaxPre - 1) / kMaxPre > 32 ? (d.E + kMaxPre - 1) / kMaxPre : 32));
-    if (head_ctas * kMaxPre < d.E) return false;
+    const int max_pre = (d.pre_dtype == EDG_F16 && d.H <= 2048) ? kMaxPre : kFW;
+    const int need = (d.E + max_pre - 1) / max_pre;
+    const int grid = d.K * kC, head_ctas = grid < 32 ? grid : (grid < need ? grid : (need > 32 ? need : 32));
+    if (head_ctas * max_pre < d.E) return false;
     if (d.group > 128 || (d.group & (d.group - 1)) != 0) return false;
     if (d.rank % 8 != 0) return false;            // adapter slices are staged by 16-byte bulk copies
     return fused_smem(d.H, d.I, d.E, d.group, d.rank).total <= kFusedSmemLimit;
@@ -1068,7 +1153,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.K * (kDownSlices / p.qpc) * kC, 1, 1);
+    cfg.gridDim = dim3(p.K / p.epc * (kDownSlices / p.qpc) * kC, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -1119,6 +1204,10 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.stale = stale;
     // a chained step shares the GPU with its neighbours: few, long-lived CTAs; a lone step wants all SMs at once
     p.qpc = flag_in >= 0 ? kDownSlices : 1;
+    // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
+    // CTAs per step, each amortising its start-up over twice the bytes
+    const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // two head rows per warp
+    p.epc = (flag_in >= 0 && d->K % 2 == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (d->K / 2) * kC * kMaxPre >= d->E) ? 2 : 1;
     p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlFin);
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;

@@ -277,7 +277,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
             uint8_t* w8 = static_cast<uint8_t*>(workspace);
             const edg::WorkspaceLayout W = edg::workspace_layout(s->d, 1);
             EDG_CUDA_TRY(cudaMemsetAsync(w8 + edg::kCtrlCounters, 0, edg::kCtrlBytes - edg::kCtrlCounters, st));
-            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.logits, 0xFF, (size_t)edg::kHandoffRing * s->d.E * sizeof(float), st));
+            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.logits, 0xFF, (size_t)edg::kHandoffRing * (s->d.E + edg::kPairWords) * sizeof(float), st));
             s->ring_ws = workspace;
             s->ring_next = 0;
             s->pub_slot = -1;

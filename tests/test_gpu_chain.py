@@ -62,8 +62,8 @@ def test_chained_steps_in_flight_match_oracle_and_unchained(name, steps, stride)
 
 def test_a_hand_off_that_never_arrives_times_out_and_falls_back():
     """Failure path of the chained hand-off, provoked from the host: after a step has published its
-    head's logits in the workspace ring, the test wipes that ring slot (back to "not yet written"), so
-    the chained next step polls for logits that never come.  Its bounded wait must run out, raise
+    head's logits and routing in the workspace ring, the test wipes that ring slot (back to "not yet
+    written"), so the chained next step polls for a routing that never comes.  Its bounded wait must run out, raise
     EDG_E_TIMEOUT in the status word, fall back to waiting for the previous kernel and to the routing
     that kernel wrote -- and still produce the right output.  Nothing faults or hangs."""
     cfg = synth.CONFIGS["cfg1"]
@@ -88,7 +88,7 @@ def test_a_hand_off_that_never_arrives_times_out_and_falls_back():
     first = (wsf == logits[1][0]).nonzero().flatten().tolist()
     hits = [i for i in first if i + cfg.E <= wsf.numel() and torch.equal(wsf[i:i + cfg.E], logits[1])]
     assert len(hits) == 1
-    ws.view(torch.int32)[hits[0]:hits[0] + cfg.E] = -1
+    ws.view(torch.int32)[hits[0]:hits[0] + cfg.E + 64] = -1     # the logits and the (expert, gate) pairs behind them
     torch.cuda.synchronize()
     edg.moe_layer_decode(store, 0, xd[1], inds[1], gates[1], W, inds[2], gates[2], logits[2], y[1], ws)   # chained
     torch.cuda.synchronize()
