@@ -44,8 +44,8 @@ namespace edg {
 
 constexpr int kC = 4;             // CTAs per cluster
 constexpr int kE16 = kC * kDownSlices;   // CTAs per expert
-constexpr int kFW = 8;            // warps per CTA
-constexpr int kStages = 4;        // gate/up copy stages per CTA
+constexpr int kFW = 4;            // warps per CTA
+constexpr int kStages = 2;        // copy stages per CTA: a quarter of the gate/up K range each, or half of the down block
 constexpr int kMaxRank = 64;
 constexpr int kTraceMarks = 32;
 constexpr int kRing = kHandoffRing;   // chained layer-steps in flight: hand-off slots for logits, reduce scratch, counters
@@ -63,7 +63,6 @@ struct FusedSmem {
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t lora0, lora_bytes;                        // two buffers of per-quarter adapter slices: B_gate rows, B_up rows, A_down columns
-    uint32_t b_down;                                   // B_down rows of this CTA
     uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
@@ -80,9 +79,8 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.d_sz = S.stage0 + rows_d * sw / 2;               // rows_d * (sw/2 + sw/group*4) == 2 * stage_bytes
     S.lora_bytes = 3 * rows_gu * (uint32_t)rank * 2;   // B_gate[rows_gu][rank], B_up[rows_gu][rank], A_down[rank][rows_gu]
     S.lora0 = o;      o += 2 * S.lora_bytes;
-    S.b_down = o;     o += rows_d * (uint32_t)rank * 2;       // B_down[n0 .. n0+rows_d][rank]
     o = (o + 15) / 16 * 16;
-    S.bars = o;       o += 8 * (kStages + 10);
+    S.bars = o;       o += 8 * 12;
     o = (o + 15) / 16 * 16;
     S.s_u = o;        o += 2 * kMaxRank * 4;
     S.s_h = o;        o += 2 * sw * 4;                // the quarter's h, double-buffered
@@ -92,9 +90,15 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_o = o;        o += rows_d * 4;
     S.s_red = o;      o += 40 * kFW * 4;              // per-warp partials: up to 32 adapter rows + 8 head rows per CTA
     S.s_hloc = o;     o += 32 * 4;
-    S.s_topk = o;     o += (uint32_t)E * 4 + 256;     // logits gathered by the warp that finishes the head, then its K winners
+    // logits gathered by the warp that finishes the head, then its K winners: in s_o when that is
+    // large enough (s_o is first written by the down phase of the first quarter, barriers later)
+    if (rows_d * 4 >= (uint32_t)E * 4 + 256) S.s_topk = S.s_o;
+    else { S.s_topk = o; o += (uint32_t)E * 4 + 256; }
     S.s_part = o;     o += kFW * 2 * rows_gu * 4;     // per-warp (k-slice) partial sums of the gate/up rows
-    S.s_table = o;    o += (uint32_t)E * 4;           // this layer's slot table, fetched before the routing is known
+    // this layer's slot table, fetched before the routing is known and used up before the first
+    // quarter starts: in s_part when that is large enough
+    if (kFW * 2 * rows_gu * 4 >= (uint32_t)E * 4) S.s_table = S.s_part;
+    else { S.s_table = o; o += (uint32_t)E * 4; }
     o = (o + 15) / 16 * 16;
     S.s_xb = o;       o += (uint32_t)H * 2;           // x as fp16 B-fragment words, k-slot order
     S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
@@ -129,7 +133,6 @@ struct FusedParams {
     unsigned long long* trace;    // optional [grid CTAs][kTraceMarks] globaltimer stamps, or null
     int32_t* done;                // [kRing] reducers of the step that has read each routing slot and are finished
     int ring;                     // ring slot of this step's reduce scratch
-    int32_t* fin;                 // [kRing] set once the head in that ring slot has been finished (its logits read)
     int flag_in;                  // -1: the routing is already in memory; else the ring slot to take it from
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
     int gshift;                   // log2(group)
@@ -286,6 +289,19 @@ __device__ __forceinline__ void store_y(void* y, int out_dtype, size_t i, float 
     else store_out<bf16_t>(static_cast<bf16_t*>(y), i, v);
 }
 
+// the same over a bf16 row in global memory (read-only path)
+__device__ __forceinline__ float gmem_b_dot(const uint16_t* B, const float* u, int r) {
+    float d = 0.f;
+    for (int j = 0; j < r; j += 8) {
+        const uint4 b = __ldg(reinterpret_cast<const uint4*>(B + j));
+        d = fmaf(bf16_lo(b.x), u[j + 0], d); d = fmaf(bf16_hi(b.x), u[j + 1], d);
+        d = fmaf(bf16_lo(b.y), u[j + 2], d); d = fmaf(bf16_hi(b.y), u[j + 3], d);
+        d = fmaf(bf16_lo(b.z), u[j + 4], d); d = fmaf(bf16_hi(b.z), u[j + 5], d);
+        d = fmaf(bf16_lo(b.w), u[j + 6], d); d = fmaf(bf16_hi(b.w), u[j + 7], d);
+    }
+    return d;
+}
+
 // sum_j B[j] * u[j] over a bf16 row in shared memory, r a multiple of 8
 __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, int r) {
     float d = 0.f;
@@ -299,10 +315,9 @@ __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, i
     return d;
 }
 
-// mbarriers: one per stage, then the down block, the adapter slices (two buffers), the B_down rows,
-// "stages 0-1 / 2-3 free after gate/up", "down block used", the adapter projections, h (two buffers)
-enum { BAR_DOWN = kStages, BAR_LORA = kStages + 1, BAR_BDOWN = kStages + 3, BAR_FREE01 = kStages + 4, BAR_FREE23 = kStages + 5,
-       BAR_DFREE = kStages + 6, BAR_U = kStages + 7, BAR_H = kStages + 8, kNumBars = kStages + 10 };
+// mbarriers: one per stage, then the down block, the adapter slices (two buffers), "stage 0 / 1
+// free after gate/up", "down block used", the adapter projections, h (two buffers)
+enum { BAR_DOWN = 2, BAR_LORA = 3, BAR_FREE0 = 5, BAR_DFREE = 7, BAR_U = 8, BAR_H = 9, kNumBars = 11 };
 
 // ---------------------------------------------------------------- head rows (a1) and top-k (a2)
 // The E rows of the head are dealt round-robin to the first CTAs of the grid; a row is split over
@@ -392,8 +407,6 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
         }
     }
     __syncwarp();
-    // the logits are in shared memory: the step that has read this ring slot may reset it
-    if (lane == 0 && p.flag_out >= 0) { __threadfence(); st_relaxed_gpu(&p.fin[ring], 1); }
     int32_t* s_i = reinterpret_cast<int32_t*>(smem + p.S.s_topk) + p.E;        // [K] winners, then [K] gates
     float* s_g = reinterpret_cast<float*>(s_i + 32);
     if (lane == 0) trace_stamp(p, 17);
@@ -401,15 +414,17 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
     else topk_large(work, p.E, p.K, lane, s_i, s_g);
     __syncwarp();
     if (lane < p.K) {
-        p.inds_next[lane] = s_i[lane];
-        p.gates_next[lane] = s_g[lane];
-        // the hand-off proper: (expert, gate) as one word per choice behind the logits of the ring
-        // slot, released after everything the publishers of the logits had observed
+        // the hand-off proper, first: (expert, gate) as one word per choice behind the logits of the
+        // ring slot, released after everything the publishers of the logits had observed.  The
+        // step that takes them resets the slot only after all of its CTAs have read them, i.e.
+        // after this warp has long finished with the logits.
         if (p.flag_out >= 0) {
             __threadfence();
             st_relaxed_gpu_u64(reinterpret_cast<unsigned long long*>(logits_ws + p.E) + lane,
                                ((unsigned long long)__float_as_uint(s_g[lane]) << 32) | (uint32_t)s_i[lane]);
         }
+        p.inds_next[lane] = s_i[lane];
+        p.gates_next[lane] = s_g[lane];
     }
     if (lane == 0) trace_stamp(p, 15);
 }
@@ -423,10 +438,10 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
 // instruction fetches compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
-constexpr int kMaxPre = 16;       // head rows per head CTA (two per warp)
+constexpr int kMaxPre = 2 * kFW;  // head rows per head CTA (two per warp)
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
-__global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_constant__ FusedParams p) {
+__global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_constant__ FusedParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
     const int cl = blockIdx.x / kC;                // cluster: an expert, or some quarters of it
     const int nq = kDownSlices / p.qpc;            // clusters per expert
@@ -469,7 +484,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     // head left unread in the ring.
     if (p.stale >= 0 && blockIdx.x == 0) {
         for (int i = tid; i < p.E + kPairWords; i += kFW * 32) st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.stale * (p.E + kPairWords) + i], kNotYet);
-        if (tid == 0) st_relaxed_gpu(&p.fin[p.stale], 0);
     }
 
     // ---- a1 for the next step, first of all: the loads of the head rows depend on nothing but x,
@@ -517,7 +531,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     //      exist, and every CTA of the cluster must be running, before anyone sends)
     if (tid == 0) {
         for (int s = 0; s < kNumBars; ++s)
-            mbar_init(&bars[s], (s == BAR_FREE01 || s == BAR_FREE23) ? kFW / 2 : (s == BAR_DFREE ? kFW : 1));
+            mbar_init(&bars[s], (s == BAR_FREE0 || s == BAR_FREE0 + 1) ? 2 : (s == BAR_DFREE ? kFW : 1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         // bytes this CTA will receive: 2r adapter projections once; per quarter, that quarter of h
@@ -539,19 +553,21 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     //      (for the zero points).
     if (p.table != nullptr && warp == 0)      // (warp 0 alone: it resolves the routing before the CTA's first barrier)
         for (int i = lane; i < p.E; i += 32) s_table[i] = __ldcg(&p.table[i]);
-    {
+    for (int t0 = 0; t0 * 8 < p.H; t0 += kFW * 32) {
+        const int t = t0 + tid;
+        const bool on = t * 8 < p.H;
         float sum = 0.f;
-        if (pre_lane) {
-            const uint4 v = *reinterpret_cast<const uint4*>(p.x + tid * 8);
+        if (on) {
+            const uint4 v = *reinterpret_cast<const uint4*>(p.x + t * 8);
             const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
                                 bf16_lo(v.z), bf16_hi(v.z), bf16_lo(v.w), bf16_hi(v.w)};
-            s_xb[tid] = permute8(f);
+            s_xb[t] = permute8(f);
             // fp16 is exact for bf16 inputs in the normal range; sum what the MMA will see
 #pragma unroll
             for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
         }
         sum = group_sum<4 * CPB>(sum);
-        if (pre_lane && (tid % (4 * CPB)) == 0) s_xsum[tid / (4 * CPB)] = sum;
+        if (on && (t % (4 * CPB)) == 0) s_xsum[t / (4 * CPB)] = sum;
     }
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
@@ -592,23 +608,25 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
     const int gps = sw >> p.gshift;       // groups of a down row-slice
 
-    // One warp issues two stages (K quarters 2 pair, 2 pair + 1) of the gate/up rows of item w (a
-    // quarter of one of the cluster's experts): lanes 0 and 8 arm the barriers, then lanes 0..7 /
-    // 8..15 issue one run each (codes or sz of a (matrix, row tile)).
-    auto issue_gu = [&](int w, int pair) {
+    // One warp issues K quarters 2 pair and 2 pair + 1 of the gate/up rows of item w (a quarter of
+    // one of the cluster's experts) into stages 0 and 1 -- or just the one that goes into stage
+    // `only`: lanes 0 and 8 arm the barriers, then lanes 0..7 / 8..15 issue one run each (codes or
+    // sz of a (matrix, row tile)).
+    auto issue_gu = [&](int w, int pair, int only) {
         const int c = c0 + w % p.qpc;
         const uint8_t* rec = item_expert(w) ? rec1 : rec0;
-        const int s = pair * 2 + (lane >> 3), run = lane & 7;
-        if (lane < 16 && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
+        const int s = lane >> 3, run = lane & 7, kq = pair * 2 + s;
+        const bool mine = lane < 16 && (only < 0 || only == s);
+        if (mine && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
         __syncwarp();
-        if (lane < 16 && run < 4 * TG) {
+        if (mine && run < 4 * TG) {
             uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
             const uint64_t pol = policy_evict_first();   // weights stream through L2 once
             const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
             const int n = c * sw + crank * rows_gu + 16 * ti;
-            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, s * cps),
+            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, kq * cps),
                                       S.mat_codes, &bars[s], pol);
-            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, s * gpst),
+            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, kq * gpst),
                                S.mat_sz, &bars[s], pol);
         }
     };
@@ -684,16 +702,8 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 take();
                 if (valid) {
                     // the copies of the first quarter, and of the adapter rows every quarter needs
-                    issue_gu(0, 0);
-                    issue_gu(0, 1);
-                    if (r > 0) {
-                        issue_lora(0);
-                        if (lane == 0) {
-                            const uint32_t bd = rows_d * r * 2;
-                            mbar_expect_tx(&bars[BAR_BDOWN], bd);
-                            bulk_g2s(smem + S.b_down, static_cast<const uint8_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r * 2, bd, &bars[BAR_BDOWN]);
-                        }
-                    }
+                    issue_gu(0, 0, -1);
+                    if (r > 0) issue_lora(0);
                 }
                 trace_mark(p, 1);
                 routed = true;
@@ -761,10 +771,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
     take();
     trace_mark(p, 10);
     cluster_wait();
-
-    float acc_lo[TD], acc_hi[TD];         // down accumulators: rows g and g+8 of TD row tiles, over all quarters
-#pragma unroll
-    for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
 
     if (valid) {
         // ---- with the weights on their way: this CTA's share of the 2r rows of A_gate / A_up, per-warp
@@ -837,8 +843,6 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             //      point are applied per block: acc += s * (c - z * sum(x)).
             {
                 const int s = warp / 2;
-                mbar_wait(&bars[s], par, p.status);
-                if (w == 0) trace_mark(p, 3);
                 const uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
                 const int ch0 = (warp & 1) * NCW;                        // first chunk of this warp inside the stage
                 constexpr int NT = 2 * TG;                               // (matrix, row tile) pairs, all independent: interleaved
@@ -846,49 +850,56 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
 #pragma unroll
                 for (int mt = 0; mt < NT; ++mt) { a_lo[mt] = 0.f; a_hi[mt] = 0.f; }
                 const uint8_t* cbase = st + ch0 * 256 + g8 * 16 + t4 * 4;
-                const uint4* xbp = s_xb + (warp * NCW) * 4 + t4;
+                // the K range in two halves: K quarters 0 and 1 fill the two stages first, quarters 2
+                // and 3 follow into the same stages as soon as their two warps are done with them
 #pragma unroll 1
-                for (int ib = 0; ib < NCW / CPB; ++ib) {                 // scaled blocks of this warp's K range
-                    float cfr[NT][4];
+                for (int half = 0; half < 2; ++half) {
+                    const int vw = warp + kFW * half;                    // this warp's K slice: chunks vw NCW .. vw NCW + NCW - 1 of a row
+                    mbar_wait(&bars[s], half, p.status);
+                    if (w == 0 && half == 0) trace_mark(p, 3);
+                    const uint4* xbp = s_xb + (vw * NCW) * 4 + t4;
+#pragma unroll 1
+                    for (int ib = 0; ib < NCW / CPB; ++ib) {             // scaled blocks of this warp's K range
+                        float cfr[NT][4];
 #pragma unroll
-                    for (int u = 0; u < CPB; ++u) {
-                        const int i = ib * CPB + u;
-                        uint4 xb = make_uint4(0, 0, 0, 0);
-                        if (g8 == 0) xb = xbp[i * 4];
+                        for (int u = 0; u < CPB; ++u) {
+                            const int i = ib * CPB + u;
+                            uint4 xb = make_uint4(0, 0, 0, 0);
+                            if (g8 == 0) xb = xbp[i * 4];
+#pragma unroll
+                            for (int mt = 0; mt < NT; ++mt) {
+                                const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
+                                uint32_t alo[4], ahi[4];
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                                if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                                else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
+                                mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
+                            }
+                        }
+                        const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
+                        const float xs = s_xsum[(vw * NCW) / CPB + ib];
 #pragma unroll
                         for (int mt = 0; mt < NT; ++mt) {
-                            const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
-                            uint32_t alo[4], ahi[4];
-                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                            if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
-                            else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
-                            mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
+                            const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
+                            const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                            const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                            a_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), a_lo[mt]);
+                            a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), a_hi[mt]);
                         }
                     }
-                    const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
-                    const float xs = s_xsum[(warp * NCW) / CPB + ib];
-#pragma unroll
-                    for (int mt = 0; mt < NT; ++mt) {
-                        const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
-                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
-                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                        a_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), a_lo[mt]);
-                        a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), a_hi[mt]);
-                    }
-                }
-                if (t4 == 0) {
-#pragma unroll
-                    for (int mt = 0; mt < NT; ++mt) {
-                        s_part[warp * 2 * rows_gu + mt * 16 + g8] = a_lo[mt];
-                        s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = a_hi[mt];
-                    }
-                }
-                // stages 0-1: the quarter's down block follows; stages 2-3: the next quarter's K quarters 2-3
-                if (warp < kFW / 2) {
-                    if (lane == 0) mbar_arrive(&bars[BAR_FREE01]);
-                    if (warp == 0) {
-                        mbar_wait(&bars[BAR_FREE01], par, p.status);
+                    // this stage is free once both of its warps are done: the second half of the K
+                    // range follows, and after that (both stages free) the quarter's down block
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&bars[BAR_FREE0 + s]);
+                    if (half == 0) {
+                        if ((warp & 1) == 0) {
+                            mbar_wait(&bars[BAR_FREE0 + s], 0, p.status);
+                            issue_gu(w, 1, s);
+                        }
+                    } else if (warp == 0) {
+                        mbar_wait(&bars[BAR_FREE0], 1, p.status);
+                        mbar_wait(&bars[BAR_FREE0 + 1], 1, p.status);
                         if (lane == 0) {
                             const uint64_t pol = policy_evict_first();
                             const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
@@ -897,11 +908,12 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                             bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
                         }
                     }
-                } else {
-                    if (lane == 0) mbar_arrive(&bars[BAR_FREE23]);
-                    if (warp == kFW / 2 && w + 1 < n_items) {
-                        mbar_wait(&bars[BAR_FREE23], par, p.status);
-                        issue_gu(w + 1, 1);
+                }
+                if (t4 == 0) {
+#pragma unroll
+                    for (int mt = 0; mt < NT; ++mt) {
+                        s_part[warp * 2 * rows_gu + mt * 16 + g8] = a_lo[mt];
+                        s_part[warp * 2 * rows_gu + mt * 16 + 8 + g8] = a_hi[mt];
                     }
                 }
             }
@@ -986,36 +998,53 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             {
                 const uint8_t* dbase = smem + S.d_codes + g8 * 16 + t4 * 4;
                 const uint8_t* dsz = smem + S.d_sz;
+                // a warp's row tiles in two passes of TD tiles (the registers of one pass); the sums
+                // over the quarters of an expert are kept in s_o, every row by the lane that owns it
 #pragma unroll 1
-                for (int ib = 0; ib < DCH / CPB; ++ib) {
-                    float cfr[TD][4];
+                for (int ps = 0; ps < 2; ++ps) {
+                    float acc_lo[TD], acc_hi[TD];                        // rows g and g+8 of TD row tiles
 #pragma unroll
-                    for (int u = 0; u < CPB; ++u) {
-                        const int i = ib * CPB + u;
-                        uint4 hb = make_uint4(0, 0, 0, 0);
-                        if (g8 < 2) hb = s_hb[(i * 2 + g8) * 4 + t4];
+                    for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
+#pragma unroll 1
+                    for (int ib = 0; ib < DCH / CPB; ++ib) {
+                        float cfr[TD][4];
+#pragma unroll
+                        for (int u = 0; u < CPB; ++u) {
+                            const int i = ib * CPB + u;
+                            uint4 hb = make_uint4(0, 0, 0, 0);
+                            if (g8 < 2) hb = s_hb[(i * 2 + g8) * 4 + t4];
+#pragma unroll
+                            for (int tt = 0; tt < TD; ++tt) {
+                                const int ti = warp + kFW * (ps * TD + tt);
+                                const uint8_t* cw = dbase + (ti * DCH + i) * 256;
+                                uint32_t alo[4], ahi[4];
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
+                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                                if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                                else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
+                                mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
+                            }
+                        }
+                        const int gi = (ib * CPB * 32) >> p.gshift;
+                        const float hs = s_hsum[ib];
 #pragma unroll
                         for (int tt = 0; tt < TD; ++tt) {
-                            const int ti = warp + kFW * tt;
-                            const uint8_t* cw = dbase + (ti * DCH + i) * 256;
-                            uint32_t alo[4], ahi[4];
-                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                            dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
-                            if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
-                            else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
-                            mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
+                            const int ti = warp + kFW * (ps * TD + tt);
+                            const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
+                            const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
+                            const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
+                            acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
+                            acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
                         }
                     }
-                    const int gi = (ib * CPB * 32) >> p.gshift;
-                    const float hs = s_hsum[ib];
+                    if (t4 == 0) {
 #pragma unroll
-                    for (int tt = 0; tt < TD; ++tt) {
-                        const int ti = warp + kFW * tt;
-                        const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
-                        const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
-                        const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                        acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
-                        acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
+                        for (int tt = 0; tt < TD; ++tt) {
+                            const int ti = warp + kFW * (ps * TD + tt);
+                            // (the first quarter of an expert starts the sums)
+                            s_o[ti * 16 + g8] = it ? s_o[ti * 16 + g8] + acc_lo[tt] : acc_lo[tt];
+                            s_o[ti * 16 + 8 + g8] = it ? s_o[ti * 16 + 8 + g8] + acc_hi[tt] : acc_hi[tt];
+                        }
                     }
                 }
             }
@@ -1025,32 +1054,30 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
                 if (lane == 0) mbar_arrive(&bars[BAR_DFREE]);
                 if (warp == 0) {
                     mbar_wait(&bars[BAR_DFREE], par, p.status);
-                    issue_gu(w + 1, 0);
+                    issue_gu(w + 1, 0, -1);
                 }
             }
             if (w == 0) trace_mark(p, 24);
 
             // ---- the last quarter of an expert: its gate-weighted output rows go to the reduce scratch
             if (it == p.qpc - 1) {
-                if (t4 == 0) {
-#pragma unroll
-                    for (int tt = 0; tt < TD; ++tt) {
-                        const int ti = warp + kFW * tt;
-                        s_o[ti * 16 + g8] = acc_lo[tt];
-                        s_o[ti * 16 + 8 + g8] = acc_hi[tt];
-                    }
-                }
-#pragma unroll
-                for (int tt = 0; tt < TD; ++tt) { acc_lo[tt] = 0.f; acc_hi[tt] = 0.f; }
-                if (r > 0) mbar_wait(&bars[BAR_BDOWN], 0, p.status);
-                __syncthreads();          // s_o, s_ud and the B_down rows complete
-                // LoRA B for down (A_down.h summed over the quarters) and the gate weight: one thread per output row
+                __syncthreads();          // s_o and s_ud complete
+                // LoRA B for down (A_down.h summed over the quarters; the rows of B_down come
+                // straight from memory, 2r bytes each) and the gate weight: one thread per output row
                 const float gate_k = e ? gate1 : gate0;
                 float* prow = partial + ((size_t)(k + e) * nq + cq) * p.H + n0_d;
-                for (int lr = tid; lr < rows_d; lr += kFW * 32) {
-                    float o = s_o[lr];
-                    if (r > 0) o = fmaf(p.sigma, smem_b_dot(reinterpret_cast<const uint16_t*>(smem + S.b_down) + lr * r, s_ud, r), o);
-                    prow[lr] = gate_k * o;
+                const uint16_t* Bd = static_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r;
+                constexpr int kRowsPerThread = rows_d / (kFW * 32);
+                float dl[kRowsPerThread];
+#pragma unroll
+                for (int q = 0; q < kRowsPerThread; ++q) {
+                    dl[q] = 0.f;
+                    if (r > 0) dl[q] = gmem_b_dot(Bd + (size_t)(tid + q * kFW * 32) * r, s_ud, r);
+                }
+#pragma unroll
+                for (int q = 0; q < kRowsPerThread; ++q) {
+                    const int lr = tid + q * kFW * 32;
+                    prow[lr] = gate_k * fmaf(p.sigma, dl[q], s_o[lr]);
                 }
                 if (w + 1 < n_items) {   // another expert follows: its A_down.h starts from zero
                     __syncthreads();
@@ -1095,16 +1122,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
             if (tid == 0) s_flag[3] = (atomicAdd(&p.done[p.flag_in], 1) == kC - 1) ? 1 : 0;
             __syncthreads();
             if (s_flag[3]) {
-                if (tid == 0) {
-                    p.done[p.flag_in] = 0;
-                    // the head that filled the slot may still be copying the logits for its own top-k
-                    uint32_t it = 0;
-                    while (ld_relaxed_gpu(&p.fin[p.flag_in]) == 0 && ++it < kSpinLimit) {}
-                    if (it >= kSpinLimit) atomicExch(p.status, EDG_E_TIMEOUT);
-                    st_relaxed_gpu(&p.fin[p.flag_in], 0);
-                    __threadfence();
-                }
-                __syncthreads();
+                if (tid == 0) p.done[p.flag_in] = 0;
                 // (the routing pairs behind the logits first: whoever finds a logit reset finds them reset too)
                 for (int i = tid; i < kPairWords; i += kFW * 32)
                     st_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_in * (p.E + kPairWords) + p.E + i], kNotYet);
@@ -1125,7 +1143,7 @@ __global__ void __launch_bounds__(kFW * 32, 2) fused_layer_kernel(const __grid_c
 
 static unsigned long long* g_trace = nullptr;     // set by edg_set_trace_buffer
 
-constexpr size_t kFusedSmemLimit = 112 * 1024;    // two CTAs per SM
+constexpr size_t kFusedSmemLimit = 56 * 1024;     // four CTAs per SM
 
 bool fused_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
@@ -1206,9 +1224,7 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.qpc = flag_in >= 0 ? kDownSlices : 1;
     // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
     // CTAs per step, each amortising its start-up over twice the bytes
-    const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // two head rows per warp
-    p.epc = (flag_in >= 0 && d->K % 2 == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (d->K / 2) * kC * kMaxPre >= d->E) ? 2 : 1;
-    p.fin = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlFin);
+    p.epc = 1;
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
