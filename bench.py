@@ -207,8 +207,8 @@ def run_b200(args):
 
     steps, warmup = args.steps, max(args.warmup, 3)
     full, rem = divmod(steps, G)
-    if rem % 32:                           # the hand-off ring has 32 slots: keep graph lengths a multiple
-        raise SystemExit("--steps must be a multiple of 32")
+    if rem % 64:                           # the hand-off ring has 64 slots: keep graph lengths a multiple
+        raise SystemExit("--steps must be a multiple of 64")
     g_full = capture(G) if full or warmup else None
     g_rem = capture(rem) if rem else None
 
@@ -320,7 +320,7 @@ def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
         st.synchronize()
 
     n = min(args.steps, args.e2e_steps)
-    n -= n % 32
+    n -= n % 64
     for s in range(max(4, min(args.warmup, 20) // 2 * 2)):
         step(s)
     base = store.stats()

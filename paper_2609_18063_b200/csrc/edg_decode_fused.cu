@@ -438,7 +438,7 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
 // instruction fetches compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
-constexpr int kMaxPre = 2 * kFW;  // head rows per head CTA (two per warp)
+constexpr int kMaxPre = 4 * kFW;  // head rows per head CTA (two batches of two per warp)
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_constant__ FusedParams p) {
@@ -497,10 +497,11 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     // Usual case (fp16 head, H <= 2048): warp w evaluates row w of this CTA's rows by itself, each
     // lane covering 8 runs of 8 elements, and publishes it without waiting for any other warp.
     const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= 2048;
-    const int my_e = (int)blockIdx.x + warp * n_head_ctas;       // fast path: this warp's row, and its second row
-    const int my_e2 = (int)blockIdx.x + (warp + kFW) * n_head_ctas;
-    const bool my_row = pre_fast && warp < n_pre && my_e < p.E;
-    const bool my_row2 = pre_fast && warp + kFW < n_pre && my_e2 < p.E;
+    // Its rows beyond the first two follow in further batches of two.
+    int my_e = (int)blockIdx.x + warp * n_head_ctas;             // fast path: this warp's row, and its second row
+    int my_e2 = (int)blockIdx.x + (warp + kFW) * n_head_ctas;
+    bool my_row = pre_fast && warp < n_pre && my_e < p.E;
+    bool my_row2 = pre_fast && warp + kFW < n_pre && my_e2 < p.E;
     uint4 lw[8], lw2[8];
     if (my_row) {
 #pragma unroll
@@ -710,9 +711,11 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
         }
         if (pass) break;
-        // ---- the head rows (their loads have been in flight since the kernel started), each published
-        //      by its warp as soon as it is summed
-        if (my_row) {
+        // ---- the head rows (the loads of the first two have been in flight since the kernel started),
+        //      published by their warp as soon as they are summed
+#pragma unroll 1
+        for (int b = 0; pre_fast && b * 2 * kFW < n_pre; ++b) {
+            if (!my_row) break;           // (a warp's rows are valid in ascending order)
             float v = 0.f, v2 = 0.f;
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
@@ -740,10 +743,34 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             v = warp_sum(v);
             v2 = warp_sum(v2);
             if (warp == 0) trace_mark(p, 12);
+            // the next two rows of this warp, if any: on their way while these are published
+            const int pe = my_e, pe2 = my_e2;
+            const bool prow2 = my_row2;
+            const uint32_t ps = pre_state, ps2 = pre_state2;
+            {
+                const int r1 = warp + kFW * 2 * (b + 1);
+                my_e = (int)blockIdx.x + r1 * n_head_ctas;
+                my_e2 = (int)blockIdx.x + (r1 + kFW) * n_head_ctas;
+                my_row = r1 < n_pre && my_e < p.E;
+                my_row2 = r1 + kFW < n_pre && my_e2 < p.E;
+                pre_state = kNotYet; pre_state2 = kNotYet;
+                if (my_row) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int i = (j * 32 + lane) * 8;
+                        lw[j] = i < p.H ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)my_e * p.H + i) : make_uint4(0, 0, 0, 0);
+                        if (my_row2) lw2[j] = i < p.H ? ld_keep16(static_cast<const __half*>(p.W_pre) + (size_t)my_e2 * p.H + i) : make_uint4(0, 0, 0, 0);
+                    }
+                    if (p.flag_out >= 0 && lane == 0) {
+                        pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e]);
+                        if (my_row2) pre_state2 = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e2]);
+                    }
+                }
+            }
             // both rows in one go: lane 0 publishes the first, lane 1 the second
-            const uint32_t st2 = __shfl_sync(0xFFFFFFFFu, pre_state2, 0);
-            head_publish(p, smem, lane == 1 ? v2 : v, lane == 1 ? my_e2 : my_e, lane == 0 || (lane == 1 && my_row2), lane,
-                         lane == 1 ? st2 : pre_state);
+            const uint32_t st2 = __shfl_sync(0xFFFFFFFFu, ps2, 0);
+            head_publish(p, smem, lane == 1 ? v2 : v, lane == 1 ? pe2 : pe, lane == 0 || (lane == 1 && prow2), lane,
+                         lane == 1 ? st2 : ps);
             if (warp == 0) trace_mark(p, 13);
         }
     }
@@ -1224,7 +1251,10 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.qpc = flag_in >= 0 ? kDownSlices : 1;
     // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
     // CTAs per step, each amortising its start-up over twice the bytes
-    p.epc = 1;
+    // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
+    // CTAs per step, each amortising its start-up over twice the bytes
+    const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // up to 4 kFW head rows per CTA
+    p.epc = (flag_in >= 0 && d->K % 2 == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (d->K / 2) * kC * kMaxPre >= d->E) ? 2 : 1;
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;
