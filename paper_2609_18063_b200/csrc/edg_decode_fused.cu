@@ -63,7 +63,7 @@ struct FusedSmem {
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t lora0, lora_bytes;                        // two buffers of per-quarter adapter slices: B_gate rows, B_up rows, A_down columns
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_hb, s_hsum, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_xbias, s_hb, s_hsum, s_hbias, flag, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
@@ -102,8 +102,10 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     o = (o + 15) / 16 * 16;
     S.s_xb = o;       o += (uint32_t)H * 2;           // x as fp16 B-fragment words, k-slot order
     S.s_xsum = o;     o += (uint32_t)(H / 32) * 4;    // sums of x per scaled block
+    S.s_xbias = o;    o += (uint32_t)(H / 32) * 4;    // what the biased codes add per scaled block: 1024 * (even positions) + 64 * (odd positions)
     S.s_hb = o;       o += (sw / 32) * 2 * 64;        // the quarter's h as (hi, lo) B-fragment words
     S.s_hsum = o;     o += (sw / 32) * 4;
+    S.s_hbias = o;    o += (sw / 32) * 4;
     S.flag = o;       o += 16;
     S.total = (o + 15) / 16 * 16;
     return S;
@@ -467,8 +469,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     int* s_table = reinterpret_cast<int*>(smem + S.s_table);        // [E]
     uint4* s_xb = reinterpret_cast<uint4*>(smem + S.s_xb);          // [H/8]  x as B-fragment words
     float* s_xsum = reinterpret_cast<float*>(smem + S.s_xsum);      // [H/(32 CPB)] block sums of x
+    float* s_xbias = reinterpret_cast<float*>(smem + S.s_xbias);    // [H/(32 CPB)] bias carried by the codes of a block
     uint4* s_hb = reinterpret_cast<uint4*>(smem + S.s_hb);          // [DCH][2][4] h (hi, lo) as B-fragment words
     float* s_hsum = reinterpret_cast<float*>(smem + S.s_hsum);      // [DCH/CPB]
+    float* s_hbias = reinterpret_cast<float*>(smem + S.s_hbias);    // [DCH/CPB]
 
     constexpr int rows_gu = 16 * TG, rows_d = 128 * TD, sw = 32 * DCH;
     const int n0_d = crank * rows_d;               // first down (= output) row of this CTA
@@ -557,7 +561,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     for (int t0 = 0; t0 * 8 < p.H; t0 += kFW * 32) {
         const int t = t0 + tid;
         const bool on = t * 8 < p.H;
-        float sum = 0.f;
+        float sum = 0.f, sodd = 0.f;
         if (on) {
             const uint4 v = *reinterpret_cast<const uint4*>(p.x + t * 8);
             const float f[8] = {bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y),
@@ -565,10 +569,17 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             s_xb[t] = permute8(f);
             // fp16 is exact for bf16 inputs in the normal range; sum what the MMA will see
 #pragma unroll
-            for (int e = 0; e < 8; ++e) sum += __half2float(__float2half_rn(f[e]));
+            for (int e = 0; e < 8; e += 2) {
+                sum += __half2float(__float2half_rn(f[e]));
+                sodd += __half2float(__float2half_rn(f[e + 1]));
+            }
         }
         sum = group_sum<4 * CPB>(sum);
-        if (on && (t % (4 * CPB)) == 0) s_xsum[t / (4 * CPB)] = sum;
+        sodd = group_sum<4 * CPB>(sodd);
+        if (on && (t % (4 * CPB)) == 0) {
+            s_xsum[t / (4 * CPB)] = sum + sodd;
+            s_xbias[t / (4 * CPB)] = fmaf(1024.f, sum, 64.f * sodd);
+        }
     }
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
@@ -897,22 +908,22 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                             for (int mt = 0; mt < NT; ++mt) {
                                 const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
                                 uint32_t alo[4], ahi[4];
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                                dequant_word_b(*reinterpret_cast<const uint32_t*>(cw), alo);
+                                dequant_word_b(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
                                 if (u == 0) mma16816_zero(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
                                 else mma16816(cfr[mt], alo[0], ahi[0], alo[1], ahi[1], xb.x, xb.y);
                                 mma16816(cfr[mt], alo[2], ahi[2], alo[3], ahi[3], xb.z, xb.w);
                             }
                         }
                         const int gi = ((ch0 + ib * CPB) * 32) >> p.gshift;
-                        const float xs = s_xsum[(vw * NCW) / CPB + ib];
+                        const float xs = s_xsum[(vw * NCW) / CPB + ib], xbias = s_xbias[(vw * NCW) / CPB + ib];
 #pragma unroll
                         for (int mt = 0; mt < NT; ++mt) {
                             const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
                             const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
                             const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                            a_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0]), a_lo[mt]);
-                            a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2]), a_hi[mt]);
+                            a_lo[mt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), xs, cfr[mt][0] - xbias), a_lo[mt]);
+                            a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2] - xbias), a_hi[mt]);
                         }
                     }
                     // this stage is free once both of its warps are done: the second half of the K
@@ -1014,9 +1025,13 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 s_hb[tid] = lo ? permute8_lo(f) : permute8(f);
             } else if (tid >= 64 && tid < 64 + DCH / CPB) {
                 const int j = tid - 64;
-                float v = 0.f;
-                for (int e = 0; e < 32 * CPB; ++e) v += hq[j * 32 * CPB + e];   // hi + lo == h up to 2^-22: sum h itself
-                s_hsum[j] = v;
+                float v = 0.f, vo = 0.f;
+                for (int e = 0; e < 32 * CPB; e += 2) {                         // hi + lo == h up to 2^-22: sum h itself
+                    v += hq[j * 32 * CPB + e];
+                    vo += hq[j * 32 * CPB + e + 1];
+                }
+                s_hsum[j] = v + vo;
+                s_hbias[j] = fmaf(1024.f, v, 64.f * vo);
             }
             __syncthreads();
             // this buffer's barrier is used again two quarters on: arm it before anyone can send
@@ -1045,23 +1060,23 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                                 const int ti = warp + kFW * (ps * TD + tt);
                                 const uint8_t* cw = dbase + (ti * DCH + i) * 256;
                                 uint32_t alo[4], ahi[4];
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw), alo);
-                                dequant_word_q(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
+                                dequant_word_b(*reinterpret_cast<const uint32_t*>(cw), alo);
+                                dequant_word_b(*reinterpret_cast<const uint32_t*>(cw + 128), ahi);
                                 if (u == 0) mma16816_zero(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
                                 else mma16816(cfr[tt], alo[0], ahi[0], alo[1], ahi[1], hb.x, hb.y);
                                 mma16816(cfr[tt], alo[2], ahi[2], alo[3], ahi[3], hb.z, hb.w);
                             }
                         }
                         const int gi = (ib * CPB * 32) >> p.gshift;
-                        const float hs = s_hsum[ib];
+                        const float hs = s_hsum[ib], hbias = s_hbias[ib];
 #pragma unroll
                         for (int tt = 0; tt < TD; ++tt) {
                             const int ti = warp + kFW * (ps * TD + tt);
                             const uint8_t* zw = dsz + (ti * gps + gi) * 64 + g8 * 4;
                             const __half2 z0 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw));
                             const __half2 z1 = u32_as_h2(*reinterpret_cast<const uint32_t*>(zw + 32));
-                            acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1]), acc_lo[tt]);
-                            acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3]), acc_hi[tt]);
+                            acc_lo[tt] = fmaf(__low2float(z0), fmaf(-__high2float(z0), hs, cfr[tt][0] + cfr[tt][1] - hbias), acc_lo[tt]);
+                            acc_hi[tt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), hs, cfr[tt][2] + cfr[tt][3] - hbias), acc_hi[tt]);
                         }
                     }
                     if (t4 == 0) {

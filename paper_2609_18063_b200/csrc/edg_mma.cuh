@@ -81,4 +81,17 @@ __device__ __forceinline__ void dequant_word_q(uint32_t w, uint32_t (&out)[4]) {
     out[3] = h2_as_u32(__hfma2(u32_as_h2(lop3_and_or(w2, 0x00F000F0u, 0x64006400u)), k16th, __hneg2(k64)));
 }
 
+// The cheapest form: the code words masked straight into fp16 with a bias -- codes 0, 2, 4, 6 of a
+// word as 1024 + q, codes 1, 3, 5, 7 as 64 + q (their nibble sits four bits higher in the
+// mantissa) -- five instructions a word.  The dot product then carries 1024 * (sum of the
+// activations at even positions) + 64 * (sum at odd positions), exactly representable products
+// summed in fp32, which the caller subtracts per scaled block along with the zero-point term.
+__device__ __forceinline__ void dequant_word_b(uint32_t w, uint32_t (&out)[4]) {
+    const uint32_t w2 = w >> 8;
+    out[0] = lop3_and_or(w, 0x000F000Fu, 0x64006400u);
+    out[1] = lop3_and_or(w, 0x00F000F0u, 0x54005400u);
+    out[2] = lop3_and_or(w2, 0x000F000Fu, 0x64006400u);
+    out[3] = lop3_and_or(w2, 0x00F000F0u, 0x54005400u);
+}
+
 }  // namespace edg
