@@ -317,9 +317,9 @@ __device__ __forceinline__ float smem_b_dot(const uint16_t* B, const float* u, i
     return d;
 }
 
-// mbarriers: one per stage, then the down block, the adapter slices (two buffers), "stage 0 / 1
-// free after gate/up", "down block used", the adapter projections, h (two buffers)
-enum { BAR_DOWN = 2, BAR_LORA = 3, BAR_FREE0 = 5, BAR_DFREE = 7, BAR_U = 8, BAR_H = 9, kNumBars = 11 };
+// mbarriers: one per stage (two arrivals: the two warps that issue its copies), then the down
+// block, the adapter slices (two buffers), the adapter projections, h (two buffers)
+enum { BAR_DOWN = 2, BAR_LORA = 3, BAR_U = 5, BAR_H = 6, kNumBars = 8 };
 
 // ---------------------------------------------------------------- head rows (a1) and top-k (a2)
 // The E rows of the head are dealt round-robin to the first CTAs of the grid; a row is split over
@@ -536,7 +536,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      exist, and every CTA of the cluster must be running, before anyone sends)
     if (tid == 0) {
         for (int s = 0; s < kNumBars; ++s)
-            mbar_init(&bars[s], (s == BAR_FREE0 || s == BAR_FREE0 + 1) ? 2 : (s == BAR_DFREE ? kFW : 1));
+            mbar_init(&bars[s], s < kStages ? 2 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         // bytes this CTA will receive: 2r adapter projections once; per quarter, that quarter of h
@@ -620,26 +620,30 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
     const int gps = sw >> p.gshift;       // groups of a down row-slice
 
-    // One warp issues K quarters 2 pair and 2 pair + 1 of the gate/up rows of item w (a quarter of
-    // one of the cluster's experts) into stages 0 and 1 -- or just the one that goes into stage
-    // `only`: lanes 0 and 8 arm the barriers, then lanes 0..7 / 8..15 issue one run each (codes or
-    // sz of a (matrix, row tile)).
-    auto issue_gu = [&](int w, int pair, int only) {
+    // K quarters 2 pair and 2 pair + 1 of the gate/up rows of item w (a quarter of one of the
+    // cluster's experts) go into stages 0 and 1 as 16 copies, one run each (codes or sz of a
+    // (matrix, row tile)); issuing a copy costs its lane some 50 ns and the lanes of a warp take
+    // turns, so the copies are dealt to the four warps: warp v issues runs 4 (v & 1) .. + 3 of
+    // stage v / 2 from its lanes 0..3, after lane 0 has armed the stage's barrier with their bytes
+    // (one arrival per issuing warp).  The calling warp plays warps v0 .. v1 - 1.
+    auto issue_gu = [&](int w, int pair, int v0, int v1) {
         const int c = c0 + w % p.qpc;
         const uint8_t* rec = item_expert(w) ? rec1 : rec0;
-        const int s = lane >> 3, run = lane & 7, kq = pair * 2 + s;
-        const bool mine = lane < 16 && (only < 0 || only == s);
-        if (mine && run == 0) mbar_expect_tx(&bars[s], S.stage_bytes);
-        __syncwarp();
-        if (mine && run < 4 * TG) {
-            uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
-            const uint64_t pol = policy_evict_first();   // weights stream through L2 once
-            const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
-            const int n = c * sw + crank * rows_gu + 16 * ti;
-            if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, kq * cps),
-                                      S.mat_codes, &bars[s], pol);
-            else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, kq * gpst),
-                               S.mat_sz, &bars[s], pol);
+        const uint64_t pol = policy_evict_first();       // weights stream through L2 once
+        for (int v = v0; v < v1; ++v) {
+            const int s = v >> 1, run = (v & 1) * 4 + lane, kq = pair * 2 + s;
+            const int n_runs = min(4, max(0, 4 * TG - (v & 1) * 4));
+            if (lane == 0) mbar_expect_tx(&bars[s], (uint32_t)(n_runs / 2) * (S.mat_codes + S.mat_sz));
+            __syncwarp();
+            if (lane < n_runs) {
+                uint8_t* st = smem + S.stage0 + s * S.stage_bytes;
+                const int mt = run >> 1, is_sz = run & 1, m = mt / TG, ti = mt % TG;
+                const int n = c * sw + crank * rows_gu + 16 * ti;
+                if (!is_sz) bulk_g2s_hint(st + mt * S.mat_codes, rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, kq * cps),
+                                          S.mat_codes, &bars[s], pol);
+                else bulk_g2s_hint(st + S.sz0 + mt * S.mat_sz, rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, kq * gpst),
+                                   S.mat_sz, &bars[s], pol);
+            }
         }
     };
     // One warp issues the adapter slices of item w into buffer w & 1: this CTA's rows of B_gate and
@@ -714,7 +718,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 take();
                 if (valid) {
                     // the copies of the first quarter, and of the adapter rows every quarter needs
-                    issue_gu(0, 0, -1);
+                    issue_gu(0, 0, 0, kFW);
                     if (r > 0) issue_lora(0);
                 }
                 trace_mark(p, 1);
@@ -872,6 +876,9 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             const int it = w % p.qpc, c = c0 + it, e = item_expert(w);
             const uint8_t* rec = e ? rec1 : rec0;
             const uint32_t par = w & 1, par2 = (w >> 1) & 1;
+            // the adapter slices of the next quarter go into the buffer the previous quarter used:
+            // a score of small copies, issued while this quarter's weights are still on their way
+            if (warp == kFW - 1 && r > 0 && w + 1 < n_items) issue_lora(w + 1);
             // ---- gate/up on the tensor cores.  Warp w owns the K range of its NCW chunks (inside
             //      stage w / 2) for every row tile of gate and up; the 16 x 32 codes of a (tile,
             //      chunk) are 256 contiguous bytes of shared memory, lane (g, t) reading word t of
@@ -926,25 +933,11 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                             a_hi[mt] = fmaf(__low2float(z1), fmaf(-__high2float(z1), xs, cfr[mt][2] - xbias), a_hi[mt]);
                         }
                     }
-                    // this stage is free once both of its warps are done: the second half of the K
-                    // range follows, and after that (both stages free) the quarter's down block
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&bars[BAR_FREE0 + s]);
+                    // the second half of the K range follows into the same stages as soon as all
+                    // four warps are done with the first
                     if (half == 0) {
-                        if ((warp & 1) == 0) {
-                            mbar_wait(&bars[BAR_FREE0 + s], 0, p.status);
-                            issue_gu(w, 1, s);
-                        }
-                    } else if (warp == 0) {
-                        mbar_wait(&bars[BAR_FREE0], 1, p.status);
-                        mbar_wait(&bars[BAR_FREE0 + 1], 1, p.status);
-                        if (lane == 0) {
-                            const uint64_t pol = policy_evict_first();
-                            const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
-                            mbar_expect_tx(&bars[BAR_DOWN], dcb + dzb);
-                            bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), dcb, &bars[BAR_DOWN], pol);
-                            bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
-                        }
+                        __syncthreads();
+                        issue_gu(w, 1, warp, warp + 1);
                     }
                 }
                 if (t4 == 0) {
@@ -956,8 +949,15 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 }
             }
             __syncthreads();
-            // the adapter slices of the next quarter go into the buffer the previous quarter used
-            if (warp == kFW - 1 && r > 0 && w + 1 < n_items) issue_lora(w + 1);
+            // both stages are free: the quarter's down block follows (a warp that has no part in the sums below issues it)
+            if (warp == kFW - 2 && lane < 2) {
+                const uint64_t pol = policy_evict_first();
+                const uint32_t dcb = (uint32_t)rows_d * sw / 2, dzb = (uint32_t)rows_d * gps * 4;
+                if (lane == 0) mbar_expect_tx(&bars[BAR_DOWN], dcb + dzb);
+                __syncwarp(0x3u);
+                if (lane == 0) bulk_g2s_hint(smem + S.d_codes, rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), dcb, &bars[BAR_DOWN], pol);
+                else bulk_g2s_hint(smem + S.d_sz, rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), dzb, &bars[BAR_DOWN], pol);
+            }
             // sum the kFW k-slices: row mt*16 + j of (matrix, tile) order == s_gu[proj * rows_gu + row]
             if (tid < 2 * rows_gu) {
                 float v = 0.f;
@@ -1090,14 +1090,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                     }
                 }
             }
-            // the next quarter's K quarters 0-1 go into stages 0-1 once every warp is done with the down block
+            // the next quarter's K quarters 0-1 go into the stages once every warp is done with the down block
             if (w + 1 < n_items) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bars[BAR_DFREE]);
-                if (warp == 0) {
-                    mbar_wait(&bars[BAR_DFREE], par, p.status);
-                    issue_gu(w + 1, 0, -1);
-                }
+                __syncthreads();
+                issue_gu(w + 1, 0, warp, warp + 1);
             }
             if (w == 0) trace_mark(p, 24);
 
