@@ -290,8 +290,11 @@ int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          float* logits_next_opt, void* y,
                          void* workspace, size_t workspace_bytes, void* stream);
 
-/* Switches the chaining of consecutive moe_layer_decode calls on (default) or off.  With chaining
- * off every layer-step is an ordinary stream-ordered launch. */
+/* Chaining of consecutive moe_layer_decode calls: 0 off -- every layer-step is an ordinary
+ * stream-ordered launch; 1 (default) a call is chained when the buffers line up and the step
+ * before it is still in flight (its completion event has not fired) or the stream is being
+ * captured -- a step that finds the GPU idle is launched on its own, across all SMs, which is
+ * several times faster for that single step; 2 chained whenever the buffers line up. */
 int32_t edg_store_set_chaining(edg_store* store, int32_t enable);
 
 #ifdef __cplusplus

@@ -277,8 +277,10 @@ class Store:
         except Exception:
             pass
 
-    def set_chaining(self, enable: bool) -> None:
-        _check(_lib.edg_store_set_chaining(self.handle, 1 if enable else 0), "edg_store_set_chaining")
+    def set_chaining(self, enable) -> None:
+        """False / 0: off; True / 1: chain a step when the one before it is still in flight (default);
+        2: chain whenever the buffers line up."""
+        _check(_lib.edg_store_set_chaining(self.handle, int(enable)), "edg_store_set_chaining")
 
     def stats(self) -> dict:
         s = StoreStats()

@@ -1,39 +1,45 @@
 // The batch-1 layer-step as ONE kernel (a1-a2 for the next step, a3 take, a4-a6 for this step).
 //
-// Work split.  CTAs of 256 threads in thread-block clusters of kC = 4 (clusters of 4 can all be placed
-// one CTA per SM on a B200; eight clusters of 16 cannot, and a cluster that shares SMs finishes last).
-// A cluster owns `qpc` quarters of the intermediate dimension of one routed expert and walks them one
-// after the other: for a quarter its CTAs compute their gate/up rows (over all of K), exchange
-// h = silu(gate) * up inside the cluster, and add the quarter's columns to the H/4 output rows each
-// CTA owns (accumulators stay in registers), so no exchange ever crosses a cluster.  A step chained
-// to its predecessor uses one cluster per expert (qpc = 4: few, long-lived CTAs, several steps share
-// the GPU); a step launched alone uses four (qpc = 1: all SMs at once).
-//   * Weights stream through four stage buffers by bulk asynchronous copies (cp.async.bulk, completion
-//     on mbarriers): the gate/up rows of a quarter fill all four (a K quarter each), the quarter's down
-//     block follows into stages 0-1 as soon as their warps are done, the next quarter's K quarters 2-3
-//     into stages 2-3 likewise, and its K quarters 0-1 once the down block has been used.
-//   * Both projections run on mma.sync.m16n8k16 fragments: exact integer codes in fp16 (one lop3 per
-//     pair of codes), the activations as column 0 of the B tile, scale and zero point applied in
-//     fp32 per 64-code block.  The loops over K blocks are rolled and the operands live in shared
-//     memory on purpose: a CTA runs most of this code once, and instruction fetch competes with the
-//     weight stream.
+// Work split.  CTAs of 128 threads in thread-block clusters of kC = 4, four CTAs to an SM.  A cluster
+// owns `qpc` quarters of the intermediate dimension of one routed expert (of two, one after the
+// other, when the experts share one adapter) and walks them in sequence: for a quarter its CTAs
+// compute their gate/up rows (over all of K), exchange h = silu(gate) * up inside the cluster, and
+// add the quarter's columns to the H/4 output rows each CTA owns, so no exchange ever crosses a
+// cluster.  A step chained to its predecessor uses one cluster per expert or pair of experts
+// (qpc = 4: few, long-lived CTAs, dozens of steps share the GPU); a step launched alone uses four
+// clusters per expert (qpc = 1: all SMs at once).
+//   * Weights stream through two stage buffers by bulk asynchronous copies (cp.async.bulk, completion
+//     on mbarriers), one 36 KB load in flight per CTA at any time: the first half of the K range of
+//     the quarter's gate/up rows (a K quarter per stage), the second half, then the quarter's down
+//     block across both stages.  The exchange of h runs while the down block is on its way.  What
+//     keeps the memory system busy is the number of such pipelines: four per SM.
+//   * Issuing a bulk copy costs its lane some 50 ns and the lanes of a warp take turns, so the 16
+//     copies of a load are dealt to the four warps behind a CTA barrier, and the score of small
+//     copies for the adapter slices is issued while the quarter's weights are still in flight.
+//   * Both projections run on mma.sync.m16n8k16 fragments: the codes masked straight into biased
+//     fp16 (1024 + q or 64 + q, five instructions a word), the activations as column 0 of the B
+//     tile; bias, zero point and scale are applied in fp32 per 64-code block.  The loops over K
+//     blocks are rolled and the operands live in shared memory on purpose: a CTA runs most of this
+//     code once, and instruction fetch competes with the weight stream.
 //   * The rank-r LoRA projections A.x are split over the CTAs of a cluster and exchanged through
 //     distributed shared memory, as are h and the partials of A_down.h (summed over the quarters,
-//     B_down applied once at the end).  The exchanges are remote stores that count their bytes on an
-//     mbarrier of the receiving CTA (st.async); the only cluster barrier is a handshake at start-up,
-//     before any copy is issued, because a cluster-scope barrier also waits for every bulk copy in
-//     flight into the SM.
-//   * The rows of the prerouter head are dealt to the first CTAs of the grid, one row per warp; every
-//     warp publishes its logit into a ring slot of the workspace by itself, and the warp that
-//     delivers the last one also computes the caller's inds_next / gates_next.
+//     B_down applied once at the end, its rows read straight from memory).  The exchanges are
+//     remote stores that count their bytes on an mbarrier of the receiving CTA (st.async); the only
+//     cluster barrier is a handshake at start-up, because a cluster-scope barrier also waits for
+//     every bulk copy in flight into the SM.
+//   * The rows of the prerouter head are dealt to the first CTAs of the grid, two rows per warp at
+//     a time; every warp publishes its logits into a ring slot of the workspace by itself, and the
+//     warp that delivers the last one selects the experts: it leaves the (expert, gate) pairs
+//     behind the logits in the ring slot and writes the caller's inds_next / gates_next.
 // The reduce y = sum_k w_k o_k goes through an fp32 scratch (one set per ring slot): each CTA writes
 // its gate-weighted partial, and the last CTA to arrive for a block of rows (one atomic counter per
 // block) sums the partials in a fixed order, so the result does not depend on arrival order.
-// Consecutive layer-steps are chained by programmatic dependent launch: the next step's kernel
-// starts early, takes the head's logits from the ring as soon as they are written, selects its
-// experts itself and streams its weights while earlier steps are still computing; it never waits
-// for the previous kernel to end.  Every wait on another CTA or kernel is bounded and falls back to
-// a safe path (or flags the result) when it gives up.
+// Consecutive layer-steps are chained by programmatic dependent launch: every CTA releases the next
+// step's kernel as soon as it runs, so steps queue up on the device as far as its CTA slots go; a
+// step evaluates its head first, then takes its routing from the ring slot of the step before it
+// and streams its weights while earlier steps are still computing.  It never waits for the
+// previous kernel to end.  Every wait on another CTA or kernel is bounded and falls back to a safe
+// path (or flags the result) when it gives up.
 #include <cooperative_groups.h>
 
 #include "edg_mma.cuh"
@@ -52,11 +58,10 @@ constexpr int kRing = kHandoffRing;   // chained layer-steps in flight: hand-off
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
 
 // ---------------------------------------------------------------- shared-memory carve-up
-// Byte offsets, identical on host and device.  The four gate/up stages (quarters of the K range)
-// come first; the down block
-// later reuses stages 0 and 1 (it is exactly half the size of the gate/up slice), which keeps a
-// CTA under half an SM's shared memory so two CTAs -- of this launch or of the next one -- can
-// share an SM.
+// Byte offsets, identical on host and device.  The two stages (a quarter of the gate/up K range
+// each) come first; the down block later takes both (it is exactly two stages large).  A CTA stays
+// under a quarter of an SM's shared memory, so four CTAs -- of this launch or of later ones -- share
+// an SM.
 struct FusedSmem {
     uint32_t stage0, stage_bytes;                      // stage s (a quarter of the K range) at stage0 + s * stage_bytes
     uint32_t mat_codes, mat_sz;                        // bytes of one (matrix, row tile) run of codes / sz inside a stage
@@ -359,8 +364,8 @@ __device__ __noinline__ void topk_large(float* work, int E, int K, int lane, int
 
 // One warp publishes head logits -- lane l owns logit `e` with value `v` when `own` is set -- into the
 // ring slot the next layer-step reads, and if they were the last ones of the head, computes the
-// top-k for the caller's inds_next / gates_next.  A chained next step does not wait for that: it
-// takes the logits from the ring and selects its experts itself.  `state` is the lane's entry of
+// top-k: the (expert, gate) pairs go behind the logits of the ring slot, where a chained next step
+// picks them up, and into the caller's inds_next / gates_next.  `state` is the lane's entry of
 // the ring slot as it was when the kernel started: a slot is written again only after the step
 // that read it has ended and has reset it.
 __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, float v, int e, bool own, int lane, uint32_t state) {
@@ -545,10 +550,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
         if (p.qpc * p.epc > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
     }
-    // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed just
-    // before the copies are issued: a cluster-scope barrier waits for every bulk copy in flight
-    // into the SM, those of a neighbouring CTA included, and that wait is hidden behind the loads
-    // below.
+    // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed
+    // before the first remote store: the arriving side of a cluster-scope barrier waits for every
+    // bulk copy in flight into the SM, those of a neighbouring CTA included, and that wait is
+    // hidden behind the loads below.
     cluster_arrive();
 
     // ---- everyone: the slot table of this layer (one coalesced read now saves a dependent trip to
@@ -867,10 +872,9 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         // ---- the four quarters of the intermediate dimension, one after the other.  For quarter c
         //      this CTA computes its rows_gu gate/up rows (over all of K), the cluster exchanges
         //      h = silu(gate) * up, and the CTA adds the quarter's columns to its rows_d output rows.
-        //      The weights stream through four stage buffers: gate/up of a quarter fills all four
-        //      (a K quarter each), its down block follows into stages 0-1 as soon as their warps
-        //      are done, the next quarter's K quarters 2-3 into stages 2-3 likewise, and its K
-        //      quarters 0-1 once the down block has been used.
+        //      The weights stream through the two stage buffers, one load at a time: the first half
+        //      of the K range of the gate/up rows (a K quarter per stage), the second half, the
+        //      quarter's down block, then the next quarter's first half.
 #pragma unroll 1
         for (int w = 0; w < n_items; ++w) {
             const int it = w % p.qpc, c = c0 + it, e = item_expert(w);
@@ -1203,7 +1207,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFusedSmemLimit);
         if (e != cudaSuccess) return e;
-        // two CTAs per SM: more clusters resident at once
+        // four CTAs per SM: more clusters resident at once
         e = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (e != cudaSuccess) return e;
         configured = true;

@@ -68,7 +68,9 @@ struct edg_store {
     const void* ring_ws = nullptr;         // workspace whose hand-off ring this store has initialised
     int ring_next = 0;                     // ring slot of the next batch-1 layer-step
     int pub_slot = -1;                     // ring slot holding logits no step has read yet, or -1
-    bool chaining = true;
+    int chaining = 1;                      // 0 off, 1 when the previous step is still in flight (or under capture), 2 always
+    cudaEvent_t step_done = nullptr;       // recorded behind every batch-1 layer-step launched outside a capture
+    bool step_done_valid = false;
 };
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
@@ -130,6 +132,7 @@ extern "C" int32_t edg_store_destroy(edg_store* s) {
     for (int i = 0; i < kRing; ++i)
         if (s->ring_ev[i]) cudaEventDestroy(s->ring_ev[i]);
     if (s->ring) cudaFreeHost(s->ring);
+    if (s->step_done) cudaEventDestroy(s->step_done);
     s->magic = 0;
     delete s;
     return EDG_OK;
@@ -267,8 +270,18 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         if (!workspace || !edg::aligned(workspace, 256) || workspace_bytes < edg::workspace_layout(s->d, 1).bytes)
             return EDG_E_WORKSPACE;
         if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
-        const bool chained = s->chaining && s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
-                             s->chain_stream == stream;
+        bool chained = s->chaining && s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
+                       s->chain_stream == stream;
+        // Chaining pays when steps queue up on the device: a chained step runs as a few long-lived
+        // CTAs that share the GPU with dozens of other steps.  A step that finds the GPU idle -- the
+        // step before it has already finished -- is launched on its own, across all SMs, which
+        // is several times faster for that one step.  Inside a stream capture nothing can be
+        // asked of the device; a captured sequence is replayed back to back, so it is chained.
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        EDG_CUDA_TRY(cudaStreamIsCapturing(st, &capturing));
+        if (chained && s->chaining == 1 && capturing == cudaStreamCaptureStatusNone && s->step_done_valid &&
+            cudaEventQuery(s->step_done) == cudaSuccess)
+            chained = false;
         // A workspace seen for the first time gets its ring cleared: counters to zero, logits to
         // "not yet written".  After that the ring looks after itself: a chained step resets the
         // slot it has read, and a step that starts over clears the slot the last head left unread.
@@ -295,6 +308,12 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
                                   logits_next_opt, workspace, flag_in, flag_out, ring, stale, st);
         if (W_pre_next != nullptr) s->pub_slot = flag_out;
         if (rc != EDG_OK) return rc;
+        s->step_done_valid = false;
+        if (capturing == cudaStreamCaptureStatusNone && s->chaining == 1) {
+            if (s->step_done == nullptr) EDG_CUDA_TRY(cudaEventCreateWithFlags(&s->step_done, cudaEventDisableTiming));
+            EDG_CUDA_TRY(cudaEventRecord(s->step_done, st));
+            s->step_done_valid = true;
+        }
         s->chain_inds = W_pre_next != nullptr ? inds_next : nullptr;
         s->chain_ws = workspace;
         s->chain_stream = stream;
@@ -312,6 +331,6 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
 
 extern "C" int32_t edg_store_set_chaining(edg_store* s, int32_t enable) {
     if (!store_ok(s)) return EDG_E_INVAL;
-    s->chaining = enable != 0;
+    s->chaining = enable < 0 ? 0 : (enable > 2 ? 2 : enable);
     return EDG_OK;
 }

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 
 
 def _run(cfg, store, d, W, xd, steps, ws, chaining):
-    store.set_chaining(chaining)
+    store.set_chaining(2 if chaining else 0)    # 2: chain whether or not the previous step is still running
     inds = torch.zeros((steps + 1, cfg.K), dtype=torch.int32, device="cuda")
     gates = torch.zeros((steps + 1, cfg.K), dtype=torch.float32, device="cuda")
     logits = torch.zeros((steps + 1, cfg.E), dtype=torch.float32, device="cuda")
@@ -75,6 +75,7 @@ def test_a_hand_off_that_never_arrives_times_out_and_falls_back():
     X = synth.hidden_states(cfg, 3, stream=29)
     xd = x_dev(X)
     ws = layer_io.new_workspace(d)
+    store.set_chaining(2)                       # the default would launch a step that finds the GPU idle on its own
     inds = torch.zeros((3, cfg.K), dtype=torch.int32, device="cuda")
     gates = torch.zeros((3, cfg.K), dtype=torch.float32, device="cuda")
     logits = torch.zeros((3, cfg.E), dtype=torch.float32, device="cuda")
