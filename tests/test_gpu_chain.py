@@ -103,3 +103,41 @@ def test_a_hand_off_that_never_arrives_times_out_and_falls_back():
         _assert_close(y_h[t], ref)
     _check_routing(logits[2].cpu().numpy(), inds_h[2], gates_h[2], W_np, X[1], cfg.K)
     store.close()
+
+
+def test_default_policy_gives_the_same_results_whether_or_not_steps_overlap():
+    """Default chaining policy: a step is chained only while the step before it is still in flight.
+    With a host synchronisation after every step each step finds the GPU idle and is launched on its
+    own; without one the steps queue up and are chained.  Indices and logits must be bit-equal in
+    both regimes and equal to those with chaining off; outputs agree far inside the tolerance."""
+    cfg = synth.CONFIGS["cfg1"]
+    steps = 24
+    store, d, hosts, slots, tables, cs, _ = _make_store(cfg, n_slots=cfg.E)
+    edg.stage_experts_to_slots(store, 0, np.arange(cfg.E, dtype=np.int32))
+    torch.cuda.synchronize()
+    W = torch.from_numpy(synth.prerouter_weights(cfg)).cuda()
+    xd = x_dev(synth.hidden_states(cfg, steps + 1, stream=31))
+    ws = layer_io.new_workspace(d)
+
+    def run(mode, sync_each):
+        store.set_chaining(mode)
+        inds = torch.zeros((steps + 1, cfg.K), dtype=torch.int32, device="cuda")
+        gates = torch.zeros((steps + 1, cfg.K), dtype=torch.float32, device="cuda")
+        logits = torch.zeros((steps + 1, cfg.E), dtype=torch.float32, device="cuda")
+        edg.prerouter_topk(d, W, xd[steps], 1, inds[0], gates[0], logits[0])
+        y = out_tensor(d, steps)
+        for t in range(steps):
+            edg.moe_layer_decode(store, 0, xd[t], inds[t], gates[t], W, inds[t + 1], gates[t + 1], logits[t + 1], y[t], ws)
+            if sync_each:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        assert edg.workspace_status(ws) == 0
+        return inds.cpu().numpy(), logits.cpu().numpy(), y.float().cpu().numpy()
+
+    ref = run(0, False)
+    for mode, sync_each in [(1, True), (1, False), (2, True)]:
+        got = run(mode, sync_each)
+        assert np.array_equal(got[0], ref[0])
+        assert np.array_equal(got[1], ref[1])
+        assert np.abs(got[2] - ref[2]).max() <= 1e-4
+    store.close()
