@@ -207,9 +207,9 @@ def run_b200(args):
 
     steps, warmup = args.steps, max(args.warmup, 3)
     full, rem = divmod(steps, G)
-    # The hand-off ring has 64 slots and a captured chain has its slots baked in, so graphs hold a
-    # multiple of 64 steps; what is left of --steps runs as direct calls at the end of the timed region.
-    tail = rem % 64
+    # The hand-off ring has 128 slots and a captured chain has its slots baked in, so graphs hold a
+    # multiple of 128 steps; what is left of --steps runs as direct calls at the end of the timed region.
+    tail = rem % 128
     rem -= tail
     g_full = capture(G) if full or warmup else None
     g_rem = capture(rem) if rem else None
@@ -234,7 +234,7 @@ def run_b200(args):
         e1.record(stream)
         stream.synchronize()
         ms = e0.elapsed_time(e1)
-        for s in range(tail, 64 if tail else 0):   # untimed: bring the ring back to where the graphs expect it
+        for s in range(tail, 128 if tail else 0):   # untimed: bring the ring back to where the graphs expect it
             step(s)
         # keep the GPU under the same load a little longer so the clock sampler sees it
         t_end = time.time() + 0.3

@@ -227,7 +227,7 @@ int32_t edg_store_mark_computed(edg_store* store, int32_t layer, void* stream);
  *   lora        host struct of dev pointers, or NULL for no adapter
  *   y           dev [T][H] of out_dtype
  *   workspace   dev, edg_ffn_workspace_bytes(desc, T) bytes, 256-byte aligned; holds the
- *               intermediate h and the rank-r projections.  Its first 2048 bytes are a control
+ *               intermediate h and the rank-r projections.  Its first 4096 bytes are a control
  *               block (sticky status word, see edg_workspace_status, and arrival counters) that
  *               the caller zeroes once before first use; the rest needs no initialisation.
  *               Calls that share a workspace must be ordered on the device.
@@ -276,13 +276,13 @@ int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* 
  * are chained: the later kernel is launched as a programmatic dependent of the earlier one, starts
  * as soon as that one is running, and takes its routing from a ring inside the workspace: the
  * earlier kernel leaves the logits of its head there and, behind them, the (expert, gate) pairs it
- * selects from them -- the same values it writes to inds_next / gates_next.  Up to 64 chained
+ * selects from them -- the same values it writes to inds_next / gates_next.  Up to 128 chained
  * steps share the GPU.  The results are those of unchained calls; what changes is the
  * contract on the inputs: a chained call reads x, W_pre_next and the slot pool as soon as it
  * starts, so they must already be valid when the call is made -- not produced by work queued
  * on the stream between the two calls.  Callers that cannot promise this switch chaining off
  * with edg_store_set_chaining.  A chain captured in a CUDA graph that is replayed back to back
- * must hold a multiple of 64 layer-steps, so that every replay finds the ring where the
+ * must hold a multiple of 128 layer-steps, so that every replay finds the ring where the
  * previous one left it. */
 int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          const int32_t* inds_cur, const float* gates_cur,

@@ -53,6 +53,7 @@ constexpr int kE16 = kC * kDownSlices;   // CTAs per expert
 constexpr int kFW = 4;            // warps per CTA
 constexpr int kStages = 2;        // copy stages per CTA: a quarter of the gate/up K range each, or half of the down block
 constexpr int kMaxRank = 64;
+constexpr int kMaxEpc = 4;         // experts a cluster may take, one after the other
 constexpr int kTraceMarks = 32;
 constexpr int kRing = kHandoffRing;   // chained layer-steps in flight: hand-off slots for logits, reduce scratch, counters
 constexpr uint32_t kSpinLimit = 1u << 22;   // bounded mbarrier polling
@@ -68,7 +69,7 @@ struct FusedSmem {
     uint32_t sz0;                                      // offset of the sz runs inside a stage
     uint32_t d_codes, d_sz;                            // down block, from stage0
     uint32_t lora0, lora_bytes;                        // two buffers of per-quarter adapter slices: B_gate rows, B_up rows, A_down columns
-    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_xbias, s_hb, s_hsum, s_hbias, flag, total;
+    uint32_t bars, s_u, s_h, s_ud_part, s_ud, s_gu, s_o, s_red, s_hloc, s_topk, s_part, s_table, s_xb, s_xsum, s_xbias, s_hb, s_hsum, s_hbias, flag, s_ex, total;
 };
 __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, int rank) {
     FusedSmem S;
@@ -112,6 +113,7 @@ __host__ __device__ inline FusedSmem fused_smem(int H, int I, int E, int group, 
     S.s_hsum = o;     o += (sw / 32) * 4;
     S.s_hbias = o;    o += (sw / 32) * 4;
     S.flag = o;       o += 16;
+    S.s_ex = o;       o += 96;                        // the cluster's experts: raw routing, then what the take made of it
     S.total = (o + 15) / 16 * 16;
     return S;
 }
@@ -144,7 +146,7 @@ struct FusedParams {
     int flag_out;                 // -1 or the ring slot that receives inds_next / gates_next
     int gshift;                   // log2(group)
     int qpc;                      // quarters of the intermediate dimension per cluster: 4 (one cluster per expert), 2 or 1
-    int epc;                      // experts per cluster, one after the other: 1, or 2 (only with qpc = 4)
+    int epc;                      // experts per cluster, one after the other: 1, or 2 or 4 (only with qpc = 4)
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     FusedSmem S;                  // shared-memory carve-up
 };
@@ -445,7 +447,7 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
 // instruction fetches compete with the weight stream for the same memory system.
 
 constexpr int kPreRed = 32;       // s_red rows 0..31: adapter projections, 32..39: head rows
-constexpr int kMaxPre = 4 * kFW;  // head rows per head CTA (two batches of two per warp)
+constexpr int kMaxPre = 8 * kFW;  // head rows per head CTA (up to four batches of two per warp)
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
 __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_constant__ FusedParams p) {
@@ -588,39 +590,37 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     }
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
-    // ---- a3: take, for the one or two experts of this cluster, as a function of the routing in
-    //      s_flag.  The decision is the same in every CTA of the cluster.  An expert that is out of
-    //      range is skipped (and flagged).  Warp 0 takes early, for the copies it issues; everyone
-    //      takes after the barrier.
-    int ad = 0;                               // two experts per cluster only with one shared adapter: ad = 0 for both
-    float gate0 = 0.f, gate1 = 0.f;
-    const uint8_t* rec0 = p.pool, *rec1 = p.pool;
-    bool ok0 = false, ok1 = false, valid = false;
-    int e_first = 0, n_items = 0;             // the items of this cluster's stream: the quarters of its valid experts, one expert after the other
-    auto take = [&]() {
-        {
-            int slot = s_flag[1];
-            gate0 = __int_as_float(s_flag[2]);
-            const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k] : 0);
-            if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
-            ad = 0;
-            if (r > 0 && p.n_adapters != 1) ad = (expert >= 0 && expert < p.E) ? expert : -1;
-            ok0 = slot >= 0 && slot < p.n_slots && ad >= 0;
-            if (ok0) rec0 = p.pool + (size_t)slot * p.L.bytes;
-            if (ad < 0) ad = 0;
+    // ---- a3: take, for the experts of this cluster (up to kMaxEpc, one after the other), as a
+    //      function of the routing warp 0 has put into s_ex.  The decision is the same in every CTA
+    //      of the cluster.  An expert that is out of range is skipped (and flagged).  Lane 0 of warp
+    //      0 resolves -- before the CTA's first barrier, for the copies warp 0 issues -- and leaves
+    //      the result in shared memory: s_ex[0..7] raw (expert or slot, gate) pairs, [8] number of
+    //      valid experts, [9] adapter, [10] mask of valid experts, [12..15] the valid experts in
+    //      order, [16..19] their slots, [20..23] their gates.
+    int* s_ex = reinterpret_cast<int*>(smem + S.s_ex);
+    auto take = [&]() {               // warp 0
+        if (lane == 0) {
+            int nv = 0, okm = 0, adv = 0;
+            for (int e = 0; e < p.epc; ++e) {
+                int slot = s_ex[2 * e];
+                const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k + e] : 0);
+                if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
+                int a_e = 0;          // several experts per cluster only with one shared adapter: 0 for all
+                if (r > 0 && p.n_adapters != 1) a_e = (expert >= 0 && expert < p.E) ? expert : -1;
+                const bool ok = slot >= 0 && slot < p.n_slots && a_e >= 0;
+                if (ok) { s_ex[12 + nv] = e; s_ex[16 + e] = slot; okm |= 1 << e; ++nv; if (e == 0) adv = a_e; }
+                s_ex[20 + e] = s_ex[2 * e + 1];
+            }
+            s_ex[8] = nv; s_ex[9] = adv; s_ex[10] = okm;
         }
-        if (p.epc == 2) {
-            int slot = s_flag[0];
-            gate1 = __int_as_float(s_flag[3]);
-            if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
-            ok1 = slot >= 0 && slot < p.n_slots;
-            if (ok1) rec1 = p.pool + (size_t)slot * p.L.bytes;
-        }
-        valid = ok0 || ok1;
-        e_first = ok0 ? 0 : 1;
-        n_items = ((ok0 ? 1 : 0) + (ok1 ? 1 : 0)) * p.qpc;
+        __syncwarp();
     };
-    auto item_expert = [&](int w) { return (ok0 && ok1) ? w / p.qpc : e_first; };
+    int ad = 0, n_items = 0;          // set from s_ex: by warp 0 right after its take, by everyone after the barrier
+    bool valid = false;
+    auto read_take = [&]() { n_items = s_ex[8] * p.qpc; ad = s_ex[9]; valid = n_items > 0; };
+    // the items of this cluster's stream: the quarters of its valid experts, one expert after the other
+    auto item_expert = [&](int w) { return s_ex[12 + w / p.qpc]; };
+    auto item_rec = [&](int w) { return p.pool + (size_t)s_ex[16 + item_expert(w)] * p.L.bytes; };
     const int cps = p.H / 128;            // chunks of a row per stage
     const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
     const int gps = sw >> p.gshift;       // groups of a down row-slice
@@ -633,7 +633,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     // (one arrival per issuing warp).  The calling warp plays warps v0 .. v1 - 1.
     auto issue_gu = [&](int w, int pair, int v0, int v1) {
         const int c = c0 + w % p.qpc;
-        const uint8_t* rec = item_expert(w) ? rec1 : rec0;
+        const uint8_t* rec = item_rec(w);
         const uint64_t pol = policy_evict_first();       // weights stream through L2 once
         for (int v = v0; v < v1; ++v) {
             const int s = v >> 1, run = (v & 1) * 4 + lane, kq = pair * 2 + s;
@@ -681,7 +681,9 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
 #pragma unroll 1
     for (int pass = 0; pass < 2; ++pass) {
         if (warp == 0 && !routed && (pass || p.flag_in < 0)) {
-            int vi[2] = {-1, -1}, vg[2] = {0, 0};
+            int vi[kMaxEpc], vg[kMaxEpc];
+#pragma unroll
+            for (int e = 0; e < kMaxEpc; ++e) { vi[e] = -1; vg[e] = 0; }
             bool got = false;
             if (p.flag_in >= 0) {
                 const unsigned long long* pr = reinterpret_cast<const unsigned long long*>(p.logits_ws + (size_t)p.flag_in * (p.E + kPairWords) + p.E);
@@ -696,7 +698,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                     // ring slot being free again, above all) is ordered before what this CTA does next
                     asm volatile("fence.acq_rel.gpu;" ::: "memory");
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
+                    for (int e = 0; e < kMaxEpc; ++e) {
                         const unsigned long long we = __shfl_sync(0xFFFFFFFFu, w, (k + e) & 31);
                         if (e < p.epc) { vi[e] = (int)(uint32_t)we; vg[e] = (int)(uint32_t)(we >> 32); }
                     }
@@ -711,16 +713,19 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
             if (p.flag_in < 0 || (!got && pass)) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e)
+                for (int e = 0; e < kMaxEpc; ++e)
                     if (e < p.epc) { vi[e] = __ldcg(&p.slots[k + e]); vg[e] = __float_as_int(__ldcg(&p.gates[k + e])); }
                 got = true;
             }
             if (got) {
-                // (the second expert's pair sits in words 0 and 3, which the end of the kernel uses for its flags)
-                if (lane == 0) { s_flag[1] = vi[0]; s_flag[2] = vg[0]; s_flag[0] = vi[1]; s_flag[3] = vg[1]; }
+                if (lane == 0) {
+#pragma unroll
+                    for (int e = 0; e < kMaxEpc; ++e) { s_ex[2 * e] = vi[e]; s_ex[2 * e + 1] = vg[e]; }
+                }
                 __syncwarp();
                 trace_mark(p, 14);
                 take();
+                read_take();
                 if (valid) {
                     // the copies of the first quarter, and of the adapter rows every quarter needs
                     issue_gu(0, 0, 0, kFW);
@@ -815,7 +820,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         head_publish(p, smem, v, e, own, lane, pre_state);
     }
 
-    take();
+    read_take();
     trace_mark(p, 10);
     cluster_wait();
 
@@ -878,7 +883,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
 #pragma unroll 1
         for (int w = 0; w < n_items; ++w) {
             const int it = w % p.qpc, c = c0 + it, e = item_expert(w);
-            const uint8_t* rec = e ? rec1 : rec0;
+            const uint8_t* rec = item_rec(w);
             const uint32_t par = w & 1, par2 = (w >> 1) & 1;
             // the adapter slices of the next quarter go into the buffer the previous quarter used:
             // a score of small copies, issued while this quarter's weights are still on their way
@@ -1106,7 +1111,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 __syncthreads();          // s_o and s_ud complete
                 // LoRA B for down (A_down.h summed over the quarters; the rows of B_down come
                 // straight from memory, 2r bytes each) and the gate weight: one thread per output row
-                const float gate_k = e ? gate1 : gate0;
+                const float gate_k = __int_as_float(s_ex[20 + e]);
                 float* prow = partial + ((size_t)(k + e) * nq + cq) * p.H + n0_d;
                 const uint16_t* Bd = static_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r;
                 constexpr int kRowsPerThread = rows_d / (kFW * 32);
@@ -1130,12 +1135,11 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         trace_mark(p, 8);
     }
     // a skipped expert contributes nothing
-    if (!ok0 || (p.epc == 2 && !ok1)) {
+    if (s_ex[8] != p.epc) {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
-        if (!ok0)
-            for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)k * nq + cq) * p.H + n0_d + i] = 0.f;
-        if (p.epc == 2 && !ok1)
-            for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)(k + 1) * nq + cq) * p.H + n0_d + i] = 0.f;
+        for (int e = 0; e < p.epc; ++e)
+            if (!((s_ex[10] >> e) & 1))
+                for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)(k + e) * nq + cq) * p.H + n0_d + i] = 0.f;
     }
 
     // ---- a6: this partial is published; the last arriver for the block of rows sums all partials
@@ -1268,8 +1272,11 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     // CTAs per step, each amortising its start-up over twice the bytes
     // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
     // CTAs per step, each amortising its start-up over twice the bytes
-    const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // up to 4 kFW head rows per CTA
-    p.epc = (flag_in >= 0 && d->K % 2 == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (d->K / 2) * kC * kMaxPre >= d->E) ? 2 : 1;
+    const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // up to 8 kFW head rows per CTA
+    p.epc = 1;
+    for (int c = 2; c <= kMaxEpc; c *= 2)
+        if (flag_in >= 0 && d->K % c == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (W_pre == nullptr || (d->K / c) * kC * kMaxPre >= d->E))
+            p.epc = c;
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
     const bool pdl = flag_in >= 0;

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 def _ffn_tokens(L, d, X_bits, inds, gates, T, use_table=True):
     if L.ws.numel() < edg.ffn_workspace_bytes(d, T):
         L.ws = layer_io.new_workspace(d, T)
-    L.ws[:2048].zero_()
+    L.ws[:4096].zero_()
     y = out_tensor(d, T)
     table = torch.arange(d.E, dtype=torch.int32, device="cuda") if use_table else None
     edg.moe_expert_ffn_int4_lora(d, L.pool, table, T, inds, inds, gates, x_dev(X_bits), L.lora, y, L.ws)
@@ -154,7 +154,7 @@ def test_grouped_reduces_to_the_decode_path_and_handles_per_expert_adapters():
     assert orc.max_abs(y1[0], Y[0]) <= TOL_MAX_ABS and orc.rel_l2(y1[0], Y[0]) <= TOL_REL_L2
     # an out-of-range expert in one pair is skipped and flagged, the other tokens are untouched
     bad = inds_h.copy(); bad[5, 1] = cfg.E
-    L.ws[:2048].zero_()
+    L.ws[:4096].zero_()
     y = out_tensor(L.desc, T)
     edg.moe_expert_ffn_int4_lora(L.desc, L.pool, torch.arange(cfg.E, dtype=torch.int32, device="cuda"), T,
                                  torch.from_numpy(bad).cuda(), None, gates, x_dev(X), L.lora, y, L.ws)

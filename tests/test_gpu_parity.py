@@ -115,7 +115,7 @@ def _run_ffn(L, d, x_bits, inds, gates, lora, T=1, use_table=False, experts="sam
     g = torch.tensor(np.asarray(gates, dtype=np.float32).reshape(T, d.K), device="cuda")
     table = torch.arange(d.E, dtype=torch.int32, device="cuda") if use_table else None
     ex = slots if experts == "same" else experts
-    L.ws[:2048].zero_()
+    L.ws[:4096].zero_()
     edg.moe_expert_ffn_int4_lora(d, L.pool, table, T, slots, ex, g, x_dev(x_bits), lora, y, L.ws)
     torch.cuda.synchronize()
     return y

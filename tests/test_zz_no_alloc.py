@@ -26,7 +26,7 @@ def test_static_scratch_entry_point_matches_the_regular_one_twice():
         gates = torch.tensor(rng.dirichlet(np.ones(cfg.K)).astype(np.float32), device="cuda")
         x = x_dev(X[call:call + 1])
         y_ref, y_new = out_tensor(d), out_tensor(d)
-        L.ws[:2048].zero_()
+        L.ws[:4096].zero_()
         edg.moe_expert_ffn_int4_lora(d, L.pool, None, 1, inds, inds, gates, x, L.lora, y_ref, L.ws)
         edg.moe_expert_ffn_int4_lora_static(d, L.pool, None, inds, inds, gates, x, L.lora, y_new)
         torch.cuda.synchronize()
