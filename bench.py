@@ -42,7 +42,7 @@ UNIT = "tok/s"
 WORKLOAD = "cfg2: one 35B-class MoE layer (H2048 I512 E256 top-8 int4 g64 LoRA r16), batch-1 decode"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised in profiles/fused_layer_kernel_cfg2.md.
-NCU_TRAFFIC_BYTES = 15_586_560
+NCU_TRAFFIC_BYTES = 15_591_424
 
 
 def _peaks():
@@ -586,7 +586,7 @@ def run_cfg3(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10000)
+    ap.add_argument("--steps", type=int, default=10240)
     ap.add_argument("--warmup", type=int, default=100)
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--instances", type=int, default=8, help="independently seeded resident layer instances")
