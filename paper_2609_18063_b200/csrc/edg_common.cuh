@@ -76,15 +76,14 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 // Workspace layout for T tokens (floats unless noted).  The first kCtrlBytes bytes are a control
 // block that must start out zero: its first int32 is the device-side status word, the rest are the
 // counters of the ring that chained batch-1 layer-steps share (arrivals of the reduce, head rows
-// delivered, reducers finished, head finished -- one set per ring slot).
+// delivered, reducers finished -- one set per ring slot).
 constexpr int kPairWords = 64;         // words behind the logits of a ring slot: 32 (expert, gate) pairs, the routing itself
 constexpr int kHandoffRing = 128;      // ring slots shared by chained batch-1 layer-steps in flight
 constexpr size_t kCtrlBytes = 4096;    // control block: status word at 0, then the ring's counters
 constexpr size_t kCtrlCounters = 64;                               // [ring][4] arrivals per block of output rows
 constexpr size_t kCtrlHead = kCtrlCounters + kHandoffRing * 16;    // [ring] head rows delivered
 constexpr size_t kCtrlDone = kCtrlHead + kHandoffRing * 4;         // [ring] reducers finished
-constexpr size_t kCtrlFin = kCtrlDone + kHandoffRing * 4;          // [ring] head finished
-static_assert(kCtrlFin + kHandoffRing * 4 <= kCtrlBytes, "control block too small");
+static_assert(kCtrlDone + kHandoffRing * 4 <= kCtrlBytes, "control block too small");
 
 struct WorkspaceLayout {
     size_t ctrl;      // kCtrlBytes control block

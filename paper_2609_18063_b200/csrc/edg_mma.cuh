@@ -70,17 +70,6 @@ __device__ __forceinline__ uint4 permute8(const float (&v)[8]) {
     return r;
 }
 
-// The same without a zero point: exact codes q (the zero point is then applied on the fp32 partial
-// sum as z * sum(x)).
-__device__ __forceinline__ void dequant_word_q(uint32_t w, uint32_t (&out)[4]) {
-    const __half2 k1024 = __float2half2_rn(1024.f), k64 = __float2half2_rn(64.f), k16th = __float2half2_rn(0.0625f);
-    const uint32_t w2 = w >> 8;
-    out[0] = h2_as_u32(__hsub2(u32_as_h2(lop3_and_or(w, 0x000F000Fu, 0x64006400u)), k1024));
-    out[1] = h2_as_u32(__hfma2(u32_as_h2(lop3_and_or(w, 0x00F000F0u, 0x64006400u)), k16th, __hneg2(k64)));
-    out[2] = h2_as_u32(__hsub2(u32_as_h2(lop3_and_or(w2, 0x000F000Fu, 0x64006400u)), k1024));
-    out[3] = h2_as_u32(__hfma2(u32_as_h2(lop3_and_or(w2, 0x00F000F0u, 0x64006400u)), k16th, __hneg2(k64)));
-}
-
 // The cheapest form: the code words masked straight into fp16 with a bias -- codes 0, 2, 4, 6 of a
 // word as 1024 + q, codes 1, 3, 5, 7 as 64 + q (their nibble sits four bits higher in the
 // mantissa) -- five instructions a word.  The dot product then carries 1024 * (sum of the
