@@ -141,3 +141,35 @@ def test_default_policy_gives_the_same_results_whether_or_not_steps_overlap():
         assert np.array_equal(got[1], ref[1])
         assert np.abs(got[2] - ref[2]).max() <= 1e-4
     store.close()
+
+
+@pytest.mark.parametrize("per_expert_adapters", [False, True])
+def test_chained_small_layer_with_an_fp16_head(per_expert_adapters):
+    """The small layer shape with an fp16 head, chained unconditionally.  With one shared adapter a
+    cluster takes both routed experts one after the other; with one adapter per expert every expert
+    has a cluster of its own and the adapter follows the expert.  Every step is checked against the
+    oracle on the routing the GPU produced."""
+    import dataclasses
+    base = synth.CONFIGS["cfg1"]
+    cfg = dataclasses.replace(base, pre_dtype="f16", n_adapters=base.E if per_expert_adapters else 1)
+    steps = 20
+    store, d, hosts, slots, tables, cs, _ = _make_store(cfg, n_slots=cfg.E)
+    edg.stage_experts_to_slots(store, 0, np.arange(cfg.E, dtype=np.int32))
+    torch.cuda.synchronize()
+    W_np = synth.prerouter_weights(cfg)
+    W = torch.from_numpy(W_np).cuda()
+    X = synth.hidden_states(cfg, steps + 1, stream=37)
+    xd = x_dev(X)
+    ws = layer_io.new_workspace(d)
+    inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, xd, steps, ws, True)
+    inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, xd, steps, ws, False)
+    assert np.array_equal(inds_c, inds_u) and np.array_equal(logits_c, logits_u) and np.array_equal(gates_c, gates_u)
+    assert np.abs(y_c - y_u).max() <= 1e-4
+    experts, adapters = {}, {}
+    get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
+    get_lora = lambda e: adapters.setdefault(e if per_expert_adapters else 0, synth.lora_tensors(cfg, 0, e if per_expert_adapters else 0))
+    for t in range(steps):
+        ref = orc.moe_ffn(X[t], inds_c[t], gates_c[t].astype(np.float64), get, get_lora, cfg.lora_scale, cfg.group)
+        _assert_close(y_c[t], ref)
+        _check_routing(logits_c[t + 1], inds_c[t + 1], gates_c[t + 1], W_np.astype(np.float32), X[t], cfg.K)
+    store.close()
