@@ -667,9 +667,9 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      step takes its routing from the hand-off ring: the (expert, gate) pairs that the head of
     //      the step before it has left behind its logits, long before that kernel ends.  Its own
     //      head rows come first (pass 0) -- nothing this kernel owes to a later step is ever held
-    //      back by a wait -- then warp 0 waits for the pairs (pass 1), takes, and issues the copies
-    //      of the first quarter by itself, ahead of the CTA's first barrier.  A step that is not
-    //      chained has its routing in memory and issues before its head rows.  Bounded wait; on a
+    //      back by a wait -- then warp 0 waits for the pairs (pass 1) and takes; the copies of the
+    //      first quarter are issued by all warps right behind the CTA's first barrier.  A step that
+    //      is not chained has its routing in memory: warp 0 issues before its head rows.  Bounded wait; on a
     //      time-out fall back to waiting for the whole previous kernel and to the routing it has
     //      written, which is always sufficient.
     bool routed = false;                  // warp 0: routing taken, first copies issued
@@ -721,8 +721,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 trace_mark(p, 14);
                 take();
                 read_take();
-                if (valid) {
-                    // the copies of the first quarter, and of the adapter rows every quarter needs
+                // A step on its own issues the copies of the first quarter here, ahead of its head
+                // rows; in a chained step the other warps are already waiting at the barrier below,
+                // and all four issue their share right behind it, which is quicker.
+                if (valid && p.flag_in < 0) {
                     issue_gu(0, 0, 0, kFW);
                     if (r > 0) issue_lora(0);
                 }
@@ -816,6 +818,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     }
 
     read_take();
+    if (valid && p.flag_in >= 0) {
+        issue_gu(0, 0, warp, warp + 1);
+        if (warp == kFW - 1 && r > 0) issue_lora(0);
+    }
     trace_mark(p, 10);
     cluster_wait();
 
