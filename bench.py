@@ -192,27 +192,34 @@ def run_b200(args):
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
 
-    def capture(n_steps):
+    # touch every instance once outside capture (an even count keeps the two-entry routing ring in
+    # phase), so that no staging event is waited on inside a graph
+    with torch.cuda.stream(stream):
+        for s in range(2 * n_inst):
+            step(s)
+        stream.synchronize()
+
+    def capture(n_steps, base=0):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
-            # touch every instance once outside capture (an even count keeps the two-entry routing
-            # ring in phase), so that no staging event is waited on inside the graph
-            for s in range(2 * n_inst):
-                step(s)
-            stream.synchronize()
             with torch.cuda.graph(g, stream=stream):
-                for s in range(n_steps):
+                for s in range(base, base + n_steps):
                     step(s)
         return g
 
     steps, warmup = args.steps, max(args.warmup, 3)
     full, rem = divmod(steps, G)
-    # The hand-off ring has 128 slots and a captured chain has its slots baked in, so graphs hold a
-    # multiple of 128 steps; what is left of --steps runs as direct calls at the end of the timed region.
+    # The hand-off ring has 128 slots and a captured chain has its slots baked in: a graph that is
+    # replayed again and again holds a multiple of 128 steps.  What is left of --steps is a graph of
+    # its own, captured and replayed last, and followed (untimed) by its complement to 128 so that
+    # the ring is back where the other graphs expect it.  The graphs are captured in the order in
+    # which they run, each starting where the one before it ends.
     tail = rem % 128
     rem -= tail
     g_full = capture(G) if full or warmup else None
     g_rem = capture(rem) if rem else None
+    g_tail = capture(tail) if tail else None
+    g_comp = capture(128 - tail, base=tail) if tail else None
 
     sampler = ClockSampler(_physical_device(local_rank))
     with torch.cuda.stream(stream):
@@ -229,13 +236,13 @@ def run_b200(args):
             g_full.replay()
         if g_rem is not None:
             g_rem.replay()
-        for s in range(tail):
-            step(s)
+        if g_tail is not None:
+            g_tail.replay()
         e1.record(stream)
         stream.synchronize()
         ms = e0.elapsed_time(e1)
-        for s in range(tail, 128 if tail else 0):   # untimed: bring the ring back to where the graphs expect it
-            step(s)
+        if g_comp is not None:
+            g_comp.replay()
         # keep the GPU under the same load a little longer so the clock sampler sees it
         t_end = time.time() + 0.3
         while time.time() < t_end and g_full is not None:
