@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(1024) build_tiles_kernel(GroupedParams p) {
 // both gate and up, so silu(g) * u is formed in registers.
 
 template <int G_NT>
-__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_gate_up_kernel(GroupedParams p) {
+__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 4 : 2) grouped_gate_up_kernel(GroupedParams p) {
     constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;
@@ -268,7 +268,7 @@ __global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_gate_
 // CTA = (tile of up to 64 pairs of one slot) x (256 rows of H).  Warp w owns rows 32w..32w+31.
 
 template <int G_NT>
-__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 3 : 2) grouped_down_kernel(GroupedParams p) {
+__global__ void __launch_bounds__(G_WARPS * 32, G_NT == 1 ? 4 : 2) grouped_down_kernel(GroupedParams p) {
     constexpr int G_NTOK = G_NT * 8;
     const int tile = blockIdx.x;
     if (tile >= *p.n_tiles) return;

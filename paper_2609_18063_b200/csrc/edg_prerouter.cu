@@ -9,6 +9,7 @@
 #include <math_constants.h>
 
 #include "edg_common.cuh"
+#include "edg_mma.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -190,6 +191,88 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_kernel(PrePar
     }
 }
 
+// The same for an fp16 head on the tensor cores: the block's 8 tokens are the 8 columns of an
+// m16n8k16 tile, 16 rows of the head its rows.  A CTA takes its share of the rows tile by tile; warp
+// w multiplies K slice w of every tile (A fragments straight from memory: the 16 k of a step are one
+// full 32-byte sector per row; B fragments from the tokens' states, fp16 in shared memory, rows
+// padded by 16 bytes so the eight token rows fall into different banks), the slices are summed
+// through shared memory, and the logits go to the leader as above.  fp16 of a bf16 state is exact in
+// the normal range; products are exact in fp32 and summed in fp32.
+__global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(PreParams p, int T) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
+    const int csize = (int)cluster.num_blocks();
+    const int t0 = blockIdx.y * kTokBlock;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
+    extern __shared__ float smem[];
+    float* s_logits = smem;                                             // [kTokBlock][E]
+    float* s_red = smem + kTokBlock * p.E;                              // [kPreWarps][16 x 8] partial tiles
+    const int xs = p.H * 2 + 16;                                        // bytes per token row
+    uint8_t* s_xh = reinterpret_cast<uint8_t*>(s_red + kPreWarps * 128);    // [kTokBlock][H + 8] fp16
+    for (int tt = 0; tt < kTokBlock; ++tt) {
+        const int t = t0 + tt;
+        for (int i = threadIdx.x; i < p.H; i += blockDim.x)
+            *reinterpret_cast<__half*>(s_xh + tt * xs + i * 2) = __float2half_rn(t < T ? bf16_bits_to_float(p.s[(size_t)t * p.H + i]) : 0.f);
+    }
+    __syncthreads();
+
+    float* leader = cluster.map_shared_rank(s_logits, 0);
+    const int per = p.E / csize;                                        // rows of this CTA: a multiple of 16
+    const int ksl = p.H / kPreWarps;                                    // k per warp: a multiple of 16
+    const __half* W = static_cast<const __half*>(p.W);
+    for (int r0 = crank * per; r0 < (crank + 1) * per; r0 += 16) {
+        const __half* wlo = W + (size_t)(r0 + g) * p.H + warp * ksl + 2 * t4;
+        const __half* whi = wlo + (size_t)8 * p.H;
+        const uint8_t* xb = s_xh + g * xs + (warp * ksl + 2 * t4) * 2;
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int k0 = 0; k0 < ksl; k0 += 64) {                          // four steps' worth of loads in flight
+            uint32_t a[4][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = k0 + 16 * u;
+                const bool on = k < ksl;
+                a[u][0] = on ? ld_stream4(wlo + k) : 0u;
+                a[u][1] = on ? ld_stream4(whi + k) : 0u;
+                a[u][2] = on ? ld_stream4(wlo + k + 8) : 0u;
+                a[u][3] = on ? ld_stream4(whi + k + 8) : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int k = k0 + 16 * u;
+                if (k < ksl) {
+                    const uint32_t b0 = *reinterpret_cast<const uint32_t*>(xb + k * 2);
+                    const uint32_t b1 = *reinterpret_cast<const uint32_t*>(xb + k * 2 + 16);
+                    mma16816(c, a[u][0], a[u][1], a[u][2], a[u][3], b0, b1);
+                }
+            }
+        }
+        // rows g / g + 8, tokens 2 t4 / 2 t4 + 1 of this warp's K slice
+        float* mine = s_red + warp * 128;
+        mine[g * 8 + 2 * t4] = c[0]; mine[g * 8 + 2 * t4 + 1] = c[1];
+        mine[(g + 8) * 8 + 2 * t4] = c[2]; mine[(g + 8) * 8 + 2 * t4 + 1] = c[3];
+        __syncthreads();
+        if (threadIdx.x < 128) {
+            float v = 0.f;
+#pragma unroll
+            for (int w = 0; w < kPreWarps; ++w) v += s_red[w * 128 + threadIdx.x];
+            const int row = threadIdx.x >> 3, tok = threadIdx.x & 7;
+            leader[tok * p.E + r0 + row] = v;
+        }
+        __syncthreads();
+    }
+    cluster.sync();                     // every CTA's logits have landed in the leader
+    if (crank != 0) return;
+
+    const int t = t0 + warp;            // kPreWarps == kTokBlock: warp w finishes token w of the block
+    if (warp < kTokBlock && t < T) {
+        float* row = s_logits + warp * p.E;
+        if (p.logits != nullptr)
+            for (int e = lane; e < p.E; e += 32) p.logits[(size_t)t * p.E + e] = row[e];
+        __syncwarp();
+        warp_softmax_topk(row, p.E, p.K, lane, p.inds + (size_t)t * p.K, p.gates + (size_t)t * p.K);
+    }
+}
+
 // a2 alone: one warp per row of given logits.
 __global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* logits, int T, int E, int K,
                                                                 int32_t* inds, float* gates) {
@@ -229,9 +312,16 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
         if (!configured) {
             EDG_CUDA_TRY(cudaFuncSetAttribute(prerouter_tokens_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
             EDG_CUDA_TRY(cudaFuncSetAttribute(prerouter_tokens_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            EDG_CUDA_TRY(cudaFuncSetAttribute(prerouter_tokens_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
             configured = true;
         }
         if (cfg.dynamicSmemBytes > 200 * 1024) return EDG_E_SHAPE;
+        // an fp16 head whose rows and columns split into whole MMA tiles goes to the tensor cores
+        if (d->pre_dtype == EDG_F16 && d->E % (16 * kPreCluster) == 0 && d->H % (16 * kPreWarps) == 0) {
+            cfg.dynamicSmemBytes = (size_t)kTokBlock * d->E * 4 + kPreWarps * 128 * 4 + (size_t)kTokBlock * (d->H * 2 + 16);
+            EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_mma_kernel, p, (int)n_heads));
+            return EDG_OK;
+        }
         if (d->pre_dtype == EDG_F16) EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_kernel<__half>, p, (int)n_heads));
         else EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_kernel<float>, p, (int)n_heads));
         return EDG_OK;
