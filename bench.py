@@ -590,6 +590,43 @@ def run_cfg3(args):
                       "arms": out}))
 
 
+def run_sigmoid_group(args):
+    """The paper's second routing family (Appendix A, sigmoid-group; 8B tier: E = 128, n = 8 groups,
+    keep 4, K = 8, scale 2.5) on given logits: rows per second and bytes per second of the one kernel."""
+    import torch
+    import paper_2609_18063_b200 as edg
+    peak, how = _peaks()
+    E, K, n, G, T = 128, 8, 8, 4, 1 << 19           # 268 MB of logits: larger than L2
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    logits = torch.randn((T, E), generator=g, device="cuda", dtype=torch.float32) * 2.0
+    bias = (torch.rand((E,), generator=g, device="cuda", dtype=torch.float32) - 0.5) * 0.1
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    steps, warmup = max(1, min(args.steps, 50)), max(args.warmup, 3)
+    for _ in range(warmup):
+        edg.sigmoid_group_topk_rows(logits, T, E, K, n, G, 2.5, bias, inds, gates)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        edg.sigmoid_group_topk_rows(logits, T, E, K, n, G, 2.5, bias, inds, gates)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert int(inds.min()) >= 0 and int(inds.max()) < E and abs(float(gates[0].sum()) - 2.5) < 1e-4
+    alg = T * (E * 4 + K * 8)
+    achieved = alg / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "sigmoid_group_routing_rows_per_s", "value": round(T / (ms * 1e-3), 1), "unit": "rows/s",
+                      "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": round(ms, 5), "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "sigmoid-group routing, 8B-tier shape: E=128, 8 groups keep 4, top-8, scale 2.5, 524288 rows of logits",
+                                 "l2": "268 MB of logits per launch exceed the 126 MB L2"},
+                      "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                                   "frac": round(achieved / peak, 4), "traffic": None, "peak_kind": how,
+                                   "algorithmic_bytes_per_launch": alg},
+                      "gpu_launches": steps}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -601,7 +638,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", choices=["cfg2", "cfg3", "cfg4", "cfg5"], default="cfg2",
+    ap.add_argument("--workload", choices=["cfg2", "cfg3", "cfg4", "cfg5", "sigmoid_group"], default="cfg2",
                     help="cfg2 is the headline line; the others print their own line")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -612,6 +649,8 @@ def main():
         run_cfg4(args)
     elif args.workload == "cfg5":
         run_cfg5(args)
+    elif args.workload == "sigmoid_group":
+        run_sigmoid_group(args)
     else:
         run_b200(args)
 

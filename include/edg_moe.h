@@ -170,6 +170,21 @@ int32_t prerouter_topk_tokens(const edg_layer_desc* desc, const void* W_pre, con
 int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,
                           int32_t* inds, float* gates, void* stream);
 
+/* The other routing family of the paper (Appendix A, "Sigmoid-group"; its 8B tier runs n = 8 groups,
+ * keep G = 4, K = 8, scale 2.5, E = 128) on given logits: sigma = sigmoid(l); a group's score is the
+ * sum of its two largest selection scores, where the selection score is sigma, plus bias_opt[e] when a
+ * bias is given (the "biased score" of the paper's remark); the keep_groups best groups survive,
+ * ties to the lower group; the K best survivors by selection score are taken, ties to the lower
+ * index; gates = scale * sigma[inds] / (sum of sigma[inds] + 1e-20) -- the raw sigmoid, not the biased
+ * score.  logits dev float [T][E]; bias_opt dev float [E] or NULL; inds dev int32 [T][K] in
+ * ascending index; gates dev float [T][K] aligned with inds.  E <= 1024, n_groups <= 32 dividing E
+ * with at least two experts a group, K <= 32 and <= keep_groups * E / n_groups; else EDG_E_SHAPE.
+ * One warp per row; no workspace; arithmetic in fp32 (the decision is taken in the kernel's
+ * precision). */
+int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32_t E, int32_t K, int32_t n_groups,
+                                int32_t keep_groups, float scale, const float* bias_opt,
+                                int32_t* inds, float* gates, void* stream);
+
 /* ---------------------------------------------------------------- a3: slot-pool expert store */
 
 /* Creates the store of n_layers layers (Sec. 3.1 "staged" path; Fig. 1: bounded streaming pool

@@ -293,8 +293,10 @@ __device__ __forceinline__ void topk_cex(uint32_t& ka, int& ia, uint32_t& kb, in
     ka = tk; kb = uk; ia = ti; ib = ui;
 }
 
+// (the selection alone: lane j < K ends up with winner j -- value myv, index myi, or myi == INT_MAX
+// when there were fewer than K candidates; entries of work[] that are NaN are not candidates)
 template <int V>
-__device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+__device__ __forceinline__ void warp_topk_reg(const float* work, int E, int K, int lane, float& myv, int& myi) {
     static_assert(V == 8, "the sorting network below is for 8 candidates per lane");
     const unsigned full = 0xFFFFFFFFu;
     uint32_t key[V];
@@ -316,8 +318,8 @@ __device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, 
     EDG_CEX(2, 4); EDG_CEX(3, 5);
     EDG_CEX(3, 4);
 #undef EDG_CEX
-    float myv = 0.f;
-    int myi = 0x7FFFFFFF;
+    myv = 0.f;
+    myi = 0x7FFFFFFF;
 #pragma unroll 1
     for (int j = 0; j < K; ++j) {
         const uint32_t best = __reduce_max_sync(full, key[0]);
@@ -333,6 +335,13 @@ __device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, 
             key[V - 1] = 0u;
         }
     }
+}
+
+template <int V>
+__device__ __forceinline__ void warp_softmax_topk_reg(const float* work, int E, int K, int lane, int32_t* inds, float* gates) {
+    float myv;
+    int myi;
+    warp_topk_reg<V>(work, E, K, lane, myv, myi);
     topk_emit(myv, myi, K, lane, inds, gates);
 }
 

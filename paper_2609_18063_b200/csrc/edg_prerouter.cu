@@ -286,6 +286,100 @@ __global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* log
     warp_softmax_topk(work, E, K, lane, inds + (size_t)t * K, gates + (size_t)t * K);
 }
 
+// Appendix A, sigmoid-group routing, one warp per row of given logits: sigma = sigmoid(l); a group's
+// score is the sum of its two largest selection scores (sigma, plus a bias when one is given); the
+// best `keep` of the `n` groups survive (ties to the lower group); top-K among the survivors by
+// selection score (ties to the lower index); w = scale * sigma[inds] / (sum sigma[inds] + 1e-20):
+// the weights use the raw sigmoid.  Winners are written in ascending index.
+__global__ void __launch_bounds__(128) sigmoid_group_topk_rows_kernel(const float* logits, const float* bias, int T, int E, int K,
+                                                                      int n, int keep, float scale, int32_t* inds, float* gates) {
+    extern __shared__ float smem[];
+    const unsigned full = 0xFFFFFFFFu;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * 4 + warp;
+    if (t >= T) return;
+    float* sig = smem + warp * 2 * E;          // [E] raw sigmoid
+    float* sel = sig + E;                      // [E] selection score; NaN = not a candidate (any more)
+    for (int e = lane; e < E; e += 32) {
+        const float sg = 1.f / (1.f + expf(-logits[(size_t)t * E + e]));
+        sig[e] = sg;
+        sel[e] = bias != nullptr ? sg + bias[e] : sg;
+    }
+    __syncwarp();
+    // group scores.  When the groups divide the warp, 32 / n lanes share a group: each scans its part,
+    // the (largest, second largest) pairs are merged by a butterfly, and every lane of the group
+    // ends up with the group's score; otherwise lane g scans group g alone.
+    const int per = E / n;
+    float gs = -CUDART_INF_F;
+    const int lpg = 32 / n;                    // lanes per group (when n divides 32)
+    const bool split = (32 % n) == 0 && (per % lpg) == 0;
+    if (split || lane < n) {
+        const int grp = split ? lane / lpg : lane, part = split ? lane % lpg : 0, cnt = split ? per / lpg : per;
+        float m1 = -CUDART_INF_F, m2 = -CUDART_INF_F;
+        for (int i = 0; i < cnt; ++i) {
+            const float v = sel[grp * per + part * cnt + i];
+            if (v > m1) { m2 = m1; m1 = v; } else if (v > m2) m2 = v;
+        }
+        if (split) {
+            for (int o = 1; o < lpg; o <<= 1) {
+                const float o1 = __shfl_xor_sync(full, m1, o), o2 = __shfl_xor_sync(full, m2, o);
+                const float hi = fmaxf(m1, o1), lo = fminf(m1, o1);
+                m2 = fmaxf(lo, fmaxf(m2, o2));
+                m1 = hi;
+            }
+        }
+        gs = m1 + m2;
+    }
+    int rank = 0;
+    const int mygrp = split ? lane / lpg : lane;
+    for (int j = 0; j < n; ++j) {
+        const float gj = __shfl_sync(full, gs, split ? j * lpg : j);
+        rank += (gj > gs || (gj == gs && j < mygrp)) ? 1 : 0;
+    }
+    const unsigned alive_l = __ballot_sync(full, (split || lane < n) && rank < keep);
+    // (one bit per group)
+    unsigned alive = 0u;
+    for (int j = 0; j < n; ++j) alive |= ((alive_l >> (split ? j * lpg : j)) & 1u) << j;
+    for (int e = lane; e < E; e += 32)
+        if (!((alive >> (e / per)) & 1u)) sel[e] = __int_as_float(0x7fffffff);
+    __syncwarp();
+    // top-K among the survivors, ties to the lower index
+    float myv = 0.f;
+    int myi = 0x7FFFFFFF;
+    if (E <= 256) {
+        warp_topk_reg<8>(sel, E, K, lane, myv, myi);
+        if (lane < K && myi != 0x7FFFFFFF) myv = sig[myi];
+    } else {
+        // every lane keeps its best remaining candidate, the owner of a round's winner rescans
+        uint32_t key;
+        int idx;
+        lane_best(sel, E, lane, key, idx);
+        for (int j = 0; j < K; ++j) {
+            const uint32_t best = __reduce_max_sync(full, idx == 0x7FFFFFFF ? 0u : key);
+            const int cand = (idx != 0x7FFFFFFF && key == best) ? idx : 0x7FFFFFFF;
+            const int win = (int)__reduce_min_sync(full, (unsigned)cand);
+            if (win == 0x7FFFFFFF) break;                   // fewer than K survivors
+            if (lane == j) { myv = sig[win]; myi = win; }
+            __syncwarp();
+            if (idx == win) {
+                sel[win] = __int_as_float(0x7fffffff);
+                lane_best(sel, E, lane, key, idx);
+            }
+            __syncwarp();
+        }
+    }
+    const float sum = warp_sum((lane < K && myi != 0x7FFFFFFF) ? myv : 0.f);
+    int pos = 0;
+    for (int i = 0; i < K; ++i) {
+        const int oi = __shfl_sync(full, myi, i);
+        pos += (oi < myi) ? 1 : 0;
+    }
+    if (lane < K && myi != 0x7FFFFFFF) {
+        inds[(size_t)t * K + pos] = myi;
+        gates[(size_t)t * K + pos] = scale * myv / (sum + 1e-20f);
+    }
+}
+
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
                       int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head = 0) {
     int32_t rc = check_desc(d);
@@ -351,6 +445,19 @@ extern "C" int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* lo
     const size_t sm = 4 * (size_t)desc->E * sizeof(float);
     edg::softmax_topk_rows_kernel<<<(T + 3) / 4, 128, sm, static_cast<cudaStream_t>(stream)>>>(
         logits, T, desc->E, desc->K, inds, gates);
+    EDG_CUDA_TRY(cudaGetLastError());
+    return EDG_OK;
+}
+
+extern "C" int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32_t E, int32_t K, int32_t n_groups,
+                                           int32_t keep_groups, float scale, const float* bias_opt,
+                                           int32_t* inds, float* gates, void* stream) {
+    if (!logits || !inds || !gates || T < 1) return EDG_E_INVAL;
+    if (E < 2 || E > 1024 || n_groups < 1 || n_groups > 32 || E % n_groups != 0 || E / n_groups < 2) return EDG_E_SHAPE;
+    if (keep_groups < 1 || keep_groups > n_groups || K < 1 || K > 32 || K > keep_groups * (E / n_groups)) return EDG_E_SHAPE;
+    const size_t sm = 4 * 2 * (size_t)E * sizeof(float);
+    edg::sigmoid_group_topk_rows_kernel<<<(T + 3) / 4, 128, sm, static_cast<cudaStream_t>(stream)>>>(
+        logits, bias_opt, T, E, K, n_groups, keep_groups, scale, inds, gates);
     EDG_CUDA_TRY(cudaGetLastError());
     return EDG_OK;
 }
