@@ -115,6 +115,48 @@ def prerouter_logits(W_pre, s_bits) -> np.ndarray:
     return np.array([np.dot(W[e], s) for e in range(W.shape[0])], dtype=np.float64)
 
 
+def gelu_erf(z) -> np.ndarray:
+    """Exact (erf) GELU: z * Phi(z) = 0.5 z (1 + erf(z / sqrt 2)), the activation of the prerouter's MLP
+    path (Sec. 3.2 "Head")."""
+    z = np.asarray(z, dtype=np.float64)
+    return np.array([0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in z.ravel()], dtype=np.float64).reshape(z.shape)
+
+
+def prerouter_mlp_logits(W1, b1, W2, b2, W_res, s_bits, cur_inds, prev_inds) -> np.ndarray:
+    """Sec. 3.2 "Head", the full head of one layer: fc1 -> erf-gelu -> fc2 plus the linear residual path.
+
+    The input feature concatenates the hidden state with two K-hot vectors over the E experts: the
+    experts this layer routed to at this token (``cur_inds``) and at the previous token
+    (``prev_inds``): f = [s ; hot(cur) ; hot(prev)], dimension d + 2E.
+        z = W1 f + b1        (W1 [D][d + 2E], D the hidden width)
+        l = W2 gelu(z) + b2 + W_res s        (W2 [E][D]; W_res [E][d], the residual path, acts on the
+                                              hidden state: it is what a router weight would be)
+    Biases and the residual path are optional (None = absent)."""
+    s = bf16_to_f64(s_bits)
+    W1 = np.asarray(W1).astype(np.float64)
+    W2 = np.asarray(W2).astype(np.float64)
+    d = s.shape[0]
+    E = W2.shape[0]
+    if W1.shape[1] != d + 2 * E or W2.shape[1] != W1.shape[0]:
+        raise ValueError("head shapes do not fit")
+    f = np.zeros(d + 2 * E, dtype=np.float64)
+    f[:d] = s
+    for e in cur_inds:
+        f[d + int(e)] = 1.0
+    for e in prev_inds:
+        f[d + E + int(e)] = 1.0
+    z = np.array([np.dot(W1[r], f) for r in range(W1.shape[0])], dtype=np.float64)
+    if b1 is not None:
+        z = z + np.asarray(b1).astype(np.float64)
+    a = gelu_erf(z)
+    l = np.array([np.dot(W2[e], a) for e in range(E)], dtype=np.float64)
+    if b2 is not None:
+        l = l + np.asarray(b2).astype(np.float64)
+    if W_res is not None:
+        l = l + prerouter_logits(W_res, s_bits)
+    return l
+
+
 def softmax_topk(logits, K: int) -> Tuple[np.ndarray, np.ndarray]:
     """Appendix A, softmax-topk with renormalisation:
     g = softmax(l); inds = top-k(g, K); w = g[inds] / sum(g[inds]).

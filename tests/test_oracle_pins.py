@@ -400,3 +400,45 @@ def test_layer_decode_is_the_composition_of_its_parts():
     assert sorted(e for e, _ in copies) == inds_cur.tolist() and slots == [0, 1]
     # magnitudes the tolerances were derived for: outputs of order 1-10, not 1e-3 or 1e3
     assert 1.0 < np.std(y) < 30.0
+
+
+# ------------------------------------------------------------------ the MLP head (Sec. 3.2 "Head")
+
+def test_gelu_erf_known_values_and_limits():
+    # z * Phi(z) with the standard normal CDF: Phi(0) = 1/2, Phi(1) = 0.8413447460685429, Phi(-1) = 1 - Phi(1)
+    g = orc.gelu_erf(np.array([0.0, 1.0, -1.0, 2.0, 8.0, -8.0]))
+    assert g[0] == 0.0
+    assert abs(g[1] - 0.8413447460685429) < 1e-15
+    assert abs(g[2] + (1.0 - 0.8413447460685429)) < 1e-15
+    assert abs(g[3] - 2.0 * 0.9772498680518208) < 1e-15
+    assert abs(g[4] - 8.0) < 1e-13 and abs(g[5]) < 1e-13          # identity far right, zero far left
+    # the identity gelu(z) - gelu(-z) = z holds for every z
+    z = np.random.default_rng(3).standard_normal(50) * 3
+    assert np.allclose(orc.gelu_erf(z) - orc.gelu_erf(-z), z, rtol=0, atol=1e-14)
+
+
+def test_mlp_head_reduces_to_the_linear_head_and_to_a_column_gather():
+    rng = np.random.default_rng(11)
+    d, E, D, K = 32, 8, 16, 2
+    s_bits = _bf16(rng.standard_normal(d))
+    W1 = rng.standard_normal((D, d + 2 * E)) * 0.3
+    b1 = rng.standard_normal(D) * 0.1
+    W2 = rng.standard_normal((E, D)) * 0.3
+    b2 = rng.standard_normal(E) * 0.1
+    Wr = rng.standard_normal((E, d)) * 0.2
+    cur, prev = [1, 6], [0, 6]
+    # with a zero fc2 the head is the residual path alone (+ b2): the linear head that is pinned above
+    l0 = orc.prerouter_mlp_logits(W1, b1, np.zeros((E, D)), None, Wr, s_bits, cur, prev)
+    assert np.array_equal(l0, orc.prerouter_logits(Wr, s_bits))
+    # the one-hot part of the feature picks columns of W1: brute force with an explicit concatenated vector
+    s = orc.bf16_to_f64(s_bits)
+    z = W1[:, :d] @ s + W1[:, d + 1] + W1[:, d + 6] + W1[:, d + E + 0] + W1[:, d + E + 6] + b1
+    a = np.array([0.5 * v * (1.0 + math.erf(v / math.sqrt(2.0))) for v in z])
+    want = W2 @ a + b2 + Wr @ s
+    got = orc.prerouter_mlp_logits(W1, b1, W2, b2, Wr, s_bits, cur, prev)
+    assert np.allclose(got, want, rtol=0, atol=1e-12)
+    # the two one-hot blocks are distinct inputs: swapping them changes the result
+    assert not np.allclose(got, orc.prerouter_mlp_logits(W1, b1, W2, b2, Wr, s_bits, prev, cur))
+    # hand example: d = 1, E = 1, D = 1: z = 2*1.5 + 0.25 (cur) + 0.5 (prev) - 0.75 = 3.0, l = 4 * gelu(3) + 1 + 0.5 * 1.5
+    one = orc.prerouter_mlp_logits([[2.0, 0.25, 0.5]], [-0.75], [[4.0]], [1.0], [[0.5]], _bf16([1.5]), [0], [0])
+    assert abs(one[0] - (4.0 * 3.0 * 0.9986501019683699 + 1.0 + 0.75)) < 1e-12
