@@ -627,6 +627,55 @@ def run_sigmoid_group(args):
                       "gpu_launches": steps}))
 
 
+def run_mlp_head(args):
+    """The full prerouter head (Sec. 3.2: fc1 -> erf-gelu -> fc2 + linear residual path; feature = hidden
+    state and two K-hot vectors) for many (head, state) pairs in one launch, as in the paper's single
+    flush: 64 heads of the 35B-tier shape (H + 2E = 2560, width 512, fp16), 252 MB of head weights."""
+    import torch
+    import paper_2609_18063_b200 as edg
+    from workloads import synth
+    from paper_2609_18063_b200 import layer_io
+    peak, how = _peaks()
+    cfg = synth.CONFIGS["cfg2"]
+    desc = edg.make_desc(cfg, n_slots=cfg.E)
+    E, K, H, D, NH = cfg.E, cfg.K, cfg.H, 512, 64
+    hw = [synth.mlp_head_weights(cfg, l % 4, D) for l in range(4)]         # four distinct heads, tiled to 64
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    tile = lambda k: dev(np.stack([hw[l % 4][k] for l in range(NH)]))
+    W1, b1, W2, b2 = tile("W1"), tile("b1"), tile("W2"), tile("b2")
+    Wr = dev(np.stack([synth.prerouter_weights(cfg, l % 4) for l in range(NH)]))
+    X = layer_io.bits_to_device(synth.hidden_states(cfg, NH, stream=600), torch.bfloat16)
+    rng = np.random.default_rng(9)
+    cur = dev(np.stack([np.sort(rng.choice(E, K, replace=False)) for _ in range(NH)]).astype(np.int32))
+    prev = dev(np.stack([np.sort(rng.choice(E, K, replace=False)) for _ in range(NH)]).astype(np.int32))
+    inds = torch.zeros((NH, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((NH, K), dtype=torch.float32, device="cuda")
+    steps, warmup = max(1, min(args.steps, 200)), max(args.warmup, 3)
+    call = lambda: edg.prerouter_mlp_topk(desc, W1, b1, W2, b2, Wr, D, X, cur, prev, NH, inds, gates, None)
+    for _ in range(warmup):
+        call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert abs(float(gates.sum()) - NH) < 1e-2
+    alg = NH * (D * (H + 2 * E) * 2 + E * D * 2 + E * H * 2 + (D + E) * 2 + H * 2)
+    achieved = alg / (ms * 1e-3) / 1e9
+    print(json.dumps({"metric": "prerouter_mlp_heads_per_s", "value": round(NH / (ms * 1e-3), 1), "unit": "heads/s",
+                      "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": round(ms, 5), "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "fp16 weights, fp32 accumulate", "data": "synthetic",
+                      "config": {"workload": "full prerouter head, 35B-tier shape (feature 2560, width 512, E=256, top-8), 64 heads per launch",
+                                 "l2": "252 MB of head weights per launch exceed the 126 MB L2"},
+                      "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                                   "frac": round(achieved / peak, 4), "traffic": None, "peak_kind": how,
+                                   "algorithmic_bytes_per_launch": alg},
+                      "gpu_launches": steps}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -638,7 +687,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", choices=["cfg2", "cfg3", "cfg4", "cfg5", "sigmoid_group"], default="cfg2",
+    ap.add_argument("--workload", choices=["cfg2", "cfg3", "cfg4", "cfg5", "sigmoid_group", "mlp_head"], default="cfg2",
                     help="cfg2 is the headline line; the others print their own line")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -651,6 +700,8 @@ def main():
         run_cfg5(args)
     elif args.workload == "sigmoid_group":
         run_sigmoid_group(args)
+    elif args.workload == "mlp_head":
+        run_mlp_head(args)
     else:
         run_b200(args)
 

@@ -181,6 +181,31 @@ int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32
  * with at least two experts a group, K <= 32 and <= keep_groups * E / n_groups; else EDG_E_SHAPE.
  * One warp per row; no workspace; arithmetic in fp32 (the decision is taken in the kernel's
  * precision). */
+/* The full prerouter head of a layer (Sec. 3.2 "Head"): fc1 -> erf-gelu -> fc2 plus a linear residual
+ * path.  The input feature is the hidden state followed by two K-hot vectors over the E experts --
+ * the experts this layer routed to at this token and at the previous token -- so its dimension is
+ * H + 2E (2560 at the 35B tier) and the hidden width D is 512 there.  With f = [s ; hot(cur) ; hot(prev)]:
+ *     z = W1 f + b1,    l = W2 gelu(z) + b2 + W_res s,    gelu(z) = z/2 (1 + erf(z / sqrt 2)),
+ * followed by the same softmax top-k with renormalised gates as prerouter_topk.  The residual path acts
+ * on the hidden state alone (it is what the paper warm-starts from the next layer's router weight).
+ * All tensors are device memory owned by the caller; biases and the residual path may be NULL. */
+typedef struct edg_mlp_head {
+    const void* W1;     /* fp16 [n_heads][D][H + 2E]                                   */
+    const void* b1;     /* fp16 [n_heads][D] or NULL                                   */
+    const void* W2;     /* fp16 [n_heads][E][D]                                        */
+    const void* b2;     /* fp16 [n_heads][E] or NULL                                   */
+    const void* W_res;  /* [n_heads][E][H] of desc->pre_dtype, or NULL                 */
+    int32_t width;      /* D: a multiple of 8, 8 <= D <= 4096                          */
+} edg_mlp_head;
+
+/* s dev bf16 [n_heads][H]; cur_inds / prev_inds dev int32 [n_heads][K] (entries outside 0..E-1 are
+ * ignored); inds dev int32 [n_heads][K] ascending; gates dev float [n_heads][K]; logits_opt dev float
+ * [n_heads][E] or NULL.  One cluster of 8 CTAs per head; fp32 accumulation; (E + H + D) * 4 bytes of
+ * shared memory must fit 48 KB, else EDG_E_SHAPE.  Pointers 16-byte aligned, else EDG_E_INVAL. */
+int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_head* head, const void* s,
+                           const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
+                           int32_t* inds, float* gates, float* logits_opt, void* stream);
+
 int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32_t E, int32_t K, int32_t n_groups,
                                 int32_t keep_groups, float scale, const float* bias_opt,
                                 int32_t* inds, float* gates, void* stream);

@@ -15,7 +15,7 @@ import numpy as np
 __all__ = [
     "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
-    "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows", "sigmoid_group_topk_rows",
+    "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows", "sigmoid_group_topk_rows", "prerouter_mlp_topk",
     "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
 ]
 
@@ -70,6 +70,7 @@ _SIG = {
     "prerouter_topk_tokens": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "softmax_topk_rows": ([_D, _P, C.c_int32, _P, _P, _P], C.c_int32),
     "sigmoid_group_topk_rows": ([_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, _P, _P], C.c_int32),
+    "prerouter_mlp_topk": ([_D, _P, _P, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
     "edg_store_get_stats": ([_P, C.POINTER(StoreStats)], C.c_int32),
@@ -223,6 +224,17 @@ def prerouter_topk(desc, W_pre, s, n_heads, inds, gates, logits_opt=None, stream
 def prerouter_topk_tokens(desc, W_pre, s, T, inds, gates, logits_opt=None, stream=None) -> None:
     _check(_lib.prerouter_topk_tokens(C.byref(desc), _ptr(W_pre), _ptr(s), T, _ptr(inds), _ptr(gates),
                                       _ptr(logits_opt), _stream(stream)), "prerouter_topk_tokens")
+
+
+class MlpHead(C.Structure):
+    _fields_ = [("W1", _P), ("b1", _P), ("W2", _P), ("b2", _P), ("W_res", _P), ("width", C.c_int32)]
+
+
+def prerouter_mlp_topk(desc, W1, b1, W2, b2, W_res, width, s, cur_inds, prev_inds, n_heads, inds, gates,
+                       logits_opt=None, stream=None) -> None:
+    head = MlpHead(_ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(W_res), int(width))
+    _check(_lib.prerouter_mlp_topk(C.byref(desc), C.byref(head), _ptr(s), _ptr(cur_inds), _ptr(prev_inds), n_heads,
+                                   _ptr(inds), _ptr(gates), _ptr(logits_opt), _stream(stream)), "prerouter_mlp_topk")
 
 
 def sigmoid_group_topk_rows(logits, T, E, K, n_groups, keep_groups, scale, bias, inds, gates, stream=None) -> None:

@@ -35,7 +35,7 @@ template <> struct RowDot<__half> {
     static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
         const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const __half*>(W) + row * H);
         float acc = 0.f;
-#pragma unroll 4
+#pragma unroll 8
         for (int c = lane; c < H / 8; c += 32) {
             const uint4 w = ld_stream16(wp + c);
             const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
@@ -286,6 +286,106 @@ __global__ void __launch_bounds__(128) softmax_topk_rows_kernel(const float* log
     warp_softmax_topk(work, E, K, lane, inds + (size_t)t * K, gates + (size_t)t * K);
 }
 
+// ---------------------------------------------------------------- the full head (Sec. 3.2 "Head")
+// fc1 -> erf-gelu -> fc2 plus the linear residual path, one cluster per head.  The feature is the
+// hidden state followed by two K-hot vectors (this layer's experts at this token and at the previous
+// one), so fc1 is a dot product over the hidden state plus a gather of 2K columns.  Phase 1: the D
+// rows of fc1 are dealt to the CTAs of the cluster, a warp per row; every activation is written
+// into the shared memory of all CTAs.  Phase 2: the E rows of fc2 (+ the residual row over the
+// hidden state) likewise; the logits land in the leader, which does softmax + top-k.
+struct MlpParams {
+    const __half* W1;       // [n_heads][D][H + 2E]
+    const __half* b1;       // [n_heads][D] or null
+    const __half* W2;       // [n_heads][E][D]
+    const __half* b2;       // [n_heads][E] or null
+    const void* Wres;       // [n_heads][E][H] (fp16 or fp32) or null
+    const uint16_t* s;      // [n_heads][H] bf16
+    const int32_t* cur;     // [n_heads][K]
+    const int32_t* prev;    // [n_heads][K]
+    int32_t* inds;          // [n_heads][K]
+    float* gates;           // [n_heads][K]
+    float* logits;          // [n_heads][E] or null
+    int H, E, K, D;
+};
+
+// dot product of an fp16 row of n (a multiple of 8) weights with fp32 activations, by one warp
+__device__ __forceinline__ float half_row_dot(const __half* row, const float* sx, int n, int lane) {
+    const uint4* wp = reinterpret_cast<const uint4*>(row);
+    float acc = 0.f;
+#pragma unroll 8
+    for (int c = lane; c < n / 8; c += 32) {
+        const uint4 w = ld_stream16(wp + c);
+        const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w.x));
+        const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&w.y));
+        const float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w.z));
+        const float2 e = __half22float2(*reinterpret_cast<const __half2*>(&w.w));
+        const float* x = sx + c * 8;
+        acc = fmaf(a.x, x[0], acc); acc = fmaf(a.y, x[1], acc);
+        acc = fmaf(b.x, x[2], acc); acc = fmaf(b.y, x[3], acc);
+        acc = fmaf(d.x, x[4], acc); acc = fmaf(d.y, x[5], acc);
+        acc = fmaf(e.x, x[6], acc); acc = fmaf(e.y, x[7], acc);
+    }
+    return acc;                          // (not yet summed over the lanes)
+}
+
+template <typename WT>
+__global__ void __launch_bounds__(kPreWarps * 32) prerouter_mlp_kernel(MlpParams p) {
+    cg::cluster_group cluster = cg::this_cluster();
+    const int crank = (int)cluster.block_rank();
+    const int csize = (int)cluster.num_blocks();
+    const int head = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    extern __shared__ float smem[];
+    float* s_logits = smem;             // [E]   (the leader's copy collects every CTA's rows)
+    float* s_x = smem + p.E;            // [H]   hidden state widened to fp32
+    float* s_a = s_x + p.H;             // [D]   gelu(fc1), complete in every CTA after the first cluster barrier
+
+    const uint16_t* sv = p.s + (size_t)head * p.H;
+    for (int i = threadIdx.x; i < p.H; i += blockDim.x) s_x[i] = bf16_bits_to_float(sv[i]);
+    __syncthreads();
+
+    const int F = p.H + 2 * p.E;
+    const int perD = (p.D + csize - 1) / csize;
+    // the K-hot parts of the feature pick columns: lane k < K holds the k-th expert of either list
+    int hc = -1, hq = -1;
+    if (lane < p.K) {
+        hc = p.cur[(size_t)head * p.K + lane];
+        hq = p.prev[(size_t)head * p.K + lane];
+        if (hc < 0 || hc >= p.E) hc = -1;
+        if (hq < 0 || hq >= p.E) hq = -1;
+    }
+    for (int r = crank * perD + warp; r < min(p.D, (crank + 1) * perD); r += kPreWarps) {
+        const __half* row = p.W1 + ((size_t)head * p.D + r) * F;
+        // (the gathered columns are fetched together with the row, not after it)
+        const __half gc = hc >= 0 ? row[p.H + hc] : __float2half(0.f);
+        const __half gq = hq >= 0 ? row[p.H + p.E + hq] : __float2half(0.f);
+        float z = half_row_dot(row, s_x, p.H, lane);
+        z += __half2float(gc) + __half2float(gq);
+        z = warp_sum(z);
+        if (p.b1 != nullptr) z += __half2float(p.b1[(size_t)head * p.D + r]);
+        const float a = 0.5f * z * (1.f + erff(z * 0.70710678118654752f));
+        if (lane < csize) cluster.map_shared_rank(s_a, lane)[r] = a;
+    }
+    cluster.sync();                     // every CTA holds all D activations
+
+    float* leader = cluster.map_shared_rank(s_logits, 0);
+    const int perE = (p.E + csize - 1) / csize;
+    for (int e = crank * perE + warp; e < min(p.E, (crank + 1) * perE); e += kPreWarps) {
+        float l = warp_sum(half_row_dot(p.W2 + ((size_t)head * p.E + e) * p.D, s_a, p.D, lane));
+        if (p.b2 != nullptr) l += __half2float(p.b2[(size_t)head * p.E + e]);
+        if (p.Wres != nullptr) l += RowDot<WT>::run(p.Wres, (size_t)head * p.E + e, s_x, p.H, lane);
+        if (lane == 0) leader[e] = l;
+    }
+    cluster.sync();                     // every CTA's logits have landed in the leader
+    if (crank != 0) return;
+
+    if (p.logits != nullptr)
+        for (int e = threadIdx.x; e < p.E; e += blockDim.x) p.logits[(size_t)head * p.E + e] = s_logits[e];
+    __syncthreads();
+    if (warp == 0)
+        warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds + (size_t)head * p.K, p.gates + (size_t)head * p.K);
+}
+
 // Appendix A, sigmoid-group routing, one warp per row of given logits: sigma = sigmoid(l); a group's
 // score is the sum of its two largest selection scores (sigma, plus a bias when one is given); the
 // best `keep` of the `n` groups survive (ties to the lower group); top-K among the survivors by
@@ -459,5 +559,39 @@ extern "C" int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32
     edg::sigmoid_group_topk_rows_kernel<<<(T + 3) / 4, 128, sm, static_cast<cudaStream_t>(stream)>>>(
         logits, bias_opt, T, E, K, n_groups, keep_groups, scale, inds, gates);
     EDG_CUDA_TRY(cudaGetLastError());
+    return EDG_OK;
+}
+
+extern "C" int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_head* head, const void* s,
+                                      const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
+                                      int32_t* inds, float* gates, float* logits_opt, void* stream) {
+    int32_t rc = edg::check_desc(desc);
+    if (rc != EDG_OK) return rc;
+    if (!head || !head->W1 || !head->W2 || !s || !cur_inds || !prev_inds || !inds || !gates || n_heads < 1 || n_heads > 65535)
+        return EDG_E_INVAL;
+    const int D = head->width;
+    if (D < 8 || D > 4096 || D % 8 != 0 || desc->H % 8 != 0 || (desc->H + 2 * desc->E) % 8 != 0) return EDG_E_SHAPE;
+    if (!edg::aligned(head->W1, 16) || !edg::aligned(head->W2, 16) || !edg::aligned(s, 16) ||
+        (head->W_res && !edg::aligned(head->W_res, 16)))
+        return EDG_E_INVAL;
+    edg::MlpParams p{static_cast<const __half*>(head->W1), static_cast<const __half*>(head->b1),
+                     static_cast<const __half*>(head->W2), static_cast<const __half*>(head->b2), head->W_res,
+                     static_cast<const uint16_t*>(s), cur_inds, prev_inds, inds, gates, logits_opt,
+                     desc->H, desc->E, desc->K, D};
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(edg::kPreCluster, n_heads, 1);
+    cfg.blockDim = dim3(edg::kPreWarps * 32, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)(desc->E + desc->H + D) * sizeof(float);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    if (cfg.dynamicSmemBytes > 48 * 1024) return EDG_E_SHAPE;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = edg::kPreCluster;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    if (desc->pre_dtype == EDG_F16) EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, edg::prerouter_mlp_kernel<__half>, p));
+    else EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, edg::prerouter_mlp_kernel<float>, p));
     return EDG_OK;
 }

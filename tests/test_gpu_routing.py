@@ -76,3 +76,49 @@ def test_sigmoid_group_rejects_shapes_it_cannot_route():
     for args in [(8, 2, 3, 1), (8, 2, 8, 1), (8, 5, 2, 1), (8, 2, 2, 3)]:      # (E, K, n, G): groups not dividing E, one expert a group, K beyond the survivors, G > n
         with pytest.raises(Exception):
             edg.sigmoid_group_topk_rows(z, 1, args[0], args[1], args[2], args[3], 2.5, None, i, g)
+
+
+# ------------------------------------------------------------------ the full head (Sec. 3.2 "Head")
+
+@pytest.mark.parametrize("name,width,n_heads,variant", [("cfg2", 512, 3, "full"), ("cfg1", 64, 2, "full"),
+                                                       ("cfg2", 512, 1, "no_residual"), ("cfg1", 64, 1, "no_bias")])
+def test_mlp_head_matches_the_oracle(name, width, n_heads, variant):
+    from workloads import synth
+    from tests._gpu_util import x_dev
+    cfg = synth.CONFIGS[name]
+    d = edg.make_desc(cfg, n_slots=cfg.E)
+    E, K, H = cfg.E, cfg.K, cfg.H
+    rng = np.random.default_rng(17)
+    heads = [synth.mlp_head_weights(cfg, layer, width) for layer in range(n_heads)]
+    Wres = [synth.prerouter_weights(cfg, layer) for layer in range(n_heads)]
+    X = synth.hidden_states(cfg, n_heads, stream=41)
+    cur = np.stack([np.sort(rng.choice(E, K, replace=False)) for _ in range(n_heads)]).astype(np.int32)
+    prev = np.stack([np.sort(rng.choice(E, K, replace=False)) for _ in range(n_heads)]).astype(np.int32)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    W1, W2 = dev(np.stack([h["W1"] for h in heads])), dev(np.stack([h["W2"] for h in heads]))
+    b1 = None if variant == "no_bias" else dev(np.stack([h["b1"] for h in heads]))
+    b2 = None if variant == "no_bias" else dev(np.stack([h["b2"] for h in heads]))
+    Wr = None if variant == "no_residual" else dev(np.stack(Wres))
+    inds = torch.zeros((n_heads, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((n_heads, K), dtype=torch.float32, device="cuda")
+    logits = torch.zeros((n_heads, E), dtype=torch.float32, device="cuda")
+    edg.prerouter_mlp_topk(d, W1, b1, W2, b2, Wr, width, x_dev(X), dev(cur), dev(prev), n_heads, inds, gates, logits)
+    torch.cuda.synchronize()
+    for h in range(n_heads):
+        want = orc.prerouter_mlp_logits(heads[h]["W1"], None if b1 is None else heads[h]["b1"], heads[h]["W2"],
+                                        None if b2 is None else heads[h]["b2"], None if Wr is None else Wres[h],
+                                        X[h], cur[h], prev[h])
+        got = logits[h].cpu().numpy().astype(np.float64)
+        assert np.abs(got - want).max() <= 2e-4 * max(1.0, np.abs(want).max())
+        # the routing is the exact top-k of the GPU's own logits, and the oracle's wherever its margin allows
+        gi, gw = orc.softmax_topk(got, K)
+        assert inds[h].cpu().numpy().tolist() == gi.tolist()
+        assert np.allclose(gates[h].cpu().numpy(), gw, rtol=1e-5, atol=1e-7)
+        srt = np.sort(want)[::-1]
+        if srt[K - 1] - srt[K] > 1e-3:
+            assert gi.tolist() == orc.softmax_topk(want, K)[0].tolist()
+    # the K-hot inputs matter: other executed routings give other logits
+    logits2 = torch.zeros_like(logits)
+    edg.prerouter_mlp_topk(d, W1, b1, W2, b2, Wr, width, x_dev(X), dev(prev), dev(cur), n_heads, inds, gates, logits2)
+    torch.cuda.synchronize()
+    assert not torch.equal(logits, logits2)

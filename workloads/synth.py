@@ -25,7 +25,7 @@ from typing import Dict, Tuple
 import numpy as np
 
 # tensor ids inside a stream key
-_T_X, _T_WPRE, _T_CODES, _T_SCALES, _T_ZEROS, _T_LORA_A, _T_LORA_B, _T_LOGITS, _T_PERM = range(9)
+_T_X, _T_WPRE, _T_CODES, _T_SCALES, _T_ZEROS, _T_LORA_A, _T_LORA_B, _T_LOGITS, _T_PERM, _T_MLP = range(10)
 _PROJ_ID = {"gate": 0, "up": 1, "down": 2}
 PROJS = ("gate", "up", "down")
 
@@ -127,6 +127,17 @@ def prerouter_weights(cfg: MoEConfig, layer: int = 0) -> np.ndarray:
     if cfg.pre_dtype == "f32":
         return w
     raise ValueError(f"pre_dtype {cfg.pre_dtype!r}")
+
+
+def mlp_head_weights(cfg: MoEConfig, layer: int = 0, width: int = 512) -> Dict[str, np.ndarray]:
+    """The MLP path of a prerouter head (fp16, the paper's export precision): W1 [width][H + 2E] and
+    W2 [E][width] ~ N(0, 0.02), biases b1 [width], b2 [E] ~ N(0, 0.01)."""
+    g = _rng(cfg.seed, layer, _T_MLP)
+    f = cfg.H + 2 * cfg.E
+    return {"W1": (g.standard_normal((width, f), dtype=np.float32) * np.float32(0.02)).astype(np.float16),
+            "b1": (g.standard_normal(width, dtype=np.float32) * np.float32(0.01)).astype(np.float16),
+            "W2": (g.standard_normal((cfg.E, width), dtype=np.float32) * np.float32(0.02)).astype(np.float16),
+            "b2": (g.standard_normal(cfg.E, dtype=np.float32) * np.float32(0.01)).astype(np.float16)}
 
 
 def expert_tensors(cfg: MoEConfig, layer: int, expert: int) -> Dict[str, Tuple[np.ndarray, np.ndarray, np.ndarray]]:
