@@ -32,7 +32,7 @@ template <typename WT> struct RowDot;
 
 // fp16 head: 8 weights (16 bytes) per lane per step
 template <> struct RowDot<__half> {
-    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+    static __device__ __forceinline__ float partial(const void* W, size_t row, const float* sx, int H, int lane) {
         const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const __half*>(W) + row * H);
         float acc = 0.f;
 #pragma unroll 8
@@ -48,13 +48,16 @@ template <> struct RowDot<__half> {
             acc = fmaf(d.x, x[4], acc); acc = fmaf(d.y, x[5], acc);
             acc = fmaf(e.x, x[6], acc); acc = fmaf(e.y, x[7], acc);
         }
-        return warp_sum(acc);
+        return acc;
+    }
+    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+        return warp_sum(partial(W, row, sx, H, lane));
     }
 };
 
 // fp32 head: 4 weights (16 bytes) per lane per step
 template <> struct RowDot<float> {
-    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+    static __device__ __forceinline__ float partial(const void* W, size_t row, const float* sx, int H, int lane) {
         const uint4* wp = reinterpret_cast<const uint4*>(static_cast<const float*>(W) + row * H);
         float acc = 0.f;
 #pragma unroll 4
@@ -64,7 +67,10 @@ template <> struct RowDot<float> {
             acc = fmaf(__uint_as_float(w.x), x[0], acc); acc = fmaf(__uint_as_float(w.y), x[1], acc);
             acc = fmaf(__uint_as_float(w.z), x[2], acc); acc = fmaf(__uint_as_float(w.w), x[3], acc);
         }
-        return warp_sum(acc);
+        return acc;
+    }
+    static __device__ __forceinline__ float run(const void* W, size_t row, const float* sx, int H, int lane) {
+        return warp_sum(partial(W, row, sx, H, lane));
     }
 };
 
@@ -328,8 +334,31 @@ __device__ __forceinline__ float half_row_dot(const __half* row, const float* sx
     return acc;                          // (not yet summed over the lanes)
 }
 
+// two rows at once against the same activations: twice the loads in flight, the activations read once
+__device__ __forceinline__ void half_row_dot2(const __half* row0, const __half* row1, const float* sx, int n, int lane,
+                                              float& acc0, float& acc1) {
+    const uint4* wp0 = reinterpret_cast<const uint4*>(row0);
+    const uint4* wp1 = reinterpret_cast<const uint4*>(row1);
+    acc0 = 0.f; acc1 = 0.f;
+#pragma unroll 8
+    for (int c = lane; c < n / 8; c += 32) {
+        const uint4 w0 = ld_stream16(wp0 + c), w1 = ld_stream16(wp1 + c);
+        const float4 x0 = *reinterpret_cast<const float4*>(sx + c * 8), x1 = *reinterpret_cast<const float4*>(sx + c * 8 + 4);
+        float2 a = __half22float2(*reinterpret_cast<const __half2*>(&w0.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&w0.y));
+        float2 d = __half22float2(*reinterpret_cast<const __half2*>(&w0.z)), e = __half22float2(*reinterpret_cast<const __half2*>(&w0.w));
+        acc0 = fmaf(a.x, x0.x, acc0); acc0 = fmaf(a.y, x0.y, acc0); acc0 = fmaf(b.x, x0.z, acc0); acc0 = fmaf(b.y, x0.w, acc0);
+        acc0 = fmaf(d.x, x1.x, acc0); acc0 = fmaf(d.y, x1.y, acc0); acc0 = fmaf(e.x, x1.z, acc0); acc0 = fmaf(e.y, x1.w, acc0);
+        a = __half22float2(*reinterpret_cast<const __half2*>(&w1.x)); b = __half22float2(*reinterpret_cast<const __half2*>(&w1.y));
+        d = __half22float2(*reinterpret_cast<const __half2*>(&w1.z)); e = __half22float2(*reinterpret_cast<const __half2*>(&w1.w));
+        acc1 = fmaf(a.x, x0.x, acc1); acc1 = fmaf(a.y, x0.y, acc1); acc1 = fmaf(b.x, x0.z, acc1); acc1 = fmaf(b.y, x0.w, acc1);
+        acc1 = fmaf(d.x, x1.x, acc1); acc1 = fmaf(d.y, x1.y, acc1); acc1 = fmaf(e.x, x1.z, acc1); acc1 = fmaf(e.y, x1.w, acc1);
+    }
+}
+
+constexpr int kMlpWarps = 8;      // warps per CTA of the full head (16 measured no faster)
+
 template <typename WT>
-__global__ void __launch_bounds__(kPreWarps * 32) prerouter_mlp_kernel(MlpParams p) {
+__global__ void __launch_bounds__(kMlpWarps * 32) prerouter_mlp_kernel(MlpParams p) {
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
     const int csize = (int)cluster.num_blocks();
@@ -354,26 +383,41 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_mlp_kernel(MlpParams
         if (hc < 0 || hc >= p.E) hc = -1;
         if (hq < 0 || hq >= p.E) hq = -1;
     }
-    for (int r = crank * perD + warp; r < min(p.D, (crank + 1) * perD); r += kPreWarps) {
-        const __half* row = p.W1 + ((size_t)head * p.D + r) * F;
-        // (the gathered columns are fetched together with the row, not after it)
-        const __half gc = hc >= 0 ? row[p.H + hc] : __float2half(0.f);
-        const __half gq = hq >= 0 ? row[p.H + p.E + hq] : __float2half(0.f);
-        float z = half_row_dot(row, s_x, p.H, lane);
-        z += __half2float(gc) + __half2float(gq);
-        z = warp_sum(z);
-        if (p.b1 != nullptr) z += __half2float(p.b1[(size_t)head * p.D + r]);
-        const float a = 0.5f * z * (1.f + erff(z * 0.70710678118654752f));
-        if (lane < csize) cluster.map_shared_rank(s_a, lane)[r] = a;
+    const int rend = min(p.D, (crank + 1) * perD);
+    for (int r = crank * perD + warp; r < rend; r += 2 * kMlpWarps) {      // two rows of this warp at a time
+        const int r1 = r + kMlpWarps;
+        const bool two = r1 < rend;
+        const __half* row0 = p.W1 + ((size_t)head * p.D + r) * F;
+        const __half* row1 = two ? row0 + (size_t)kMlpWarps * F : row0;
+        // (the gathered columns are fetched together with the rows, not after them)
+        const __half gc0 = hc >= 0 ? row0[p.H + hc] : __float2half(0.f), gq0 = hq >= 0 ? row0[p.H + p.E + hq] : __float2half(0.f);
+        const __half gc1 = hc >= 0 ? row1[p.H + hc] : __float2half(0.f), gq1 = hq >= 0 ? row1[p.H + p.E + hq] : __float2half(0.f);
+        float z0, z1;
+        half_row_dot2(row0, row1, s_x, p.H, lane, z0, z1);
+        z0 = warp_sum(z0 + __half2float(gc0) + __half2float(gq0));
+        z1 = warp_sum(z1 + __half2float(gc1) + __half2float(gq1));
+        if (p.b1 != nullptr) {
+            z0 += __half2float(p.b1[(size_t)head * p.D + r]);
+            if (two) z1 += __half2float(p.b1[(size_t)head * p.D + r1]);
+        }
+        const float a0 = 0.5f * z0 * (1.f + erff(z0 * 0.70710678118654752f));
+        const float a1 = 0.5f * z1 * (1.f + erff(z1 * 0.70710678118654752f));
+        if (lane < csize) {
+            float* dst = cluster.map_shared_rank(s_a, lane);
+            dst[r] = a0;
+            if (two) dst[r1] = a1;
+        }
     }
     cluster.sync();                     // every CTA holds all D activations
 
     float* leader = cluster.map_shared_rank(s_logits, 0);
     const int perE = (p.E + csize - 1) / csize;
-    for (int e = crank * perE + warp; e < min(p.E, (crank + 1) * perE); e += kPreWarps) {
-        float l = warp_sum(half_row_dot(p.W2 + ((size_t)head * p.E + e) * p.D, s_a, p.D, lane));
+    for (int e = crank * perE + warp; e < min(p.E, (crank + 1) * perE); e += kMlpWarps) {
+        // (both dot products' loads are issued before either sum is reduced)
+        float l = half_row_dot(p.W2 + ((size_t)head * p.E + e) * p.D, s_a, p.D, lane);
+        if (p.Wres != nullptr) l += RowDot<WT>::partial(p.Wres, (size_t)head * p.E + e, s_x, p.H, lane);
+        l = warp_sum(l);
         if (p.b2 != nullptr) l += __half2float(p.b2[(size_t)head * p.E + e]);
-        if (p.Wres != nullptr) l += RowDot<WT>::run(p.Wres, (size_t)head * p.E + e, s_x, p.H, lane);
         if (lane == 0) leader[e] = l;
     }
     cluster.sync();                     // every CTA's logits have landed in the leader
@@ -580,7 +624,7 @@ extern "C" int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_
                      desc->H, desc->E, desc->K, D};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(edg::kPreCluster, n_heads, 1);
-    cfg.blockDim = dim3(edg::kPreWarps * 32, 1, 1);
+    cfg.blockDim = dim3(edg::kMlpWarps * 32, 1, 1);
     cfg.dynamicSmemBytes = (size_t)(desc->E + desc->H + D) * sizeof(float);
     cfg.stream = static_cast<cudaStream_t>(stream);
     if (cfg.dynamicSmemBytes > 48 * 1024) return EDG_E_SHAPE;
