@@ -212,9 +212,9 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(Pr
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t4 = lane & 3;
     extern __shared__ float smem[];
     float* s_logits = smem;                                             // [kTokBlock][E]
-    float* s_red = smem + kTokBlock * p.E;                              // [kPreWarps][16 x 8] partial tiles
+    float* s_red = smem + kTokBlock * p.E;                              // [kPreWarps][2 x 16 x 8] partial tiles
     const int xs = p.H * 2 + 16;                                        // bytes per token row
-    uint8_t* s_xh = reinterpret_cast<uint8_t*>(s_red + kPreWarps * 128);    // [kTokBlock][H + 8] fp16
+    uint8_t* s_xh = reinterpret_cast<uint8_t*>(s_red + kPreWarps * 256);    // [kTokBlock][H + 8] fp16
     for (int tt = 0; tt < kTokBlock; ++tt) {
         const int t = t0 + tt;
         for (int i = threadIdx.x; i < p.H; i += blockDim.x)
@@ -226,13 +226,17 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(Pr
     const int per = p.E / csize;                                        // rows of this CTA: a multiple of 16
     const int ksl = p.H / kPreWarps;                                    // k per warp: a multiple of 16
     const __half* W = static_cast<const __half*>(p.W);
-    for (int r0 = crank * per; r0 < (crank + 1) * per; r0 += 16) {
+    // two row tiles at a time: twice the loads in flight for the same B fragments
+    for (int r0 = crank * per; r0 < (crank + 1) * per; r0 += 32) {
+        const bool two = r0 + 16 < (crank + 1) * per;
         const __half* wlo = W + (size_t)(r0 + g) * p.H + warp * ksl + 2 * t4;
         const __half* whi = wlo + (size_t)8 * p.H;
+        const __half* vlo = two ? wlo + (size_t)16 * p.H : wlo;
+        const __half* vhi = vlo + (size_t)8 * p.H;
         const uint8_t* xb = s_xh + g * xs + (warp * ksl + 2 * t4) * 2;
-        float c[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int k0 = 0; k0 < ksl; k0 += 64) {                          // four steps' worth of loads in flight
-            uint32_t a[4][4];
+        float c[4] = {0.f, 0.f, 0.f, 0.f}, d[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int k0 = 0; k0 < ksl; k0 += 64) {                          // four steps' worth of loads in flight per tile
+            uint32_t a[4][4], b[4][4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int k = k0 + 16 * u;
@@ -241,6 +245,10 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(Pr
                 a[u][1] = on ? ld_stream4(whi + k) : 0u;
                 a[u][2] = on ? ld_stream4(wlo + k + 8) : 0u;
                 a[u][3] = on ? ld_stream4(whi + k + 8) : 0u;
+                b[u][0] = on ? ld_stream4(vlo + k) : 0u;
+                b[u][1] = on ? ld_stream4(vhi + k) : 0u;
+                b[u][2] = on ? ld_stream4(vlo + k + 8) : 0u;
+                b[u][3] = on ? ld_stream4(vhi + k + 8) : 0u;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -249,19 +257,22 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(Pr
                     const uint32_t b0 = *reinterpret_cast<const uint32_t*>(xb + k * 2);
                     const uint32_t b1 = *reinterpret_cast<const uint32_t*>(xb + k * 2 + 16);
                     mma16816(c, a[u][0], a[u][1], a[u][2], a[u][3], b0, b1);
+                    mma16816(d, b[u][0], b[u][1], b[u][2], b[u][3], b0, b1);
                 }
             }
         }
-        // rows g / g + 8, tokens 2 t4 / 2 t4 + 1 of this warp's K slice
-        float* mine = s_red + warp * 128;
+        // rows g / g + 8, tokens 2 t4 / 2 t4 + 1 of this warp's K slice, for both tiles
+        float* mine = s_red + warp * 256;
         mine[g * 8 + 2 * t4] = c[0]; mine[g * 8 + 2 * t4 + 1] = c[1];
         mine[(g + 8) * 8 + 2 * t4] = c[2]; mine[(g + 8) * 8 + 2 * t4 + 1] = c[3];
+        mine[128 + g * 8 + 2 * t4] = d[0]; mine[128 + g * 8 + 2 * t4 + 1] = d[1];
+        mine[128 + (g + 8) * 8 + 2 * t4] = d[2]; mine[128 + (g + 8) * 8 + 2 * t4 + 1] = d[3];
         __syncthreads();
-        if (threadIdx.x < 128) {
+        if (threadIdx.x < 128 || two) {
             float v = 0.f;
 #pragma unroll
-            for (int w = 0; w < kPreWarps; ++w) v += s_red[w * 128 + threadIdx.x];
-            const int row = threadIdx.x >> 3, tok = threadIdx.x & 7;
+            for (int w = 0; w < kPreWarps; ++w) v += s_red[w * 256 + threadIdx.x];
+            const int row = threadIdx.x >> 3, tok = threadIdx.x & 7;      // row 0..31 over the two tiles
             leader[tok * p.E + r0 + row] = v;
         }
         __syncthreads();
@@ -556,7 +567,7 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
         if (cfg.dynamicSmemBytes > 200 * 1024) return EDG_E_SHAPE;
         // an fp16 head whose rows and columns split into whole MMA tiles goes to the tensor cores
         if (d->pre_dtype == EDG_F16 && d->E % (16 * kPreCluster) == 0 && d->H % (16 * kPreWarps) == 0) {
-            cfg.dynamicSmemBytes = (size_t)kTokBlock * d->E * 4 + kPreWarps * 128 * 4 + (size_t)kTokBlock * (d->H * 2 + 16);
+            cfg.dynamicSmemBytes = (size_t)kTokBlock * d->E * 4 + kPreWarps * 256 * 4 + (size_t)kTokBlock * (d->H * 2 + 16);
             EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_mma_kernel, p, (int)n_heads));
             return EDG_OK;
         }
