@@ -10,12 +10,20 @@ call ``moe_layer_decode``.
 Default arm (``--impl b200``):
   value : layer-steps per second with everything resident in HBM.  The workload rotates over
           several independently seeded instances of the layer (each with all E experts resident),
-          so the bytes a step streams are far outside the L2 and come from HBM.  Steps are chained
-          through the routing (step t+1 consumes the top-k that step t produced) and launched from
-          CUDA graphs; timed with CUDA events on the launching stream.
+          so the bytes a step streams are far outside the L2 and come from HBM.  Steps depend on
+          one another through the routing only (step t+1 consumes the top-k that step t produced;
+          the hidden states are independent draws, as the configuration states) and are launched
+          from CUDA graphs.  Whatever ``--steps`` says, the timed region is WINDOWS windows of
+          WINDOW_STEPS steps each, timed with CUDA events on the launching stream; the median
+          window is reported (``config.timed_steps`` / ``config.windows``), so the number does not
+          depend on the flag.
+  dependent : the same layer-steps when the hidden state of step t+1 is produced on the device from
+          step t's output, x(t+1) = bf16(rmsnorm(x(t) + y(t))): no step can start its arithmetic
+          before the previous one has finished -- the latency a decoder sees.
   e2e   : the same metric with HOST buffers: the experts live in a pinned-host store, the HBM pool
           has the configuration's 8 slots, every step copies its hidden state host->device, stages
           the missing experts with cudaMemcpyAsync, runs the layer-step and reads y back.
+  secondary : batched decode (cfg4 shape) and prefill (cfg5 shape) on the same resident layer.
   roofline / cpu_baseline / clocks: see the keys of the JSON line.
 Reference arm (``--impl reference``): the fp64 CPU oracle, as it stands, on the host cores.
 """
@@ -40,9 +48,11 @@ from workloads import synth  # noqa: E402
 METRIC = "moe_layer_decode_tok_per_s_batch1"
 UNIT = "tok/s"
 WORKLOAD = "cfg2: one 35B-class MoE layer (H2048 I512 E256 top-8 int4 g64 LoRA r16), batch-1 decode"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised in profiles/fused_layer_kernel_cfg2.md.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from an ncu
+# capture of this workload (not measured by this run: reported as "from profile").
 NCU_TRAFFIC_BYTES = 15_591_424
+WINDOWS = 5            # timed windows; the median is reported
+WINDOW_STEPS = 2560    # layer-steps per window: ten replays of a 256-step graph
 
 
 def _peaks():
@@ -208,44 +218,40 @@ def run_b200(args):
         return g
 
     steps, warmup = args.steps, max(args.warmup, 3)
-    full, rem = divmod(steps, G)
-    # The hand-off ring has 128 slots and a captured chain has its slots baked in: a graph that is
-    # replayed again and again holds a multiple of 128 steps.  What is left of --steps is a graph of
-    # its own, captured and replayed last, and followed (untimed) by its complement to 128 so that
-    # the ring is back where the other graphs expect it.  The graphs are captured in the order in
-    # which they run, each starting where the one before it ends.
-    tail = rem % 128
-    rem -= tail
-    g_full = capture(G) if full or warmup else None
-    g_rem = capture(rem) if rem else None
-    g_tail = capture(tail) if tail else None
-    g_comp = capture(128 - tail, base=tail) if tail else None
+    # The hand-off ring has 128 slots and a captured chain has its slots baked in, so a graph that is
+    # replayed again and again holds a multiple of 128 steps: one graph of 256 steps, replayed.
+    store.set_chaining(1)                  # opt in: the captured steps are chained through the routing
+    g_full = capture(G)
+    reps = WINDOW_STEPS // G
+
+    def timed_windows(graph):
+        """WINDOWS windows of `reps` replays each, one event pair per window; ms per window, max over ranks."""
+        out = []
+        with torch.cuda.stream(stream):
+            for _ in range(WINDOWS):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(reps):
+                    graph.replay()
+                e1.record(stream)
+                out.append((e0, e1))
+            stream.synchronize()
+        return [replicas.max_over_ranks(a.elapsed_time(b), "cuda") for a, b in out]
 
     sampler = ClockSampler(_physical_device(local_rank))
     with torch.cuda.stream(stream):
-        for _ in range((warmup + G - 1) // G):
+        for _ in range(max(2, (warmup + G - 1) // G)):
             g_full.replay()
         stream.synchronize()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        sampler.start()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(full):
-            g_full.replay()
-        if g_rem is not None:
-            g_rem.replay()
-        if g_tail is not None:
-            g_tail.replay()
-        e1.record(stream)
-        stream.synchronize()
-        ms = e0.elapsed_time(e1)
-        if g_comp is not None:
-            g_comp.replay()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    window_ms = timed_windows(g_full)
+    with torch.cuda.stream(stream):
         # keep the GPU under the same load a little longer so the clock sampler sees it
         t_end = time.time() + 0.3
-        while time.time() < t_end and g_full is not None:
+        while time.time() < t_end:
             g_full.replay()
         stream.synchronize()
     clocks = sampler.stop()
@@ -254,9 +260,52 @@ def run_b200(args):
     if status != 0 or not bool(torch.isfinite(y).all()):
         raise SystemExit(f"bench: bad device status {status} or non-finite output")
 
-    ms_max = replicas.max_over_ranks(ms, "cuda")
-    value = replicas.whole_job_rate(world, steps, ms_max)
-    ms_per_step = ms_max / steps
+    ms_med = statistics.median(window_ms)
+    value = replicas.whole_job_rate(world, WINDOW_STEPS, ms_med)
+    ms_per_step = ms_med / WINDOW_STEPS
+
+    # ---- dependent arm: x(t+1) = bf16(rmsnorm(x(t) + y(t))) on the device, chaining off
+    dependent = None
+    if not args.no_dependent:
+        store.set_chaining(0)
+        xdep = torch.zeros((2, H), dtype=torch.bfloat16, device="cuda")
+        xdep[0] = xd[0]
+        ydep = torch.zeros((H,), dtype=torch.float32, device="cuda")
+
+        def dep_step(s_):
+            i = s_ % n_inst
+            edg.moe_layer_decode(store, i, xdep[s_ % 2], inds[s_ % 2], gates[s_ % 2], W[(s_ + 1) % n_inst],
+                                 inds[(s_ + 1) % 2], gates[(s_ + 1) % 2], None, ydep, ws)
+            edg.next_hidden_state(desc, xdep[s_ % 2], ydep, xdep[(s_ + 1) % 2], 1e-6)
+
+        with torch.cuda.stream(stream):
+            for s_ in range(2 * n_inst):
+                dep_step(s_)
+            stream.synchronize()
+        g_dep = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g_dep, stream=stream):
+                for s_ in range(G):
+                    dep_step(s_)
+            g_dep.replay()
+            stream.synchronize()
+        dep_ms = statistics.median(timed_windows(g_dep))
+        status = edg.workspace_status(ws)
+        if status != 0 or not bool(torch.isfinite(ydep).all()) or not bool(torch.isfinite(xdep.float()).all()):
+            raise SystemExit(f"bench: dependent arm: bad device status {status} or non-finite state")
+        dep_step_ms = dep_ms / WINDOW_STEPS
+        dependent = {"value": round(replicas.whole_job_rate(world, WINDOW_STEPS, dep_ms), 1), "unit": UNIT,
+                     "ms_per_step": round(dep_step_ms, 6),
+                     "hbm_gbs_on_expert_bytes": round(K * R / (dep_step_ms * 1e-3) / 1e9, 1),
+                     "frac_of_peak": round(K * R / (dep_step_ms * 1e-3) / 1e9 / _peaks()[0], 4),
+                     "dependency": "x(t+1) = bf16(rmsnorm(x(t) + y(t))) computed on the device: every step waits for the one before it",
+                     "launch": f"two kernels per step (layer-step, next-state norm), CUDA graphs of {G} steps, chaining off",
+                     "timed_steps": WINDOWS * WINDOW_STEPS, "windows": WINDOWS}
+
+    # ---- batched decode and prefill on the same resident layer (secondary figures)
+    secondary = None
+    if not args.no_secondary and world == 1:
+        secondary = run_secondary(edg, layer_io, cfg, desc, pool[0], loras[0], W[0], R)
 
     # ---- e2e arm: pinned-host store, 8 slots, copies inside the timed region
     e2e = None
@@ -269,7 +318,9 @@ def run_b200(args):
     launches_per_step = 1                  # one fused kernel: prerouter + take + FFN + reduce
     achieved = alg_bytes / (ms_per_step * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
-                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES, "peak_kind": how + " (burst copy)",
+                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES,
+                "traffic_source": "from profile (ncu capture of this kernel and workload), not measured by this run",
+                "peak_kind": how + " (burst copy)",
                 "kernel": "fused_layer_kernel (one launch per layer-step; duration = timed region / launches)",
                 "algorithmic_bytes_per_launch": alg_bytes}
 
@@ -287,14 +338,96 @@ def run_b200(args):
                        "hbm_working_set_bytes": n_inst * E * R,
                        "l2": "inputs larger than L2: steps rotate over the instances, routing iid from the prerouter",
                        "routing": "redrawn every step from the prerouter (step t+1 consumes step t's top-k)",
-                       "launch": f"CUDA graphs of {G} steps", "parallelism": "replicas only" if world > 1 else "1 GPU"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * steps,
+                       "dependency": "routing only: hidden states are independent draws, so steps overlap on the GPU; see 'dependent' for data-dependent steps",
+                       "timed_steps": WINDOWS * WINDOW_STEPS, "windows": WINDOWS,
+                       "window_ms": [round(m, 4) for m in window_ms],
+                       "timing": f"median of {WINDOWS} windows of {WINDOW_STEPS} steps, whatever --steps says",
+                       "launch": f"CUDA graphs of {G} steps, chained (edg_store_set_chaining 1)",
+                       "parallelism": "replicas only" if world > 1 else "1 GPU"},
+            "clocks": clocks, "e2e": e2e, "dependent": dependent, "secondary": secondary,
+            "gpu_launches": launches_per_step * WINDOWS * WINDOW_STEPS,
             "roofline": roofline, "cpu_baseline": cpu,
         }
         print(json.dumps(line))
     store.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def _event_ms(fn, iters, warmup=3):
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def run_secondary(edg, layer_io, cfg, desc, pool, lora, W, R):
+    """Batched decode (cfg4 shape: 64 concurrent tokens) and prefill (cfg5 shape: 4096 tokens, Zipf(1.1)
+    popularity) on one resident layer of the headline workload (same layer shape; `--workload cfg4` /
+    `cfg5` print the full lines on their own seeds)."""
+    import torch
+    K, E, H, I = cfg.K, cfg.E, cfg.H, cfg.I
+    peak_hbm, how = _peaks()
+    peak_tf = 1385.0
+    pk = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pk):
+        peak_tf = float(json.load(open(pk))["bf16_tflops_sustained"])
+    table = torch.arange(E, dtype=torch.int32, device="cuda")
+    out = {}
+    # ---- cfg4 shape
+    c4 = synth.CONFIGS["cfg4"]
+    T = c4.T
+    X = [layer_io.bits_to_device(synth.hidden_states(c4, T, stream=200 + i), torch.bfloat16) for i in range(4)]
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    y = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+    ws = layer_io.new_workspace(desc, T)
+    it, unions = [0], []
+
+    def step4():
+        x = X[it[0] % 4]; it[0] += 1
+        edg.prerouter_topk_tokens(desc, W, x, T, inds, gates, None)
+        edg.moe_expert_ffn_int4_lora(desc, pool, table, T, inds, None, gates, x, lora, y, ws)
+
+    for _ in range(4):
+        step4(); torch.cuda.synchronize(); unions.append(len(torch.unique(inds)))
+    ms = _event_ms(step4, 20)
+    ok = edg.workspace_status(ws) == 0 and bool(torch.isfinite(y).all())
+    union = float(np.mean(unions))
+    ach = union * R / (ms * 1e-3) / 1e9
+    out["cfg4_shape"] = {"tokens": T, "ms_per_step": round(ms, 5), "tok_per_s": round(T / (ms * 1e-3), 1),
+                         "experts_touched": union, "hbm_gbs_on_union_bytes": round(ach, 1),
+                         "frac_of_hbm_peak": round(ach / peak_hbm, 4), "ok": ok}
+    del ws, y
+    # ---- cfg5 shape
+    c5 = synth.CONFIGS["cfg5"]
+    T = c5.T
+    x = layer_io.bits_to_device(synth.hidden_states(c5, T, stream=300), torch.bfloat16)
+    logits = torch.from_numpy(synth.zipf_router_logits(c5, T)).cuda()
+    inds = torch.zeros((T, K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    y = torch.zeros((T, H), dtype=torch.float32, device="cuda")
+    ws = layer_io.new_workspace(desc, T)
+
+    def step5():
+        edg.softmax_topk_rows(desc, logits, T, inds, gates)
+        edg.moe_expert_ffn_int4_lora(desc, pool, table, T, inds, None, gates, x, lora, y, ws)
+
+    ms = _event_ms(step5, 10)
+    ok = edg.workspace_status(ws) == 0 and bool(torch.isfinite(y).all())
+    flops = T * K * (6.0 * H * I + 2.0 * cfg.rank * (2 * H + 3 * I + H))
+    tf = flops / (ms * 1e-3) / 1e12
+    out["cfg5_shape"] = {"tokens": T, "ms_per_step": round(ms, 4), "tok_per_s": round(T / (ms * 1e-3), 1),
+                         "tflops_algorithmic": round(tf, 1), "frac_of_tensor_peak": round(tf / peak_tf, 4),
+                         "peak_kind": "measured sustained bf16 GEMM", "ok": ok}
+    return out
 
 
 def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
@@ -318,21 +451,26 @@ def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
     y_host = torch.empty((H,), dtype=torch.float32).pin_memory()
     inds = torch.zeros((2, K), dtype=torch.int32, device="cuda")
     gates = torch.zeros((2, K), dtype=torch.float32, device="cuda")
-    inds_host = torch.empty((K,), dtype=torch.int32).pin_memory()
+    # the predicted routing is mirrored into pinned host memory by the kernels: the stager reads it
+    # there, without a device-to-host copy
+    mirror = torch.full((2, K), -1, dtype=torch.int32).pin_memory()
+    mir = mirror.numpy()
     st = torch.cuda.current_stream()
-    edg.prerouter_topk(desc, W, layer_io.bits_to_device(X_bits[NX - 1], torch.bfloat16), 1, inds[0], gates[0], None)
+    edg.prerouter_topk(desc, W, layer_io.bits_to_device(X_bits[NX - 1], torch.bfloat16), 1, inds[0], gates[0], None,
+                       inds_host_mirror_opt=mirror[0])
+    st.synchronize()
 
     def step(s):
         x_dev.copy_(x_host[s % NX], non_blocking=True)
-        inds_host.copy_(inds[s % 2], non_blocking=True)           # the prediction made one step earlier
-        st.synchronize()
-        edg.stage_experts_to_slots(store, 0, inds_host.numpy())
-        edg.moe_layer_decode(store, 0, x_dev, inds[s % 2], gates[s % 2], W, inds[(s + 1) % 2], gates[(s + 1) % 2],
-                             None, y_dev, ws)
+        cur, nxt = s % 2, (s + 1) % 2
+        edg.stage_experts_to_slots(store, 0, mir[cur])             # the prediction made one step earlier
+        mir[nxt] = -1
+        edg.moe_layer_decode(store, 0, x_dev, inds[cur], gates[cur], W, inds[nxt], gates[nxt],
+                             None, y_dev, ws, inds_next_host_mirror_opt=mirror[nxt])
         y_host.copy_(y_dev, non_blocking=True)
         st.synchronize()
 
-    n = max(2, min(args.steps, args.e2e_steps) // 2 * 2)   # an even count: the routing alternates between two buffers
+    n = max(64, min(args.steps, args.e2e_steps) // 2 * 2)  # an even count: the routing alternates between two buffers
     for s in range(max(4, min(args.warmup, 20) // 2 * 2)):
         step(s)
     base = store.stats()
@@ -353,6 +491,7 @@ def run_e2e(edg, layer_io, cfg, host_layer, lora, W, X_bits, args, world):
     table_bytes = (after["table_updates"] - base["table_updates"]) * E * 4 / n
     out = {"value": round(replicas.whole_job_rate(world, n, ms_max), 1), "unit": UNIT,
            "h2d_bytes_per_step": int(H * 2 + miss_bytes + table_bytes), "d2h_bytes_per_step": H * 4 + K * 4,
+           "d2h_note": "y by cudaMemcpyAsync; the K predicted indices by the kernel's own stores into mapped pinned memory",
            "steps": n, "slots": cfg.n_slots,
            "misses_per_step": round((after["misses"] - base["misses"]) / n, 3),
            "note": "pinned-host expert store, 8 slots, experts staged on demand by cudaMemcpyAsync: bound by host->device copy bandwidth"}
@@ -686,6 +825,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=400)
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dependent", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", choices=["cfg2", "cfg3", "cfg4", "cfg5", "sigmoid_group", "mlp_head"], default="cfg2",
                     help="cfg2 is the headline line; the others print their own line")

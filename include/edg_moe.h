@@ -29,7 +29,10 @@
  *
  * Quantised weight format (Sec. 3.1: int4, group-wise affine, one scale and one second parameter
  * per group of `group` consecutive input elements):  w[n][k] = scale[n][k/group] * (q[n][k] -
- * zero[n][k/group]),  q in 0..15, scale and zero stored as fp16.  Canonical interchange layout:
+ * zero[n][k/group]),  q in 0..15, scale and zero stored as fp16.  Zero points are values in
+ * [0, 16] that are multiples of 1/128 (integers 0..15 in the usual asymmetric scheme): for those
+ * every kernel forms q - zero without rounding, whichever precision it subtracts in;
+ * edg_pack_expert rejects any other zero point with EDG_E_RANGE.  Canonical interchange layout:
  * row-major [out][in]; byte j of a row holds q[2j] in its low nibble and q[2j+1] in its high nibble.
  * One expert = gate [I][H], up [I][H], down [H][I].  edg_pack_expert turns canonical tensors into
  * the record the kernels read; its size is edg_record_bytes (1,769,472 B at H=2048, I=512,
@@ -115,7 +118,9 @@ int32_t edg_record_bytes(const edg_layer_desc* desc, size_t* bytes);
 
 /* One-time host repack of canonical tensors (layout above; scales/zeros as fp16 bit patterns,
  * [out][in/group]) into the record the kernels read.  `record` is host memory of
- * edg_record_bytes bytes.  Never on the hot path.  edg_unpack_expert is its exact inverse. */
+ * edg_record_bytes bytes.  Never on the hot path.  edg_unpack_expert is its exact inverse.
+ * Returns EDG_E_RANGE (and writes nothing) when a zero point is outside [0, 16] or is not a
+ * multiple of 1/128. */
 int32_t edg_pack_expert(const edg_layer_desc* desc,
                         const uint8_t* codes_gate, const uint16_t* scales_gate, const uint16_t* zeros_gate,
                         const uint8_t* codes_up,   const uint16_t* scales_up,   const uint16_t* zeros_up,
@@ -156,9 +161,16 @@ int32_t edg_set_trace_buffer(void* dev_buffer);
  *   inds    dev int32 [n_heads][K], ascending expert index, distinct
  *   gates   dev float [n_heads][K], aligned with inds, sum to 1
  *   logits_opt  dev float [n_heads][E] or NULL: the fp32 logits the selection was made on
+ *   inds_host_mirror_opt  int32 [n_heads][K] in mapped pinned host memory (cudaHostAlloc; with
+ *               unified addressing the host pointer is what the kernel is given), or NULL: the
+ *               kernel stores the indices there too, so that the stager on the host can read the
+ *               prediction without a device-to-host copy and without synchronising the stream.
+ *               Protocol: the caller fills the mirror with -1 before the call; every entry is final
+ *               by itself once it is >= 0; a head's prediction is complete when its K entries are.
  * Equal logits go to the lower expert index. */
 int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
-                       int32_t* inds, float* gates, float* logits_opt, void* stream);
+                       int32_t* inds, float* gates, float* logits_opt, int32_t* inds_host_mirror_opt,
+                       void* stream);
 
 /* The same for T hidden states that all use ONE head (batched decode of one layer):
  * W_pre dev [E][H]; s dev bf16 [T][H]; outputs [T][K] / [T][E]. */
@@ -170,17 +182,6 @@ int32_t prerouter_topk_tokens(const edg_layer_desc* desc, const void* W_pre, con
 int32_t softmax_topk_rows(const edg_layer_desc* desc, const float* logits, int32_t T,
                           int32_t* inds, float* gates, void* stream);
 
-/* The other routing family of the paper (Appendix A, "Sigmoid-group"; its 8B tier runs n = 8 groups,
- * keep G = 4, K = 8, scale 2.5, E = 128) on given logits: sigma = sigmoid(l); a group's score is the
- * sum of its two largest selection scores, where the selection score is sigma, plus bias_opt[e] when a
- * bias is given (the "biased score" of the paper's remark); the keep_groups best groups survive,
- * ties to the lower group; the K best survivors by selection score are taken, ties to the lower
- * index; gates = scale * sigma[inds] / (sum of sigma[inds] + 1e-20) -- the raw sigmoid, not the biased
- * score.  logits dev float [T][E]; bias_opt dev float [E] or NULL; inds dev int32 [T][K] in
- * ascending index; gates dev float [T][K] aligned with inds.  E <= 1024, n_groups <= 32 dividing E
- * with at least two experts a group, K <= 32 and <= keep_groups * E / n_groups; else EDG_E_SHAPE.
- * One warp per row; no workspace; arithmetic in fp32 (the decision is taken in the kernel's
- * precision). */
 /* The full prerouter head of a layer (Sec. 3.2 "Head"): fc1 -> erf-gelu -> fc2 plus a linear residual
  * path.  The input feature is the hidden state followed by two K-hot vectors over the E experts --
  * the experts this layer routed to at this token and at the previous token -- so its dimension is
@@ -206,6 +207,17 @@ int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_head* head,
                            const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
                            int32_t* inds, float* gates, float* logits_opt, void* stream);
 
+/* The other routing family of the paper (Appendix A, "Sigmoid-group"; its 8B tier runs n = 8 groups,
+ * keep G = 4, K = 8, scale 2.5, E = 128) on given logits: sigma = sigmoid(l); a group's score is the
+ * sum of its two largest selection scores, where the selection score is sigma, plus bias_opt[e] when a
+ * bias is given (the "biased score" of the paper's remark); the keep_groups best groups survive,
+ * ties to the lower group; the K best survivors by selection score are taken, ties to the lower
+ * index; gates = scale * sigma[inds] / (sum of sigma[inds] + 1e-20) -- the raw sigmoid, not the biased
+ * score.  logits dev float [T][E]; bias_opt dev float [E] or NULL; inds dev int32 [T][K] in
+ * ascending index; gates dev float [T][K] aligned with inds.  E <= 1024, n_groups <= 32 dividing E
+ * with at least two experts a group, K <= 32 and <= keep_groups * E / n_groups; else EDG_E_SHAPE.
+ * One warp per row; no workspace; arithmetic in fp32 (the decision is taken in the kernel's
+ * precision). */
 int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32_t E, int32_t K, int32_t n_groups,
                                 int32_t keep_groups, float scale, const float* bias_opt,
                                 int32_t* inds, float* gates, void* stream);
@@ -308,10 +320,12 @@ int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* 
  * layer-step's routing (a1-a2); then marks the layer's slots free for restaging.
  *   x dev bf16 [H]; inds_cur dev int32 [K]; gates_cur dev float [K];
  *   W_pre_next dev [E][H] (NULL skips the prediction); inds_next dev int32 [K];
- *   gates_next dev float [K]; logits_next_opt dev float [E] or NULL; y dev [H] of out_dtype;
- *   workspace as for moe_expert_ffn_int4_lora with T = 1.
+ *   gates_next dev float [K]; logits_next_opt dev float [E] or NULL;
+ *   inds_next_host_mirror_opt int32 [K] in mapped pinned host memory or NULL: a second copy of
+ *   inds_next for the host-side stager, same protocol as in prerouter_topk;
+ *   y dev [H] of out_dtype; workspace as for moe_expert_ffn_int4_lora with T = 1.
  *
- * Chained calls.  When a call's inds_cur / gates_cur are the very buffers the previous call on this
+ * Chained calls (opt-in, see edg_store_set_chaining).  When chaining is on and a call's inds_cur / gates_cur are the very buffers the previous call on this
  * store wrote as inds_next / gates_next, with the same workspace and stream, the two layer-steps
  * are chained: the later kernel is launched as a programmatic dependent of the earlier one, starts
  * as soon as that one is running, and takes its routing from a ring inside the workspace: the
@@ -320,21 +334,60 @@ int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* 
  * steps share the GPU.  The results are those of unchained calls; what changes is the
  * contract on the inputs: a chained call reads x, W_pre_next and the slot pool as soon as it
  * starts, so they must already be valid when the call is made -- not produced by work queued
- * on the stream between the two calls.  Callers that cannot promise this switch chaining off
- * with edg_store_set_chaining.  A chain captured in a CUDA graph that is replayed back to back
+ * on the stream between the two calls.  Callers that cannot promise this leave chaining off
+ * (the default).  A chain captured in a CUDA graph that is replayed back to back
  * must hold a multiple of 128 layer-steps, so that every replay finds the ring where the
  * previous one left it. */
 int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          const int32_t* inds_cur, const float* gates_cur,
                          const void* W_pre_next, int32_t* inds_next, float* gates_next,
-                         float* logits_next_opt, void* y,
+                         float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
                          void* workspace, size_t workspace_bytes, void* stream);
 
-/* Chaining of consecutive moe_layer_decode calls: 0 off -- every layer-step is an ordinary
- * stream-ordered launch; 1 (default) a call is chained when the buffers line up and the step
- * before it is still in flight (its completion event has not fired) or the stream is being
- * captured -- a step that finds the GPU idle is launched on its own, across all SMs, which is
- * several times faster for that single step; 2 chained whenever the buffers line up. */
+/* One token through all n_layers layers of the store (the paper's decode timeline, Sec. 3.2
+ * "Motivation": full-token lead, one hand-off per token).  On the host: waits (bounded, 5 s) until the
+ * previous token's kernels have mirrored the routing of every layer into mirror_cur; resets
+ * mirror_next to -1; with prefetch != 0 stages the missing experts of ALL layers first, so that the
+ * copies of later layers overlap the compute of earlier ones (prefetch == 0: each layer is staged
+ * right before it runs -- the on-demand arm); then enqueues the n_layers layer-steps.  The head
+ * owned by layer l, evaluated on layer l's input, predicts layer (l + 1) mod n_layers at the next
+ * token (the double shift).  No stream synchronisation.
+ *   x dev bf16 [L][H] layer inputs; inds_cur dev int32 [L][K], gates_cur dev float [L][K]: this
+ *   token's routing; W_pre dev [L][E][H]; inds_next / gates_next dev [L][K], logits_next_opt dev
+ *   [L][E] or NULL: the next token's routing (row (l+1) mod L written by layer l);
+ *   mirror_cur / mirror_next int32 [L][K] in mapped pinned host memory: host copies of inds_cur
+ *   (complete when all entries are >= 0) and of inds_next; y dev [L][H] of out_dtype;
+ *   n_miss_out host, may be NULL: experts copied for this token.
+ * Returns EDG_E_TIMEOUT when the routing does not arrive, EDG_E_RANGE on an expert id >= E. */
+int32_t edg_stack_decode_token(edg_store* store, const void* x, const int32_t* inds_cur, const float* gates_cur,
+                               const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next_opt,
+                               const int32_t* mirror_cur, int32_t* mirror_next, void* y,
+                               void* workspace, size_t workspace_bytes, void* stream,
+                               int32_t prefetch, int32_t* n_miss_out);
+
+/* Measurement of exposed staging time: with edg_store_time_waits(store, 1) every wait that
+ * edg_store_wait_staged / moe_layer_decode actually enqueues on a compute stream is bracketed by a
+ * pair of timing events (outside stream capture); edg_store_exposed_wait_ms synchronises on them,
+ * returns the summed time the compute streams were held up by staging copies since the last call
+ * and the number of waits, and resets both.  Enabling allocates events: not a hot call. */
+int32_t edg_store_time_waits(edg_store* store, int32_t enable);
+int32_t edg_store_exposed_wait_ms(edg_store* store, double* ms_out, int64_t* n_waits_out);
+
+/* The hidden state a decoder would hand to the next layer-step: x_next = bf16(rmsnorm(x + y)),
+ * unit gain, rmsnorm(v) = v / sqrt(mean(v^2) + eps) -- residual connection plus the next block's
+ * input norm.  The paper's method has no such step (attention and the shared expert sit between
+ * two MoE blocks there); this is the benchmark's stand-in that makes consecutive layer-steps
+ * data-dependent.  x dev bf16 [H]; y dev [H] of desc->out_dtype; x_next dev bf16 [H]; H <= 4096. */
+int32_t edg_next_hidden_state(const edg_layer_desc* desc, const void* x, const void* y, void* x_next,
+                              float eps, void* stream);
+
+/* Chaining of consecutive moe_layer_decode calls: 0 (default) off -- every layer-step is an
+ * ordinary stream-ordered launch and the usual stream semantics hold for every input; 1 a call is
+ * chained when the buffers line up and the step before it is still in flight (its completion
+ * event has not fired) or the stream is being captured -- a step that finds the GPU idle is
+ * launched on its own, across all SMs, which is several times faster for that single step;
+ * 2 chained whenever the buffers line up.  Switching it on accepts the contract on the inputs of
+ * chained calls stated above. */
 int32_t edg_store_set_chaining(edg_store* store, int32_t enable);
 
 #ifdef __cplusplus

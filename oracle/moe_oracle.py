@@ -316,6 +316,16 @@ def moe_layer_decode(x_bits, inds_cur, gates_cur, W_pre_next, K: int, get_expert
     return y, slots, copies, inds_next, gates_next, logits
 
 
+# ------------------------------------------------------------------ chaining consecutive layer-steps (benchmark construct)
+
+def next_hidden_state(x_bits, y, eps: float = 1e-6) -> np.ndarray:
+    """x_next = bf16(rmsnorm(x + y)), unit gain, rmsnorm(v) = v / sqrt(mean(v^2) + eps): residual
+    connection plus the next block's input norm.  Not a step of the paper's method; the stand-in by
+    which the dependent-chain measurement makes step t+1 wait for step t's output.  Returns bf16 bits."""
+    v = bf16_to_f64(x_bits) + np.asarray(y, dtype=np.float64)
+    return f64_to_bf16_bits(v / math.sqrt(float(np.mean(v * v)) + eps))
+
+
 # ------------------------------------------------------------------ error measures used by the parity tests
 
 def rel_l2(a, b) -> float:

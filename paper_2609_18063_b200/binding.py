@@ -16,7 +16,8 @@ __all__ = [
     "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
     "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows", "sigmoid_group_topk_rows", "prerouter_mlp_topk",
-    "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots", "EXPORTS",
+    "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots",
+    "stack_decode_token", "next_hidden_state", "EXPORTS",
 ]
 
 F32, F16, BF16 = 0, 1, 2
@@ -66,7 +67,7 @@ _SIG = {
     "edg_ffn_workspace_bytes": ([_D, C.c_int32, C.POINTER(C.c_size_t)], C.c_int32),
     "edg_workspace_status": ([_P, _P, C.POINTER(C.c_int32)], C.c_int32),
     "edg_set_trace_buffer": ([_P], C.c_int32),
-    "prerouter_topk": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
+    "prerouter_topk": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P, _P], C.c_int32),
     "prerouter_topk_tokens": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "softmax_topk_rows": ([_D, _P, C.c_int32, _P, _P, _P], C.c_int32),
     "sigmoid_group_topk_rows": ([_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, _P, _P], C.c_int32),
@@ -77,11 +78,15 @@ _SIG = {
     "edg_store_set_chaining": ([_P, C.c_int32], C.c_int32),
     "edg_store_snapshot": ([_P, C.c_int32, _P, _P], C.c_int32),
     "edg_store_wait_staged": ([_P, C.c_int32, _P], C.c_int32),
+    "edg_store_time_waits": ([_P, C.c_int32], C.c_int32),
+    "edg_store_exposed_wait_ms": ([_P, C.POINTER(C.c_double), C.POINTER(C.c_int64)], C.c_int32),
+    "edg_stack_decode_token": ([_P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, C.c_size_t, _P, C.c_int32, C.POINTER(C.c_int32)], C.c_int32),
+    "edg_next_hidden_state": ([_D, _P, _P, _P, C.c_float, _P], C.c_int32),
     "edg_store_mark_computed": ([_P, C.c_int32, _P], C.c_int32),
     "stage_experts_to_slots": ([_P, C.c_int32, _P, C.c_int32, _P, C.POINTER(C.c_int32)], C.c_int32),
     "moe_expert_ffn_int4_lora": ([_D, _P, _P, C.c_int32, _P, _P, _P, _P, C.POINTER(Lora), _P, _P, C.c_size_t, _P], C.c_int32),
     "moe_expert_ffn_int4_lora_static": ([_D, _P, _P, _P, _P, _P, _P, C.POINTER(Lora), _P, _P], C.c_int32),
-    "moe_layer_decode": ([_P, C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, C.c_size_t, _P], C.c_int32),
+    "moe_layer_decode": ([_P, C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, C.c_size_t, _P], C.c_int32),
 }
 EXPORTS = tuple(_SIG)
 for _name, (_args, _res) in _SIG.items():
@@ -216,9 +221,9 @@ def set_trace_buffer(dev_buffer) -> None:
     _check(_lib.edg_set_trace_buffer(_ptr(dev_buffer)), "edg_set_trace_buffer")
 
 
-def prerouter_topk(desc, W_pre, s, n_heads, inds, gates, logits_opt=None, stream=None) -> None:
+def prerouter_topk(desc, W_pre, s, n_heads, inds, gates, logits_opt=None, stream=None, inds_host_mirror_opt=None) -> None:
     _check(_lib.prerouter_topk(C.byref(desc), _ptr(W_pre), _ptr(s), n_heads, _ptr(inds), _ptr(gates),
-                               _ptr(logits_opt), _stream(stream)), "prerouter_topk")
+                               _ptr(logits_opt), _ptr(inds_host_mirror_opt), _stream(stream)), "prerouter_topk")
 
 
 def prerouter_topk_tokens(desc, W_pre, s, T, inds, gates, logits_opt=None, stream=None) -> None:
@@ -296,7 +301,7 @@ class Store:
             pass
 
     def set_chaining(self, enable) -> None:
-        """False / 0: off; True / 1: chain a step when the one before it is still in flight (default);
+        """False / 0: off (default); True / 1: chain a step when the one before it is still in flight;
         2: chain whenever the buffers line up."""
         _check(_lib.edg_store_set_chaining(self.handle, int(enable)), "edg_store_set_chaining")
 
@@ -314,6 +319,15 @@ class Store:
     def wait_staged(self, layer: int, stream=None) -> None:
         _check(_lib.edg_store_wait_staged(self.handle, layer, _stream(stream)), "edg_store_wait_staged")
 
+    def time_waits(self, enable: bool) -> None:
+        _check(_lib.edg_store_time_waits(self.handle, int(bool(enable))), "edg_store_time_waits")
+
+    def exposed_wait_ms(self):
+        """(ms the compute streams waited for staging copies since the last call, number of waits)."""
+        ms, n = C.c_double(), C.c_int64()
+        _check(_lib.edg_store_exposed_wait_ms(self.handle, C.byref(ms), C.byref(n)), "edg_store_exposed_wait_ms")
+        return ms.value, n.value
+
     def mark_computed(self, layer: int, stream=None) -> None:
         _check(_lib.edg_store_mark_computed(self.handle, layer, _stream(stream)), "edg_store_mark_computed")
 
@@ -330,9 +344,29 @@ def stage_experts_to_slots(store: Store, layer: int, inds_host, n: Optional[int]
 
 
 def moe_layer_decode(store: Store, layer, x, inds_cur, gates_cur, W_pre_next, inds_next, gates_next,
-                     logits_next_opt, y, workspace, workspace_bytes=None, stream=None) -> None:
+                     logits_next_opt, y, workspace, workspace_bytes=None, stream=None,
+                     inds_next_host_mirror_opt=None) -> None:
     if workspace_bytes is None:
         workspace_bytes = workspace.numel() * workspace.element_size()
     _check(_lib.moe_layer_decode(store.handle, layer, _ptr(x), _ptr(inds_cur), _ptr(gates_cur), _ptr(W_pre_next),
-                                 _ptr(inds_next), _ptr(gates_next), _ptr(logits_next_opt), _ptr(y),
+                                 _ptr(inds_next), _ptr(gates_next), _ptr(logits_next_opt),
+                                 _ptr(inds_next_host_mirror_opt), _ptr(y),
                                  _ptr(workspace), workspace_bytes, _stream(stream)), "moe_layer_decode")
+
+
+def stack_decode_token(store: Store, x, inds_cur, gates_cur, W_pre, inds_next, gates_next, logits_next_opt,
+                       mirror_cur, mirror_next, y, workspace, workspace_bytes=None, stream=None, prefetch=True) -> int:
+    """edg_stack_decode_token; returns the number of experts copied for this token."""
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    miss = C.c_int32()
+    _check(_lib.edg_stack_decode_token(store.handle, _ptr(x), _ptr(inds_cur), _ptr(gates_cur), _ptr(W_pre),
+                                       _ptr(inds_next), _ptr(gates_next), _ptr(logits_next_opt), _ptr(mirror_cur),
+                                       _ptr(mirror_next), _ptr(y), _ptr(workspace), workspace_bytes, _stream(stream),
+                                       int(bool(prefetch)), C.byref(miss)), "edg_stack_decode_token")
+    return miss.value
+
+
+def next_hidden_state(desc, x, y, x_next, eps=1e-6, stream=None) -> None:
+    _check(_lib.edg_next_hidden_state(C.byref(desc), _ptr(x), _ptr(y), _ptr(x_next), float(eps), _stream(stream)),
+           "edg_next_hidden_state")

@@ -140,6 +140,29 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
 
 int32_t check_desc(const edg_layer_desc* d);   // EDG_OK or EDG_E_INVAL / EDG_E_SHAPE
 
+// ---------------------------------------------------------------- host entry points shared by the translation units
+
+// What the batch-1 layer kernel can do beyond the plain layer-step; all optional.
+struct FusedExtras {
+    int32_t* inds_mirror = nullptr;        // [K] copy of inds_next in mapped pinned host memory
+};
+
+bool fused_supported(const edg_layer_desc& d);
+// One fused launch for a batch-1 layer-step (edg_decode_fused.cu).  W_pre may be null (no prediction).
+int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
+                        const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
+                        const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st,
+                        const FusedExtras* extras = nullptr);
+// a4-a6 for T tokens on whatever kernels fit the shape (edg_ffn.cu)
+int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots,
+                const int32_t* table, const int32_t* experts, const float* gates, const void* x,
+                const edg_lora* lora, void* y, void* workspace, size_t workspace_bytes, cudaStream_t st);
+// a1-a2 for n_heads (head, state) pairs, or for n_heads states of one head (edg_prerouter.cu)
+int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head = 0,
+                      int32_t* mirror = nullptr);
+
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 
@@ -376,6 +399,17 @@ __device__ __forceinline__ void warp_softmax_topk(float* work, int E, int K, int
         __syncwarp();
     }
     topk_emit(myv, myi, K, lane, inds, gates);
+}
+
+// A warp's K freshly written indices, copied to a mirror in mapped pinned host memory with
+// system-scope stores.  Each entry is final by itself: a host that has filled the mirror with -1
+// beforehand may poll it and take the prediction as complete once all K entries are >= 0.
+__device__ __forceinline__ void mirror_inds(int32_t* mirror, const int32_t* inds, int K, int lane) {
+    __syncwarp();
+    if (mirror != nullptr && lane < K) {
+        const int v = inds[lane];
+        asm volatile("st.relaxed.sys.global.s32 [%0], %1;" ::"l"(mirror + lane), "r"(v) : "memory");
+    }
 }
 
 template <typename T> __device__ __forceinline__ void store_out(T* y, size_t i, float v);

@@ -148,6 +148,7 @@ struct FusedParams {
     int qpc;                      // quarters of the intermediate dimension per cluster: 4 (one cluster per expert), 2 or 1
     int epc;                      // experts per cluster, one after the other: 1, or 2 or 4 (only with qpc = 4)
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
+    int32_t* inds_mirror;         // [K] copy of inds_next in mapped pinned host memory, or null
     FusedSmem S;                  // shared-memory carve-up
 };
 
@@ -429,6 +430,9 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
         }
         p.inds_next[lane] = s_i[lane];
         p.gates_next[lane] = s_g[lane];
+        // (each entry is final by itself: the host polls the mirror until all K are >= 0)
+        if (p.inds_mirror != nullptr)
+            asm volatile("st.relaxed.sys.global.s32 [%0], %1;" ::"l"(p.inds_mirror + lane), "r"(s_i[lane]) : "memory");
     }
     if (lane == 0) trace_stamp(p, 15);
 }
@@ -1238,7 +1242,8 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
 int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
                         const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                         const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st) {
+                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st,
+                        const FusedExtras* extras) {
     const bool has_lora = lora != nullptr && d->rank > 0;
     FusedParams p{};
     p.pool = static_cast<const uint8_t*>(slot_pool);
@@ -1267,12 +1272,11 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlDone);
     p.ring = ring;
     p.stale = stale;
+    if (extras != nullptr) p.inds_mirror = extras->inds_mirror;
     // a chained step shares the GPU with its neighbours: few, long-lived CTAs; a lone step wants all SMs at once
     p.qpc = flag_in >= 0 ? kDownSlices : 1;
-    // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
-    // CTAs per step, each amortising its start-up over twice the bytes
-    // ... and when the experts share one adapter a cluster takes two experts, one after the other: half as many
-    // CTAs per step, each amortising its start-up over twice the bytes
+    // ... and when the experts share one adapter a cluster takes two or four experts, one after the other:
+    // fewer CTAs per step, each amortising its start-up over more bytes
     const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // up to 8 kFW head rows per CTA
     p.epc = 1;
     for (int c = 2; c <= kMaxEpc; c *= 2)

@@ -8,12 +8,6 @@
 
 namespace edg {
 
-bool fused_supported(const edg_layer_desc& d);
-int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
-                        const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
-                        const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st);
-
 int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots, const int32_t* table,
                     const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
                     void* workspace, cudaStream_t st);

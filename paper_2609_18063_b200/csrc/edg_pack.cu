@@ -45,6 +45,27 @@ static void repack(const edg_layer_desc& d, int N, int Kd, bool down, uint8_t* r
     }
 }
 
+// A zero point the kernels can subtract from a code without rounding: an fp16 value in [0, 16]
+// that is a multiple of 1/128 (then q - z, |q - z| <= 16, fits the 11 significant bits of fp16).
+static bool zero_point_ok(uint16_t bits) {
+    if (bits & 0x8000u) return (bits & 0x7FFFu) == 0;          // -0 only
+    const int exp = (bits >> 10) & 0x1F, man = bits & 0x3FF;
+    if (exp == 0) return man == 0;                               // subnormals are below 1/128
+    if (exp == 0x1F) return false;                               // inf / nan
+    const int e = exp - 15;                                      // value = (1024 + man) * 2^(e - 10)
+    if (e > 4 || (e == 4 && man != 0)) return false;             // above 16
+    const int shift = 3 - e;                                     // low bits that must be clear for a multiple of 2^-7
+    if (shift <= 0) return true;
+    if (shift > 10) return false;                                // below 1/128 and not zero
+    return (man & ((1 << shift) - 1)) == 0;
+}
+
+static bool zero_points_ok(const uint16_t* z, size_t n) {
+    for (size_t i = 0; i < n; ++i)
+        if (!zero_point_ok(z[i])) return false;
+    return true;
+}
+
 }  // namespace edg
 
 extern "C" int32_t edg_version(void) { return 1000; }
@@ -70,6 +91,9 @@ extern "C" int32_t edg_pack_expert(const edg_layer_desc* desc,
     int32_t rc = edg::check_desc(desc);
     if (rc != EDG_OK) return rc;
     if (!cg || !sg || !zg || !cu || !su || !zu || !cd || !sd || !zd || !record) return EDG_E_INVAL;
+    const size_t n_groups = (size_t)desc->H * desc->I / desc->group;
+    if (!edg::zero_points_ok(zg, n_groups) || !edg::zero_points_ok(zu, n_groups) || !edg::zero_points_ok(zd, n_groups))
+        return EDG_E_RANGE;
     const edg::RecordLayout L = edg::record_layout(desc->H, desc->I, desc->group);
     uint8_t* r = static_cast<uint8_t*>(record);
     // Inside every 16-byte chunk the canonical nibble order is kept (a 32-bit word holds code k in

@@ -26,6 +26,7 @@ struct PreParams {
     float* logits;          // [n_heads][E] or null
     int H, E, K;
     int shared_head;        // 1: every state uses head 0 (batched tokens of one layer)
+    int32_t* mirror;        // [n_heads][K] in mapped pinned host memory, or null
 };
 
 template <typename WT> struct RowDot;
@@ -103,8 +104,10 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_kernel(PreParams p) 
     if (p.logits != nullptr)
         for (int e = threadIdx.x; e < p.E; e += blockDim.x) p.logits[(size_t)head * p.E + e] = s_logits[e];
     __syncthreads();
-    if (warp == 0)
+    if (warp == 0) {
         warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds + (size_t)head * p.K, p.gates + (size_t)head * p.K);
+        mirror_inds(p.mirror != nullptr ? p.mirror + (size_t)head * p.K : nullptr, p.inds + (size_t)head * p.K, p.K, lane);
+    }
 }
 
 // One head, T hidden states (batched decode of one layer): a cluster handles kTokBlock tokens, so
@@ -536,12 +539,13 @@ __global__ void __launch_bounds__(128) sigmoid_group_topk_rows_kernel(const floa
 }
 
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
-                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head = 0) {
+                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head,
+                      int32_t* mirror) {
     int32_t rc = check_desc(d);
     if (rc != EDG_OK) return rc;
     if (!W_pre || !s || !inds || !gates || n_heads < 1 || n_heads > 65535) return EDG_E_INVAL;
     if (!aligned(W_pre, 16) || !aligned(s, 16)) return EDG_E_INVAL;
-    PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K, shared_head};
+    PreParams p{W_pre, static_cast<const uint16_t*>(s), inds, gates, logits_opt, d->H, d->E, d->K, shared_head, mirror};
 
     const bool batched = shared_head != 0 && n_heads > 1;     // one head, several tokens: a cluster per block of tokens
     cudaLaunchConfig_t cfg = {};
@@ -583,8 +587,10 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
 }  // namespace edg
 
 extern "C" int32_t prerouter_topk(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t n_heads,
-                                  int32_t* inds, float* gates, float* logits_opt, void* stream) {
-    return edg::run_prerouter(desc, W_pre, s, n_heads, inds, gates, logits_opt, static_cast<cudaStream_t>(stream));
+                                  int32_t* inds, float* gates, float* logits_opt, int32_t* inds_host_mirror_opt,
+                                  void* stream) {
+    return edg::run_prerouter(desc, W_pre, s, n_heads, inds, gates, logits_opt, static_cast<cudaStream_t>(stream), 0,
+                              inds_host_mirror_opt);
 }
 
 extern "C" int32_t prerouter_topk_tokens(const edg_layer_desc* desc, const void* W_pre, const void* s, int32_t T,

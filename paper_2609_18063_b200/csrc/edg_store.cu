@@ -7,23 +7,12 @@
 // stream, ordered after the layer's last compute by an event, so that the copies of the next
 // token overlap the compute of the current one.  Slots are sticky: an expert that stays routed
 // is never copied again, and a step rewrites only the slots whose expert changed.
+#include <chrono>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "edg_common.cuh"
-
-namespace edg {
-int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const int32_t* slots,
-                const int32_t* table, const int32_t* experts, const float* gates, const void* x,
-                const edg_lora* lora, void* y, void* workspace, size_t workspace_bytes, cudaStream_t st);
-bool fused_supported(const edg_layer_desc& d);
-int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const int32_t* slots, const int32_t* table,
-                        const int32_t* experts, const float* gates, const void* x, const edg_lora* lora, void* y,
-                        const void* W_pre, int32_t* inds_next, float* gates_next, float* logits_next,
-                        void* workspace, int flag_in, int flag_out, int ring, int stale, cudaStream_t st);
-int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
-                      int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head);
-}  // namespace edg
 
 namespace {
 
@@ -68,10 +57,32 @@ struct edg_store {
     const void* ring_ws = nullptr;         // workspace whose hand-off ring this store has initialised
     int ring_next = 0;                     // ring slot of the next batch-1 layer-step
     int pub_slot = -1;                     // ring slot holding logits no step has read yet, or -1
-    int chaining = 1;                      // 0 off, 1 when the previous step is still in flight (or under capture), 2 always
+    int chaining = 0;                      // 0 off (default), 1 when the previous step is still in flight (or under capture), 2 always
     cudaEvent_t step_done = nullptr;       // recorded behind every batch-1 layer-step launched outside a capture
     bool step_done_valid = false;
+    // optional measurement of the time compute streams spend waiting for staging copies: an event
+    // pair around every wait that is actually enqueued
+    bool time_waits = false;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> wait_events;
+    size_t wait_used = 0;
+    double wait_ms = 0.0;
+    int64_t wait_count = 0;
 };
+
+constexpr size_t kWaitPairs = 2048;
+
+// adds up the pairs recorded so far (synchronising on the last of them) and frees the pool
+static int32_t drain_waits(edg_store* s) {
+    for (size_t i = 0; i < s->wait_used; ++i) {
+        EDG_CUDA_TRY(cudaEventSynchronize(s->wait_events[i].second));
+        float ms = 0.f;
+        EDG_CUDA_TRY(cudaEventElapsedTime(&ms, s->wait_events[i].first, s->wait_events[i].second));
+        s->wait_ms += ms;
+    }
+    s->wait_count += (int64_t)s->wait_used;
+    s->wait_used = 0;
+    return EDG_OK;
+}
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
 
@@ -133,6 +144,10 @@ extern "C" int32_t edg_store_destroy(edg_store* s) {
         if (s->ring_ev[i]) cudaEventDestroy(s->ring_ev[i]);
     if (s->ring) cudaFreeHost(s->ring);
     if (s->step_done) cudaEventDestroy(s->step_done);
+    for (auto& pr : s->wait_events) {
+        if (pr.first) cudaEventDestroy(pr.first);
+        if (pr.second) cudaEventDestroy(pr.second);
+    }
     s->magic = 0;
     delete s;
     return EDG_OK;
@@ -231,9 +246,46 @@ extern "C" int32_t edg_store_wait_staged(edg_store* s, int32_t layer, void* stre
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     LayerState& L = s->layers[layer];
     if (L.copy_pending) {
-        EDG_CUDA_TRY(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), L.copy_done, 0));
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (s->time_waits) EDG_CUDA_TRY(cudaStreamIsCapturing(st, &capturing));
+        const bool timed = s->time_waits && capturing == cudaStreamCaptureStatusNone;
+        if (timed && s->wait_used == s->wait_events.size()) {
+            int32_t rc = drain_waits(s);
+            if (rc != EDG_OK) return rc;
+        }
+        if (timed) EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].first, st));
+        EDG_CUDA_TRY(cudaStreamWaitEvent(st, L.copy_done, 0));
+        if (timed) {
+            EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].second, st));
+            s->wait_used += 1;
+        }
         L.copy_pending = false;
     }
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_time_waits(edg_store* s, int32_t enable) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (enable && s->wait_events.empty()) {
+        s->wait_events.assign(kWaitPairs, std::make_pair((cudaEvent_t) nullptr, (cudaEvent_t) nullptr));
+        for (auto& pr : s->wait_events) {
+            EDG_CUDA_TRY(cudaEventCreate(&pr.first));
+            EDG_CUDA_TRY(cudaEventCreate(&pr.second));
+        }
+    }
+    s->time_waits = enable != 0;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_exposed_wait_ms(edg_store* s, double* ms_out, int64_t* n_waits_out) {
+    if (!store_ok(s) || !ms_out) return EDG_E_INVAL;
+    int32_t rc = drain_waits(s);
+    if (rc != EDG_OK) return rc;
+    *ms_out = s->wait_ms;
+    if (n_waits_out) *n_waits_out = s->wait_count;
+    s->wait_ms = 0.0;
+    s->wait_count = 0;
     return EDG_OK;
 }
 
@@ -252,7 +304,7 @@ extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* st
 extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
                                     const int32_t* inds_cur, const float* gates_cur,
                                     const void* W_pre_next, int32_t* inds_next, float* gates_next,
-                                    float* logits_next_opt, void* y,
+                                    float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
                                     void* workspace, size_t workspace_bytes, void* stream) {
     if (!store_ok(s) || !x || !inds_cur || !gates_cur || !y) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
@@ -303,9 +355,11 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         const int ring = s->ring_next;                               // ring slot of this step's scratch and of the head it evaluates
         const int flag_out = W_pre_next != nullptr ? ring : -1;
         s->ring_next = (ring + 1) % edg::kHandoffRing;
+        edg::FusedExtras extras;
+        extras.inds_mirror = W_pre_next != nullptr ? inds_next_host_mirror_opt : nullptr;
         rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
-                                  logits_next_opt, workspace, flag_in, flag_out, ring, stale, st);
+                                  logits_next_opt, workspace, flag_in, flag_out, ring, stale, st, &extras);
         if (W_pre_next != nullptr) s->pub_slot = flag_out;
         if (rc != EDG_OK) return rc;
         s->step_done_valid = false;
@@ -322,11 +376,69 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         rc = edg::run_ffn(&s->d, pool, 1, inds_cur, table, nullptr, gates_cur, x, lora, y, workspace, workspace_bytes, st);
         if (rc != EDG_OK) return rc;
         if (W_pre_next != nullptr) {
-            rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st, 0);
+            rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st, 0,
+                                    inds_next_host_mirror_opt);
             if (rc != EDG_OK) return rc;
         }
     }
     return edg_store_mark_computed(s, layer, stream);
+}
+
+extern "C" int32_t edg_stack_decode_token(edg_store* s, const void* x, const int32_t* inds_cur, const float* gates_cur,
+                                          const void* W_pre, int32_t* inds_next, float* gates_next,
+                                          float* logits_next_opt, const int32_t* mirror_cur, int32_t* mirror_next,
+                                          void* y, void* workspace, size_t workspace_bytes, void* stream,
+                                          int32_t prefetch, int32_t* n_miss_out) {
+    if (!store_ok(s) || !x || !inds_cur || !gates_cur || !W_pre || !inds_next || !gates_next || !mirror_cur ||
+        !mirror_next || !y)
+        return EDG_E_INVAL;
+    const int L = s->n_layers, K = s->d.K, E = s->d.E, H = s->d.H;
+    // (1) the single hand-off of the token: the routing of every layer, predicted during the previous
+    //     token, as the kernels have mirrored it into host memory.  Bounded wait.
+    {
+        const volatile int32_t* m = mirror_cur;
+        const auto t0 = std::chrono::steady_clock::now();
+        int done = 0;
+        for (uint64_t spin = 0; done < L * K; ++spin) {
+            while (done < L * K && m[done] >= 0) ++done;
+            if (done < L * K && (spin & 0xFFF) == 0xFFF &&
+                std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count() > 5.0)
+                return EDG_E_TIMEOUT;
+        }
+    }
+    for (int i = 0; i < L * K; ++i) {
+        if (mirror_cur[i] >= E) return EDG_E_RANGE;
+        mirror_next[i] = -1;
+    }
+    int32_t slots_tmp[32];
+    int32_t miss = 0, total_miss = 0, rc;
+    // (2) prediction-driven staging: every layer's missing experts are queued on the copy stream
+    //     before the first layer runs, so later layers' copies overlap earlier layers' compute
+    if (prefetch)
+        for (int l = 0; l < L; ++l) {
+            rc = stage_experts_to_slots(s, l, mirror_cur + (size_t)l * K, K, slots_tmp, &miss);
+            if (rc != EDG_OK) return rc;
+            total_miss += miss;
+        }
+    // (3) the layer-steps; the head owned by layer l predicts layer (l + 1) mod L at the next token
+    const size_t wb = (size_t)E * H * (s->d.pre_dtype == EDG_F16 ? 2 : 4);
+    const size_t yb = (size_t)H * (s->d.out_dtype == EDG_F32 ? 4 : 2);
+    for (int l = 0; l < L; ++l) {
+        if (!prefetch) {
+            rc = stage_experts_to_slots(s, l, mirror_cur + (size_t)l * K, K, slots_tmp, &miss);
+            if (rc != EDG_OK) return rc;
+            total_miss += miss;
+        }
+        const int ln = (l + 1) % L;
+        rc = moe_layer_decode(s, l, static_cast<const uint16_t*>(x) + (size_t)l * H, inds_cur + (size_t)l * K,
+                              gates_cur + (size_t)l * K, static_cast<const uint8_t*>(W_pre) + (size_t)l * wb,
+                              inds_next + (size_t)ln * K, gates_next + (size_t)ln * K,
+                              logits_next_opt ? logits_next_opt + (size_t)ln * E : nullptr, mirror_next + (size_t)ln * K,
+                              static_cast<uint8_t*>(y) + (size_t)l * yb, workspace, workspace_bytes, stream);
+        if (rc != EDG_OK) return rc;
+    }
+    if (n_miss_out) *n_miss_out = total_miss;
+    return EDG_OK;
 }
 
 extern "C" int32_t edg_store_set_chaining(edg_store* s, int32_t enable) {

@@ -1,15 +1,16 @@
-"""Host loop of the expert stack: one token through L MoE layers with prediction-driven staging.
+"""The expert stack: one token through L MoE layers with prediction-driven staging.
 
-Orchestration only -- every arithmetic step runs in the CUDA library.  Per token the loop does what
-the paper's decode timeline shows: the routing of every layer was predicted one token earlier (the
-head owned by layer l, evaluated on that layer's input at token t, predicts layer (l+1) mod L at
-token t+1); it is handed to the host once per token (the single flush), the stager enqueues the
+A thin owner of the buffers around ``edg_stack_decode_token`` -- the per-token host loop itself (wait
+for the mirrored routing, stage, enqueue the L layer-steps) runs inside the C library.  Per token
+it does what the paper's decode timeline shows: the routing of every layer was predicted one token
+earlier (the head owned by layer l, evaluated on that layer's input at token t, predicts layer
+(l+1) mod L at token t+1); the kernels mirror it into pinned host memory, so the single hand-off of
+a token needs neither a device-to-host copy nor a stream synchronisation; the stager enqueues the
 copies of the missing experts on the side stream, and each layer's kernel waits only for its own
 layer's copies, so later layers' copies overlap earlier layers' compute.
 """
 from __future__ import annotations
 
-import numpy as np
 import torch
 
 from . import binding as B
@@ -24,7 +25,8 @@ class StackDecoder:
         K = desc.K
         self.inds = torch.zeros((2, self.L, K), dtype=torch.int32, device="cuda")
         self.gates = torch.zeros((2, self.L, K), dtype=torch.float32, device="cuda")
-        self.inds_host = torch.zeros((self.L, K), dtype=torch.int32).pin_memory()
+        # host mirrors of the two routing buffers, written by the kernels themselves (-1 = not yet)
+        self.mirror = torch.full((2, self.L, K), -1, dtype=torch.int32).pin_memory()
         self.ws = layer_io.new_workspace(desc)
         self.misses = 0
 
@@ -38,22 +40,12 @@ class StackDecoder:
         # head l feeds layer (l+1) % L
         self.inds[0] = torch.roll(tmp_i, 1, dims=0)
         self.gates[0] = torch.roll(tmp_g, 1, dims=0)
+        self.mirror[0].copy_(self.inds[0])
+        torch.cuda.current_stream().synchronize()
 
     def step(self, t: int, X: torch.Tensor, Y: torch.Tensor, logits_out=None) -> None:
         """Token t: X device bf16 [L][H] (layer inputs), Y device [L][H] (layer outputs)."""
         cur, nxt = t % 2, (t + 1) % 2
-        stream = torch.cuda.current_stream()
-        # one hand-off per token: the predictions made during the previous token
-        self.inds_host.copy_(self.inds[cur], non_blocking=True)
-        stream.synchronize()
-        ih = self.inds_host.numpy()
-        if self.prefetch:
-            for l in range(self.L):
-                self.misses += B.stage_experts_to_slots(self.store, l, ih[l])[1]
-        for l in range(self.L):
-            if not self.prefetch:
-                self.misses += B.stage_experts_to_slots(self.store, l, ih[l])[1]
-            ln = (l + 1) % self.L
-            B.moe_layer_decode(self.store, l, X[l], self.inds[cur, l], self.gates[cur, l], self.W_pre[l],
-                               self.inds[nxt, ln], self.gates[nxt, ln],
-                               None if logits_out is None else logits_out[ln], Y[l], self.ws)
+        self.misses += B.stack_decode_token(self.store, X, self.inds[cur], self.gates[cur], self.W_pre,
+                                            self.inds[nxt], self.gates[nxt], logits_out, self.mirror[cur],
+                                            self.mirror[nxt], Y, self.ws, prefetch=self.prefetch)

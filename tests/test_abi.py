@@ -88,6 +88,28 @@ def test_pack_unpack_identity_and_layout(lib):
         lib.pack_expert(lib.make_desc(synth.CONFIGS["cfg2"]), ex)
 
 
+def test_pack_accepts_exactly_the_zero_points_the_kernels_subtract_without_rounding(lib):
+    """Zero points are fp16 values in [0, 16] that are multiples of 1/128: q - z then fits fp16's 11
+    significant bits, whichever kernel forms it.  Anything else is refused and nothing is written."""
+    cfg = synth.CONFIGS["cfg1"]
+    d = lib.make_desc(cfg)
+    ex = synth.expert_tensors(cfg, 0, 1)
+    def with_zero(v, proj="up"):
+        out = {p: tuple(np.array(a, copy=True) for a in t) for p, t in ex.items()}
+        out[proj][2][3, 2] = np.float16(v)
+        return out
+    for ok in (0.0, 7.5, 3.25, 15.0, 16.0, 1.0 / 128, 9 + 5.0 / 128, 0.0078125 * 3):
+        back = lib.unpack_expert(d, lib.pack_expert(d, with_zero(ok)))
+        assert float(back["up"][2][3, 2]) == float(np.float16(ok))
+    for bad, proj in ((0.1, "gate"), (17.0, "up"), (-1.0, "down"), (1.0 / 256, "up"), (4 + 1.0 / 256, "gate"),
+                      (float("inf"), "down"), (float("nan"), "up")):
+        rec = np.full(cfg.record_bytes, 0xA5, dtype=np.uint8)
+        with pytest.raises(lib.EdgError) as ei:
+            lib.pack_expert(d, with_zero(bad, proj), rec)
+        assert ei.value.code == -4
+        assert (rec == 0xA5).all()
+
+
 def test_host_calls_reject_bad_handles(lib):
     import paper_2609_18063_b200.binding as b
     assert b._lib.edg_store_destroy(None) == -1

@@ -109,6 +109,12 @@ def test_prefill_cfg5_full_size_sampled_tokens():
     hot, cold = int(np.argmax(counts)), int(np.argmin(np.where(counts > 0, counts, 1 << 30)))
     pick = {0, T - 1, int(np.nonzero((inds_h == hot).any(axis=1))[0][-1]), int(np.nonzero((inds_h == cold).any(axis=1))[0][0])}
     pick |= set(rng.choice(T, 12, replace=False).tolist())
+    # an expert of middling popularity that spans a few 128-token tiles: the tokens on both sides of
+    # its first tile boundary, its first and its last token (the ragged tail of its last tile)
+    mid = int(np.argmin(np.where((counts > 256) & (counts < 1024), np.abs(counts - 400), 1 << 30)))
+    assert 256 < counts[mid] < 1024
+    toks = np.nonzero((inds_h == mid).any(axis=1))[0]          # ascending, the order of the expert's token list
+    pick |= {int(toks[0]), int(toks[127]), int(toks[128]), int(toks[255]), int(toks[256]), int(toks[-1])}
     _check_tokens(L, X, inds_h, gates_h, Y, sorted(pick))
     # a second run is bit-identical (fixed reduction order, no atomics on the data path)
     Y2 = _ffn_tokens(L, L.desc, X, inds, gates, T)

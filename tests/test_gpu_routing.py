@@ -80,6 +80,10 @@ def test_sigmoid_group_rejects_shapes_it_cannot_route():
 
 # ------------------------------------------------------------------ the full head (Sec. 3.2 "Head")
 
+# fp32 accumulation of ~3000 fp16 x bf16 products per logit, logits of order 1: the same bar as the
+# linear head's logits (measured errors are printed by the test)
+MLP_LOGIT_TOL = 1e-5
+
 @pytest.mark.parametrize("name,width,n_heads,variant", [("cfg2", 512, 3, "full"), ("cfg1", 64, 2, "full"),
                                                        ("cfg2", 512, 1, "no_residual"), ("cfg1", 64, 1, "no_bias")])
 def test_mlp_head_matches_the_oracle(name, width, n_heads, variant):
@@ -109,7 +113,9 @@ def test_mlp_head_matches_the_oracle(name, width, n_heads, variant):
                                         None if b2 is None else heads[h]["b2"], None if Wr is None else Wres[h],
                                         X[h], cur[h], prev[h])
         got = logits[h].cpu().numpy().astype(np.float64)
-        assert np.abs(got - want).max() <= 2e-4 * max(1.0, np.abs(want).max())
+        err = np.abs(got - want).max()
+        print(f"mlp head {name}/{variant} head {h}: max |logit error| = {err:.3e}, max |logit| = {np.abs(want).max():.3f}")
+        assert err <= MLP_LOGIT_TOL
         # the routing is the exact top-k of the GPU's own logits, and the oracle's wherever its margin allows
         gi, gw = orc.softmax_topk(got, K)
         assert inds[h].cpu().numpy().tolist() == gi.tolist()

@@ -189,6 +189,43 @@ def test_sigmoid_group_hand_example():
     assert np.allclose(w, [2.5 * 0.75 / 1.25, 2.5 * 0.5 / 1.25], rtol=0, atol=1e-12)
 
 
+def _sig_logit(p):
+    return math.log(p / (1.0 - p))
+
+
+def test_sigmoid_group_score_is_the_top2_sum_not_the_max_nor_the_group_sum():
+    # Three groups of three whose sigmoids are chosen so that the three candidate group scores rank
+    # the groups differently (Appendix A: a group is ranked by the sum of its two largest scores):
+    #   group 0: .9  .15 .1    max .9   top-2 sum 1.05  whole sum 1.15
+    #   group 1: .6  .6  .05   max .6   top-2 sum 1.2   whole sum 1.25
+    #   group 2: .5  .5  .45   max .5   top-2 sum 1.0   whole sum 1.45
+    # keep 1 group: top-2 sum -> group 1; the max would keep group 0; the whole sum group 2.
+    sig = [.9, .15, .1, .6, .6, .05, .5, .5, .45]
+    l = np.array([_sig_logit(p) for p in sig])
+    inds, w = orc.sigmoid_group_topk(l, K=2, n_groups=3, keep_groups=1, scale=1.0)
+    assert inds.tolist() == [3, 4]
+    assert np.allclose(w, [0.5, 0.5], rtol=0, atol=1e-12)
+    # keep 2 of 3 groups.  top-2 sums 1.05 / 1.2 / 1.0: groups 1 and 0.  (The max would keep {0, 1} as
+    # well, the whole sum {1, 2}: expert 0 tells them apart.)
+    inds, w = orc.sigmoid_group_topk(l, K=3, n_groups=3, keep_groups=2, scale=2.0)
+    assert inds.tolist() == [0, 3, 4]
+    assert np.allclose(w, [2.0 * .9 / 2.1, 2.0 * .6 / 2.1, 2.0 * .6 / 2.1], rtol=0, atol=1e-12)
+    # keep 2 of 3 where the second survivor differs between top-2 sum and max:
+    #   group 0: .7 .1 .1 (max .7, top-2 .8)   group 1: .6 .6 .1 (max .6, top-2 1.2)   group 2: .5 .45 .1 (max .5, top-2 .95)
+    # top-2 sum keeps {1, 2}; the max would keep {0, 1}.  K = 4 of the six survivors by score.
+    sig = [.7, .1, .1, .6, .6, .1, .5, .45, .1]
+    l = np.array([_sig_logit(p) for p in sig])
+    inds, w = orc.sigmoid_group_topk(l, K=4, n_groups=3, keep_groups=2, scale=2.5)
+    assert inds.tolist() == [3, 4, 6, 7]
+    tot = .6 + .6 + .5 + .45
+    assert np.allclose(w, [2.5 * .6 / tot, 2.5 * .6 / tot, 2.5 * .5 / tot, 2.5 * .45 / tot], rtol=0, atol=1e-12)
+    # an off-by-one in the number of kept groups (1 or 3 instead of 2) changes the answer:
+    assert orc.sigmoid_group_topk(l, K=4, n_groups=3, keep_groups=3, scale=2.5)[0].tolist() == [0, 3, 4, 6]
+    # K as large as the survivors: every expert of the kept groups, none of the dropped group
+    inds, _ = orc.sigmoid_group_topk(l, K=6, n_groups=3, keep_groups=2, scale=2.5)
+    assert inds.tolist() == [3, 4, 5, 6, 7, 8]
+
+
 # ------------------------------------------------------------------ FFN, LoRA, reduce
 
 def _tiny_expert(rng, H, I, g):
@@ -442,3 +479,24 @@ def test_mlp_head_reduces_to_the_linear_head_and_to_a_column_gather():
     # hand example: d = 1, E = 1, D = 1: z = 2*1.5 + 0.25 (cur) + 0.5 (prev) - 0.75 = 3.0, l = 4 * gelu(3) + 1 + 0.5 * 1.5
     one = orc.prerouter_mlp_logits([[2.0, 0.25, 0.5]], [-0.75], [[4.0]], [1.0], [[0.5]], _bf16([1.5]), [0], [0])
     assert abs(one[0] - (4.0 * 3.0 * 0.9986501019683699 + 1.0 + 0.75)) < 1e-12
+
+
+# ------------------------------------------------------------------ the benchmark's chain construct
+
+def test_next_hidden_state_closed_forms():
+    # x + y = (3, 4, 0, 0): mean square 25/4, rms 2.5 -> (1.2, 1.6, 0, 0), rounded to bf16
+    x = _bf16([1.0, 1.0, 0.5, -2.0])
+    y = np.array([2.0, 3.0, -0.5, 2.0])
+    out = orc.next_hidden_state(x, y, eps=0.0)
+    assert out.tolist() == [0x3F9A, 0x3FCD, 0x0000, 0x0000]          # 1.203125, 1.6015625 (nearest bf16 of 1.2, 1.6)
+    # a constant vector normalises to ones whatever its size; the sign survives
+    assert orc.next_hidden_state(_bf16([0.0] * 8), np.full(8, -7.25), eps=0.0).tolist() == [0xBF80] * 8
+    # scale invariance without eps, and eps in the right place: v = (1e-3,)*4, eps = 1e-6 -> 1e-3 / sqrt(2e-6)
+    rng = np.random.default_rng(11)
+    xb, yv = _bf16(rng.standard_normal(64)), rng.standard_normal(64)
+    a = orc.next_hidden_state(xb, yv, eps=0.0)
+    xs = orc.bf16_to_f64(xb) * 4.0
+    b = orc.next_hidden_state(_bf16(xs), yv * 4.0, eps=0.0)
+    assert np.array_equal(a, b)
+    got = orc.bf16_to_f64(orc.next_hidden_state(_bf16([0.0] * 4), np.full(4, 1e-3), eps=1e-6))
+    assert np.allclose(got, 1e-3 / math.sqrt(2e-6), rtol=2.0 ** -8)

@@ -34,6 +34,10 @@ def test_static_scratch_entry_point_matches_the_regular_one_twice():
         assert np.isfinite(a).all()
         assert orc.max_abs(a, b) <= TOL_MAX_ABS and orc.rel_l2(a, b) <= TOL_REL_L2
         assert np.array_equal(a, b)          # same kernel, same arithmetic: in fact bit-identical
+        # ... and against the fp64 oracle, like every other entry point
+        ref = orc.moe_ffn(X[call], inds.cpu().numpy(), gates.cpu().numpy().astype(np.float64), L.expert, L.get_lora,
+                          cfg.lora_scale, cfg.group)
+        assert orc.max_abs(a, ref) <= TOL_MAX_ABS and orc.rel_l2(a, ref) <= TOL_REL_L2
     # a shape whose scratch cannot fit the fixed array, or that the batch-1 kernel does not cover, is rejected
     bad = edg.make_desc(cfg, n_slots=cfg.E, H=4096)
     with pytest.raises(edg.EdgError) as ei:
