@@ -238,6 +238,61 @@ int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers, const voi
                          void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
                          void* copy_stream, edg_store** out);
 int32_t edg_store_destroy(edg_store* store);
+
+/* What the store asks of the machine when it stages: copies, events, stream ordering, a little
+ * pinned memory.  The default engine is the CUDA runtime.  A caller may pass its own -- the
+ * host-side tests do, with an engine that runs on plain host memory, completes operations late and
+ * out of order across streams (honouring only the orderings the store has asked for) and so shows
+ * whether the store asks for every ordering it needs.  All functions return 0 on success; `ctx` is
+ * passed back as given.  With a foreign engine only the host-side calls are usable
+ * (stage_experts_to_slots, edg_store_wait_staged, edg_store_mark_computed, snapshots, stats):
+ * moe_layer_decode and edg_stack_decode_token launch kernels and return EDG_E_INVAL. */
+typedef struct edg_copy_engine {
+    void* ctx;
+    int32_t (*copy_h2d)(void* ctx, void* dst, const void* src, size_t bytes, void* stream);   /* asynchronous on stream */
+    int32_t (*fill)(void* ctx, void* dst, int32_t byte, size_t bytes, void* stream);          /* asynchronous memset    */
+    int32_t (*event_create)(void* ctx, void** event_out);
+    int32_t (*event_destroy)(void* ctx, void* event);
+    int32_t (*event_record)(void* ctx, void* event, void* stream);
+    int32_t (*stream_wait_event)(void* ctx, void* stream, void* event);
+    int32_t (*event_synchronize)(void* ctx, void* event);       /* host waits */
+    int32_t (*stream_synchronize)(void* ctx, void* stream);     /* host waits */
+    int32_t (*host_alloc)(void* ctx, void** ptr_out, size_t bytes);   /* page-locked where that means something */
+    int32_t (*host_free)(void* ctx, void* ptr);
+} edg_copy_engine;
+
+/* edg_store_create with a caller-supplied engine (NULL = the CUDA runtime, i.e. edg_store_create). */
+int32_t edg_store_create_ex(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
+                            void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
+                            void* copy_stream, const edg_copy_engine* engine_opt, edg_store** out);
+
+/* The "hot" executor path (Sec. 3.1: a fixed set of LRU-resident hot experts per layer; hits run
+ * from their slots, misses fall to the on-demand path).  Switch it on before the first staging call.
+ * Each layer's pool of n_slots slots is then split: the first n_slots - K slots hold the hot set,
+ * the last K are transient slots, one per routed expert of the step in flight.
+ *   - stage_experts_to_slots(layer, P) becomes the hot set's bookkeeping for one step: resident
+ *     experts are hits (returned slot >= 0); the others are misses (returned slot -1) that the step
+ *     serves on demand.  A miss whose expert has by now been routed `admit_after` times (1 = plain
+ *     LRU, more = a popularity cache) also enters the hot set for LATER steps, in place of the
+ *     least recently used slot this step neither hits nor has given away; its copy (copy engine,
+ *     side stream) is queued by the layer's next edg_store_mark_computed, i.e. behind this step's
+ *     compute, so the step never waits for it.
+ *   - moe_layer_decode serves the misses itself, on the compute stream: a fetch kernel maps the
+ *     routed experts through the device slot table and, for each one that is not resident, the SMs
+ *     read its record straight from the pinned-host tier (plain 16-byte loads of mapped host
+ *     memory) into a transient slot -- device-initiated, no host round trip, the indices never
+ *     leave the GPU; the layer kernel then runs over hot and transient slots alike.  host_layers
+ *     must be device-accessible (cudaHostAlloc memory is, under unified addressing).
+ * Chaining does not apply to hot-path steps.  n_slots must exceed K; admit_after >= 1. */
+int32_t edg_store_set_hot(edg_store* store, int32_t enable, int32_t admit_after);
+
+typedef struct edg_hot_stats {
+    int64_t hits;         /* routed experts found in the hot set                      */
+    int64_t misses;       /* routed experts served on demand                          */
+    int64_t admitted;     /* misses that entered the hot set for later steps          */
+    int64_t bytes_direct; /* record bytes the SMs fetched from the host tier          */
+} edg_hot_stats;
+int32_t edg_store_get_hot_stats(const edg_store* store, edg_hot_stats* out);
 int32_t edg_store_get_stats(const edg_store* store, edg_store_stats* out);
 
 /* Host side of a3.  `inds_host` holds n distinct experts (n <= n_slots; n = K for one token, up to

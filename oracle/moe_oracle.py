@@ -250,6 +250,67 @@ class SlotAllocator:
         return [self.slot_of_expert[e] for e in P], copies
 
 
+class HotSetAllocator:
+    """The "hot" executor path of one layer (Sec. 3.1): a fixed pool of S_hot slots holds the
+    least-recently-used-resident hot experts; a routed expert that is resident is a hit and is run
+    from its slot; one that is not is a miss and is served on demand for this step (the paper's
+    misses "fall to exact"), without waiting for any staging.
+
+    Readings taken (the paper gives the path one sentence): a miss also enters the hot set for
+    *later* steps once the expert has been routed ``admit_after`` times in total (1 = plain LRU
+    cache; larger values make it a popularity cache), replacing the least recently used slot that
+    this step neither hit nor has already given away; if every slot is spoken for, the miss is only
+    served.  ``step(P)`` takes the routed experts in ascending index and returns
+    (slot per expert, -1 for a miss served on demand; the (expert, slot) admissions that take
+    effect after this step's compute).
+    """
+
+    def __init__(self, E: int, S_hot: int, admit_after: int = 1):
+        self.E, self.S, self.admit_after = E, S_hot, admit_after
+        self.expert_of_slot = [-1] * S_hot
+        self.slot_of_expert = [-1] * E
+        self.last_use = [-1] * S_hot
+        self.uses = [0] * E
+        self.n = 0
+        self.hits = self.misses = self.admitted = 0
+
+    def step(self, P: Sequence[int]) -> Tuple[List[int], List[Tuple[int, int]]]:
+        P = [int(e) for e in P]
+        if len(set(P)) != len(P) or any(e < 0 or e >= self.E for e in P):
+            raise ValueError("bad expert set")
+        for e in P:
+            self.uses[e] += 1
+        spoken = [False] * self.S
+        now = [self.slot_of_expert[e] for e in P]           # what this step's compute sees
+        for s in now:
+            if s >= 0:
+                spoken[s] = True
+                self.last_use[s] = self.n
+        admissions = []
+        for e, s in zip(P, now):
+            if s >= 0:
+                self.hits += 1
+                continue
+            self.misses += 1
+            if self.uses[e] < self.admit_after:
+                continue
+            free = [v for v in range(self.S) if not spoken[v]]
+            if not free:
+                continue
+            victim = min(free, key=lambda v: (self.last_use[v], v))
+            old = self.expert_of_slot[victim]
+            if old >= 0:
+                self.slot_of_expert[old] = -1
+            self.expert_of_slot[victim] = e
+            self.slot_of_expert[e] = victim
+            self.last_use[victim] = self.n
+            spoken[victim] = True
+            admissions.append((e, victim))
+            self.admitted += 1
+        self.n += 1
+        return now, admissions
+
+
 # ------------------------------------------------------------------ expert FFN + LoRA + reduce
 
 def silu(v):

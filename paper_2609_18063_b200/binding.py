@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 import numpy as np
 
 __all__ = [
-    "EdgError", "LayerDesc", "Lora", "StoreStats", "Store", "F32", "F16", "BF16", "LIB_PATH",
+    "EdgError", "LayerDesc", "Lora", "StoreStats", "HotStats", "CopyEngine", "make_copy_engine", "Store", "F32", "F16", "BF16", "LIB_PATH",
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
     "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows", "sigmoid_group_topk_rows", "prerouter_mlp_topk",
     "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots",
@@ -50,6 +50,38 @@ class Lora(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("A_gate", "B_gate", "A_up", "B_up", "A_down", "B_down")]
 
 
+class HotStats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("hits", "misses", "admitted", "bytes_direct")]
+
+
+_ENG_FN = {
+    "copy_h2d": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p),
+    "fill": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_size_t, C.c_void_p),
+    "event_create": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.POINTER(C.c_void_p)),
+    "event_destroy": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p),
+    "event_record": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p),
+    "stream_wait_event": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p),
+    "event_synchronize": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p),
+    "stream_synchronize": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p),
+    "host_alloc": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.POINTER(C.c_void_p), C.c_size_t),
+    "host_free": C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_void_p),
+}
+
+
+class CopyEngine(C.Structure):
+    """edg_copy_engine: ``ctx`` plus ten callbacks, in the header's order."""
+    _fields_ = [("ctx", C.c_void_p)] + [(n, t) for n, t in _ENG_FN.items()]
+
+
+def make_copy_engine(obj) -> CopyEngine:
+    """Wraps an object that has the ten methods of edg_copy_engine (same arguments, ctx first).
+    The returned struct keeps the callbacks alive through its ``_keep`` attribute."""
+    fns = {n: t(getattr(obj, n)) for n, t in _ENG_FN.items()}
+    eng = CopyEngine(None, *[fns[n] for n in _ENG_FN])
+    eng._keep = (obj, fns)
+    return eng
+
+
 class StoreStats(C.Structure):
     _fields_ = [(n, C.c_int64) for n in ("stage_calls", "hits", "misses", "bytes_copied", "table_updates")]
 
@@ -73,7 +105,10 @@ _SIG = {
     "sigmoid_group_topk_rows": ([_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, _P, _P], C.c_int32),
     "prerouter_mlp_topk": ([_D, _P, _P, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
+    "edg_store_create_ex": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(CopyEngine), C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
+    "edg_store_set_hot": ([_P, C.c_int32, C.c_int32], C.c_int32),
+    "edg_store_get_hot_stats": ([_P, C.POINTER(HotStats)], C.c_int32),
     "edg_store_get_stats": ([_P, C.POINTER(StoreStats)], C.c_int32),
     "edg_store_set_chaining": ([_P, C.c_int32], C.c_int32),
     "edg_store_snapshot": ([_P, C.c_int32, _P, _P], C.c_int32),
@@ -276,17 +311,22 @@ class Store:
     """Owner of an ``edg_store`` handle.  Keeps references to the caller's buffers alive."""
 
     def __init__(self, desc: LayerDesc, host_layers: Sequence, dev_slots, dev_tables,
-                 loras: Optional[Sequence[Lora]] = None, copy_stream=None):
+                 loras: Optional[Sequence[Lora]] = None, copy_stream=None, engine: Optional[CopyEngine] = None):
         self.desc = desc
         self.n_layers = len(host_layers)
-        self._keep = (list(host_layers), dev_slots, dev_tables, loras, copy_stream)
+        self._keep = (list(host_layers), dev_slots, dev_tables, loras, copy_stream, engine)
         ptrs = (_P * self.n_layers)(*[_ptr(h) for h in host_layers])
         lor = None
         if loras is not None:
             lor = (Lora * self.n_layers)(*loras)
         h = _P()
-        _check(_lib.edg_store_create(C.byref(desc), self.n_layers, ptrs, _ptr(dev_slots), _ptr(dev_tables),
-                                     lor, _stream(copy_stream), C.byref(h)), "edg_store_create")
+        if engine is None:
+            _check(_lib.edg_store_create(C.byref(desc), self.n_layers, ptrs, _ptr(dev_slots), _ptr(dev_tables),
+                                         lor, _stream(copy_stream), C.byref(h)), "edg_store_create")
+        else:                       # a caller's engine: streams are whatever that engine understands
+            _check(_lib.edg_store_create_ex(C.byref(desc), self.n_layers, ptrs, _ptr(dev_slots), _ptr(dev_tables),
+                                            lor, copy_stream, C.byref(engine), C.byref(h)), "edg_store_create_ex")
+        self._foreign = engine is not None
         self.handle = h
 
     def close(self) -> None:
@@ -316,8 +356,19 @@ class Store:
         _check(_lib.edg_store_snapshot(self.handle, layer, _ptr(eos), _ptr(soe)), "edg_store_snapshot")
         return eos, soe
 
+    def set_hot(self, enable: bool = True, admit_after: int = 1) -> None:
+        _check(_lib.edg_store_set_hot(self.handle, int(bool(enable)), int(admit_after)), "edg_store_set_hot")
+
+    def hot_stats(self) -> dict:
+        s = HotStats()
+        _check(_lib.edg_store_get_hot_stats(self.handle, C.byref(s)), "edg_store_get_hot_stats")
+        return {n: getattr(s, n) for n, _ in HotStats._fields_}
+
+    def _st(self, stream):
+        return stream if self._foreign else _stream(stream)
+
     def wait_staged(self, layer: int, stream=None) -> None:
-        _check(_lib.edg_store_wait_staged(self.handle, layer, _stream(stream)), "edg_store_wait_staged")
+        _check(_lib.edg_store_wait_staged(self.handle, layer, self._st(stream)), "edg_store_wait_staged")
 
     def time_waits(self, enable: bool) -> None:
         _check(_lib.edg_store_time_waits(self.handle, int(bool(enable))), "edg_store_time_waits")
@@ -329,7 +380,7 @@ class Store:
         return ms.value, n.value
 
     def mark_computed(self, layer: int, stream=None) -> None:
-        _check(_lib.edg_store_mark_computed(self.handle, layer, _stream(stream)), "edg_store_mark_computed")
+        _check(_lib.edg_store_mark_computed(self.handle, layer, self._st(stream)), "edg_store_mark_computed")
 
 
 def stage_experts_to_slots(store: Store, layer: int, inds_host, n: Optional[int] = None):

@@ -14,7 +14,82 @@
 
 #include "edg_common.cuh"
 
+namespace edg {
+
+// The hot path's on-demand fetch, initiated by the device: block row k looks routed expert k up in the
+// layer's slot table; a resident expert only has its slot noted; for one that is not, the SMs copy
+// its record from the pinned-host tier (mapped host memory, plain 16-byte loads, four in flight per
+// thread) into transient slot S_hot + k.  slots_eff[k] is what the layer kernel then runs over.
+constexpr int kFetchBlocks = 32, kFetchThreads = 256;
+
+__device__ __forceinline__ uint4 ld_host16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__global__ void __launch_bounds__(kFetchThreads) hot_fetch_kernel(const int32_t* inds, const int32_t* table,
+                                                                  const uint8_t* host_layer, uint8_t* pool,
+                                                                  int32_t* slots_eff, int E, int S_hot, int n_slots,
+                                                                  size_t R) {
+    const int k = blockIdx.y;
+    const int e = inds[k];
+    const bool first = blockIdx.x == 0 && threadIdx.x == 0;
+    if (e < 0 || e >= E) {                       // the layer kernel skips and flags it
+        if (first) slots_eff[k] = -1;
+        return;
+    }
+    const int s = table[e];
+    if (s >= 0 && s < n_slots) {                 // a hit: run from the hot set
+        if (first) slots_eff[k] = s;
+        return;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(host_layer + (size_t)e * R);
+    uint4* dst = reinterpret_cast<uint4*>(pool + (size_t)(S_hot + k) * R);
+    const size_t n16 = R / 16, stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += 4 * stride) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i + u * stride < n16) v[u] = ld_host16(src + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (i + u * stride < n16) dst[i + u * stride] = v[u];
+    }
+    if (first) slots_eff[k] = S_hot + k;
+}
+
+}  // namespace edg
+
 namespace {
+
+// ---- the default copy engine: the CUDA runtime
+int32_t cu_rc(cudaError_t e) { if (e != cudaSuccess) { edg::set_cuda_error(e); return EDG_E_CUDA; } return EDG_OK; }
+int32_t cu_copy(void*, void* dst, const void* src, size_t n, void* st) {
+    return cu_rc(cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, static_cast<cudaStream_t>(st)));
+}
+int32_t cu_fill(void*, void* dst, int32_t b, size_t n, void* st) { return cu_rc(cudaMemsetAsync(dst, b, n, static_cast<cudaStream_t>(st))); }
+int32_t cu_ev_create(void*, void** ev) {
+    cudaEvent_t e = nullptr;
+    const int32_t rc = cu_rc(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    *ev = e;
+    return rc;
+}
+int32_t cu_ev_destroy(void*, void* ev) { return cu_rc(cudaEventDestroy(static_cast<cudaEvent_t>(ev))); }
+int32_t cu_ev_record(void*, void* ev, void* st) { return cu_rc(cudaEventRecord(static_cast<cudaEvent_t>(ev), static_cast<cudaStream_t>(st))); }
+int32_t cu_wait(void*, void* st, void* ev) { return cu_rc(cudaStreamWaitEvent(static_cast<cudaStream_t>(st), static_cast<cudaEvent_t>(ev), 0)); }
+int32_t cu_ev_sync(void*, void* ev) { return cu_rc(cudaEventSynchronize(static_cast<cudaEvent_t>(ev))); }
+int32_t cu_st_sync(void*, void* st) { return cu_rc(cudaStreamSynchronize(static_cast<cudaStream_t>(st))); }
+int32_t cu_halloc(void*, void** p, size_t n) { return cu_rc(cudaHostAlloc(p, n, cudaHostAllocDefault)); }
+int32_t cu_hfree(void*, void* p) { return cu_rc(cudaFreeHost(p)); }
+const edg_copy_engine kCudaEngine = {nullptr, cu_copy, cu_fill, cu_ev_create, cu_ev_destroy, cu_ev_record, cu_wait,
+                                     cu_ev_sync, cu_st_sync, cu_halloc, cu_hfree};
+
+#define EDG_ENG_TRY(expr)                          \
+    do {                                           \
+        const int32_t _rc = (expr);                \
+        if (_rc != EDG_OK) return _rc;             \
+    } while (0)
 
 constexpr uint32_t kMagic = 0x45444731u;   // "EDG1"
 constexpr int kRing = 64;                  // pinned staging rows for slot-table updates
@@ -24,7 +99,10 @@ struct LayerState {
     std::vector<int64_t> last_use;
     std::vector<uint8_t> taken;
     int64_t n = 0;                         // stage calls so far (the LRU clock)
-    cudaEvent_t copy_done = nullptr, compute_done = nullptr;
+    std::vector<int64_t> uses;             // hot path: times each expert has been routed
+    std::vector<std::pair<int32_t, int32_t>> pending;   // hot path: (expert, slot) admissions waiting for this step's compute
+    void* copy_done = nullptr;             // engine events
+    void* compute_done = nullptr;
     bool copy_pending = false;             // copy_done recorded and not yet waited on by compute
     bool compute_recorded = false;
 };
@@ -40,10 +118,16 @@ struct edg_store {
     uint8_t* dev_slots = nullptr;
     int32_t* dev_tables = nullptr;
     std::vector<edg_lora> loras;
-    cudaStream_t copy_stream = nullptr;
+    void* copy_stream = nullptr;
+    edg_copy_engine eng{};                 // what staging runs on: the CUDA runtime, or a caller's engine
+    bool cuda_engine = true;
+    bool hot = false;                      // the hot executor path (edg_store_set_hot)
+    int admit_after = 1;
+    edg_hot_stats hot_stats{};
+    int32_t* slots_eff = nullptr;          // dev [n_layers][K]: slots of a hot-path step after the fetch kernel
     std::vector<LayerState> layers;
     int32_t* ring = nullptr;               // pinned [kRing][E]
-    cudaEvent_t ring_ev[kRing] = {};
+    void* ring_ev[kRing] = {};
     bool ring_used[kRing] = {};
     int ring_pos = 0;
     edg_store_stats stats{};
@@ -86,15 +170,20 @@ static int32_t drain_waits(edg_store* s) {
 
 static bool store_ok(const edg_store* s) { return s != nullptr && s->magic == kMagic; }
 
-extern "C" int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
-                                    void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
-                                    void* copy_stream, edg_store** out) {
+extern "C" int32_t edg_store_create_ex(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
+                                       void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
+                                       void* copy_stream, const edg_copy_engine* engine_opt, edg_store** out) {
     int32_t rc = edg::check_desc(desc);
     if (rc != EDG_OK) return rc;
     if (!host_layers || !dev_slots || !dev_tables || !out || n_layers < 1) return EDG_E_INVAL;
     if (!edg::aligned(dev_slots, 256) || !edg::aligned(dev_tables, 16)) return EDG_E_INVAL;
     for (int l = 0; l < n_layers; ++l)
         if (!host_layers[l] || !edg::aligned(host_layers[l], 16)) return EDG_E_INVAL;
+    if (engine_opt != nullptr &&
+        (!engine_opt->copy_h2d || !engine_opt->fill || !engine_opt->event_create || !engine_opt->event_destroy ||
+         !engine_opt->event_record || !engine_opt->stream_wait_event || !engine_opt->event_synchronize ||
+         !engine_opt->stream_synchronize || !engine_opt->host_alloc || !engine_opt->host_free))
+        return EDG_E_INVAL;
     edg_store* s = new (std::nothrow) edg_store();
     if (!s) return EDG_E_INVAL;
     s->d = *desc;
@@ -105,45 +194,52 @@ extern "C" int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers
     s->dev_slots = static_cast<uint8_t*>(dev_slots);
     s->dev_tables = dev_tables;
     if (loras) s->loras.assign(loras, loras + n_layers);
-    s->copy_stream = static_cast<cudaStream_t>(copy_stream);
+    s->copy_stream = copy_stream;
+    s->eng = engine_opt ? *engine_opt : kCudaEngine;
+    s->cuda_engine = engine_opt == nullptr;
     s->layers.resize(n_layers);
-    auto fail = [&](cudaError_t e) { edg::set_cuda_error(e); edg_store_destroy(s); return EDG_E_CUDA; };
+    const edg_copy_engine& g = s->eng;
+    auto fail = [&](int32_t code) { edg_store_destroy(s); return code; };
     for (auto& L : s->layers) {
         L.expert_of_slot.assign(desc->n_slots, -1);
         L.slot_of_expert.assign(desc->E, -1);
         L.last_use.assign(desc->n_slots, -1);
         L.taken.assign(desc->n_slots, 0);
-        cudaError_t e = cudaEventCreateWithFlags(&L.copy_done, cudaEventDisableTiming);
-        if (e != cudaSuccess) return fail(e);
-        e = cudaEventCreateWithFlags(&L.compute_done, cudaEventDisableTiming);
-        if (e != cudaSuccess) return fail(e);
+        L.uses.assign(desc->E, 0);
+        if ((rc = g.event_create(g.ctx, &L.copy_done)) != EDG_OK) return fail(rc);
+        if ((rc = g.event_create(g.ctx, &L.compute_done)) != EDG_OK) return fail(rc);
     }
-    cudaError_t e = cudaHostAlloc(reinterpret_cast<void**>(&s->ring), (size_t)kRing * desc->E * sizeof(int32_t), cudaHostAllocDefault);
-    if (e != cudaSuccess) return fail(e);
-    for (int i = 0; i < kRing; ++i) {
-        e = cudaEventCreateWithFlags(&s->ring_ev[i], cudaEventDisableTiming);
-        if (e != cudaSuccess) return fail(e);
-    }
+    void* ring = nullptr;
+    if ((rc = g.host_alloc(g.ctx, &ring, (size_t)kRing * desc->E * sizeof(int32_t))) != EDG_OK) return fail(rc);
+    s->ring = static_cast<int32_t*>(ring);
+    for (int i = 0; i < kRing; ++i)
+        if ((rc = g.event_create(g.ctx, &s->ring_ev[i])) != EDG_OK) return fail(rc);
     // every expert starts non-resident
-    e = cudaMemsetAsync(dev_tables, 0xFF, (size_t)n_layers * desc->E * sizeof(int32_t), s->copy_stream);
-    if (e != cudaSuccess) return fail(e);
-    e = cudaStreamSynchronize(s->copy_stream);
-    if (e != cudaSuccess) return fail(e);
+    if ((rc = g.fill(g.ctx, dev_tables, 0xFF, (size_t)n_layers * desc->E * sizeof(int32_t), s->copy_stream)) != EDG_OK) return fail(rc);
+    if ((rc = g.stream_synchronize(g.ctx, s->copy_stream)) != EDG_OK) return fail(rc);
     *out = s;
     return EDG_OK;
 }
 
+extern "C" int32_t edg_store_create(const edg_layer_desc* desc, int32_t n_layers, const void* const* host_layers,
+                                    void* dev_slots, int32_t* dev_tables, const edg_lora* loras,
+                                    void* copy_stream, edg_store** out) {
+    return edg_store_create_ex(desc, n_layers, host_layers, dev_slots, dev_tables, loras, copy_stream, nullptr, out);
+}
+
 extern "C" int32_t edg_store_destroy(edg_store* s) {
     if (!store_ok(s)) return EDG_E_INVAL;
-    cudaStreamSynchronize(s->copy_stream);
+    const edg_copy_engine& g = s->eng;
+    g.stream_synchronize(g.ctx, s->copy_stream);
     for (auto& L : s->layers) {
-        if (L.copy_done) cudaEventDestroy(L.copy_done);
-        if (L.compute_done) cudaEventDestroy(L.compute_done);
+        if (L.copy_done) g.event_destroy(g.ctx, L.copy_done);
+        if (L.compute_done) g.event_destroy(g.ctx, L.compute_done);
     }
     for (int i = 0; i < kRing; ++i)
-        if (s->ring_ev[i]) cudaEventDestroy(s->ring_ev[i]);
-    if (s->ring) cudaFreeHost(s->ring);
+        if (s->ring_ev[i]) g.event_destroy(g.ctx, s->ring_ev[i]);
+    if (s->ring) g.host_free(g.ctx, s->ring);
     if (s->step_done) cudaEventDestroy(s->step_done);
+    if (s->slots_eff) cudaFree(s->slots_eff);
     for (auto& pr : s->wait_events) {
         if (pr.first) cudaEventDestroy(pr.first);
         if (pr.second) cudaEventDestroy(pr.second);
@@ -168,19 +264,94 @@ extern "C" int32_t edg_store_snapshot(const edg_store* s, int32_t layer, int32_t
     return EDG_OK;
 }
 
+// Queues, on the copy stream, the copies of the given (expert, slot) pairs of a layer -- behind the
+// layer's last recorded compute, which may still be reading the slots -- then the layer's new
+// expert -> slot row for the device table, then the layer's copy-done event.
+static int32_t queue_copies(edg_store* s, int layer, const std::pair<int32_t, int32_t>* pairs, int n_pairs) {
+    if (n_pairs <= 0) return EDG_OK;
+    const edg_copy_engine& g = s->eng;
+    const int S = s->d.n_slots, E = s->d.E;
+    LayerState& L = s->layers[layer];
+    if (L.compute_recorded) EDG_ENG_TRY(g.stream_wait_event(g.ctx, s->copy_stream, L.compute_done));
+    for (int i = 0; i < n_pairs; ++i)
+        EDG_ENG_TRY(g.copy_h2d(g.ctx, s->dev_slots + ((size_t)layer * S + pairs[i].second) * s->R,
+                               s->host_layers[layer] + (size_t)pairs[i].first * s->R, s->R, s->copy_stream));
+    // publish the new expert -> slot row to the device table, after the record copies
+    const int r = s->ring_pos;
+    s->ring_pos = (r + 1) % kRing;
+    if (s->ring_used[r]) EDG_ENG_TRY(g.event_synchronize(g.ctx, s->ring_ev[r]));
+    int32_t* row = s->ring + (size_t)r * E;
+    for (int e = 0; e < E; ++e) row[e] = L.slot_of_expert[e];
+    EDG_ENG_TRY(g.copy_h2d(g.ctx, s->dev_tables + (size_t)layer * E, row, (size_t)E * sizeof(int32_t), s->copy_stream));
+    EDG_ENG_TRY(g.event_record(g.ctx, s->ring_ev[r], s->copy_stream));
+    s->ring_used[r] = true;
+    EDG_ENG_TRY(g.event_record(g.ctx, L.copy_done, s->copy_stream));
+    L.copy_pending = true;
+    s->stats.table_updates += 1;
+    s->stats.bytes_copied += (int64_t)n_pairs * (int64_t)s->R;
+    return EDG_OK;
+}
+
+// least recently used slot among the first `n_pool` that this call has not spoken for, or -1
+static int lru_victim(const LayerState& L, int n_pool) {
+    int victim = -1;
+    for (int sl = 0; sl < n_pool; ++sl)
+        if (!L.taken[sl] && (victim < 0 || L.last_use[sl] < L.last_use[victim])) victim = sl;
+    return victim;
+}
+
 extern "C" int32_t stage_experts_to_slots(edg_store* s, int32_t layer, const int32_t* inds, int32_t n,
                                           int32_t* slots_out, int32_t* n_miss_out) {
     if (!store_ok(s) || !inds || !slots_out) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     const int S = s->d.n_slots, E = s->d.E;
     if (n < 0) return EDG_E_INVAL;
-    if (n > S) return EDG_E_SLOTS;
+    if (n > (s->hot ? s->d.K : S)) return EDG_E_SLOTS;
     LayerState& L = s->layers[layer];
 
     // validate before touching any state: in range and distinct
     for (int i = 0; i < n; ++i) {
         if (inds[i] < 0 || inds[i] >= E) return EDG_E_RANGE;
         for (int j = 0; j < i; ++j) if (inds[j] == inds[i]) return EDG_E_RANGE;
+    }
+    s->stats.stage_calls += 1;
+
+    if (s->hot) {
+        // The hot path: this step runs its hits from the hot set as it stands and serves its misses
+        // on demand; what a miss changes in the hot set takes effect after this step's compute.
+        const int S_hot = S - s->d.K;
+        for (int i = 0; i < n; ++i) L.uses[inds[i]] += 1;
+        for (int i = 0; i < S_hot; ++i) L.taken[i] = 0;
+        for (int i = 0; i < n; ++i) {
+            const int sl = L.slot_of_expert[inds[i]];
+            slots_out[i] = sl;
+            if (sl >= 0) { L.taken[sl] = 1; L.last_use[sl] = L.n; }
+        }
+        int n_miss = 0;
+        for (int i = 0; i < n; ++i) {
+            if (slots_out[i] >= 0) continue;
+            ++n_miss;
+            const int e = inds[i];
+            if (L.uses[e] < s->admit_after) continue;
+            const int victim = lru_victim(L, S_hot);
+            if (victim < 0) continue;                      // every slot is spoken for: served only
+            const int old = L.expert_of_slot[victim];
+            if (old >= 0) L.slot_of_expert[old] = -1;
+            L.expert_of_slot[victim] = e;
+            L.slot_of_expert[e] = victim;
+            L.last_use[victim] = L.n;
+            L.taken[victim] = 1;
+            L.pending.emplace_back(e, victim);
+            s->hot_stats.admitted += 1;
+        }
+        L.n += 1;
+        s->hot_stats.hits += n - n_miss;
+        s->hot_stats.misses += n_miss;
+        s->hot_stats.bytes_direct += (int64_t)n_miss * (int64_t)s->R;
+        s->stats.hits += n - n_miss;
+        s->stats.misses += n_miss;
+        if (n_miss_out) *n_miss_out = n_miss;
+        return EDG_OK;
     }
 
     // (i) residents keep their slot and are touched
@@ -190,55 +361,26 @@ extern "C" int32_t stage_experts_to_slots(edg_store* s, int32_t layer, const int
         if (sl >= 0) { L.taken[sl] = 1; L.last_use[sl] = L.n; }
     }
     // (ii) each missing expert takes the least recently used slot this call does not need
+    std::pair<int32_t, int32_t> copies[1024];
     int n_miss = 0;
-    bool waited = false;
     for (int i = 0; i < n; ++i) {
         const int e = inds[i];
         if (L.slot_of_expert[e] >= 0) continue;
-        int victim = -1;
-        for (int sl = 0; sl < S; ++sl)
-            if (!L.taken[sl] && (victim < 0 || L.last_use[sl] < L.last_use[victim])) victim = sl;
-        // n <= S guarantees a free slot
+        const int victim = lru_victim(L, S);               // n <= S guarantees a free slot
         const int old = L.expert_of_slot[victim];
         if (old >= 0) L.slot_of_expert[old] = -1;
         L.expert_of_slot[victim] = e;
         L.slot_of_expert[e] = victim;
         L.last_use[victim] = L.n;
         L.taken[victim] = 1;
-        if (!waited && L.compute_recorded) {
-            // do not overwrite a slot the layer's last compute may still be reading
-            EDG_CUDA_TRY(cudaStreamWaitEvent(s->copy_stream, L.compute_done, 0));
-            waited = true;
-        }
-        EDG_CUDA_TRY(cudaMemcpyAsync(s->dev_slots + ((size_t)layer * S + victim) * s->R,
-                                     s->host_layers[layer] + (size_t)e * s->R, s->R,
-                                     cudaMemcpyHostToDevice, s->copy_stream));
-        ++n_miss;
+        copies[n_miss++] = std::make_pair(e, victim);
     }
     L.n += 1;
     for (int i = 0; i < n; ++i) slots_out[i] = L.slot_of_expert[inds[i]];
     if (n_miss_out) *n_miss_out = n_miss;
-    s->stats.stage_calls += 1;
     s->stats.hits += n - n_miss;
     s->stats.misses += n_miss;
-    s->stats.bytes_copied += (int64_t)n_miss * (int64_t)s->R;
-
-    if (n_miss > 0) {
-        // publish the new expert -> slot row to the device table, after the record copies
-        const int r = s->ring_pos;
-        s->ring_pos = (r + 1) % kRing;
-        if (s->ring_used[r]) EDG_CUDA_TRY(cudaEventSynchronize(s->ring_ev[r]));
-        int32_t* row = s->ring + (size_t)r * E;
-        for (int e = 0; e < E; ++e) row[e] = L.slot_of_expert[e];
-        EDG_CUDA_TRY(cudaMemcpyAsync(s->dev_tables + (size_t)layer * E, row, (size_t)E * sizeof(int32_t),
-                                     cudaMemcpyHostToDevice, s->copy_stream));
-        EDG_CUDA_TRY(cudaEventRecord(s->ring_ev[r], s->copy_stream));
-        s->ring_used[r] = true;
-        EDG_CUDA_TRY(cudaEventRecord(L.copy_done, s->copy_stream));
-        L.copy_pending = true;
-        s->stats.table_updates += 1;
-    }
-    return EDG_OK;
+    return queue_copies(s, layer, copies, n_miss);
 }
 
 extern "C" int32_t edg_store_wait_staged(edg_store* s, int32_t layer, void* stream) {
@@ -246,18 +388,21 @@ extern "C" int32_t edg_store_wait_staged(edg_store* s, int32_t layer, void* stre
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     LayerState& L = s->layers[layer];
     if (L.copy_pending) {
-        cudaStream_t st = static_cast<cudaStream_t>(stream);
-        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
-        if (s->time_waits) EDG_CUDA_TRY(cudaStreamIsCapturing(st, &capturing));
-        const bool timed = s->time_waits && capturing == cudaStreamCaptureStatusNone;
+        const edg_copy_engine& g = s->eng;
+        bool timed = false;
+        if (s->time_waits && s->cuda_engine) {
+            cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+            EDG_CUDA_TRY(cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &capturing));
+            timed = capturing == cudaStreamCaptureStatusNone;
+        }
         if (timed && s->wait_used == s->wait_events.size()) {
             int32_t rc = drain_waits(s);
             if (rc != EDG_OK) return rc;
         }
-        if (timed) EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].first, st));
-        EDG_CUDA_TRY(cudaStreamWaitEvent(st, L.copy_done, 0));
+        if (timed) EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].first, static_cast<cudaStream_t>(stream)));
+        EDG_ENG_TRY(g.stream_wait_event(g.ctx, stream, L.copy_done));
         if (timed) {
-            EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].second, st));
+            EDG_CUDA_TRY(cudaEventRecord(s->wait_events[s->wait_used].second, static_cast<cudaStream_t>(stream)));
             s->wait_used += 1;
         }
         L.copy_pending = false;
@@ -293,11 +438,38 @@ extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* st
     if (!store_ok(s)) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     // Only a pool that can evict needs the ordering: with n_slots == E nothing is ever overwritten.
-    if (s->d.n_slots < s->d.E) {
-        LayerState& L = s->layers[layer];
-        EDG_CUDA_TRY(cudaEventRecord(L.compute_done, static_cast<cudaStream_t>(stream)));
+    LayerState& L = s->layers[layer];
+    if (s->d.n_slots < s->d.E || s->hot) {
+        const edg_copy_engine& g = s->eng;
+        EDG_ENG_TRY(g.event_record(g.ctx, L.compute_done, stream));
         L.compute_recorded = true;
     }
+    // hot path: the admissions decided while this step was staged go out now, behind its compute
+    if (!L.pending.empty()) {
+        const int32_t rc = queue_copies(s, layer, L.pending.data(), (int)L.pending.size());
+        L.pending.clear();
+        if (rc != EDG_OK) return rc;
+    }
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_set_hot(edg_store* s, int32_t enable, int32_t admit_after) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (!enable) { s->hot = false; return EDG_OK; }
+    if (admit_after < 1) return EDG_E_INVAL;
+    if (s->d.n_slots <= s->d.K) return EDG_E_SLOTS;
+    for (const auto& L : s->layers)
+        if (L.n != 0) return EDG_E_INVAL;                  // before the first staging call
+    if (s->cuda_engine && s->slots_eff == nullptr)
+        EDG_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s->slots_eff), (size_t)s->n_layers * s->d.K * sizeof(int32_t)));
+    s->hot = true;
+    s->admit_after = admit_after;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_get_hot_stats(const edg_store* s, edg_hot_stats* out) {
+    if (!store_ok(s) || !out) return EDG_E_INVAL;
+    *out = s->hot_stats;
     return EDG_OK;
 }
 
@@ -308,6 +480,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
                                     void* workspace, size_t workspace_bytes, void* stream) {
     if (!store_ok(s) || !x || !inds_cur || !gates_cur || !y) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    if (!s->cuda_engine) return EDG_E_INVAL;               // kernels need the real machine
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int32_t rc = edg_store_wait_staged(s, layer, stream);
     if (rc != EDG_OK) return rc;
@@ -315,6 +488,19 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
     if (W_pre_next != nullptr && (!inds_next || !gates_next)) return EDG_E_INVAL;
     const void* pool = s->dev_slots + (size_t)layer * s->d.n_slots * s->R;
     const int32_t* table = s->dev_tables + (size_t)layer * s->d.E;
+    const int32_t* slot_arg = inds_cur;                    // expert ids, mapped through the table by the kernels
+    const int32_t* expert_arg = nullptr;
+    if (s->hot) {
+        // hits from the hot set, misses fetched by the SMs from the host tier into transient slots
+        int32_t* eff = s->slots_eff + (size_t)layer * s->d.K;
+        edg::hot_fetch_kernel<<<dim3(edg::kFetchBlocks, s->d.K), edg::kFetchThreads, 0, st>>>(
+            inds_cur, table, s->host_layers[layer], s->dev_slots + (size_t)layer * s->d.n_slots * s->R, eff,
+            s->d.E, s->d.n_slots - s->d.K, s->d.n_slots, s->R);
+        EDG_CUDA_TRY(cudaGetLastError());
+        slot_arg = eff;
+        expert_arg = inds_cur;
+        table = nullptr;
+    }
     if (edg::fused_supported(s->d)) {
         // one launch: prerouter for the next step, take, FFN and reduce for this one
         rc = edg::check_desc(&s->d);
@@ -322,8 +508,8 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         if (!workspace || !edg::aligned(workspace, 256) || workspace_bytes < edg::workspace_layout(s->d, 1).bytes)
             return EDG_E_WORKSPACE;
         if (!edg::aligned(x, 16) || !edg::aligned(y, 16) || (W_pre_next && !edg::aligned(W_pre_next, 16))) return EDG_E_INVAL;
-        bool chained = s->chaining && s->chain_inds != nullptr && s->chain_inds == inds_cur && s->chain_ws == workspace &&
-                       s->chain_stream == stream;
+        bool chained = s->chaining && !s->hot && s->chain_inds != nullptr && s->chain_inds == inds_cur &&
+                       s->chain_ws == workspace && s->chain_stream == stream;
         // Chaining pays when steps queue up on the device: a chained step runs as a few long-lived
         // CTAs that share the GPU with dozens of other steps.  A step that finds the GPU idle -- the
         // step before it has already finished -- is launched on its own, across all SMs, which
@@ -357,7 +543,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         s->ring_next = (ring + 1) % edg::kHandoffRing;
         edg::FusedExtras extras;
         extras.inds_mirror = W_pre_next != nullptr ? inds_next_host_mirror_opt : nullptr;
-        rc = edg::run_fused_layer(&s->d, pool, inds_cur, table, nullptr, gates_cur, x,
+        rc = edg::run_fused_layer(&s->d, pool, slot_arg, table, expert_arg, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
                                   logits_next_opt, workspace, flag_in, flag_out, ring, stale, st, &extras);
         if (W_pre_next != nullptr) s->pub_slot = flag_out;
@@ -373,7 +559,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         s->chain_stream = stream;
         s->chain_flag = flag_out;
     } else {
-        rc = edg::run_ffn(&s->d, pool, 1, inds_cur, table, nullptr, gates_cur, x, lora, y, workspace, workspace_bytes, st);
+        rc = edg::run_ffn(&s->d, pool, 1, slot_arg, table, expert_arg, gates_cur, x, lora, y, workspace, workspace_bytes, st);
         if (rc != EDG_OK) return rc;
         if (W_pre_next != nullptr) {
             rc = edg::run_prerouter(&s->d, W_pre_next, x, 1, inds_next, gates_next, logits_next_opt, st, 0,

@@ -500,3 +500,46 @@ def test_next_hidden_state_closed_forms():
     assert np.array_equal(a, b)
     got = orc.bf16_to_f64(orc.next_hidden_state(_bf16([0.0] * 4), np.full(4, 1e-3), eps=1e-6))
     assert np.allclose(got, 1e-3 / math.sqrt(2e-6), rtol=2.0 ** -8)
+
+
+# ------------------------------------------------------------------ the hot executor path
+
+def test_hot_set_hand_worked_sequence():
+    # 3 hot slots, plain LRU admission.  Step by step, by hand:
+    a = orc.HotSetAllocator(E=8, S_hot=3)
+    assert a.step([1, 2]) == ([-1, -1], [(1, 0), (2, 1)])          # cold start: both served on demand, both admitted
+    assert a.step([1, 5]) == ([0, -1], [(5, 2)])                   # 1 hits slot 0; 5 takes the last empty slot
+    assert a.step([2, 5]) == ([1, 2], [])                          # two hits, nothing moves
+    # 6 and 7 miss; slot 0 (expert 1, last used at step 1) is the LRU, then slot 1 (expert 2, used at step 2)
+    # -- but slots used by THIS step are never given away: here none is, so 6 -> slot 0, 7 -> slot 1
+    assert a.step([6, 7]) == ([-1, -1], [(6, 0), (7, 1)])
+    assert a.expert_of_slot == [6, 7, 5] and a.slot_of_expert[1] == -1 and a.slot_of_expert[2] == -1
+    # a step that hits two slots and misses two more: only one slot is free to give away
+    assert a.step([0, 3, 5, 6]) == ([-1, -1, 2, 0], [(0, 1)])      # 0 takes slot 1 (expert 7); 3 is only served
+    assert a.expert_of_slot == [6, 0, 5]
+    assert (a.hits, a.misses, a.admitted) == (5, 7, 6)
+
+
+def test_hot_set_popularity_admission_and_invariants():
+    # admit_after = 3: an expert enters the hot set only on its third routing
+    a = orc.HotSetAllocator(E=6, S_hot=2, admit_after=3)
+    assert a.step([4]) == ([-1], [])
+    assert a.step([4]) == ([-1], [])
+    assert a.step([4]) == ([-1], [(4, 0)])
+    assert a.step([4]) == ([0], [])
+    rng = np.random.default_rng(12)
+    b = orc.HotSetAllocator(E=32, S_hot=6, admit_after=2)
+    for _ in range(300):
+        P = sorted(rng.choice(32, 4, replace=False).tolist())
+        before = list(b.slot_of_expert)
+        now, adm = b.step(P)
+        assert now == [before[e] for e in P]                         # this step sees the table as it was
+        for e, v in adm:
+            assert before[e] < 0 and v not in [s for s in now if s >= 0]    # a slot hit by this step is never given away
+        res = [e for e in b.expert_of_slot if e >= 0]
+        assert len(res) == len(set(res))
+        for v, e in enumerate(b.expert_of_slot):
+            if e >= 0:
+                assert b.slot_of_expert[e] == v
+        assert sum(1 for s in b.slot_of_expert if s >= 0) == len(res)
+    assert b.hits + b.misses == 1200 and b.admitted <= b.misses
