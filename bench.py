@@ -733,15 +733,21 @@ def run_cfg3(args):
     arms = {}
     order = [("iid", "resident_S256", E, True), ("iid", "prefetch_S8", 8, True), ("iid", "on_demand_S8", 8, False),
              ("iid", "prefetch_S32", 32, True), ("ar1", "prefetch_S8", 8, True), ("ar1", "on_demand_S8", 8, False),
-             ("ar1", "prefetch_S32", 32, True), ("ar1", "lru_S256", E, True)]
+             ("ar1", "prefetch_S32", 32, True), ("ar1", "lru_S256", E, True),
+             # the hot executor path (LRU-resident hot set, misses fetched by the SMs inside the step)
+             ("ar1", "hot_S64", 64 + K, True), ("iid", "hot_S64", 64 + K, True), ("ar1", "hot_S64_k4", 64 + 4, True)]
     for routing, name, S, prefetch in order:
         Xn = X_iid if routing == "iid" else X_ar1
         X = layer_io.bits_to_device(Xn, torch.bfloat16)                     # [L][n_x][H]
         Xt = [X[:, t].contiguous() for t in range(n_x)]
-        d = edg.make_desc(cfg, n_slots=S, out_dtype="f32")
+        hot = name.startswith("hot")
+        Kd = 4 if name.endswith("k4") else K                                # K = 4: the 35B tier's shipped profile
+        d = edg.make_desc(cfg, n_slots=S, out_dtype="f32", K=Kd)
         slots = torch.empty((L, S, R), dtype=torch.uint8, device="cuda")
         tables = torch.empty((L, E), dtype=torch.int32, device="cuda")
         store = edg.Store(d, hosts, slots, tables, loras, torch.cuda.Stream())
+        if hot:
+            store.set_hot(True, 1)
         if name == "resident_S256":
             for l in range(L):
                 for e0 in range(0, E, 64):
@@ -774,7 +780,11 @@ def run_cfg3(args):
             "copies_per_token": round((st["misses"] - base["misses"]) / tokens, 2),
             "hit_rate": round((st["hits"] - base["hits"]) / max(1, staged), 4),
             "MiB_copied_per_token": round((st["bytes_copied"] - base["bytes_copied"]) / tokens / 2 ** 20, 1),
-            "hbm_GBps_on_expert_bytes": round(L * K * R / (ms * 1e-3) / 1e9, 1)}
+            "hbm_GBps_on_expert_bytes": round(L * Kd * R / (ms * 1e-3) / 1e9, 1)}
+        if hot:
+            hs = store.hot_stats()
+            arms[f"{routing}/{name}"].update({"K": Kd, "hot_slots": S - Kd, "admitted_per_token": round(hs["admitted"] / (tokens + warm), 2),
+                                              "MiB_fetched_by_SMs_per_token": round(hs["bytes_direct"] / (tokens + warm) / 2 ** 20, 1)})
         assert edg.workspace_status(dec.ws) == 0 and bool(torch.isfinite(Y).all())
         store.close()
         del slots, tables, dec, X, Xt
