@@ -286,6 +286,21 @@ int32_t edg_store_create_ex(const edg_layer_desc* desc, int32_t n_layers, const 
  * Chaining does not apply to hot-path steps.  n_slots must exceed K; admit_after >= 1. */
 int32_t edg_store_set_hot(edg_store* store, int32_t enable, int32_t admit_after);
 
+/* The layer's shared expert (Sec. 3.1 "Problem" lists it beside the routed experts; Sec. 4 "Phase 2"
+ * attaches the recovery adapter to its projections): one more SwiGLU expert of the same shape and
+ * record format that every token runs, whatever the routing.  With a shared expert set,
+ * moe_layer_decode computes
+ *     y = sum_k w_k expert_k(x) + shared(x),
+ * the shared expert in the same kernel launch as the routed ones (K + 1 experts, the last with
+ * weight 1 and an adapter of its own), each projection again int4 base + lora_scale * B (A .).
+ *   dev_record  dev, one record as written by edg_pack_expert, 256-byte aligned, resident for the
+ *               lifetime of the store (never staged or evicted); NULL removes the shared expert
+ *   lora_opt    its adapter: A/B tensors with leading dimension 1 and the descriptor's rank, or NULL.
+ *               Routed experts may run without an adapter (store created with loras == NULL) while
+ *               the shared expert has one -- the placement the paper trains.
+ * Only for shapes the batch-1 layer kernel covers (else EDG_E_SHAPE); not used by the T > 1 calls. */
+int32_t edg_store_set_shared_expert(edg_store* store, int32_t layer, const void* dev_record, const edg_lora* lora_opt);
+
 typedef struct edg_hot_stats {
     int64_t hits;         /* routed experts found in the hot set                      */
     int64_t misses;       /* routed experts served on demand                          */

@@ -355,6 +355,17 @@ def moe_ffn(x_bits, inds, gates, get_expert: Callable[[int], Dict[str, tuple]],
     return y
 
 
+def moe_ffn_with_shared(x_bits, inds, gates, get_expert, get_lora, shared_expert, shared_lora,
+                        sigma: float, group: int) -> np.ndarray:
+    """y = sum_k w_k * expert_k(x) + shared(x): the routed experts plus the layer's always-on shared
+    expert (Sec. 3.1 lists it beside the routed experts; Sec. 4 "Phase 2" puts the adapter on its
+    projections).  Reading taken: the shared expert obeys the same math contract and enters with
+    weight 1 (the paper states no gate for it).  Summed routed experts first, the shared one last."""
+    y = moe_ffn(x_bits, inds, gates, get_expert, get_lora, sigma, group) if len(inds) else None
+    o = expert_ffn(bf16_to_f64(x_bits), shared_expert, shared_lora, sigma, group)
+    return o if y is None else y + o
+
+
 def moe_ffn_tokens(X_bits, inds, gates, get_expert, get_lora, sigma: float, group: int) -> np.ndarray:
     """Batched decode / prefill: the batch-1 definition applied token by token.
     X_bits [T][H], inds [T][K], gates [T][K] -> Y [T][H]."""

@@ -108,6 +108,7 @@ _SIG = {
     "edg_store_create_ex": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(CopyEngine), C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
     "edg_store_set_hot": ([_P, C.c_int32, C.c_int32], C.c_int32),
+    "edg_store_set_shared_expert": ([_P, C.c_int32, _P, C.POINTER(Lora)], C.c_int32),
     "edg_store_get_hot_stats": ([_P, C.POINTER(HotStats)], C.c_int32),
     "edg_store_get_stats": ([_P, C.POINTER(StoreStats)], C.c_int32),
     "edg_store_set_chaining": ([_P, C.c_int32], C.c_int32),
@@ -355,6 +356,12 @@ class Store:
         soe = np.empty(self.desc.E, np.int32)
         _check(_lib.edg_store_snapshot(self.handle, layer, _ptr(eos), _ptr(soe)), "edg_store_snapshot")
         return eos, soe
+
+    def set_shared_expert(self, layer: int, dev_record, lora: Optional[Lora] = None) -> None:
+        """The caller keeps `dev_record` and the adapter's tensors alive."""
+        self._keep = self._keep + (dev_record, lora)
+        _check(_lib.edg_store_set_shared_expert(self.handle, layer, _ptr(dev_record), None if lora is None else C.byref(lora)),
+               "edg_store_set_shared_expert")
 
     def set_hot(self, enable: bool = True, admit_after: int = 1) -> None:
         _check(_lib.edg_store_set_hot(self.handle, int(bool(enable)), int(admit_after)), "edg_store_set_hot")

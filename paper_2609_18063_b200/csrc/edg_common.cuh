@@ -91,7 +91,7 @@ struct WorkspaceLayout {
     size_t h;         // [T][K][I] float            : silu(gate) * up
     size_t u_d;       // [T][K][rank] float         : A_down h
     size_t logits;    // [ring][E + 64] float     : next-step head logits, then the (expert, gate) pairs chosen from them, handed to the chained next step; one set per ring slot
-    size_t partial;   // [ring][4K][H] float      : gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
+    size_t partial;   // [ring][4(K+1)][H] float  : gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
     size_t lone_bytes;// what a batch-1 call that never chains needs: everything up to the first set of partials
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
@@ -118,7 +118,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.logits = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
     W.partial = round_up(W.logits + (size_t)kHandoffRing * (d.E + kPairWords) * sizeof(float), 256);
-    const size_t one_set = (size_t)kDownSlices * d.K * d.H * sizeof(float);
+    const size_t one_set = (size_t)kDownSlices * (d.K + 1) * d.H * sizeof(float);   // K routed experts and the shared expert
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = W.hq = W.xq = end;
@@ -145,6 +145,8 @@ int32_t check_desc(const edg_layer_desc* d);   // EDG_OK or EDG_E_INVAL / EDG_E_
 // What the batch-1 layer kernel can do beyond the plain layer-step; all optional.
 struct FusedExtras {
     int32_t* inds_mirror = nullptr;        // [K] copy of inds_next in mapped pinned host memory
+    const void* shared_rec = nullptr;      // device record of the layer's shared expert: runs as one more expert with gate 1
+    const edg_lora* shared_lora = nullptr; // its adapter (leading dimension 1), or null
 };
 
 bool fused_supported(const edg_layer_desc& d);

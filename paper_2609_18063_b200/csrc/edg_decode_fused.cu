@@ -149,6 +149,10 @@ struct FusedParams {
     int epc;                      // experts per cluster, one after the other: 1, or 2 or 4 (only with qpc = 4)
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     int32_t* inds_mirror;         // [K] copy of inds_next in mapped pinned host memory, or null
+    const uint8_t* shared_rec;    // record of the layer's always-on shared expert (one more expert with gate 1), or null
+    edg_lora shared_lora;         // its own adapter, leading dimension 1 (null pointers with rank_shared == 0)
+    int n_shared;                 // 0 or 1
+    int rank_shared;
     FusedSmem S;                  // shared-memory carve-up
 };
 
@@ -453,8 +457,14 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     extern __shared__ __align__(128) uint8_t smem[];
     const int cl = blockIdx.x / kC;                // cluster: an expert, or some quarters of it
     const int nq = kDownSlices / p.qpc;            // clusters per expert
-    const int k = (cl / nq) * p.epc;               // position of the cluster's (first) expert in the routing
-    const int cq = cl % nq;                        // which of the expert's clusters this is
+    // the clusters behind those of the routed experts take the shared expert: an expert like the
+    // others, always on (gate 1), with a record and an adapter of its own, partial number K
+    const int n_routed_cl = (p.K / p.epc) * nq;
+    const bool is_shared = cl >= n_routed_cl;
+    const int epc_l = is_shared ? 1 : p.epc;       // experts this cluster takes, one after the other
+    const int k = is_shared ? p.K : (cl / nq) * p.epc;   // position of the cluster's (first) expert in the routing
+    const int cq = is_shared ? cl - n_routed_cl : cl % nq;   // which of the expert's clusters this is
+    const edg_lora& lo = is_shared ? p.shared_lora : p.lora;
     const int c0 = cq * p.qpc;                     // first quarter of the intermediate dimension of this cluster
     const int crank = blockIdx.x % kC;             // rank inside the cluster
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
@@ -482,11 +492,11 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
 
     constexpr int rows_gu = 16 * TG, rows_d = 128 * TD, sw = 32 * DCH;
     const int n0_d = crank * rows_d;               // first down (= output) row of this CTA
-    const int r = p.rank;
+    const int r = is_shared ? p.rank_shared : p.rank;
     // reduce scratch of this step's ring slot: a chained step never waits for the previous kernel to
     // end, so steps in flight must not share it
-    const int np = p.K * nq;                       // partial outputs per output row
-    float* partial = p.partial + (size_t)p.ring * kDownSlices * p.K * p.H;
+    const int np = (p.K + p.n_shared) * nq;        // partial outputs per output row
+    float* partial = p.partial + (size_t)p.ring * kDownSlices * (p.K + 1) * p.H;
     int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
     if (tid == 0) pdl_launch_dependents();
@@ -549,7 +559,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         // and kC partials of A_down.h (the barriers of quarters 2 and 3 are re-armed below)
         if (r > 0) mbar_expect_tx(&bars[BAR_U], 2u * r * 4u);
         mbar_expect_tx(&bars[BAR_H], (uint32_t)(sw + kC * r) * 4u);
-        if (p.qpc * p.epc > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
+        if (p.qpc * epc_l > 1) mbar_expect_tx(&bars[BAR_H + 1], (uint32_t)(sw + kC * r) * 4u);
     }
     // The cluster handshake starts here (thread 0 after its barrier set-up) and is completed
     // before the first remote store: the arriving side of a cluster-scope barrier waits for every
@@ -600,12 +610,13 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     auto take = [&]() {               // warp 0
         if (lane == 0) {
             int nv = 0, okm = 0, adv = 0;
-            for (int e = 0; e < p.epc; ++e) {
+            for (int e = 0; e < epc_l; ++e) {
                 int slot = s_ex[2 * e];
-                const int expert = p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k + e] : 0);
-                if (p.table != nullptr) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
+                const int expert = is_shared ? 0 : (p.table != nullptr ? slot : (p.experts != nullptr ? p.experts[k + e] : 0));
+                if (p.table != nullptr && !is_shared) slot = (slot >= 0 && slot < p.E) ? s_table[slot] : -1;
                 int a_e = 0;          // several experts per cluster only with one shared adapter: 0 for all
                 if (r > 0 && p.n_adapters != 1) a_e = (expert >= 0 && expert < p.E) ? expert : -1;
+                if (is_shared) { slot = 0; a_e = 0; }
                 const bool ok = slot >= 0 && slot < p.n_slots && a_e >= 0;
                 if (ok) { s_ex[12 + nv] = e; s_ex[16 + e] = slot; okm |= 1 << e; ++nv; if (e == 0) adv = a_e; }
                 s_ex[20 + e] = s_ex[2 * e + 1];
@@ -619,7 +630,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     auto read_take = [&]() { n_items = s_ex[8] * p.qpc; ad = s_ex[9]; valid = n_items > 0; };
     // the items of this cluster's stream: the quarters of its valid experts, one expert after the other
     auto item_expert = [&](int w) { return s_ex[12 + w / p.qpc]; };
-    auto item_rec = [&](int w) { return p.pool + (size_t)s_ex[16 + item_expert(w)] * p.L.bytes; };
+    auto item_rec = [&](int w) { return is_shared ? p.shared_rec : p.pool + (size_t)s_ex[16 + item_expert(w)] * p.L.bytes; };
     const int cps = p.H / 128;            // chunks of a row per stage
     const int gpst = (p.H / 4) >> p.gshift;   // groups of a row per stage
     const int gps = sw >> p.gshift;       // groups of a down row-slice
@@ -660,10 +671,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         if (lane == 0) mbar_expect_tx(&bars[BAR_LORA + (it & 1)], 2 * bgu + r * ad_row);
         __syncwarp();
         const size_t bo = ((size_t)ad * p.I + n0) * r * 2;
-        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(p.lora.B_gate) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
-        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(p.lora.B_up) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
+        if (lane == 0) bulk_g2s(buf, static_cast<const uint8_t*>(lo.B_gate) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
+        if (lane == 1) bulk_g2s(buf + bgu, static_cast<const uint8_t*>(lo.B_up) + bo, bgu, &bars[BAR_LORA + (it & 1)]);
         for (int j = lane; j < r; j += 32)
-            bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(p.lora.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
+            bulk_g2s(buf + 2 * bgu + j * ad_row, static_cast<const uint8_t*>(lo.A_down) + (((size_t)ad * r + j) * p.I + n0) * 2,
                      ad_row, &bars[BAR_LORA + (it & 1)]);
     };
 
@@ -699,7 +710,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
 #pragma unroll
                     for (int e = 0; e < kMaxEpc; ++e) {
                         const unsigned long long we = __shfl_sync(0xFFFFFFFFu, w, (k + e) & 31);
-                        if (e < p.epc) { vi[e] = (int)(uint32_t)we; vg[e] = (int)(uint32_t)(we >> 32); }
+                        if (e < epc_l) { vi[e] = (int)(uint32_t)we; vg[e] = (int)(uint32_t)(we >> 32); }
                     }
                     trace_mark(p, 19);
                 } else if (pass) {
@@ -713,9 +724,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             if (p.flag_in < 0 || (!got && pass)) {
 #pragma unroll
                 for (int e = 0; e < kMaxEpc; ++e)
-                    if (e < p.epc) { vi[e] = __ldcg(&p.slots[k + e]); vg[e] = __float_as_int(__ldcg(&p.gates[k + e])); }
+                    if (e < epc_l && !is_shared) { vi[e] = __ldcg(&p.slots[k + e]); vg[e] = __float_as_int(__ldcg(&p.gates[k + e])); }
                 got = true;
             }
+            if (is_shared) { vi[0] = 0; vg[0] = __float_as_int(1.f); }      // not routed: always on, weight 1
             if (got) {
                 if (lane == 0) {
 #pragma unroll
@@ -847,7 +859,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                     for (int u = 0; u < 8; ++u) {
                         const int q = min(crank * per + min(q0 + u, per - 1), 2 * r - 1);
                         const int up = q >= r ? 1 : 0;
-                        const uint16_t* A = reinterpret_cast<const uint16_t*>(up ? p.lora.A_up : p.lora.A_gate) +
+                        const uint16_t* A = reinterpret_cast<const uint16_t*>(up ? lo.A_up : lo.A_gate) +
                                             ((size_t)ad * r + (q - up * r)) * p.H;
                         ua[u] = ld_keep16(A + cc);
                     }
@@ -1118,7 +1130,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 // straight from memory, 2r bytes each) and the gate weight: one thread per output row
                 const float gate_k = __int_as_float(s_ex[20 + e]);
                 float* prow = partial + ((size_t)(k + e) * nq + cq) * p.H + n0_d;
-                const uint16_t* Bd = static_cast<const uint16_t*>(p.lora.B_down) + ((size_t)ad * p.H + n0_d) * r;
+                const uint16_t* Bd = static_cast<const uint16_t*>(lo.B_down) + ((size_t)ad * p.H + n0_d) * r;
                 constexpr int kRowsPerThread = rows_d / (kFW * 32);
                 float dl[kRowsPerThread];
 #pragma unroll
@@ -1140,9 +1152,9 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         trace_mark(p, 8);
     }
     // a skipped expert contributes nothing
-    if (s_ex[8] != p.epc) {
+    if (s_ex[8] != epc_l) {
         if (tid == 0) atomicExch(p.status, EDG_E_RANGE);
-        for (int e = 0; e < p.epc; ++e)
+        for (int e = 0; e < epc_l; ++e)
             if (!((s_ex[10] >> e) & 1))
                 for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)(k + e) * nq + cq) * p.H + n0_d + i] = 0.f;
     }
@@ -1222,7 +1234,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.K / p.epc * (kDownSlices / p.qpc) * kC, 1, 1);
+    cfg.gridDim = dim3((p.K / p.epc + p.n_shared) * (kDownSlices / p.qpc) * kC, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -1261,11 +1273,16 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.W_pre = W_pre; p.inds_next = inds_next; p.gates_next = gates_next; p.logits_next = logits_next;
     p.H = d->H; p.I = d->I; p.E = d->E; p.K = d->K; p.group = d->group;
     p.rank = has_lora ? d->rank : 0;
+    if (extras != nullptr && extras->shared_rec != nullptr) {
+        p.shared_rec = static_cast<const uint8_t*>(extras->shared_rec);
+        p.n_shared = 1;
+        if (extras->shared_lora != nullptr && d->rank > 0) { p.shared_lora = *extras->shared_lora; p.rank_shared = d->rank; }
+    }
     p.n_adapters = d->n_adapters; p.n_slots = d->n_slots;
     p.pre_dtype = d->pre_dtype; p.out_dtype = d->out_dtype;
     p.sigma = d->lora_scale;
     p.L = record_layout(d->H, d->I, d->group);
-    p.S = fused_smem(d->H, d->I, d->E, d->group, p.rank);
+    p.S = fused_smem(d->H, d->I, d->E, d->group, p.rank > p.rank_shared ? p.rank : p.rank_shared);
     p.gshift = 0;
     while ((1 << p.gshift) < d->group) ++p.gshift;
     p.trace = g_trace;

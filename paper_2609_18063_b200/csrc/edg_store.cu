@@ -118,6 +118,9 @@ struct edg_store {
     uint8_t* dev_slots = nullptr;
     int32_t* dev_tables = nullptr;
     std::vector<edg_lora> loras;
+    std::vector<const void*> shared_rec;   // per layer: device record of the shared expert, or null
+    std::vector<edg_lora> shared_lora;     // per layer: its adapter
+    std::vector<uint8_t> shared_has_lora;
     void* copy_stream = nullptr;
     edg_copy_engine eng{};                 // what staging runs on: the CUDA runtime, or a caller's engine
     bool cuda_engine = true;
@@ -453,6 +456,25 @@ extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* st
     return EDG_OK;
 }
 
+extern "C" int32_t edg_store_set_shared_expert(edg_store* s, int32_t layer, const void* dev_record, const edg_lora* lora_opt) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    if (dev_record != nullptr && !edg::aligned(dev_record, 256)) return EDG_E_INVAL;
+    if (dev_record != nullptr && !edg::fused_supported(s->d)) return EDG_E_SHAPE;
+    if (lora_opt != nullptr && s->d.rank > 0 &&
+        (!lora_opt->A_gate || !lora_opt->B_gate || !lora_opt->A_up || !lora_opt->B_up || !lora_opt->A_down || !lora_opt->B_down))
+        return EDG_E_INVAL;
+    if (s->shared_rec.empty()) {
+        s->shared_rec.assign(s->n_layers, nullptr);
+        s->shared_lora.assign(s->n_layers, edg_lora{});
+        s->shared_has_lora.assign(s->n_layers, 0);
+    }
+    s->shared_rec[layer] = dev_record;
+    s->shared_has_lora[layer] = (dev_record != nullptr && lora_opt != nullptr && s->d.rank > 0) ? 1 : 0;
+    if (s->shared_has_lora[layer]) s->shared_lora[layer] = *lora_opt;
+    return EDG_OK;
+}
+
 extern "C" int32_t edg_store_set_hot(edg_store* s, int32_t enable, int32_t admit_after) {
     if (!store_ok(s)) return EDG_E_INVAL;
     if (!enable) { s->hot = false; return EDG_OK; }
@@ -543,6 +565,10 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         s->ring_next = (ring + 1) % edg::kHandoffRing;
         edg::FusedExtras extras;
         extras.inds_mirror = W_pre_next != nullptr ? inds_next_host_mirror_opt : nullptr;
+        if (!s->shared_rec.empty() && s->shared_rec[layer] != nullptr) {
+            extras.shared_rec = s->shared_rec[layer];
+            extras.shared_lora = s->shared_has_lora[layer] ? &s->shared_lora[layer] : nullptr;
+        }
         rc = edg::run_fused_layer(&s->d, pool, slot_arg, table, expert_arg, gates_cur, x,
                                   (lora && s->d.rank > 0) ? lora : nullptr, y, W_pre_next, inds_next, gates_next,
                                   logits_next_opt, workspace, flag_in, flag_out, ring, stale, st, &extras);
@@ -559,6 +585,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         s->chain_stream = stream;
         s->chain_flag = flag_out;
     } else {
+        if (!s->shared_rec.empty() && s->shared_rec[layer] != nullptr) return EDG_E_SHAPE;   // the shared expert rides in the fused kernel only
         rc = edg::run_ffn(&s->d, pool, 1, slot_arg, table, expert_arg, gates_cur, x, lora, y, workspace, workspace_bytes, st);
         if (rc != EDG_OK) return rc;
         if (W_pre_next != nullptr) {

@@ -543,3 +543,31 @@ def test_hot_set_popularity_admission_and_invariants():
                 assert b.slot_of_expert[e] == v
         assert sum(1 for s in b.slot_of_expert if s >= 0) == len(res)
     assert b.hits + b.misses == 1200 and b.admitted <= b.misses
+
+
+# ------------------------------------------------------------------ the shared expert
+
+def test_shared_expert_is_one_more_expert_with_weight_one():
+    rng = np.random.default_rng(21)
+    H, I, g, r = 32, 32, 32, 4
+    experts = [_tiny_expert(rng, H, I, g) for _ in range(3)]
+    shared, lo, slo = _tiny_expert(rng, H, I, g), _tiny_lora(rng, H, I, r), _tiny_lora(rng, H, I, r)
+    x = _bf16(rng.standard_normal(H))
+    xv = orc.bf16_to_f64(x)
+    # brute force: the scalar-loop projections of this file, composed by hand
+    def brute_ffn(ex, lora):
+        gt = _brute_proj(xv, ex["gate"], lora["gate"], 2.0, g)
+        up = _brute_proj(xv, ex["up"], lora["up"], 2.0, g)
+        h = np.array([a / (1.0 + math.exp(-a)) * b for a, b in zip(gt, up)])
+        return np.array(_brute_proj(h, ex["down"], lora["down"], 2.0, g))
+    want = 0.25 * brute_ffn(experts[0], lo) + 0.75 * brute_ffn(experts[2], lo) + brute_ffn(shared, slo)
+    got = orc.moe_ffn_with_shared(x, [0, 2], [0.25, 0.75], experts.__getitem__, lambda e: lo, shared, slo, 2.0, g)
+    assert np.allclose(got, want, rtol=1e-12, atol=1e-12)
+    # no routed expert at all: the layer is the shared expert; routed part and shared part add
+    only = orc.moe_ffn_with_shared(x, [], [], experts.__getitem__, None, shared, slo, 2.0, g)
+    assert np.allclose(only, brute_ffn(shared, slo), rtol=1e-12, atol=1e-12)
+    routed = orc.moe_ffn(x, [0, 2], [0.25, 0.75], experts.__getitem__, lambda e: lo, 2.0, g)
+    assert np.allclose(got - routed, only, rtol=1e-10, atol=1e-12)
+    # the shared expert's adapter is its own: swapping it for the routed adapter changes the result
+    other = orc.moe_ffn_with_shared(x, [0, 2], [0.25, 0.75], experts.__getitem__, lambda e: lo, shared, lo, 2.0, g)
+    assert np.abs(other - got).max() > 1e-6
