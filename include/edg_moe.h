@@ -286,6 +286,16 @@ int32_t edg_store_create_ex(const edg_layer_desc* desc, int32_t n_layers, const 
  * Chaining does not apply to hot-path steps.  n_slots must exceed K; admit_after >= 1. */
 int32_t edg_store_set_hot(edg_store* store, int32_t enable, int32_t admit_after);
 
+/* The whole-layer executor path (Sec. 3.1: "all experts of a layer loaded in one shot for prefill
+ * ... CPU load overlaps the previous layer's GPU execution").  Needs a pool as large as the layer
+ * (n_slots == E, else EDG_E_SLOTS).  Queues on the copy stream, behind the last compute recorded for
+ * this pool layer (edg_store_mark_computed), ONE copy of all E records -- from host_layer_opt
+ * (pinned [E][record bytes]) if given, else from the layer's own host tier -- then the identity
+ * slot table and the layer's copy-done event; edg_store_wait_staged makes the compute stream wait
+ * for it.  With host_layer_opt a store of two pool layers serves a model of any depth as a double
+ * buffer: load layer l+1 into pool (l+1) % 2 while layer l computes in pool l % 2. */
+int32_t edg_store_load_whole_layer(edg_store* store, int32_t layer, const void* host_layer_opt);
+
 /* The layer's shared expert (Sec. 3.1 "Problem" lists it beside the routed experts; Sec. 4 "Phase 2"
  * attaches the recovery adapter to its projections): one more SwiGLU expert of the same shape and
  * record format that every token runs, whatever the routing.  With a shared expert set,

@@ -107,6 +107,7 @@ _SIG = {
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
     "edg_store_create_ex": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(CopyEngine), C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
+    "edg_store_load_whole_layer": ([_P, C.c_int32, _P], C.c_int32),
     "edg_store_set_hot": ([_P, C.c_int32, C.c_int32], C.c_int32),
     "edg_store_set_shared_expert": ([_P, C.c_int32, _P, C.POINTER(Lora)], C.c_int32),
     "edg_store_get_hot_stats": ([_P, C.POINTER(HotStats)], C.c_int32),
@@ -356,6 +357,9 @@ class Store:
         soe = np.empty(self.desc.E, np.int32)
         _check(_lib.edg_store_snapshot(self.handle, layer, _ptr(eos), _ptr(soe)), "edg_store_snapshot")
         return eos, soe
+
+    def load_whole_layer(self, layer: int, host_layer=None) -> None:
+        _check(_lib.edg_store_load_whole_layer(self.handle, layer, _ptr(host_layer)), "edg_store_load_whole_layer")
 
     def set_shared_expert(self, layer: int, dev_record, lora: Optional[Lora] = None) -> None:
         """The caller keeps `dev_record` and the adapter's tensors alive."""

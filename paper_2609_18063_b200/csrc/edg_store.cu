@@ -124,6 +124,7 @@ struct edg_store {
     void* copy_stream = nullptr;
     edg_copy_engine eng{};                 // what staging runs on: the CUDA runtime, or a caller's engine
     bool cuda_engine = true;
+    bool whole_layer_loads = false;        // edg_store_load_whole_layer has been used: a full pool gets overwritten too
     bool hot = false;                      // the hot executor path (edg_store_set_hot)
     int admit_after = 1;
     edg_hot_stats hot_stats{};
@@ -442,7 +443,7 @@ extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* st
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     // Only a pool that can evict needs the ordering: with n_slots == E nothing is ever overwritten.
     LayerState& L = s->layers[layer];
-    if (s->d.n_slots < s->d.E || s->hot) {
+    if (s->d.n_slots < s->d.E || s->hot || s->whole_layer_loads) {
         const edg_copy_engine& g = s->eng;
         EDG_ENG_TRY(g.event_record(g.ctx, L.compute_done, stream));
         L.compute_recorded = true;
@@ -453,6 +454,43 @@ extern "C" int32_t edg_store_mark_computed(edg_store* s, int32_t layer, void* st
         L.pending.clear();
         if (rc != EDG_OK) return rc;
     }
+    return EDG_OK;
+}
+
+// The whole-layer path (Sec. 3.1, executor path 4): every expert of a layer in one shot, for prefill,
+// where each expert is hit and there is nothing to predict.  The pinned-host layer is laid out as
+// the pool is, so the load is ONE copy of E records (the paper's per-layer stacked layout makes it
+// nine direct reads instead of 256 x 9 builds), queued on the copy stream behind the pool layer's
+// last compute; the table becomes the identity.  The next layer's load runs while this layer computes.
+extern "C" int32_t edg_store_load_whole_layer(edg_store* s, int32_t layer, const void* host_layer_opt) {
+    if (!store_ok(s)) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    if (s->d.n_slots != s->d.E || s->hot) return EDG_E_SLOTS;
+    if (host_layer_opt != nullptr && !edg::aligned(host_layer_opt, 16)) return EDG_E_INVAL;
+    const edg_copy_engine& g = s->eng;
+    const int E = s->d.E;
+    LayerState& L = s->layers[layer];
+    const uint8_t* src = host_layer_opt ? static_cast<const uint8_t*>(host_layer_opt) : s->host_layers[layer];
+    s->whole_layer_loads = true;
+    for (int e = 0; e < E; ++e) { L.expert_of_slot[e] = e; L.slot_of_expert[e] = e; L.last_use[e] = L.n; }
+    L.n += 1;
+    L.pending.clear();
+    if (L.compute_recorded) EDG_ENG_TRY(g.stream_wait_event(g.ctx, s->copy_stream, L.compute_done));
+    EDG_ENG_TRY(g.copy_h2d(g.ctx, s->dev_slots + (size_t)layer * E * s->R, src, (size_t)E * s->R, s->copy_stream));
+    const int r = s->ring_pos;
+    s->ring_pos = (r + 1) % kRing;
+    if (s->ring_used[r]) EDG_ENG_TRY(g.event_synchronize(g.ctx, s->ring_ev[r]));
+    int32_t* row = s->ring + (size_t)r * E;
+    for (int e = 0; e < E; ++e) row[e] = e;
+    EDG_ENG_TRY(g.copy_h2d(g.ctx, s->dev_tables + (size_t)layer * E, row, (size_t)E * sizeof(int32_t), s->copy_stream));
+    EDG_ENG_TRY(g.event_record(g.ctx, s->ring_ev[r], s->copy_stream));
+    s->ring_used[r] = true;
+    EDG_ENG_TRY(g.event_record(g.ctx, L.copy_done, s->copy_stream));
+    L.copy_pending = true;
+    s->stats.stage_calls += 1;
+    s->stats.misses += E;
+    s->stats.table_updates += 1;
+    s->stats.bytes_copied += (int64_t)E * (int64_t)s->R;
     return EDG_OK;
 }
 

@@ -189,3 +189,44 @@ def test_hot_path_needs_room_and_an_early_switch(lib):
     with pytest.raises(lib.EdgError):
         rig.store.set_hot(True, 1)                           # after the first staging call
     rig.store.close()
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_whole_layer_loads_as_a_double_buffer(lib, seed):
+    """The whole-layer path on the host: a store of two pool layers serves a deeper model.  Layer l+1 is
+    loaded into the other pool layer while the "kernel" of layer l runs; each kernel must find all E
+    records of ITS model layer, whatever the schedule, and a pool layer is only overwritten behind the
+    compute that last read it."""
+    E = 8
+    rig = Rig(lib, seed, S=E, E=E, K=2, n_layers=2)
+    rng = np.random.default_rng(seed)
+    depth = 7
+    model = [np.ascontiguousarray(rng.integers(0, 256, (E, rig.R), dtype=np.uint8)) for _ in range(depth)]
+
+    def kernel(pool_layer, l):
+        def run():
+            if rig.tables[pool_layer].tolist() != list(range(E)):
+                rig.violations.append(("table", l))
+            elif not np.array_equal(rig.pool[pool_layer], model[l]):
+                rig.violations.append(("bytes", l))
+        rig.eng.kernel(COMPUTE, run)
+
+    rig.store.load_whole_layer(0, model[0])
+    for l in range(depth):
+        if l + 1 < depth:
+            rig.store.load_whole_layer((l + 1) % 2, model[l + 1])     # runs while layer l computes
+        rig.store.wait_staged(l % 2, COMPUTE)
+        kernel(l % 2, l)
+        rig.store.mark_computed(l % 2, COMPUTE)
+        rig.eng.run_some(int(rng.integers(0, 5)))
+    assert rig.eng.drain() and rig.violations == [] and rig.canaries_ok()
+    assert rig.store.stats()["bytes_copied"] == depth * E * rig.R
+    eos, soe = rig.store.snapshot(1)
+    assert eos.tolist() == list(range(E)) and soe.tolist() == list(range(E))
+    # a pool smaller than the layer cannot take a whole layer
+    small = Rig(lib, seed, S=4, E=E, K=2, n_layers=1)
+    with pytest.raises(lib.EdgError) as ei:
+        small.store.load_whole_layer(0)
+    assert ei.value.code == -3
+    small.store.close()
+    rig.store.close()
