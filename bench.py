@@ -846,7 +846,8 @@ def run_prefill_stream(args):
             if overlap and l + 1 < depth:
                 store.load_whole_layer((l + 1) % 2, hosts[l + 1])
             layer(l)
-            if not overlap and l + 1 < depth:
+            if not overlap and l + 1 < depth:                 # serial: the load starts when the layer has finished
+                torch.cuda.synchronize()
                 store.load_whole_layer((l + 1) % 2, hosts[l + 1])
         e1.record()
         torch.cuda.synchronize()
