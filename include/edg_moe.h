@@ -286,6 +286,19 @@ int32_t edg_store_create_ex(const edg_layer_desc* desc, int32_t n_layers, const 
  * Chaining does not apply to hot-path steps.  n_slots must exceed K; admit_after >= 1. */
 int32_t edg_store_set_hot(edg_store* store, int32_t enable, int32_t admit_after);
 
+/* The full prerouter head inside the layer-step (Sec. 3.2 "Head" and "Feature drift": a head's input
+ * includes the routing its layer actually executed -- at decode, the head's own earlier prediction).
+ * With a head set for a layer, moe_layer_decode of that layer predicts inds_next / gates_next with
+ *     l = W2 gelu(W1 [x ; hot(cur) ; hot(prev)] + b1) + b2 + W_res x
+ * where cur is the routing this call executes (inds_cur) and prev the routing the layer executed at
+ * its previous call, which the store keeps on the device and updates after every call (empty before
+ * the first call and after edg_store_reset_feedback: a new sequence).  W_pre_next is then ignored;
+ * the prediction is made whenever inds_next is non-NULL.  The struct is copied; its tensors stay
+ * the caller's (one head: leading dimension 1).  NULL removes the head (back to the linear path).
+ * Steps of such a layer are never chained.  Allocates a small device buffer on first use: not hot. */
+int32_t edg_store_set_mlp_head(edg_store* store, int32_t layer, const edg_mlp_head* head);
+int32_t edg_store_reset_feedback(edg_store* store, int32_t layer);
+
 /* The whole-layer executor path (Sec. 3.1: "all experts of a layer loaded in one shot for prefill
  * ... CPU load overlaps the previous layer's GPU execution").  Needs a pool as large as the layer
  * (n_slots == E, else EDG_E_SLOTS).  Queues on the copy stream, behind the last compute recorded for

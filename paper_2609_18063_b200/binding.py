@@ -108,6 +108,8 @@ _SIG = {
     "edg_store_create_ex": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(CopyEngine), C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
     "edg_store_load_whole_layer": ([_P, C.c_int32, _P], C.c_int32),
+    "edg_store_set_mlp_head": ([_P, C.c_int32, _P], C.c_int32),
+    "edg_store_reset_feedback": ([_P, C.c_int32], C.c_int32),
     "edg_store_set_hot": ([_P, C.c_int32, C.c_int32], C.c_int32),
     "edg_store_set_shared_expert": ([_P, C.c_int32, _P, C.POINTER(Lora)], C.c_int32),
     "edg_store_get_hot_stats": ([_P, C.POINTER(HotStats)], C.c_int32),
@@ -357,6 +359,18 @@ class Store:
         soe = np.empty(self.desc.E, np.int32)
         _check(_lib.edg_store_snapshot(self.handle, layer, _ptr(eos), _ptr(soe)), "edg_store_snapshot")
         return eos, soe
+
+    def set_mlp_head(self, layer: int, W1=None, b1=None, W2=None, b2=None, W_res=None, width: int = 0) -> None:
+        """The full prerouter head of a layer (tensors of ONE head; the caller keeps them alive); W1 None removes it."""
+        if W1 is None:
+            _check(_lib.edg_store_set_mlp_head(self.handle, layer, None), "edg_store_set_mlp_head")
+            return
+        self._keep = self._keep + (W1, b1, W2, b2, W_res)
+        head = MlpHead(_ptr(W1), _ptr(b1), _ptr(W2), _ptr(b2), _ptr(W_res), int(width))
+        _check(_lib.edg_store_set_mlp_head(self.handle, layer, C.byref(head)), "edg_store_set_mlp_head")
+
+    def reset_feedback(self, layer: int) -> None:
+        _check(_lib.edg_store_reset_feedback(self.handle, layer), "edg_store_reset_feedback")
 
     def load_whole_layer(self, layer: int, host_layer=None) -> None:
         _check(_lib.edg_store_load_whole_layer(self.handle, layer, _ptr(host_layer)), "edg_store_load_whole_layer")

@@ -164,6 +164,10 @@ int32_t run_ffn(const edg_layer_desc* d, const void* slot_pool, int32_t T, const
 int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s, int32_t n_heads,
                       int32_t* inds, float* gates, float* logits_opt, cudaStream_t st, int shared_head = 0,
                       int32_t* mirror = nullptr);
+// the full head (fc1 -> gelu -> fc2 + residual path) for n_heads (head, state) pairs
+int32_t run_prerouter_mlp(const edg_layer_desc* desc, const edg_mlp_head* head, const void* s,
+                          const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
+                          int32_t* inds, float* gates, float* logits_opt, cudaStream_t stream, int32_t* mirror);
 
 // ---------------------------------------------------------------- device helpers
 #ifdef __CUDACC__

@@ -326,6 +326,7 @@ struct MlpParams {
     float* gates;           // [n_heads][K]
     float* logits;          // [n_heads][E] or null
     int H, E, K, D;
+    int32_t* mirror;        // [n_heads][K] in mapped pinned host memory, or null
 };
 
 // dot product of an fp16 row of n (a multiple of 8) weights with fp32 activations, by one warp
@@ -440,8 +441,10 @@ __global__ void __launch_bounds__(kMlpWarps * 32) prerouter_mlp_kernel(MlpParams
     if (p.logits != nullptr)
         for (int e = threadIdx.x; e < p.E; e += blockDim.x) p.logits[(size_t)head * p.E + e] = s_logits[e];
     __syncthreads();
-    if (warp == 0)
+    if (warp == 0) {
         warp_softmax_topk(s_logits, p.E, p.K, lane, p.inds + (size_t)head * p.K, p.gates + (size_t)head * p.K);
+        mirror_inds(p.mirror != nullptr ? p.mirror + (size_t)head * p.K : nullptr, p.inds + (size_t)head * p.K, p.K, lane);
+    }
 }
 
 // Appendix A, sigmoid-group routing, one warp per row of given logits: sigma = sigmoid(l); a group's
@@ -626,6 +629,13 @@ extern "C" int32_t sigmoid_group_topk_rows(const float* logits, int32_t T, int32
 extern "C" int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_head* head, const void* s,
                                       const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
                                       int32_t* inds, float* gates, float* logits_opt, void* stream) {
+    return edg::run_prerouter_mlp(desc, head, s, cur_inds, prev_inds, n_heads, inds, gates, logits_opt,
+                                  static_cast<cudaStream_t>(stream), nullptr);
+}
+
+int32_t edg::run_prerouter_mlp(const edg_layer_desc* desc, const edg_mlp_head* head, const void* s,
+                               const int32_t* cur_inds, const int32_t* prev_inds, int32_t n_heads,
+                               int32_t* inds, float* gates, float* logits_opt, cudaStream_t stream, int32_t* mirror) {
     int32_t rc = edg::check_desc(desc);
     if (rc != EDG_OK) return rc;
     if (!head || !head->W1 || !head->W2 || !s || !cur_inds || !prev_inds || !inds || !gates || n_heads < 1 || n_heads > 65535)
@@ -638,12 +648,12 @@ extern "C" int32_t prerouter_mlp_topk(const edg_layer_desc* desc, const edg_mlp_
     edg::MlpParams p{static_cast<const __half*>(head->W1), static_cast<const __half*>(head->b1),
                      static_cast<const __half*>(head->W2), static_cast<const __half*>(head->b2), head->W_res,
                      static_cast<const uint16_t*>(s), cur_inds, prev_inds, inds, gates, logits_opt,
-                     desc->H, desc->E, desc->K, D};
+                     desc->H, desc->E, desc->K, D, mirror};
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(edg::kPreCluster, n_heads, 1);
     cfg.blockDim = dim3(edg::kMlpWarps * 32, 1, 1);
     cfg.dynamicSmemBytes = (size_t)(desc->E + desc->H + D) * sizeof(float);
-    cfg.stream = static_cast<cudaStream_t>(stream);
+    cfg.stream = stream;
     if (cfg.dynamicSmemBytes > 48 * 1024) return EDG_E_SHAPE;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;

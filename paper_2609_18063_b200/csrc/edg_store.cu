@@ -118,6 +118,8 @@ struct edg_store {
     uint8_t* dev_slots = nullptr;
     int32_t* dev_tables = nullptr;
     std::vector<edg_lora> loras;
+    std::vector<edg_mlp_head> mlp_heads;   // per layer: the full prerouter head (W1 == null: none)
+    int32_t* prev_inds = nullptr;          // dev [n_layers][K]: the routing each layer executed at its previous step (-1: none yet)
     std::vector<const void*> shared_rec;   // per layer: device record of the shared expert, or null
     std::vector<edg_lora> shared_lora;     // per layer: its adapter
     std::vector<uint8_t> shared_has_lora;
@@ -244,6 +246,7 @@ extern "C" int32_t edg_store_destroy(edg_store* s) {
     if (s->ring) g.host_free(g.ctx, s->ring);
     if (s->step_done) cudaEventDestroy(s->step_done);
     if (s->slots_eff) cudaFree(s->slots_eff);
+    if (s->prev_inds) cudaFree(s->prev_inds);
     for (auto& pr : s->wait_events) {
         if (pr.first) cudaEventDestroy(pr.first);
         if (pr.second) cudaEventDestroy(pr.second);
@@ -494,6 +497,31 @@ extern "C" int32_t edg_store_load_whole_layer(edg_store* s, int32_t layer, const
     return EDG_OK;
 }
 
+extern "C" int32_t edg_store_set_mlp_head(edg_store* s, int32_t layer, const edg_mlp_head* head) {
+    if (!store_ok(s) || !s->cuda_engine) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    if (s->mlp_heads.empty()) s->mlp_heads.assign(s->n_layers, edg_mlp_head{});
+    if (head == nullptr) { s->mlp_heads[layer] = edg_mlp_head{}; return EDG_OK; }
+    if (!head->W1 || !head->W2) return EDG_E_INVAL;
+    if (head->width < 8 || head->width > 4096 || head->width % 8 != 0) return EDG_E_SHAPE;
+    if ((size_t)(s->d.E + s->d.H + head->width) * sizeof(float) > 48 * 1024) return EDG_E_SHAPE;
+    if (s->prev_inds == nullptr) {
+        const size_t n = (size_t)s->n_layers * s->d.K * sizeof(int32_t);
+        EDG_CUDA_TRY(cudaMalloc(reinterpret_cast<void**>(&s->prev_inds), n));
+        EDG_CUDA_TRY(cudaMemset(s->prev_inds, 0xFF, n));   // no previous step yet: an empty K-hot vector
+    }
+    s->mlp_heads[layer] = *head;
+    return EDG_OK;
+}
+
+extern "C" int32_t edg_store_reset_feedback(edg_store* s, int32_t layer) {
+    if (!store_ok(s) || !s->cuda_engine) return EDG_E_INVAL;
+    if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
+    if (s->prev_inds != nullptr)
+        EDG_CUDA_TRY(cudaMemset(s->prev_inds + (size_t)layer * s->d.K, 0xFF, (size_t)s->d.K * sizeof(int32_t)));
+    return EDG_OK;
+}
+
 extern "C" int32_t edg_store_set_shared_expert(edg_store* s, int32_t layer, const void* dev_record, const edg_lora* lora_opt) {
     if (!store_ok(s)) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
@@ -545,6 +573,19 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
     int32_t rc = edg_store_wait_staged(s, layer, stream);
     if (rc != EDG_OK) return rc;
     const edg_lora* lora = s->loras.empty() ? nullptr : &s->loras[layer];
+    // A layer with a full (MLP) head predicts with it: fc1 -> gelu -> fc2 + residual path on the feature
+    // [x ; K-hot(routing executed now) ; K-hot(routing executed at this layer's previous step)].
+    const bool mlp = !s->mlp_heads.empty() && s->mlp_heads[layer].W1 != nullptr && inds_next != nullptr;
+    if (mlp) {
+        if (!gates_next) return EDG_E_INVAL;
+        int32_t* prev = s->prev_inds + (size_t)layer * s->d.K;
+        rc = edg::run_prerouter_mlp(&s->d, &s->mlp_heads[layer], x, inds_cur, prev, 1, inds_next, gates_next,
+                                    logits_next_opt, st, inds_next_host_mirror_opt);
+        if (rc != EDG_OK) return rc;
+        // what this step executes is the next step's "previous routing"
+        EDG_CUDA_TRY(cudaMemcpyAsync(prev, inds_cur, (size_t)s->d.K * sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+        W_pre_next = nullptr;                              // the layer kernel evaluates no head of its own
+    }
     if (W_pre_next != nullptr && (!inds_next || !gates_next)) return EDG_E_INVAL;
     const void* pool = s->dev_slots + (size_t)layer * s->d.n_slots * s->R;
     const int32_t* table = s->dev_tables + (size_t)layer * s->d.E;
