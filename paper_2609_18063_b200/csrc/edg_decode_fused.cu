@@ -511,9 +511,18 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      round-robin to the first CTAs of the grid; a row is split over all threads of its CTA
     //      (8 elements each).
     const int max_pre = (p.pre_dtype == EDG_F16 && p.H <= 2048) ? kMaxPre : kFW;     // two rows per warp only on the fast path below
-    const int n_head_ctas = p.W_pre != nullptr ? min((int)gridDim.x, max(32, (p.E + max_pre - 1) / max_pre)) : 0;
+    // An fp16 head whose rows split into blocks of 32 goes to the tensor cores: CTA b of the first
+    // E / 32 takes rows 32 b .. 32 b + 31 as two 16-row MMA tiles, warp w computing tile (w & 1) over
+    // K half (w >> 1) with the hidden state as column 0 of the B operand -- an eighth of the
+    // instructions of the FMA form below, and the head is bound by its instructions.
+    const bool pre_mma = p.W_pre != nullptr && p.pre_dtype == EDG_F16 && (p.E % 32) == 0 && (p.H % 512) == 0 &&
+                         p.E / 32 <= (int)gridDim.x && p.qpc == kDownSlices;   // (a step launched alone spreads the rows over more CTAs instead)
+    const int n_head_ctas = p.W_pre == nullptr ? 0 : pre_mma ? p.E / 32 : min((int)gridDim.x, max(32, (p.E + max_pre - 1) / max_pre));
     const bool head_cta = (int)blockIdx.x < n_head_ctas;
-    const int n_pre = head_cta ? min(max_pre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
+    const int n_pre = (head_cta && !pre_mma) ? min(max_pre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
+    const bool mma_head = pre_mma && head_cta;
+    const int mrow0 = (int)blockIdx.x * 32 + (warp & 1) * 16;     // first row of this warp's tile
+    const int mk0 = (warp >> 1) * (p.H / 2);                      // first k of this warp's K half
     // Usual case (fp16 head, H <= 2048): warp w evaluates row w of this CTA's rows by itself, each
     // lane covering 8 runs of 8 elements, and publishes it without waiting for any other warp.
     const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= 2048;
@@ -523,6 +532,15 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     bool my_row = pre_fast && warp < n_pre && my_e < p.E;
     bool my_row2 = pre_fast && warp + kFW < n_pre && my_e2 < p.E;
     uint4 lw[8], lw2[8];
+    // (tensor-core form: rows g and g + 8 of the tile, 8 k per lane and chunk of 32 k; the first 8 chunks now)
+    const __half* mwa = static_cast<const __half*>(p.W_pre) + (size_t)(mrow0 + g8) * p.H + mk0 + t4 * 8;
+    if (mma_head) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            lw[j] = ld_keep16(mwa + j * 32);
+            lw2[j] = ld_keep16(mwa + (size_t)8 * p.H + j * 32);
+        }
+    }
     if (my_row) {
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -540,6 +558,8 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     const bool pre_lane = tid * 8 < p.H;
     uint32_t pre_state = kNotYet, pre_state2 = kNotYet;   // the ring-slot entries this lane will publish into, as the kernel finds them
     if (p.flag_out >= 0) {
+        if (mma_head && warp < 2 && lane < 16)
+            pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + mrow0 + lane]);
         if (my_row && lane == 0) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e]);
         if (my_row2 && lane == 0) pre_state2 = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e2]);
         if (n_pre > 0 && !pre_fast && warp == kFW - 1 && lane < n_pre) {
@@ -749,6 +769,50 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
         }
         if (pass) break;
+        // ---- the head on the tensor cores: 16 rows x this warp's K half, the hidden state as column 0
+        //      of B (from s_xb, whose words hold (x0,x4) (x1,x5) (x2,x6) (x3,x7): the natural pairs
+        //      the fp16 rows need are byte permutations of them)
+        if (pre_mma) {
+            __syncthreads();                               // s_xb is complete (every CTA passes here: the condition is grid-uniform)
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+            if (mma_head) {
+                const int nb = p.H / 512;                  // batches of 8 chunks in a K half
+#pragma unroll 1
+                for (int b = 0; b < nb; ++b) {
+                    const uint4* xbp = s_xb + (mk0 + b * 256) / 8 + t4;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint4 xb = make_uint4(0, 0, 0, 0);
+                        if (g8 == 0) xb = xbp[j * 4];
+                        mma16816(c, lw[j].x, lw2[j].x, lw[j].y, lw2[j].y, __byte_perm(xb.x, xb.y, 0x5410), __byte_perm(xb.z, xb.w, 0x5410));
+                        mma16816(c, lw[j].z, lw2[j].z, lw[j].w, lw2[j].w, __byte_perm(xb.x, xb.y, 0x7632), __byte_perm(xb.z, xb.w, 0x7632));
+                    }
+                    if (b + 1 < nb) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            lw[j] = ld_keep16(mwa + (b + 1) * 256 + j * 32);
+                            lw2[j] = ld_keep16(mwa + (size_t)8 * p.H + (b + 1) * 256 + j * 32);
+                        }
+                    }
+                }
+                // the upper K half hands its 16 sums to the warp of the lower one
+                if (warp >= 2 && t4 == 0) {
+                    s_red[kPreRed * kFW + (warp & 1) * 16 + g8] = c[0];
+                    s_red[kPreRed * kFW + (warp & 1) * 16 + 8 + g8] = c[2];
+                }
+            }
+            __syncthreads();
+            if (mma_head && warp < 2) {
+                // rows g and g + 8 sit in the lanes with t4 == 0; lane L < 16 publishes row L of the tile
+                const float lo_ = c[0] + s_red[kPreRed * kFW + warp * 16 + g8];
+                const float hi_ = c[2] + s_red[kPreRed * kFW + warp * 16 + 8 + g8];
+                const float v_lo = __shfl_sync(0xFFFFFFFFu, lo_, (lane & 7) * 4);
+                const float v_hi = __shfl_sync(0xFFFFFFFFu, hi_, (lane & 7) * 4);
+                if (warp == 0) trace_mark(p, 12);
+                head_publish(p, smem, lane < 8 ? v_lo : v_hi, mrow0 + lane, lane < 16, lane, pre_state);
+                if (warp == 0) trace_mark(p, 13);
+            }
+        }
         // ---- the head rows (the loads of the first two have been in flight since the kernel started),
         //      published by their warp as soon as they are summed
 #pragma unroll 1
