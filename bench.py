@@ -294,12 +294,42 @@ def run_b200(args):
         if status != 0 or not bool(torch.isfinite(ydep).all()) or not bool(torch.isfinite(xdep.float()).all()):
             raise SystemExit(f"bench: dependent arm: bad device status {status} or non-finite state")
         dep_step_ms = dep_ms / WINDOW_STEPS
-        dependent = {"value": round(replicas.whole_job_rate(world, WINDOW_STEPS, dep_ms), 1), "unit": UNIT,
-                     "ms_per_step": round(dep_step_ms, 6),
-                     "hbm_gbs_on_expert_bytes": round(K * R / (dep_step_ms * 1e-3) / 1e9, 1),
-                     "frac_of_peak": round(K * R / (dep_step_ms * 1e-3) / 1e9 / _peaks()[0], 4),
+        # the same chain with the next state written by the layer kernel itself and the steps chained:
+        # step t+1 is resident, routed and has its first weights when x(t+1) is written
+        store.set_chaining(1)
+
+        def dep2_step(s_):
+            i = s_ % n_inst
+            edg.moe_layer_decode_dependent(store, i, xdep[s_ % 2], inds[s_ % 2], gates[s_ % 2], W[(s_ + 1) % n_inst],
+                                           inds[(s_ + 1) % 2], gates[(s_ + 1) % 2], None, ydep, xdep[(s_ + 1) % 2], ws, 1e-6)
+
+        with torch.cuda.stream(stream):
+            for s_ in range(2 * n_inst):
+                dep2_step(s_)
+            stream.synchronize()
+        g_dep2 = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(g_dep2, stream=stream):
+                for s_ in range(G):
+                    dep2_step(s_)
+            g_dep2.replay()
+            stream.synchronize()
+        dep2_ms = statistics.median(timed_windows(g_dep2))
+        status = edg.workspace_status(ws)
+        if status != 0 or not bool(torch.isfinite(ydep).all()) or not bool(torch.isfinite(xdep.float()).all()):
+            raise SystemExit(f"bench: fused dependent arm: bad device status {status} or non-finite state")
+        store.set_chaining(0)
+        dep2_step_ms = dep2_ms / WINDOW_STEPS
+        dependent = {"value": round(replicas.whole_job_rate(world, WINDOW_STEPS, dep2_ms), 1), "unit": UNIT,
+                     "ms_per_step": round(dep2_step_ms, 6),
+                     "hbm_gbs_on_expert_bytes": round(K * R / (dep2_step_ms * 1e-3) / 1e9, 1),
+                     "frac_of_peak": round(K * R / (dep2_step_ms * 1e-3) / 1e9 / _peaks()[0], 4),
                      "dependency": "x(t+1) = bf16(rmsnorm(x(t) + y(t))) computed on the device: every step waits for the one before it",
-                     "launch": f"two kernels per step (layer-step, next-state norm), CUDA graphs of {G} steps, chaining off",
+                     "launch": f"moe_layer_decode_dependent: one kernel per step writes y and x(t+1); steps chained (the next step "
+                               f"is resident, routed and streaming its first weights while it waits for x); CUDA graphs of {G} steps",
+                     "unchained_two_kernels": {"ms_per_step": round(dep_step_ms, 6),
+                                               "value": round(replicas.whole_job_rate(world, WINDOW_STEPS, dep_ms), 1),
+                                               "launch": "layer-step + next-state norm as two stream-ordered kernels, chaining off"},
                      "timed_steps": WINDOWS * WINDOW_STEPS, "windows": WINDOWS}
 
     # ---- batched decode and prefill on the same resident layer (secondary figures)

@@ -142,7 +142,7 @@ int32_t edg_ffn_workspace_bytes(const edg_layer_desc* desc, int32_t T, size_t* b
 int32_t edg_workspace_status(const void* workspace, void* stream, int32_t* status);
 
 /* Tracing: with a dev buffer of (CTAs in the grid) x 32 uint64 (the batch-1 layer kernel launches
- * 4K CTAs for a chained step and 16K for a lone one), every CTA stamps the GPU's nanosecond timer
+ * at most 16 (K + 1) + E / 16 + 3 CTAs), every CTA stamps the GPU's nanosecond timer
  * at its phase boundaries, in slot 0 start, 1 first copies issued, 2 adapter projections sent,
  * 3 first weights landed, 4 gate/up of the first quarter done, 5 peers' projections in, 6 h sent,
  * 7 h of the quarter in, 8 partial output written, 9 end, 10 slot taken, 12 head row summed,
@@ -436,6 +436,23 @@ int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          const void* W_pre_next, int32_t* inds_next, float* gates_next,
                          float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* The same layer-step for a chain of data-dependent steps: besides y the kernel writes
+ *     x_next = bf16(rmsnorm(x + y)),   rmsnorm(v) = v / sqrt(mean(v^2) + eps),  unit gain
+ * (what edg_next_hidden_state computes, folded into the layer kernel's reduce: no second launch).
+ * x_next dev bf16 [H], 16-byte aligned, not x itself.  With chaining switched on
+ * (edg_store_set_chaining), a following call whose x is this call's x_next and whose inds_cur /
+ * gates_cur are this call's inds_next / gates_next (same workspace and stream) is launched as a
+ * programmatic dependent in the all-SM form: it starts while this step is still computing, takes
+ * its routing from the hand-off ring, streams the first weights of its experts, and only then waits
+ * (bounded, on a device flag) for this step to write x_next -- the overlap the paper's lead buys:
+ * the routing is known a step ahead, the hidden state is not.  Results equal those of unchained calls. */
+int32_t moe_layer_decode_dependent(edg_store* store, int32_t layer, const void* x,
+                                   const int32_t* inds_cur, const float* gates_cur,
+                                   const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                                   float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
+                                   void* x_next, float eps,
+                                   void* workspace, size_t workspace_bytes, void* stream);
 
 /* One token through all n_layers layers of the store (the paper's decode timeline, Sec. 3.2
  * "Motivation": full-token lead, one hand-off per token).  On the host: waits (bounded, 5 s) until the

@@ -17,7 +17,7 @@ __all__ = [
     "make_desc", "make_lora", "version", "check_desc", "record_bytes", "pack_expert", "unpack_expert",
     "ffn_workspace_bytes", "workspace_status", "set_trace_buffer", "prerouter_topk", "prerouter_topk_tokens", "softmax_topk_rows", "sigmoid_group_topk_rows", "prerouter_mlp_topk",
     "moe_expert_ffn_int4_lora", "moe_expert_ffn_int4_lora_static", "moe_layer_decode", "stage_experts_to_slots",
-    "stack_decode_token", "next_hidden_state", "EXPORTS",
+    "moe_layer_decode_dependent", "stack_decode_token", "next_hidden_state", "EXPORTS",
 ]
 
 F32, F16, BF16 = 0, 1, 2
@@ -104,6 +104,7 @@ _SIG = {
     "softmax_topk_rows": ([_D, _P, C.c_int32, _P, _P, _P], C.c_int32),
     "sigmoid_group_topk_rows": ([_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, _P, _P], C.c_int32),
     "prerouter_mlp_topk": ([_D, _P, _P, _P, _P, C.c_int32, _P, _P, _P, _P], C.c_int32),
+    "moe_layer_decode_dependent": ([_P, C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, _P, _P, C.c_float, _P, C.c_size_t, _P], C.c_int32),
     "edg_store_create": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(_P)], C.c_int32),
     "edg_store_create_ex": ([_D, C.c_int32, C.POINTER(_P), _P, _P, C.POINTER(Lora), _P, C.POINTER(CopyEngine), C.POINTER(_P)], C.c_int32),
     "edg_store_destroy": ([_P], C.c_int32),
@@ -446,3 +447,14 @@ def stack_decode_token(store: Store, x, inds_cur, gates_cur, W_pre, inds_next, g
 def next_hidden_state(desc, x, y, x_next, eps=1e-6, stream=None) -> None:
     _check(_lib.edg_next_hidden_state(C.byref(desc), _ptr(x), _ptr(y), _ptr(x_next), float(eps), _stream(stream)),
            "edg_next_hidden_state")
+
+
+def moe_layer_decode_dependent(store: Store, layer, x, inds_cur, gates_cur, W_pre_next, inds_next, gates_next,
+                               logits_next_opt, y, x_next, workspace, eps=1e-6, workspace_bytes=None, stream=None,
+                               inds_next_host_mirror_opt=None) -> None:
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size()
+    _check(_lib.moe_layer_decode_dependent(store.handle, layer, _ptr(x), _ptr(inds_cur), _ptr(gates_cur), _ptr(W_pre_next),
+                                           _ptr(inds_next), _ptr(gates_next), _ptr(logits_next_opt),
+                                           _ptr(inds_next_host_mirror_opt), _ptr(y), _ptr(x_next), float(eps),
+                                           _ptr(workspace), workspace_bytes, _stream(stream)), "moe_layer_decode_dependent")

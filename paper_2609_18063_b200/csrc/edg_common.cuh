@@ -83,7 +83,8 @@ constexpr size_t kCtrlBytes = 4096;    // control block: status word at 0, then 
 constexpr size_t kCtrlCounters = 64;                               // [ring][4] arrivals per block of output rows
 constexpr size_t kCtrlHead = kCtrlCounters + kHandoffRing * 16;    // [ring] head rows delivered
 constexpr size_t kCtrlDone = kCtrlHead + kHandoffRing * 4;         // [ring] reducers finished
-static_assert(kCtrlDone + kHandoffRing * 4 <= kCtrlBytes, "control block too small");
+constexpr size_t kCtrlNorm = kCtrlDone + kHandoffRing * 4;         // [ring] reducers that have delivered their sum of squares (dependent chain)
+static_assert(kCtrlNorm + kHandoffRing * 4 <= kCtrlBytes, "control block too small");
 
 struct WorkspaceLayout {
     size_t ctrl;      // kCtrlBytes control block
@@ -92,6 +93,7 @@ struct WorkspaceLayout {
     size_t u_d;       // [T][K][rank] float         : A_down h
     size_t logits;    // [ring][E + 64] float     : next-step head logits, then the (expert, gate) pairs chosen from them, handed to the chained next step; one set per ring slot
     size_t partial;   // [ring][4(K+1)][H] float  : gate-weighted partial expert outputs of the fused batch-1 kernel, one set per ring slot
+    size_t dep;       // [ring][8] float          : dependent chain: kC partial sums of squares of x + y, then the "next state written" flag
     size_t lone_bytes;// what a batch-1 call that never chains needs: everything up to the first set of partials
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
@@ -117,7 +119,8 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.h = round_up(W.u_gu + (size_t)T * n_sets * 2 * r * sizeof(float), 256);
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.logits = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
-    W.partial = round_up(W.logits + (size_t)kHandoffRing * (d.E + kPairWords) * sizeof(float), 256);
+    W.dep = round_up(W.logits + (size_t)kHandoffRing * (d.E + kPairWords) * sizeof(float), 256);
+    W.partial = round_up(W.dep + (size_t)kHandoffRing * 8 * sizeof(float), 256);
     const size_t one_set = (size_t)kDownSlices * (d.K + 1) * d.H * sizeof(float);   // K routed experts and the shared expert
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);
@@ -145,6 +148,9 @@ int32_t check_desc(const edg_layer_desc* d);   // EDG_OK or EDG_E_INVAL / EDG_E_
 // What the batch-1 layer kernel can do beyond the plain layer-step; all optional.
 struct FusedExtras {
     int32_t* inds_mirror = nullptr;        // [K] copy of inds_next in mapped pinned host memory
+    void* x_next = nullptr;                // [H] bf16: bf16(rmsnorm(x + y)) written by the kernel's last reducer
+    float eps = 1e-6f;
+    int dep_wait = -1;                     // ring slot whose flag announces this step's x (chained dependent steps)
     const void* shared_rec = nullptr;      // device record of the layer's shared expert: runs as one more expert with gate 1
     const edg_lora* shared_lora = nullptr; // its adapter (leading dimension 1), or null
 };

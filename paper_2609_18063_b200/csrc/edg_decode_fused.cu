@@ -149,6 +149,12 @@ struct FusedParams {
     int epc;                      // experts per cluster, one after the other: 1, or 2 or 4 (only with qpc = 4)
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     int32_t* inds_mirror;         // [K] copy of inds_next in mapped pinned host memory, or null
+    uint16_t* x_next;             // [H] bf16 or null: bf16(rmsnorm(x + y)), the next layer-step's hidden state in a dependent chain
+    float* dep_ws;                // [kRing][8]: per ring slot, kC partial sums of squares and (word 4) the "x_next is written" flag
+    int32_t* norm_cnt;            // [kRing] reducers that have delivered their sum of squares
+    float eps;
+    int head_extra;               // CTAs behind those of the experts that evaluate the head and nothing else (0: the first CTAs of the grid do)
+    int dep_wait;                 // -1, or the ring slot whose flag says that this step's x has been written
     const uint8_t* shared_rec;    // record of the layer's always-on shared expert (one more expert with gate 1), or null
     edg_lora shared_lora;         // its own adapter, leading dimension 1 (null pointers with rank_shared == 0)
     int n_shared;                 // 0 or 1
@@ -296,6 +302,25 @@ __device__ __forceinline__ void store_y(void* y, int out_dtype, size_t i, float 
     if (out_dtype == EDG_F32) store_out<float>(static_cast<float*>(y), i, v);
     else if (out_dtype == EDG_F16) store_out<__half>(static_cast<__half*>(y), i, v);
     else store_out<bf16_t>(static_cast<bf16_t*>(y), i, v);
+}
+
+// four consecutive stored outputs (i a multiple of 4) as floats, read past the L1 (another CTA wrote them)
+__device__ __forceinline__ float4 load_y4_cg(const void* y, int out_dtype, size_t i) {
+    if (out_dtype == EDG_F32) return __ldcg(reinterpret_cast<const float4*>(static_cast<const float*>(y) + i));
+    const uint2 w = __ldcg(reinterpret_cast<const uint2*>(static_cast<const unsigned short*>(y) + i));
+    if (out_dtype == EDG_F16) {
+        const float2 a = __half22float2(u32_as_h2(w.x)), b = __half22float2(u32_as_h2(w.y));
+        return make_float4(a.x, a.y, b.x, b.y);
+    }
+    return make_float4(bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y));
+}
+// a value as it reads back after being stored in the output type
+__device__ __forceinline__ float round_out(float v, int out_dtype) {
+    if (out_dtype == EDG_F32) return v;
+    if (out_dtype == EDG_F16) return __half2float(__float2half_rn(v));
+    uint32_t u = __float_as_uint(v);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return __uint_as_float(u & 0xFFFF0000u);
 }
 
 // the same over a bf16 row in global memory (read-only path)
@@ -499,6 +524,12 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     float* partial = p.partial + (size_t)p.ring * kDownSlices * (p.K + 1) * p.H;
     int32_t* counters = p.counters + p.ring * kC;
     trace_mark(p, 0);
+    // A step that produces the next hidden state clears its "written" flag before it releases the
+    // next kernel, which may start polling it at once.
+    if (p.x_next != nullptr && blockIdx.x == 0 && tid == 0) {
+        st_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + 4, 0u);
+        __threadfence();
+    }
     if (tid == 0) pdl_launch_dependents();
     // A call that does not continue a chain runs alone on its workspace: it clears what the last
     // head left unread in the ring.
@@ -511,18 +542,24 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      round-robin to the first CTAs of the grid; a row is split over all threads of its CTA
     //      (8 elements each).
     const int max_pre = (p.pre_dtype == EDG_F16 && p.H <= 2048) ? kMaxPre : kFW;     // two rows per warp only on the fast path below
-    // An fp16 head whose rows split into blocks of 32 goes to the tensor cores: CTA b of the first
-    // E / 32 takes rows 32 b .. 32 b + 31 as two 16-row MMA tiles, warp w computing tile (w & 1) over
-    // K half (w >> 1) with the hidden state as column 0 of the B operand -- an eighth of the
-    // instructions of the FMA form below, and the head is bound by its instructions.
-    const bool pre_mma = p.W_pre != nullptr && p.pre_dtype == EDG_F16 && (p.E % 32) == 0 && (p.H % 512) == 0 &&
-                         p.E / 32 <= (int)gridDim.x && p.qpc == kDownSlices;   // (a step launched alone spreads the rows over more CTAs instead)
-    const int n_head_ctas = p.W_pre == nullptr ? 0 : pre_mma ? p.E / 32 : min((int)gridDim.x, max(32, (p.E + max_pre - 1) / max_pre));
-    const bool head_cta = (int)blockIdx.x < n_head_ctas;
+    // An fp16 head whose rows split into 16-row tiles goes to the tensor cores, the hidden state as
+    // column 0 of the B operand -- an eighth of the instructions of the FMA form below.  A chained step
+    // (few CTAs) gives a head CTA two tiles, each over half of K per warp; a step that runs alone one
+    // tile over a quarter of K per warp, and there the head has CTAs of its own behind those of the
+    // experts (p.head_extra of them, on SMs the experts leave idle), so that no expert waits for it.
+    const int n_expert_ctas = (int)gridDim.x - p.head_extra;
+    const bool head_only = (int)blockIdx.x >= n_expert_ctas;
+    const int head_idx = p.head_extra > 0 ? (int)blockIdx.x - n_expert_ctas : (int)blockIdx.x;
+    const int tpc = p.qpc == kDownSlices ? 2 : 1;                 // tiles per head CTA
+    const int ksplit = kFW / tpc;                                 // warps sharing the K range of a tile
+    const bool pre_mma = p.W_pre != nullptr && p.pre_dtype == EDG_F16 && (p.E % (16 * tpc)) == 0 && (p.H % (256 * ksplit)) == 0 &&
+                         p.E / (16 * tpc) <= (p.head_extra > 0 ? p.head_extra : (int)gridDim.x);
+    const int n_head_ctas = p.W_pre == nullptr ? 0 : pre_mma ? p.E / (16 * tpc) : min((int)gridDim.x, max(32, (p.E + max_pre - 1) / max_pre));
+    const bool head_cta = head_idx >= 0 && head_idx < n_head_ctas;
     const int n_pre = (head_cta && !pre_mma) ? min(max_pre, (p.E - (int)blockIdx.x + n_head_ctas - 1) / n_head_ctas) : 0;
     const bool mma_head = pre_mma && head_cta;
-    const int mrow0 = (int)blockIdx.x * 32 + (warp & 1) * 16;     // first row of this warp's tile
-    const int mk0 = (warp >> 1) * (p.H / 2);                      // first k of this warp's K half
+    const int mrow0 = (head_idx * tpc + warp % tpc) * 16;         // first row of this warp's tile
+    const int mk0 = (warp / tpc) * (p.H / ksplit);                // first k of this warp's share of K
     // Usual case (fp16 head, H <= 2048): warp w evaluates row w of this CTA's rows by itself, each
     // lane covering 8 runs of 8 elements, and publishes it without waiting for any other warp.
     const bool pre_fast = n_pre > 0 && p.pre_dtype == EDG_F16 && p.H <= 2048;
@@ -558,7 +595,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     const bool pre_lane = tid * 8 < p.H;
     uint32_t pre_state = kNotYet, pre_state2 = kNotYet;   // the ring-slot entries this lane will publish into, as the kernel finds them
     if (p.flag_out >= 0) {
-        if (mma_head && warp < 2 && lane < 16)
+        if (mma_head && warp < tpc && lane < 16)
             pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + mrow0 + lane]);
         if (my_row && lane == 0) pre_state = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e]);
         if (my_row2 && lane == 0) pre_state2 = ld_relaxed_gpu_u32(&p.logits_ws[(size_t)p.flag_out * (p.E + kPairWords) + my_e2]);
@@ -594,6 +631,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      (for the zero points).
     if (p.table != nullptr && warp == 0)      // (warp 0 alone: it resolves the routing before the CTA's first barrier)
         for (int i = lane; i < p.E; i += 32) s_table[i] = __ldcg(&p.table[i]);
+    auto convert_x = [&]() {
     for (int t0 = 0; t0 * 8 < p.H; t0 += kFW * 32) {
         const int t = t0 + tid;
         const bool on = t * 8 < p.H;
@@ -617,6 +655,8 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             s_xbias[t / (4 * CPB)] = fmaf(1024.f, sum, 64.f * sodd);
         }
     }
+    };
+    if (p.dep_wait < 0) convert_x();          // (a step that waits for its hidden state converts it once it is there)
     if (tid < kMaxRank) s_ud[tid] = 0.f;
 
     // ---- a3: take, for the experts of this cluster (up to kMaxEpc, one after the other), as a
@@ -707,10 +747,13 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     //      is not chained has its routing in memory: warp 0 issues before its head rows.  Bounded wait; on a
     //      time-out fall back to waiting for the whole previous kernel and to the routing it has
     //      written, which is always sufficient.
+    // A step whose hidden state is still being produced (dependent chain) routes first as well: its
+    // routing is known long before its x, and the first quarter's weights stream in meanwhile.
+    const bool early_route = p.flag_in < 0 || p.dep_wait >= 0;
     bool routed = false;                  // warp 0: routing taken, first copies issued
 #pragma unroll 1
     for (int pass = 0; pass < 2; ++pass) {
-        if (warp == 0 && !routed && (pass || p.flag_in < 0)) {
+        if (warp == 0 && !routed && !head_only && (pass || early_route)) {
             int vi[kMaxEpc], vg[kMaxEpc];
 #pragma unroll
             for (int e = 0; e < kMaxEpc; ++e) { vi[e] = -1; vg[e] = 0; }
@@ -760,7 +803,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 // A step on its own issues the copies of the first quarter here, ahead of its head
                 // rows; in a chained step the other warps are already waiting at the barrier below,
                 // and all four issue their share right behind it, which is quicker.
-                if (valid && p.flag_in < 0) {
+                if (valid && early_route) {
                     issue_gu(0, 0, 0, kFW);
                     if (r > 0) issue_lora(0);
                 }
@@ -769,6 +812,25 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
         }
         if (pass) break;
+        // ---- a dependent step: everything that does not need the hidden state is on its way; now
+        //      wait (bounded) until the step before this one has written it
+        if (p.dep_wait >= 0) {
+            if (tid == 0) {
+                const float* flag = p.dep_ws + p.dep_wait * 8 + 4;
+                uint32_t it = 0, v = 0;
+                do {
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+                    if (v == 0u) __nanosleep(40);
+                } while (v == 0u && ++it < kSpinLimit);
+                if (v == 0u) {                         // never seen: the previous kernel's end is always sufficient
+                    atomicExch(p.status, EDG_E_TIMEOUT);
+                    pdl_wait_prior_grid();
+                }
+                trace_mark(p, 20);
+            }
+            __syncthreads();
+            convert_x();
+        }
         // ---- the head on the tensor cores: 16 rows x this warp's K half, the hidden state as column 0
         //      of B (from s_xb, whose words hold (x0,x4) (x1,x5) (x2,x6) (x3,x7): the natural pairs
         //      the fp16 rows need are byte permutations of them)
@@ -776,7 +838,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             __syncthreads();                               // s_xb is complete (every CTA passes here: the condition is grid-uniform)
             float c[4] = {0.f, 0.f, 0.f, 0.f};
             if (mma_head) {
-                const int nb = p.H / 512;                  // batches of 8 chunks in a K half
+                const int nb = p.H / ksplit / 256;         // batches of 8 chunks in this warp's share of K
 #pragma unroll 1
                 for (int b = 0; b < nb; ++b) {
                     const uint4* xbp = s_xb + (mk0 + b * 256) / 8 + t4;
@@ -795,17 +857,21 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                         }
                     }
                 }
-                // the upper K half hands its 16 sums to the warp of the lower one
-                if (warp >= 2 && t4 == 0) {
-                    s_red[kPreRed * kFW + (warp & 1) * 16 + g8] = c[0];
-                    s_red[kPreRed * kFW + (warp & 1) * 16 + 8 + g8] = c[2];
+                // the warps of the upper K shares hand their 16 sums to the warp of the lowest one
+                // (s_red is free until the adapter projections, behind the next barriers)
+                if (warp >= tpc && t4 == 0) {
+                    s_red[(warp / tpc - 1) * 32 + (warp % tpc) * 16 + g8] = c[0];
+                    s_red[(warp / tpc - 1) * 32 + (warp % tpc) * 16 + 8 + g8] = c[2];
                 }
             }
             __syncthreads();
-            if (mma_head && warp < 2) {
+            if (mma_head && warp < tpc) {
                 // rows g and g + 8 sit in the lanes with t4 == 0; lane L < 16 publishes row L of the tile
-                const float lo_ = c[0] + s_red[kPreRed * kFW + warp * 16 + g8];
-                const float hi_ = c[2] + s_red[kPreRed * kFW + warp * 16 + 8 + g8];
+                float lo_ = c[0], hi_ = c[2];
+                for (int q = 0; q + 1 < ksplit; ++q) {       // fixed order
+                    lo_ += s_red[q * 32 + warp * 16 + g8];
+                    hi_ += s_red[q * 32 + warp * 16 + 8 + g8];
+                }
                 const float v_lo = __shfl_sync(0xFFFFFFFFu, lo_, (lane & 7) * 4);
                 const float v_hi = __shfl_sync(0xFFFFFFFFu, hi_, (lane & 7) * 4);
                 if (warp == 0) trace_mark(p, 12);
@@ -877,6 +943,13 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         }
     }
 
+    // a CTA that is there for the head alone is done (its cluster's handshake completed first)
+    if (head_only) {
+        cluster_wait();
+        trace_mark(p, 9);
+        return;
+    }
+
     // ---- any other head (fp32 weights, wider rows): every row is split over all threads of the CTA
     //      and published by one warp after the barrier below
     if (n_pre > 0 && !pre_fast) {
@@ -898,7 +971,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     }
 
     read_take();
-    if (valid && p.flag_in >= 0) {
+    if (valid && !early_route) {
         issue_gu(0, 0, warp, warp + 1);
         if (warp == kFW - 1 && r > 0) issue_lora(0);
     }
@@ -1226,20 +1299,86 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     // ---- a6: this partial is published; the last arriver for the block of rows sums all partials
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == (int)gridDim.x / kC - 1) ? 1 : 0;   // one arrival per cluster
+    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == n_expert_ctas / kC - 1) ? 1 : 0;   // one arrival per cluster of experts
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
+        // (eight partials in flight per thread and round: this sum is on the critical path of a step that runs alone)
+        float ss = 0.f;
         for (int i = tid; i < rows_d / 4; i += kFW * 32) {
+            uint2 xr = make_uint2(0u, 0u);
+            if (p.x_next != nullptr) xr = *reinterpret_cast<const uint2*>(p.x + n0_d + 4 * i);
             float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 4
-            for (int kk = 0; kk < np; ++kk) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)kk * p.H + n0_d + 4 * i]));
-                yv.x += t.x; yv.y += t.y; yv.z += t.z; yv.w += t.w;
+#pragma unroll 1
+            for (int k0 = 0; k0 < np; k0 += 8) {
+                float4 t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    t[u] = k0 + u < np ? __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)(k0 + u) * p.H + n0_d + 4 * i]))
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { yv.x += t[u].x; yv.y += t[u].y; yv.z += t[u].z; yv.w += t[u].w; }
             }
             store_y4(p.y, p.out_dtype, (size_t)n0_d + 4 * i, yv);
+            if (p.x_next != nullptr) {           // squares of x + y, y as stored (rounded to the output type)
+                const float v0 = bf16_lo(xr.x) + round_out(yv.x, p.out_dtype), v1 = bf16_hi(xr.x) + round_out(yv.y, p.out_dtype);
+                const float v2 = bf16_lo(xr.y) + round_out(yv.z, p.out_dtype), v3 = bf16_hi(xr.y) + round_out(yv.w, p.out_dtype);
+                ss = fmaf(v0, v0, ss); ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
+            }
         }
         if (tid == 0) counters[crank] = 0;
+        if (p.x_next != nullptr) {
+            // ---- the next hidden state of a dependent chain, x_next = bf16(rmsnorm(x + y)): each of the
+            //      kC reducers has summed the squares of its rows, the last one adds the kC sums in a
+            //      fixed order, normalises all H rows and raises the flag the next step waits for.
+            ss = warp_sum(ss);
+            if (lane == 0) s_red[warp] = ss;
+            __syncthreads();                      // (also: this CTA's rows of y are written)
+            if (tid == 0) {
+                float tot = 0.f;
+                for (int w = 0; w < kFW; ++w) tot += s_red[w];
+                st_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + crank, __float_as_uint(tot));
+                __threadfence();
+                s_flag[2] = (atomicAdd(&p.norm_cnt[p.ring], 1) == kC - 1) ? 1 : 0;
+            }
+            __syncthreads();
+            if (s_flag[2]) {
+                __threadfence();
+                // all loads of this thread's 16 elements first, then the arithmetic
+                constexpr int kPer = 4;           // float4 groups per thread for H = 2048 (fewer are active for smaller H)
+                float4 yq[kPer];
+                uint2 xq[kPer];
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) {
+                    const int i4 = (u * kFW * 32 + tid) * 4;
+                    if (i4 < p.H) {
+                        xq[u] = *reinterpret_cast<const uint2*>(p.x + i4);
+                        yq[u] = load_y4_cg(p.y, p.out_dtype, (size_t)i4);
+                    }
+                }
+                float tot = 0.f;
+                for (int c = 0; c < kC; ++c) tot += __uint_as_float(ld_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + c));
+                const float inv = rsqrtf(tot / (float)p.H + p.eps);
+                bf16_t* xn = reinterpret_cast<bf16_t*>(p.x_next);
+#pragma unroll
+                for (int u = 0; u < kPer; ++u) {
+                    const int i4 = (u * kFW * 32 + tid) * 4;
+                    if (i4 < p.H) {
+                        store_out<bf16_t>(xn, i4 + 0, (bf16_lo(xq[u].x) + yq[u].x) * inv);
+                        store_out<bf16_t>(xn, i4 + 1, (bf16_hi(xq[u].x) + yq[u].y) * inv);
+                        store_out<bf16_t>(xn, i4 + 2, (bf16_lo(xq[u].y) + yq[u].z) * inv);
+                        store_out<bf16_t>(xn, i4 + 3, (bf16_hi(xq[u].y) + yq[u].w) * inv);
+                    }
+                }
+                __threadfence();
+                __syncthreads();
+                if (tid == 0) {
+                    p.norm_cnt[p.ring] = 0;
+                    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.dep_ws + p.ring * 8 + 4), "r"(1u) : "memory");
+                    trace_stamp(p, 21);
+                }
+            }
+        }
         if (p.flag_in >= 0) {
             // The last of the kC reducers resets the ring slot this step has taken its logits from.
             // By then every CTA has read them and the reduce scratch of this ring slot is free
@@ -1298,7 +1437,7 @@ static cudaError_t launch_fused(const FusedParams& p, size_t smem, bool pdl, cud
         configured = true;
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.K / p.epc + p.n_shared) * (kDownSlices / p.qpc) * kC, 1, 1);
+    cfg.gridDim = dim3((p.K / p.epc + p.n_shared) * (kDownSlices / p.qpc) * kC + p.head_extra, 1, 1);
     cfg.blockDim = dim3(kFW * 32, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -1353,18 +1492,31 @@ int32_t run_fused_layer(const edg_layer_desc* d, const void* slot_pool, const in
     p.done = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlDone);
     p.ring = ring;
     p.stale = stale;
-    if (extras != nullptr) p.inds_mirror = extras->inds_mirror;
+    p.dep_wait = -1;
+    if (extras != nullptr) {
+        p.inds_mirror = extras->inds_mirror;
+        p.x_next = static_cast<uint16_t*>(extras->x_next);
+        p.eps = extras->eps;
+        p.dep_wait = flag_in >= 0 ? extras->dep_wait : -1;
+    }
+    p.dep_ws = reinterpret_cast<float*>(ws + W.dep);
+    p.norm_cnt = reinterpret_cast<int32_t*>(ws + W.ctrl + kCtrlNorm);
     // a chained step shares the GPU with its neighbours: few, long-lived CTAs; a lone step wants all SMs at once
-    p.qpc = flag_in >= 0 ? kDownSlices : 1;
+    // (a step of a dependent chain runs one after the other however it is launched: all SMs at once too)
+    p.qpc = (flag_in >= 0 && p.dep_wait < 0) ? kDownSlices : 1;
     // ... and when the experts share one adapter a cluster takes two or four experts, one after the other:
     // fewer CTAs per step, each amortising its start-up over more bytes
     const bool fast_head = W_pre == nullptr || (d->pre_dtype == EDG_F16 && d->H <= 2048);   // up to 8 kFW head rows per CTA
     p.epc = 1;
     for (int c = 2; c <= kMaxEpc; c *= 2)
-        if (flag_in >= 0 && d->K % c == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (W_pre == nullptr || (d->K / c) * kC * kMaxPre >= d->E))
+        if (flag_in >= 0 && p.qpc == kDownSlices && d->K % c == 0 && (p.rank == 0 || d->n_adapters == 1) && fast_head && (W_pre == nullptr || (d->K / c) * kC * kMaxPre >= d->E))
             p.epc = c;
     p.flag_in = flag_in;
     p.flag_out = W_pre != nullptr ? flag_out : -1;
+    // a step that runs alone gives an fp16 head CTAs of its own: one 16-row MMA tile each, whole clusters
+    p.head_extra = 0;
+    if (p.qpc == 1 && W_pre != nullptr && d->pre_dtype == EDG_F16 && d->E % 16 == 0 && d->H % 1024 == 0)
+        p.head_extra = (d->E / 16 + kC - 1) / kC * kC;
     const bool pdl = flag_in >= 0;
     const size_t smem = p.S.total;
     cudaError_t e;

@@ -140,6 +140,7 @@ struct edg_store {
     // chaining of consecutive batch-1 layer-steps: when a call consumes the routing that the
     // previous call on the same stream and workspace produced, its kernel is launched as a
     // programmatic dependent of that one and waits on a device flag instead of the kernel's end
+    const void* chain_x_next = nullptr;    // the hidden state the last batch-1 layer-step produces for its successor, or null
     const void* chain_inds = nullptr;
     const void* chain_ws = nullptr;
     void* chain_stream = nullptr;
@@ -561,11 +562,12 @@ extern "C" int32_t edg_store_get_hot_stats(const edg_store* s, edg_hot_stats* ou
     return EDG_OK;
 }
 
-extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
-                                    const int32_t* inds_cur, const float* gates_cur,
-                                    const void* W_pre_next, int32_t* inds_next, float* gates_next,
-                                    float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
-                                    void* workspace, size_t workspace_bytes, void* stream) {
+static int32_t layer_decode(edg_store* s, int32_t layer, const void* x,
+                            const int32_t* inds_cur, const float* gates_cur,
+                            const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                            float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
+                            void* x_next, float eps,
+                            void* workspace, size_t workspace_bytes, void* stream) {
     if (!store_ok(s) || !x || !inds_cur || !gates_cur || !y) return EDG_E_INVAL;
     if (layer < 0 || layer >= s->n_layers) return EDG_E_RANGE;
     if (!s->cuda_engine) return EDG_E_INVAL;               // kernels need the real machine
@@ -630,12 +632,15 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
             const edg::WorkspaceLayout W = edg::workspace_layout(s->d, 1);
             EDG_CUDA_TRY(cudaMemsetAsync(w8 + edg::kCtrlCounters, 0, edg::kCtrlBytes - edg::kCtrlCounters, st));
             EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.logits, 0xFF, (size_t)edg::kHandoffRing * (s->d.E + edg::kPairWords) * sizeof(float), st));
+            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.dep, 0, (size_t)edg::kHandoffRing * 8 * sizeof(float), st));
             s->ring_ws = workspace;
             s->ring_next = 0;
             s->pub_slot = -1;
         }
         const bool chain = chained && !fresh;
         const int flag_in = chain ? s->chain_flag : -1;              // ring slot this step's logits arrive in
+        // a chained step whose x is the state the previous step is still producing waits for it on the device
+        const bool dep_chain = chain && s->chain_x_next != nullptr && s->chain_x_next == x;
         int stale = -1;
         if (!chain && s->pub_slot >= 0) stale = s->pub_slot;         // nobody will read that head's logits
         s->pub_slot = -1;
@@ -644,6 +649,9 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
         s->ring_next = (ring + 1) % edg::kHandoffRing;
         edg::FusedExtras extras;
         extras.inds_mirror = W_pre_next != nullptr ? inds_next_host_mirror_opt : nullptr;
+        extras.x_next = x_next;
+        extras.eps = eps;
+        extras.dep_wait = dep_chain ? flag_in : -1;
         if (!s->shared_rec.empty() && s->shared_rec[layer] != nullptr) {
             extras.shared_rec = s->shared_rec[layer];
             extras.shared_lora = s->shared_has_lora[layer] ? &s->shared_lora[layer] : nullptr;
@@ -659,6 +667,7 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
             EDG_CUDA_TRY(cudaEventRecord(s->step_done, st));
             s->step_done_valid = true;
         }
+        s->chain_x_next = x_next;
         s->chain_inds = W_pre_next != nullptr ? inds_next : nullptr;
         s->chain_ws = workspace;
         s->chain_stream = stream;
@@ -673,7 +682,31 @@ extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
             if (rc != EDG_OK) return rc;
         }
     }
+    if (x_next != nullptr && !edg::fused_supported(s->d)) {
+        rc = edg_next_hidden_state(&s->d, x, y, x_next, eps, stream);
+        if (rc != EDG_OK) return rc;
+    }
     return edg_store_mark_computed(s, layer, stream);
+}
+
+extern "C" int32_t moe_layer_decode(edg_store* s, int32_t layer, const void* x,
+                                    const int32_t* inds_cur, const float* gates_cur,
+                                    const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                                    float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+    return layer_decode(s, layer, x, inds_cur, gates_cur, W_pre_next, inds_next, gates_next, logits_next_opt,
+                        inds_next_host_mirror_opt, y, nullptr, 0.f, workspace, workspace_bytes, stream);
+}
+
+extern "C" int32_t moe_layer_decode_dependent(edg_store* s, int32_t layer, const void* x,
+                                              const int32_t* inds_cur, const float* gates_cur,
+                                              const void* W_pre_next, int32_t* inds_next, float* gates_next,
+                                              float* logits_next_opt, int32_t* inds_next_host_mirror_opt, void* y,
+                                              void* x_next, float eps,
+                                              void* workspace, size_t workspace_bytes, void* stream) {
+    if (!x_next || !edg::aligned(x_next, 16) || x_next == x) return EDG_E_INVAL;
+    return layer_decode(s, layer, x, inds_cur, gates_cur, W_pre_next, inds_next, gates_next, logits_next_opt,
+                        inds_next_host_mirror_opt, y, x_next, eps, workspace, workspace_bytes, stream);
 }
 
 extern "C" int32_t edg_stack_decode_token(edg_store* s, const void* x, const int32_t* inds_cur, const float* gates_cur,

@@ -45,10 +45,11 @@ def test_chained_steps_in_flight_match_oracle_and_unchained(name, steps, stride)
     ws = layer_io.new_workspace(d)
     inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, xd, steps, ws, True)
     inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, xd, steps, ws, False)
-    # integer work is bit-exact between the two launch modes, floats agree far inside the tolerance
+    # the routing is the same in both launch modes, floats agree far inside the tolerance
     assert np.array_equal(inds_c, inds_u)
-    assert np.array_equal(logits_c, logits_u)
-    assert np.array_equal(gates_c, gates_u)
+    # (the two launch forms split a head row's K range differently: same logits up to fp32 rounding)
+    assert np.abs(logits_c - logits_u).max() <= 1e-5
+    assert np.abs(gates_c - gates_u).max() <= 1e-5
     assert np.abs(y_c - y_u).max() <= 1e-4
     experts = {}
     get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
@@ -138,7 +139,7 @@ def test_default_policy_gives_the_same_results_whether_or_not_steps_overlap():
     for mode, sync_each in [(1, True), (1, False), (2, True)]:
         got = run(mode, sync_each)
         assert np.array_equal(got[0], ref[0])
-        assert np.array_equal(got[1], ref[1])
+        assert np.abs(got[1] - ref[1]).max() <= 1e-5
         assert np.abs(got[2] - ref[2]).max() <= 1e-4
     store.close()
 
@@ -163,7 +164,7 @@ def test_chained_small_layer_with_an_fp16_head(per_expert_adapters):
     ws = layer_io.new_workspace(d)
     inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, xd, steps, ws, True)
     inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, xd, steps, ws, False)
-    assert np.array_equal(inds_c, inds_u) and np.array_equal(logits_c, logits_u) and np.array_equal(gates_c, gates_u)
+    assert np.array_equal(inds_c, inds_u) and np.abs(logits_c - logits_u).max() <= 1e-5 and np.abs(gates_c - gates_u).max() <= 1e-5
     assert np.abs(y_c - y_u).max() <= 1e-4
     experts, adapters = {}, {}
     get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))

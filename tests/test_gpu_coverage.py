@@ -62,7 +62,7 @@ def test_fused_kernel_shapes_chained_and_alone(H, I, group, pre):
     ws = layer_io.new_workspace(d)
     inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, x_dev(X), steps, ws, True)
     inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, x_dev(X), steps, ws, False)
-    assert np.array_equal(inds_c, inds_u) and np.array_equal(logits_c, logits_u)
+    assert np.array_equal(inds_c, inds_u) and np.abs(logits_c - logits_u).max() <= 1e-5
     assert np.abs(y_c - y_u).max() <= 1e-4
     _check_steps(cfg, X, W_np, inds_c, gates_c, logits_c, y_c, range(steps))
     store.close()
@@ -195,6 +195,6 @@ def test_chained_steps_wrap_the_hand_off_ring(name, steps, stride):
     # a second lap on the same workspace, not chained this time, continues from the ring where it stands
     # (step 0 is routed from another "last prompt" state in the shorter run: compare from step 1)
     inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, x_dev(X), 140, ws, False)
-    assert np.array_equal(inds_u[1:], inds[1:141]) and np.array_equal(logits_u[1:], logits[1:141])
+    assert np.array_equal(inds_u[1:], inds[1:141]) and np.abs(logits_u[1:] - logits[1:141]).max() <= 1e-5
     assert np.abs(y_u[1:] - y[1:140]).max() <= 1e-4
     store.close()

@@ -144,3 +144,58 @@ def test_exposed_wait_measurement_counts_the_waits_it_brackets():
     assert n == staged_with_copies and n >= 1 and 0.0 <= ms < 1000.0
     assert store.exposed_wait_ms() == (0.0, 0)                       # reading resets
     store.close()
+
+
+@pytest.mark.parametrize("name,steps,chaining,out_dtype", [("cfg1", 300, 2, "f32"), ("cfg2", 40, 2, "f32"), ("cfg1", 40, 0, "f32"),
+                                                          ("cfg2", 12, 1, "f32"), ("cfg1", 30, 2, "f16"), ("cfg1", 30, 2, "bf16")])
+def test_dependent_chain_with_the_state_produced_inside_the_layer_kernel(name, steps, chaining, out_dtype):
+    """moe_layer_decode_dependent: the kernel's last reducer writes x(t+1) itself, and with chaining on
+    step t+1 is already resident, has its routing and its first weights, and waits on a device flag
+    for x(t+1).  No host synchronisation inside the loop (300 steps wrap the 128-slot ring twice).
+    Step-local parity against the oracle on the GPU's own x(t)."""
+    cfg = synth.CONFIGS[name]
+    d_out = edg.make_desc(cfg, n_slots=cfg.E, out_dtype=out_dtype)
+    store, d, hosts, slots, tables, cs, _ = _make_store(cfg, n_slots=cfg.E)
+    store.close()
+    # (a store whose descriptor carries the output type under test)
+    loras = [layer_io.lora_to_device(d_out, [synth.lora_tensors(cfg, 0, a) for a in range(cfg.n_adapters)])]
+    store = edg.Store(d_out, hosts, slots, tables, [loras[0][0]], cs)
+    d = d_out
+    for e0 in range(0, cfg.E, 64):
+        edg.stage_experts_to_slots(store, 0, np.arange(e0, min(cfg.E, e0 + 64), dtype=np.int32))
+    torch.cuda.synchronize()
+    store.set_chaining(chaining)
+    W_np = synth.prerouter_weights(cfg)
+    W = torch.from_numpy(W_np).cuda()
+    x0 = synth.hidden_states(cfg, 2, stream=65)
+    xs = torch.zeros((steps + 1, cfg.H), dtype=torch.bfloat16, device="cuda")
+    xs[0] = x_dev(x0[0])
+    inds = torch.zeros((steps + 1, cfg.K), dtype=torch.int32, device="cuda")
+    gates = torch.zeros((steps + 1, cfg.K), dtype=torch.float32, device="cuda")
+    logits = torch.zeros((steps + 1, cfg.E), dtype=torch.float32, device="cuda")
+    ydt = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}[out_dtype]
+    y = torch.zeros((steps, cfg.H), dtype=ydt, device="cuda")
+    ws = layer_io.new_workspace(d)
+    edg.prerouter_topk(d, W, x_dev(x0[1]), 1, inds[0], gates[0], logits[0])
+    for t in range(steps):
+        edg.moe_layer_decode_dependent(store, 0, xs[t], inds[t], gates[t], W, inds[t + 1], gates[t + 1], logits[t + 1],
+                                       y[t], xs[t + 1], ws, 1e-6)
+    torch.cuda.synchronize()
+    assert edg.workspace_status(ws) == 0
+    X = xs.view(torch.int16).cpu().numpy().view(np.uint16)
+    ih, gh, lh = inds.cpu().numpy(), gates.cpu().numpy(), logits.cpu().numpy()
+    yh = y.float().cpu().numpy()
+    experts = {}
+    get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
+    lora = synth.lora_tensors(cfg, 0, 0)
+    check = range(steps) if name == "cfg1" else sorted(set(range(0, steps, 5)) | {steps - 1})
+    for t in range(steps):
+        _check_routing(lh[t + 1], ih[t + 1], gh[t + 1], W_np.astype(np.float32), X[t], cfg.K)
+        want = orc.next_hidden_state(X[t], yh[t].astype(np.float64), 1e-6)      # from the GPU's own stored y: step-local
+        assert _bf16_ulps(X[t + 1], want).max() <= 1, t
+        assert (X[t + 1] == want).mean() > 0.98
+        if t in check and out_dtype != "bf16":
+            ref = orc.moe_ffn(X[t], ih[t], gh[t].astype(np.float64), get, lambda e: lora, cfg.lora_scale, cfg.group)
+            _assert_close(yh[t], ref)
+    assert len({tuple(r) for r in ih.tolist()}) > min(steps // 2, 60)       # (cfg1 has only 120 possible routings)
+    store.close()

@@ -48,7 +48,7 @@ def test_shared_expert_in_the_layer_step(name, routed_lora, shared_lora, steps):
     ws = layer_io.new_workspace(d)
     inds_c, gates_c, logits_c, y_c = _run(cfg, store, d, W, x_dev(X), steps, ws, True)      # chained: steps in flight
     inds_u, gates_u, logits_u, y_u = _run(cfg, store, d, W, x_dev(X), steps, ws, False)     # each step alone
-    assert np.array_equal(inds_c, inds_u) and np.array_equal(logits_c, logits_u)
+    assert np.array_equal(inds_c, inds_u) and np.abs(logits_c - logits_u).max() <= 1e-5
     assert np.abs(y_c - y_u).max() <= 1e-4
     experts = {}
     get = lambda e: experts.setdefault(e, synth.expert_tensors(cfg, 0, e))
