@@ -179,6 +179,9 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
 // L2 policies: expert weights are read once per step and must not push the small tensors that
 // every step reuses (adapters, head, hidden state) out of the L2.
 __device__ __forceinline__ uint64_t policy_evict_first() {
@@ -721,6 +724,23 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
         }
     };
+    // A step that waits for its hidden state has time to spare: it asks the L2 for the rest of its
+    // first item (second half of K, down block), so that those loads later come from the L2.
+    auto prefetch_rest = [&](int w) {
+        const int c = c0 + w % p.qpc;
+        const uint8_t* rec = item_rec(w);
+        if (lane < 4 * TG) {
+            const int mt = lane >> 1, is_sz = lane & 1, m = mt / TG, ti = mt % TG;
+            const int n = c * sw + crank * rows_gu + 16 * ti;
+            // (K quarters 2 and 3 of a (matrix, row tile) follow each other in memory: one run of twice the size)
+            if (!is_sz) bulk_prefetch_l2(rec + (m ? p.L.codes_up : p.L.codes_gate) + code_off(p.H, n, 2 * cps), 2 * S.mat_codes);
+            else bulk_prefetch_l2(rec + (m ? p.L.sz_up : p.L.sz_gate) + sz_off(p.H, p.group, n, 2 * gpst), 2 * S.mat_sz);
+        } else if (lane == 4 * TG) {
+            bulk_prefetch_l2(rec + p.L.codes_down + down_code_off(p.H, p.I, n0_d, c * (sw / 32)), (uint32_t)rows_d * sw / 2);
+        } else if (lane == 4 * TG + 1) {
+            bulk_prefetch_l2(rec + p.L.sz_down + down_sz_off(p.H, p.I, p.group, n0_d, c * gps), (uint32_t)rows_d * gps * 4);
+        }
+    };
     // One warp issues the adapter slices of item w into buffer w & 1: this CTA's rows of B_gate and
     // B_up for the item's quarter, and its columns of A_down (one 16-byte-multiple run per rank index).
     auto issue_lora = [&](int w) {
@@ -806,6 +826,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 if (valid && early_route) {
                     issue_gu(0, 0, 0, kFW);
                     if (r > 0) issue_lora(0);
+                    if (p.dep_wait >= 0) prefetch_rest(0);
                 }
                 trace_mark(p, 1);
                 routed = true;
@@ -984,6 +1005,10 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         //      row per sweep; the loads of up to 8 rows are in flight together, so the share costs one
         //      trip to memory.
         const int per = (2 * r + kC - 1) / kC;
+        // (a step that has waited for its hidden state finds its first weights landed: it starts on
+        // them at once and computes these projections while the second half of K is on its way)
+        const bool late_ax = p.dep_wait >= 0;
+        auto lora_ax = [&]() {
         if (r > 0) {
 #pragma unroll 1
             for (int q0 = 0; q0 < per; q0 += 8) {
@@ -1027,6 +1052,8 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             }
         }
         trace_mark(p, 2);
+        };
+        if (!late_ax) lora_ax();
 
         // ---- the four quarters of the intermediate dimension, one after the other.  For quarter c
         //      this CTA computes its rows_gu gate/up rows (over all of K), the cluster exchanges
@@ -1101,6 +1128,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                     if (half == 0) {
                         __syncthreads();
                         issue_gu(w, 1, warp, warp + 1);
+                        if (late_ax && w == 0) lora_ax();
                     }
                 }
                 if (t4 == 0) {
@@ -1303,21 +1331,21 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     __syncthreads();
     if (s_flag[0]) {
         __threadfence();
-        // (eight partials in flight per thread and round: this sum is on the critical path of a step that runs alone)
+        // (sixteen partials in flight per thread and round: this sum is on the critical path of a step that runs alone)
         float ss = 0.f;
         for (int i = tid; i < rows_d / 4; i += kFW * 32) {
             uint2 xr = make_uint2(0u, 0u);
             if (p.x_next != nullptr) xr = *reinterpret_cast<const uint2*>(p.x + n0_d + 4 * i);
             float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-            for (int k0 = 0; k0 < np; k0 += 8) {
-                float4 t[8];
+            for (int k0 = 0; k0 < np; k0 += 16) {
+                float4 t[16];
 #pragma unroll
-                for (int u = 0; u < 8; ++u)
+                for (int u = 0; u < 16; ++u)
                     t[u] = k0 + u < np ? __ldcg(reinterpret_cast<const float4*>(&partial[(size_t)(k0 + u) * p.H + n0_d + 4 * i]))
                                        : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) { yv.x += t[u].x; yv.y += t[u].y; yv.z += t[u].z; yv.w += t[u].w; }
+                for (int u = 0; u < 16; ++u) { yv.x += t[u].x; yv.y += t[u].y; yv.z += t[u].z; yv.w += t[u].w; }
             }
             store_y4(p.y, p.out_dtype, (size_t)n0_d + 4 * i, yv);
             if (p.x_next != nullptr) {           // squares of x + y, y as stored (rounded to the output type)
