@@ -97,6 +97,8 @@ struct WorkspaceLayout {
     size_t lone_bytes;// what a batch-1 call that never chains needs: everything up to the first set of partials
     // grouped path (T > 1) only:
     size_t o;         // [T*K][H] float             : gate-weighted output of every (token, choice) pair
+    size_t o_part;    // [T*K][4][H] float          : the same per quarter of the intermediate dimension (small groups only)
+    size_t xt;        // [T*K/8 + n_slots] tile records of the streaming small-group kernel: x fragments, block sums, projections, pair table
     size_t pair_slot; // [T*K] int32                : resolved slot of every pair (-1: skipped)
     size_t pair_ad;   // [T*K] int32                : adapter of every pair
     size_t counts;    // [n_slots] int32            : pairs per slot
@@ -124,10 +126,17 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     const size_t one_set = (size_t)kDownSlices * (d.K + 1) * d.H * sizeof(float);   // K routed experts and the shared expert
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);
+    W.o_part = W.xt = end;
     W.o = W.pair_slot = W.pair_ad = W.counts = W.n_tiles = W.tiles = W.lists = W.hq = W.xq = end;
     if (T > 1) {
         const size_t P = (size_t)T * d.K;
         W.o = end;                 end = round_up(W.o + P * d.H * sizeof(float), 256);
+        const bool small = P <= 8 * (size_t)d.n_slots;
+        W.o_part = end;            end = round_up(W.o_part + (small ? P * 4 * d.H * sizeof(float) : 0), 256);
+        // a tile record: 8 tokens of fp16 state, two sums per 32 activations and token, 2 x rank projections per token, pair table
+        const size_t rr = d.rank > 0 ? (size_t)d.rank : 8;
+        const size_t tile_rec = (size_t)8 * d.H * 2 + 2 * 8 * (size_t)(d.H / 32) * 4 + 8 * 2 * rr * 4 + 128;
+        W.xt = end;                end = round_up(W.xt + (small ? (P / 8 + 1 + d.n_slots) * tile_rec : 0), 256);
         W.pair_slot = end;         end = round_up(W.pair_slot + P * 4, 256);
         W.pair_ad = end;           end = round_up(W.pair_ad + P * 4, 256);
         W.counts = end;            end = round_up(W.counts + (size_t)d.n_slots * 4, 256);

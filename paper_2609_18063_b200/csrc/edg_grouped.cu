@@ -466,6 +466,10 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     build_tiles_kernel<<<1, 1024, 0, st>>>(p);
     if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 0, st);
 
+    // small groups on the shapes the batch-1 kernel covers: one streaming kernel for the whole FFN
+    if (small && grouped_stream_supported(*d))
+        return run_grouped_stream(d, p, reinterpret_cast<float*>(ws + W.o_part), ws + W.xt, max_tiles, st);
+
     const int ng = G_KC / d->group, ngd = G_KD / d->group;
     const size_t sm_gu = (size_t)p.ntok * G_XS + 2 * 128 * G_CS + 2 * 128 * ng * 4 + p.ntok * 4;
     const size_t sm_d = (size_t)2 * p.ntok * G_XSD + 256 * G_CSD + 256 * ngd * 4 + p.ntok * 4;

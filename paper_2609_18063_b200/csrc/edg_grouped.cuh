@@ -40,4 +40,8 @@ bool umma_grouped_supported(const edg_layer_desc& d);
 cudaError_t launch_umma_gate_up(const GroupedParams& p, int max_tiles, cudaStream_t st);
 cudaError_t launch_umma_down(const GroupedParams& p, int max_tiles, cudaStream_t st);
 
+// streaming path for small groups (batched decode): tiles of 8 tokens through the batch-1 kernel's pipeline
+bool grouped_stream_supported(const edg_layer_desc& d);
+int32_t run_grouped_stream(const edg_layer_desc* d, const GroupedParams& g, float* o_part, uint8_t* xt, int max_tiles, cudaStream_t st);
+
 }  // namespace edg
