@@ -30,7 +30,9 @@ constexpr int SMaxRank = 64;
 struct StreamSmem {
     uint32_t stage0, stage_bytes, mat_codes, mat_sz, sz0, d_codes, d_sz;
     uint32_t lora0, lora_bytes;
-    uint32_t bars, xb, xsum, xbias, part, gu, hloc, h, hb, hsum, hbias, u, udp, ud, info, rec_bytes, total;
+    uint32_t bars, part, gu, hloc, h, hb, hsum, hbias, u, udp, ud, info, total;
+    // the tile record in global memory (pre-pass): x fragments, block sums, then what an item copies in: projections, pair table
+    uint32_t g_xsum, g_xbias, g_u, g_small, g_bytes;
 };
 
 // byte offsets, identical on host and device (rows_gu = I/16 gate/up rows per CTA and matrix, rows_d = H/4, sw = I/4)
@@ -49,14 +51,17 @@ __host__ __device__ inline StreamSmem stream_smem(int H, int I, int group, int r
     S.lora0 = o;   o += 2 * S.lora_bytes;
     o = (o + 15) / 16 * 16;
     S.bars = o;    o += 8 * 8;
-    // the tile record as the pre-pass writes it, one bulk copy per item: x fragments, block sums, adapter projections
+    // The tile record as the pre-pass writes it: [token][H/8] uint4 x as fp16 B words in k-slot order, [block][token]
+    // sums (plain, and as the biased codes weigh them) -- these are read by the MMA loops straight from the L2 -- then
+    // [token][2][rank] projections and the pair table, which an item copies into shared memory.
     const uint32_t rr = rank > 0 ? (uint32_t)rank : 8u;
-    S.xb = o;      o += ST * (uint32_t)H * 2;                 // [token][H/8] uint4: x as fp16 B words, k-slot order
-    S.xsum = o;    o += ST * (uint32_t)(H / 32) * 4;          // [block][token]
-    S.xbias = o;   o += ST * (uint32_t)(H / 32) * 4;
-    S.u = o;       o += ST * 2 * rr * 4;                      // [token][2][rank]: A_gate x, A_up x
-    S.rec_bytes = o - S.xb;
-    S.info = o;    o += 2 * 128;                              // two buffers of [8] pair, [8] gate, [8] adapter, [8] token
+    S.g_xsum = ST * (uint32_t)H * 2;
+    S.g_xbias = S.g_xsum + ST * (uint32_t)(H / 32) * 4;
+    S.g_u = S.g_xbias + ST * (uint32_t)(H / 32) * 4;
+    S.g_small = ST * 2 * rr * 4 + 128;                        // projections + pair table
+    S.g_bytes = S.g_u + S.g_small;
+    S.u = o;       o += 2 * S.g_small;                        // two buffers of ([token][2][rank] projections, [8] pair, [8] gate, [8] adapter, [8] token)
+    S.info = S.u + ST * 2 * rr * 4;
     S.part = o;    o += SW_ * 2 * rows_gu * ST * 4;           // [warp][2 rows_gu][token]
     S.gu = o;      o += 2 * rows_gu * ST * 4;                 // [2 rows_gu][token]
     S.hloc = o;    o += rows_gu * ST * 4;                     // [rows_gu][token]
@@ -104,7 +109,7 @@ __device__ __forceinline__ void lora_bwords(const float* v, int kr, int rank, in
 }
 
 template <int NCW, int DCH, int TG, int TD, int CPB>
-__global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __grid_constant__ StreamParams sp) {
+__global__ void __launch_bounds__(SW_ * 32, 3) grouped_stream_kernel(const __grid_constant__ StreamParams sp) {
     extern __shared__ __align__(128) uint8_t smem[];
     const GroupedParams& p = sp.g;
     const StreamSmem& S = sp.S;
@@ -116,9 +121,6 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
     const int cps = p.H / 128, gpst = (p.H / 4) >> sp.gshift, gps = sw >> sp.gshift;
 
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S.bars);
-    uint4* s_xb = reinterpret_cast<uint4*>(smem + S.xb);             // [ST][H/8]
-    float* s_xsum = reinterpret_cast<float*>(smem + S.xsum);         // [block][ST]
-    float* s_xbias = reinterpret_cast<float*>(smem + S.xbias);
     float* s_part = reinterpret_cast<float*>(smem + S.part);         // [warp][2 rows_gu][ST]
     float* s_gu = reinterpret_cast<float*>(smem + S.gu);             // [2 rows_gu][ST]
     float* s_hloc = reinterpret_cast<float*>(smem + S.hloc);         // [rows_gu][ST]
@@ -126,10 +128,9 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
     uint4* s_hb = reinterpret_cast<uint4*>(smem + S.hb);             // [chunk][2][ST][4]
     float* s_hsum = reinterpret_cast<float*>(smem + S.hsum);         // [block][ST]
     float* s_hbias = reinterpret_cast<float*>(smem + S.hbias);
-    float* s_u = reinterpret_cast<float*>(smem + S.u);               // [ST][2][r]
     float* s_udp = reinterpret_cast<float*>(smem + S.udp);           // [2][SC][ST][r]
     float* s_ud = reinterpret_cast<float*>(smem + S.ud);             // [ST][r]
-    const size_t xt_stride = (size_t)S.rec_bytes + 128;
+    const size_t xt_stride = S.g_bytes;
 
     const int n_items = 4 * *p.n_tiles;
     const int my_items = cl < n_items ? (n_items - cl + n_cl - 1) / n_cl : 0;
@@ -193,9 +194,8 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
     auto issue_x = [&](int j) {
         if (warp == SW_ - 2 && lane == 2) {
             const uint8_t* src = sp.xt + (size_t)((cl + j * n_cl) >> 2) * xt_stride;
-            mbar_expect_tx(&bars[SB_X], S.rec_bytes + 128);
-            bulk_g2s(smem + S.xb, src, S.rec_bytes, &bars[SB_X]);
-            bulk_g2s(smem + S.info + (j & 1) * 128, src + S.rec_bytes, 128, &bars[SB_X]);
+            mbar_expect_tx(&bars[SB_X], S.g_small);
+            bulk_g2s(smem + S.u + (j & 1) * S.g_small, src + S.g_u, S.g_small, &bars[SB_X]);
         }
     };
     issue_gu(0, 0);
@@ -212,7 +212,9 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
         // ---- the tile's pairs, their tokens' states as the B operand (fp16, k-slot order), block sums
         // ---- the tile's record (pairs, their tokens' states as the B operand, block sums, projections) has been on its way
         mbar_wait(&bars[SB_X], par, p.status);
-        const int* s_pair = reinterpret_cast<const int*>(smem + S.info + par * 128);      // [8] pair, [8] gate bits, [8] adapter, [8] token
+        const float* s_u = reinterpret_cast<const float*>(smem + S.u + par * S.g_small);                // [ST][2][r]
+        const int* s_pair = reinterpret_cast<const int*>(smem + S.info + par * S.g_small);   // [8] pair, [8] gate bits, [8] adapter, [8] token
+        const uint8_t* trec = sp.xt + (size_t)tile * xt_stride;                               // the tile's x fragments and sums, in the L2
         const int* s_gate = s_pair + 8;
         const int ad = s_pair[16];
         // ---- gate/up: warp w owns K slice w of each half for every (matrix, row tile); 8 token columns
@@ -227,15 +229,30 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
                 const int vw = warp + SW_ * half;
+                // this warp's B words of the half (token g8) and the block sums of its two tokens: asked for before the
+                // wait for the weights, so both trips overlap
+                uint4 xbw[NCW];
+                float2 xsw[NCW / CPB], xbw2[NCW / CPB];
+                {
+                    const uint4* xbp = reinterpret_cast<const uint4*>(trec) + g8 * (p.H / 8) + (vw * NCW) * 4 + t4;
+#pragma unroll
+                    for (int i = 0; i < NCW; ++i) xbw[i] = __ldg(xbp + i * 4);
+                    const float* xsp = reinterpret_cast<const float*>(trec + S.g_xsum) + ((vw * NCW) / CPB) * ST + 2 * t4;
+                    const float* xbp2 = reinterpret_cast<const float*>(trec + S.g_xbias) + ((vw * NCW) / CPB) * ST + 2 * t4;
+#pragma unroll
+                    for (int i = 0; i < NCW / CPB; ++i) {
+                        xsw[i] = __ldg(reinterpret_cast<const float2*>(xsp + i * ST));
+                        xbw2[i] = __ldg(reinterpret_cast<const float2*>(xbp2 + i * ST));
+                    }
+                }
                 mbar_wait(&bars[s], half, p.status);
-                const uint4* xbp = s_xb + g8 * (p.H / 8) + (vw * NCW) * 4 + t4;
-#pragma unroll 1
+#pragma unroll
                 for (int ib = 0; ib < NCW / CPB; ++ib) {
                     float cfr[NT][4];
 #pragma unroll
                     for (int u = 0; u < CPB; ++u) {
                         const int i = ib * CPB + u;
-                        const uint4 xb = xbp[i * 4];
+                        const uint4 xb = xbw[i];
 #pragma unroll
                         for (int mt = 0; mt < NT; ++mt) {
                             const uint8_t* cw = cbase + mt * S.mat_codes + i * 256;
@@ -248,9 +265,7 @@ __global__ void __launch_bounds__(SW_ * 32, 2) grouped_stream_kernel(const __gri
                         }
                     }
                     const int gi = ((ch0 + ib * CPB) * 32) >> sp.gshift;
-                    const int blk = (vw * NCW) / CPB + ib;
-                    const float2 xs = *reinterpret_cast<const float2*>(&s_xsum[blk * ST + 2 * t4]);
-                    const float2 xbi = *reinterpret_cast<const float2*>(&s_xbias[blk * ST + 2 * t4]);
+                    const float2 xs = xsw[ib], xbi = xbw2[ib];
 #pragma unroll
                     for (int mt = 0; mt < NT; ++mt) {
                         const uint8_t* zw = st + S.sz0 + mt * S.mat_sz + gi * 64 + g8 * 4;
@@ -511,12 +526,12 @@ __global__ void __launch_bounds__(256) stream_tile_kernel(StreamParams sp) {
     if (tile >= *p.n_tiles) return;
     const int slot = p.tiles[2 * tile], first = p.tiles[2 * tile + 1];
     const int cnt = min(ST, p.counts[slot] - first);
-    uint8_t* rec = sp.xt + (size_t)tile * ((size_t)S.rec_bytes + 128);
+    uint8_t* rec = sp.xt + (size_t)tile * S.g_bytes;
     uint4* xb = reinterpret_cast<uint4*>(rec);
-    float* xsum = reinterpret_cast<float*>(rec + (S.xsum - S.xb));
-    float* xbias = reinterpret_cast<float*>(rec + (S.xbias - S.xb));
-    float* u = reinterpret_cast<float*>(rec + (S.u - S.xb));
-    int* info = reinterpret_cast<int*>(rec + S.rec_bytes);
+    float* xsum = reinterpret_cast<float*>(rec + S.g_xsum);
+    float* xbias = reinterpret_cast<float*>(rec + S.g_xbias);
+    float* u = reinterpret_cast<float*>(rec + S.g_u);
+    int* info = reinterpret_cast<int*>(rec + S.g_u + S.g_small - 128);
     __shared__ int s_pr[ST];
     const int tid = threadIdx.x;
     if (tid < ST) {
@@ -581,7 +596,7 @@ __global__ void __launch_bounds__(256) reduce_parts_kernel(StreamParams sp) {
     store_out<OutT>(reinterpret_cast<OutT*>(p.y), i, v);
 }
 
-constexpr size_t kStreamSmemLimit = 113 * 1024;    // two CTAs per SM
+constexpr size_t kStreamSmemLimit = 113 * 1024;    // two CTAs per SM at the largest ranks, three up to rank 16
 
 bool grouped_stream_supported(const edg_layer_desc& d) {
     if (!((d.H == 1024 || d.H == 2048) && (d.I == 256 || d.I == 512))) return false;
@@ -656,6 +671,6 @@ int32_t run_grouped_stream(const edg_layer_desc* d, const GroupedParams& g, floa
 
 namespace edg {
 size_t grouped_stream_tile_bytes(const edg_layer_desc& d) {
-    return (size_t)stream_smem(d.H, d.I, d.group, d.rank).rec_bytes + 128;
+    return stream_smem(d.H, d.I, d.group, d.rank).g_bytes;
 }
 }  // namespace edg
