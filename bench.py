@@ -50,7 +50,7 @@ UNIT = "tok/s"
 WORKLOAD = "cfg2: one 35B-class MoE layer (H2048 I512 E256 top-8 int4 g64 LoRA r16), batch-1 decode"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from an ncu
 # capture of this workload (not measured by this run: reported as "from profile").
-NCU_TRAFFIC_BYTES = 15_591_424
+NCU_TRAFFIC_BYTES = 15_621_120
 WINDOWS = 5            # timed windows; the median is reported
 WINDOW_STEPS = 2560    # layer-steps per window: ten replays of a 256-step graph
 
