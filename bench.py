@@ -52,7 +52,7 @@ WORKLOAD = "cfg2: one 35B-class MoE layer (H2048 I512 E256 top-8 int4 g64 LoRA r
 # capture of this workload (not measured by this run: reported as "from profile").
 NCU_TRAFFIC_BYTES = 15_621_120
 WINDOWS = 5            # timed windows; the median is reported
-WINDOW_STEPS = 2560    # layer-steps per window: ten replays of a 256-step graph
+WINDOW_STEPS = 2560    # layer-steps per window: one replay of a 2560-step graph
 
 
 def _peaks():
@@ -196,8 +196,9 @@ def run_b200(args):
     edg.prerouter_topk(desc, W[0], xd[NX - 1], 1, inds[0], gates[0], None)
     torch.cuda.synchronize()
 
-    G = NX                                 # steps per CUDA graph
-    if G % n_inst or n_inst % 2 and n_inst != 1:
+    G = WINDOW_STEPS                       # steps per CUDA graph: a window is one replay
+    G_DEP = 256                            # the dependent arms: nothing overlaps across steps, so the graph size is immaterial
+    if NX % n_inst or n_inst % 2 and n_inst != 1:
         raise SystemExit("--instances must be even (or 1) and divide 256")
     stream = torch.cuda.Stream()
     stream.wait_stream(torch.cuda.current_stream())
@@ -219,12 +220,14 @@ def run_b200(args):
 
     steps, warmup = args.steps, max(args.warmup, 3)
     # The hand-off ring has 128 slots and a captured chain has its slots baked in, so a graph that is
-    # replayed again and again holds a multiple of 128 steps: one graph of 256 steps, replayed.
+    # replayed again and again holds a multiple of 128 steps.  A replay is stream-ordered behind the
+    # one before it, so the chain drains and refills once per replay (about half the lifetime of a
+    # CTA, 0.1 ms): the graph holds a whole window of 2560 steps (64 tokens x 40 layers' worth), not 256.
     store.set_chaining(1)                  # opt in: the captured steps are chained through the routing
     g_full = capture(G)
     reps = WINDOW_STEPS // G
 
-    def timed_windows(graph):
+    def timed_windows(graph, reps=reps):
         """WINDOWS windows of `reps` replays each, one event pair per window; ms per window, max over ranks."""
         out = []
         with torch.cuda.stream(stream):
@@ -285,11 +288,11 @@ def run_b200(args):
         g_dep = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             with torch.cuda.graph(g_dep, stream=stream):
-                for s_ in range(G):
+                for s_ in range(G_DEP):
                     dep_step(s_)
             g_dep.replay()
             stream.synchronize()
-        dep_ms = statistics.median(timed_windows(g_dep))
+        dep_ms = statistics.median(timed_windows(g_dep, WINDOW_STEPS // G_DEP))
         status = edg.workspace_status(ws)
         if status != 0 or not bool(torch.isfinite(ydep).all()) or not bool(torch.isfinite(xdep.float()).all()):
             raise SystemExit(f"bench: dependent arm: bad device status {status} or non-finite state")
@@ -310,11 +313,11 @@ def run_b200(args):
         g_dep2 = torch.cuda.CUDAGraph()
         with torch.cuda.stream(stream):
             with torch.cuda.graph(g_dep2, stream=stream):
-                for s_ in range(G):
+                for s_ in range(G_DEP):
                     dep2_step(s_)
             g_dep2.replay()
             stream.synchronize()
-        dep2_ms = statistics.median(timed_windows(g_dep2))
+        dep2_ms = statistics.median(timed_windows(g_dep2, WINDOW_STEPS // G_DEP))
         status = edg.workspace_status(ws)
         if status != 0 or not bool(torch.isfinite(ydep).all()) or not bool(torch.isfinite(xdep.float()).all()):
             raise SystemExit(f"bench: fused dependent arm: bad device status {status} or non-finite state")
@@ -326,7 +329,7 @@ def run_b200(args):
                      "frac_of_peak": round(K * R / (dep2_step_ms * 1e-3) / 1e9 / _peaks()[0], 4),
                      "dependency": "x(t+1) = bf16(rmsnorm(x(t) + y(t))) computed on the device: every step waits for the one before it",
                      "launch": f"moe_layer_decode_dependent: one kernel per step writes y and x(t+1); steps chained (the next step "
-                               f"is resident, routed and streaming its first weights while it waits for x); CUDA graphs of {G} steps",
+                               f"is resident, routed and streaming its first weights while it waits for x); CUDA graphs of {G_DEP} steps",
                      "unchained_two_kernels": {"ms_per_step": round(dep_step_ms, 6),
                                                "value": round(replicas.whole_job_rate(world, WINDOW_STEPS, dep_ms), 1),
                                                "launch": "layer-step + next-state norm as two stream-ordered kernels, chaining off"},

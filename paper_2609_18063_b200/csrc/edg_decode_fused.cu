@@ -341,6 +341,7 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
     if (p.E <= 256) warp_softmax_topk_reg<8>(work, p.E, p.K, lane, s_i, s_g);
     else topk_large(work, p.E, p.K, lane, s_i, s_g);
     __syncwarp();
+    if (lane == 0) trace_stamp(p, 25);
     if (lane < p.K) {
         // the hand-off proper, first: (expert, gate) as one word per choice behind the logits of the
         // ring slot, released after everything the publishers of the logits had observed.  The
@@ -348,6 +349,7 @@ __device__ __noinline__ void head_publish(const FusedParams& p, uint8_t* smem, f
         // after this warp has long finished with the logits.
         if (p.flag_out >= 0) {
             __threadfence();
+            if (lane == 0) trace_stamp(p, 26);
             st_relaxed_gpu_u64(reinterpret_cast<unsigned long long*>(logits_ws + p.E) + lane,
                                ((unsigned long long)__float_as_uint(s_g[lane]) << 32) | (uint32_t)s_i[lane]);
         }
