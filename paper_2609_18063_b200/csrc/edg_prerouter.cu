@@ -201,12 +201,16 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_kernel(PrePar
 }
 
 // The same for an fp16 head on the tensor cores: the block's 8 tokens are the 8 columns of an
-// m16n8k16 tile, 16 rows of the head its rows.  A CTA takes its share of the rows tile by tile; warp
-// w multiplies K slice w of every tile (A fragments straight from memory: the 16 k of a step are one
-// full 32-byte sector per row; B fragments from the tokens' states, fp16 in shared memory, rows
-// padded by 16 bytes so the eight token rows fall into different banks), the slices are summed
-// through shared memory, and the logits go to the leader as above.  fp16 of a bf16 state is exact in
-// the normal range; products are exact in fp32 and summed in fp32.
+// m16n8k16 tile, 16 rows of the head its rows.  A CTA takes its share of the rows two tiles at a
+// time; warp w multiplies K slice w of both.  Operands are fetched 16 bytes at a time: lane (g, t4)
+// reads k = 8 t4 .. 8 t4 + 7 of every 32-k block, of head rows g and g + 8 (straight from memory) and
+// of token g (fp16 in shared memory, rows padded by 64 bytes against bank conflicts), and feeds words
+// 0, 1 of each to one MMA and words 2, 3 to a second one -- a permutation of k that A and B share, so
+// the dot products are unchanged.  All loads of a warp's slice are issued before the first MMA (one
+// trip to memory); the slices are summed through shared memory, and the logits go to the leader as
+// above.  fp16 of a bf16 state is exact in the normal range; products are exact in fp32 and summed
+// in fp32.
+constexpr int kMmaHeadKs = 256;        // k per warp and pass: 8 blocks of 32
 __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(PreParams p, int T) {
     cg::cluster_group cluster = cg::this_cluster();
     const int crank = (int)cluster.block_rank();
@@ -216,51 +220,57 @@ __global__ void __launch_bounds__(kPreWarps * 32) prerouter_tokens_mma_kernel(Pr
     extern __shared__ float smem[];
     float* s_logits = smem;                                             // [kTokBlock][E]
     float* s_red = smem + kTokBlock * p.E;                              // [kPreWarps][2 x 16 x 8] partial tiles
-    const int xs = p.H * 2 + 16;                                        // bytes per token row
-    uint8_t* s_xh = reinterpret_cast<uint8_t*>(s_red + kPreWarps * 256);    // [kTokBlock][H + 8] fp16
-    for (int tt = 0; tt < kTokBlock; ++tt) {
-        const int t = t0 + tt;
-        for (int i = threadIdx.x; i < p.H; i += blockDim.x)
-            *reinterpret_cast<__half*>(s_xh + tt * xs + i * 2) = __float2half_rn(t < T ? bf16_bits_to_float(p.s[(size_t)t * p.H + i]) : 0.f);
+    const int xs = p.H * 2 + 64;                                        // bytes per token row
+    uint8_t* s_xh = reinterpret_cast<uint8_t*>(s_red + kPreWarps * 256);    // [kTokBlock][H + 32] fp16
+    const __half* W = static_cast<const __half*>(p.W);
+    const int per = p.E / csize;                                        // rows of this CTA: a multiple of 16
+    const int ksl = p.H / kPreWarps;                                    // k per warp: a multiple of 32
+
+    // the head rows of the first pass are on their way while the tokens' states are converted
+    uint4 a[2][kMmaHeadKs / 32][2];
+    auto load_a = [&](int r0, int k0, bool two) {
+#pragma unroll
+        for (int tile = 0; tile < 2; ++tile) {
+            const __half* w = W + (size_t)(r0 + (two ? 16 * tile : 0) + g) * p.H + warp * ksl + k0 + 8 * t4;
+#pragma unroll
+            for (int j = 0; j < kMmaHeadKs / 32; ++j) {
+                const bool on = k0 + 32 * j < ksl;
+                a[tile][j][0] = on ? ld_stream16(w + 32 * j) : make_uint4(0, 0, 0, 0);
+                a[tile][j][1] = on ? ld_stream16(w + (size_t)8 * p.H + 32 * j) : make_uint4(0, 0, 0, 0);
+            }
+        }
+    };
+    const int r_first = crank * per;
+    load_a(r_first, 0, r_first + 16 < (crank + 1) * per);
+    for (int i = threadIdx.x; i < kTokBlock * (p.H / 8); i += blockDim.x) {
+        const int tt = i / (p.H / 8), c = i % (p.H / 8), t = t0 + tt;
+        uint4 o = make_uint4(0, 0, 0, 0);
+        if (t < T) {
+            const uint4 v = *reinterpret_cast<const uint4*>(p.s + (size_t)t * p.H + c * 8);
+            o.x = h2_as_u32(__floats2half2_rn(bf16_lo(v.x), bf16_hi(v.x)));
+            o.y = h2_as_u32(__floats2half2_rn(bf16_lo(v.y), bf16_hi(v.y)));
+            o.z = h2_as_u32(__floats2half2_rn(bf16_lo(v.z), bf16_hi(v.z)));
+            o.w = h2_as_u32(__floats2half2_rn(bf16_lo(v.w), bf16_hi(v.w)));
+        }
+        *reinterpret_cast<uint4*>(s_xh + tt * xs + c * 16) = o;
     }
     __syncthreads();
 
     float* leader = cluster.map_shared_rank(s_logits, 0);
-    const int per = p.E / csize;                                        // rows of this CTA: a multiple of 16
-    const int ksl = p.H / kPreWarps;                                    // k per warp: a multiple of 16
-    const __half* W = static_cast<const __half*>(p.W);
-    // two row tiles at a time: twice the loads in flight for the same B fragments
-    for (int r0 = crank * per; r0 < (crank + 1) * per; r0 += 32) {
+    for (int r0 = r_first; r0 < (crank + 1) * per; r0 += 32) {
         const bool two = r0 + 16 < (crank + 1) * per;
-        const __half* wlo = W + (size_t)(r0 + g) * p.H + warp * ksl + 2 * t4;
-        const __half* whi = wlo + (size_t)8 * p.H;
-        const __half* vlo = two ? wlo + (size_t)16 * p.H : wlo;
-        const __half* vhi = vlo + (size_t)8 * p.H;
-        const uint8_t* xb = s_xh + g * xs + (warp * ksl + 2 * t4) * 2;
+        const uint8_t* xb = s_xh + g * xs + (warp * ksl + 8 * t4) * 2;
         float c[4] = {0.f, 0.f, 0.f, 0.f}, d[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int k0 = 0; k0 < ksl; k0 += 64) {                          // four steps' worth of loads in flight per tile
-            uint32_t a[4][4], b[4][4];
+        for (int k0 = 0; k0 < ksl; k0 += kMmaHeadKs) {
+            if (k0 > 0 || r0 > r_first) load_a(r0, k0, two);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int k = k0 + 16 * u;
-                const bool on = k < ksl;
-                a[u][0] = on ? ld_stream4(wlo + k) : 0u;
-                a[u][1] = on ? ld_stream4(whi + k) : 0u;
-                a[u][2] = on ? ld_stream4(wlo + k + 8) : 0u;
-                a[u][3] = on ? ld_stream4(whi + k + 8) : 0u;
-                b[u][0] = on ? ld_stream4(vlo + k) : 0u;
-                b[u][1] = on ? ld_stream4(vhi + k) : 0u;
-                b[u][2] = on ? ld_stream4(vlo + k + 8) : 0u;
-                b[u][3] = on ? ld_stream4(vhi + k + 8) : 0u;
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int k = k0 + 16 * u;
-                if (k < ksl) {
-                    const uint32_t b0 = *reinterpret_cast<const uint32_t*>(xb + k * 2);
-                    const uint32_t b1 = *reinterpret_cast<const uint32_t*>(xb + k * 2 + 16);
-                    mma16816(c, a[u][0], a[u][1], a[u][2], a[u][3], b0, b1);
-                    mma16816(d, b[u][0], b[u][1], b[u][2], b[u][3], b0, b1);
+            for (int j = 0; j < kMmaHeadKs / 32; ++j) {
+                if (k0 + 32 * j < ksl) {
+                    const uint4 b = *reinterpret_cast<const uint4*>(xb + (k0 + 32 * j) * 2);
+                    mma16816(c, a[0][j][0].x, a[0][j][1].x, a[0][j][0].y, a[0][j][1].y, b.x, b.y);
+                    mma16816(c, a[0][j][0].z, a[0][j][1].z, a[0][j][0].w, a[0][j][1].w, b.z, b.w);
+                    mma16816(d, a[1][j][0].x, a[1][j][1].x, a[1][j][0].y, a[1][j][1].y, b.x, b.y);
+                    mma16816(d, a[1][j][0].z, a[1][j][1].z, a[1][j][0].w, a[1][j][1].w, b.z, b.w);
                 }
             }
         }
@@ -573,8 +583,8 @@ int32_t run_prerouter(const edg_layer_desc* d, const void* W_pre, const void* s,
         }
         if (cfg.dynamicSmemBytes > 200 * 1024) return EDG_E_SHAPE;
         // an fp16 head whose rows and columns split into whole MMA tiles goes to the tensor cores
-        if (d->pre_dtype == EDG_F16 && d->E % (16 * kPreCluster) == 0 && d->H % (16 * kPreWarps) == 0) {
-            cfg.dynamicSmemBytes = (size_t)kTokBlock * d->E * 4 + kPreWarps * 256 * 4 + (size_t)kTokBlock * (d->H * 2 + 16);
+        if (d->pre_dtype == EDG_F16 && d->E % (16 * kPreCluster) == 0 && d->H % (32 * kPreWarps) == 0) {
+            cfg.dynamicSmemBytes = (size_t)kTokBlock * d->E * 4 + kPreWarps * 256 * 4 + (size_t)kTokBlock * (d->H * 2 + 64);
             EDG_CUDA_TRY(cudaLaunchKernelEx(&cfg, prerouter_tokens_mma_kernel, p, (int)n_heads));
             return EDG_OK;
         }
