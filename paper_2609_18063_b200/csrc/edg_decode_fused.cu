@@ -1217,19 +1217,22 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 for (int i = tid; i < rows_d; i += kFW * 32) partial[((size_t)(k + e) * nq + cq) * p.H + n0_d + i] = 0.f;
     }
 
-    // ---- a6: this partial is published; the last arriver for the block of rows sums all partials
-    __threadfence();
+    // ---- a6: this partial is published; the last arriver for the block of rows sums all partials.
+    //      The counting atomic of thread 0, behind the CTA's barrier, releases the partial rows of all its
+    //      threads and, in the last arriver, acquires everyone else's (read past the L1 below).
     __syncthreads();
-    if (tid == 0) s_flag[0] = (atomicAdd(&counters[crank], 1) == n_expert_ctas / kC - 1) ? 1 : 0;   // one arrival per cluster of experts
+    if (tid == 0) s_flag[0] = (atom_add_acq_rel_gpu(&counters[crank], 1) == n_expert_ctas / kC - 1) ? 1 : 0;   // one arrival per cluster of experts
     __syncthreads();
     if (s_flag[0]) {
-        __threadfence();
-        // (sixteen partials in flight per thread and round: this sum is on the critical path of a step that runs alone)
+        // (sixteen partials in flight per thread and round: this sum is on the critical path of a step that runs alone;
+        //  a thread owns one group of four rows: rows_d / 4 <= 128)
+        const int i = tid;
+        const bool on = i < rows_d / 4;
+        uint2 xr = make_uint2(0u, 0u);
+        float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
         float ss = 0.f;
-        for (int i = tid; i < rows_d / 4; i += kFW * 32) {
-            uint2 xr = make_uint2(0u, 0u);
+        if (on) {
             if (p.x_next != nullptr) xr = *reinterpret_cast<const uint2*>(p.x + n0_d + 4 * i);
-            float4 yv = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
             for (int k0 = 0; k0 < np; k0 += 16) {
                 float4 t[16];
@@ -1241,63 +1244,53 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 for (int u = 0; u < 16; ++u) { yv.x += t[u].x; yv.y += t[u].y; yv.z += t[u].z; yv.w += t[u].w; }
             }
             store_y4(p.y, p.out_dtype, (size_t)n0_d + 4 * i, yv);
-            if (p.x_next != nullptr) {           // squares of x + y, y as stored (rounded to the output type)
-                const float v0 = bf16_lo(xr.x) + round_out(yv.x, p.out_dtype), v1 = bf16_hi(xr.x) + round_out(yv.y, p.out_dtype);
-                const float v2 = bf16_lo(xr.y) + round_out(yv.z, p.out_dtype), v3 = bf16_hi(xr.y) + round_out(yv.w, p.out_dtype);
-                ss = fmaf(v0, v0, ss); ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
+            if (p.x_next != nullptr) {           // x + y with y as stored (rounded to the output type), and its squares
+                yv.x = bf16_lo(xr.x) + round_out(yv.x, p.out_dtype); yv.y = bf16_hi(xr.x) + round_out(yv.y, p.out_dtype);
+                yv.z = bf16_lo(xr.y) + round_out(yv.z, p.out_dtype); yv.w = bf16_hi(xr.y) + round_out(yv.w, p.out_dtype);
+                ss = fmaf(yv.x, yv.x, ss); ss = fmaf(yv.y, yv.y, ss); ss = fmaf(yv.z, yv.z, ss); ss = fmaf(yv.w, yv.w, ss);
             }
         }
         if (tid == 0) counters[crank] = 0;
         if (p.x_next != nullptr) {
-            // ---- the next hidden state of a dependent chain, x_next = bf16(rmsnorm(x + y)): each of the
-            //      kC reducers has summed the squares of its rows, the last one adds the kC sums in a
-            //      fixed order, normalises all H rows and raises the flag the next step waits for.
+            // ---- the next hidden state of a dependent chain, x_next = bf16(rmsnorm(x + y)).  Each of the kC
+            //      reducers sums the squares of its rows, publishes the sum, waits (bounded) until all kC
+            //      sums are there -- the reducers are running CTAs that publish before they wait --, adds
+            //      them in a fixed order and normalises the rows it still holds in registers.  The last one
+            //      to have written its rows raises the flag the next step waits for.
+            int32_t* norm_done = reinterpret_cast<int32_t*>(p.dep_ws + p.ring * 8 + 5);
             ss = warp_sum(ss);
             if (lane == 0) s_red[warp] = ss;
-            __syncthreads();                      // (also: this CTA's rows of y are written)
+            __syncthreads();
             if (tid == 0) {
                 float tot = 0.f;
                 for (int w = 0; w < kFW; ++w) tot += s_red[w];
                 st_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + crank, __float_as_uint(tot));
-                __threadfence();
-                s_flag[2] = (atomicAdd(&p.norm_cnt[p.ring], 1) == kC - 1) ? 1 : 0;
+                int seen = atom_add_acq_rel_gpu(&p.norm_cnt[p.ring], 1) + 1;
+                uint32_t it = 0;
+                while (seen < kC && ++it < kSpinLimit) {
+                    __nanosleep(20);
+                    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(p.norm_cnt + p.ring) : "memory");
+                }
+                if (seen < kC) atomicExch(p.status, EDG_E_TIMEOUT);
+                float all = 0.f;
+                for (int c = 0; c < kC; ++c) all += __uint_as_float(ld_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + c));
+                s_red[kFW] = rsqrtf(all / (float)p.H + p.eps);
             }
             __syncthreads();
-            if (s_flag[2]) {
-                __threadfence();
-                // all loads of this thread's 16 elements first, then the arithmetic
-                constexpr int kPer = 4;           // float4 groups per thread for H = 2048 (fewer are active for smaller H)
-                float4 yq[kPer];
-                uint2 xq[kPer];
-#pragma unroll
-                for (int u = 0; u < kPer; ++u) {
-                    const int i4 = (u * kFW * 32 + tid) * 4;
-                    if (i4 < p.H) {
-                        xq[u] = *reinterpret_cast<const uint2*>(p.x + i4);
-                        yq[u] = load_y4_cg(p.y, p.out_dtype, (size_t)i4);
-                    }
-                }
-                float tot = 0.f;
-                for (int c = 0; c < kC; ++c) tot += __uint_as_float(ld_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + c));
-                const float inv = rsqrtf(tot / (float)p.H + p.eps);
-                bf16_t* xn = reinterpret_cast<bf16_t*>(p.x_next);
-#pragma unroll
-                for (int u = 0; u < kPer; ++u) {
-                    const int i4 = (u * kFW * 32 + tid) * 4;
-                    if (i4 < p.H) {
-                        store_out<bf16_t>(xn, i4 + 0, (bf16_lo(xq[u].x) + yq[u].x) * inv);
-                        store_out<bf16_t>(xn, i4 + 1, (bf16_hi(xq[u].x) + yq[u].y) * inv);
-                        store_out<bf16_t>(xn, i4 + 2, (bf16_lo(xq[u].y) + yq[u].z) * inv);
-                        store_out<bf16_t>(xn, i4 + 3, (bf16_hi(xq[u].y) + yq[u].w) * inv);
-                    }
-                }
-                __threadfence();
-                __syncthreads();
-                if (tid == 0) {
-                    p.norm_cnt[p.ring] = 0;
-                    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.dep_ws + p.ring * 8 + 4), "r"(1u) : "memory");
-                    trace_stamp(p, 21);
-                }
+            if (on) {
+                const float inv = s_red[kFW];
+                bf16_t* xn = reinterpret_cast<bf16_t*>(p.x_next) + n0_d + 4 * i;
+                store_out<bf16_t>(xn, 0, yv.x * inv);
+                store_out<bf16_t>(xn, 1, yv.y * inv);
+                store_out<bf16_t>(xn, 2, yv.z * inv);
+                store_out<bf16_t>(xn, 3, yv.w * inv);
+            }
+            __syncthreads();                      // this CTA's rows of the next state are written
+            if (tid == 0 && atom_add_acq_rel_gpu(norm_done, 1) == kC - 1) {
+                st_relaxed_gpu(p.norm_cnt + p.ring, 0);
+                st_relaxed_gpu(norm_done, 0);
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.dep_ws + p.ring * 8 + 4), "r"(1u) : "memory");
+                trace_stamp(p, 21);
             }
         }
         if (p.flag_in >= 0) {
