@@ -47,7 +47,7 @@ def bf16_to_f64(bits) -> np.ndarray:
 
 
 def f64_to_bf16_bits(v) -> np.ndarray:
-    """Nearest-even rounding of float64 values to bf16 bit patterns (used to judge a bf16 store)."""
+    """Nearest-even rounding of float64 values to bf16 bit patterns (used to check a bf16 store)."""
     v = np.asarray(v, dtype=np.float64)
     a = np.abs(v)
     # Going through float32 would round twice, so pick the nearest of the three bf16

@@ -187,7 +187,7 @@ def test_ffn_output_dtypes(out_dtype):
     if out_dtype == "f16":
         _assert_close(y.float().cpu().numpy(), ref)
     else:
-        # judged against the oracle rounded to bf16: the stored value is that rounding, or its
+        # compared with the oracle rounded to bf16: the stored value is that rounding, or its
         # neighbour where the fp32 result sits next to a rounding boundary
         got_bits = y.view(torch.int16).cpu().numpy().view(np.uint16)
         want_bits = orc.f64_to_bf16_bits(ref)
