@@ -118,6 +118,26 @@ def test_batched_head_with_fp32_weights():
     assert decided >= T - 2
 
 
+@pytest.mark.parametrize("H,E,K,T", [(2048, 256, 8, 20), (1024, 128, 4, 13), (1024, 256, 8, 64), (512, 128, 2, 9)])
+def test_batched_head_with_fp16_weights_on_mma_tiles(H, E, K, T):
+    """prerouter_topk_tokens with an fp16 head (MMA tiles, 16-byte operand loads under a shared k
+    permutation): logits of every token against the oracle, ragged last block of tokens, one and two
+    row tiles per CTA (E = 128 / 256), K slices of 64, 128 and 256 per warp (H = 512, 1024, 2048)."""
+    cfg = dataclasses.replace(synth.CONFIGS["cfg2"], H=H, E=E, K=K, pre_dtype="f16")
+    d = edg.make_desc(cfg, n_slots=E)
+    assert d.pre_dtype == edg.F16
+    W_np = synth.prerouter_weights(cfg)
+    S = synth.hidden_states(cfg, T, stream=57)
+    inds = torch.full((T, K), -1, dtype=torch.int32, device="cuda")
+    gates = torch.zeros((T, K), dtype=torch.float32, device="cuda")
+    logits = torch.zeros((T, E), dtype=torch.float32, device="cuda")
+    edg.prerouter_topk_tokens(d, torch.from_numpy(W_np).cuda(), x_dev(S), T, inds, gates, logits)
+    torch.cuda.synchronize()
+    decided = sum(_check_routing(logits[t].cpu().numpy(), inds[t].cpu().numpy(), gates[t].cpu().numpy(),
+                                 W_np.astype(np.float32), S[t], K) for t in range(T))
+    assert decided >= T - 2
+
+
 # ------------------------------------------------------------------ zero points that are not integers
 
 class _FractionalZeroLayer(DeviceLayer):
