@@ -430,7 +430,9 @@ int32_t moe_expert_ffn_int4_lora_static(const edg_layer_desc* desc, const void* 
  * on the stream between the two calls.  Callers that cannot promise this leave chaining off
  * (the default).  A chain captured in a CUDA graph that is replayed back to back
  * must hold a multiple of 128 layer-steps, so that every replay finds the ring where the
- * previous one left it. */
+ * previous one left it.  A replay is ordered behind the one before it like any other work on the
+ * stream, so the chain of overlapping steps drains and refills once per replay (about half the
+ * lifetime of a CTA): capture long chains (thousands of steps), not short ones. */
 int32_t moe_layer_decode(edg_store* store, int32_t layer, const void* x,
                          const int32_t* inds_cur, const float* gates_cur,
                          const void* W_pre_next, int32_t* inds_next, float* gates_next,
