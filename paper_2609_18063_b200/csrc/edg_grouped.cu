@@ -464,7 +464,8 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     resolve_pairs_kernel<<<(P + 255) / 256, 256, 0, st>>>(p);
     build_lists_kernel<<<d->n_slots, kListWarps * 32, 0, st>>>(p);
     build_tiles_kernel<<<1, 1024, 0, st>>>(p);
-    if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 0, st);
+    if (has_lora && !launch_lora_ax_tokens(d, x, lora, p.u_gu, T, st))
+        launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 0, st);
 
     // small groups on the shapes the batch-1 kernel covers: one streaming kernel for the whole FFN
     if (small && grouped_stream_supported(*d))
@@ -484,7 +485,8 @@ int32_t run_grouped(const edg_layer_desc* d, const void* slot_pool, int32_t T, c
     if (umma) EDG_CUDA_TRY(launch_umma_gate_up(p, max_tiles, st));
     else if (small) grouped_gate_up_kernel<1><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
     else grouped_gate_up_kernel<8><<<dim3(max_tiles, d->I / 128), G_WARPS * 32, sm_gu, st>>>(p);
-    if (has_lora) launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 1, st);
+    if (has_lora && !launch_lora_adh_pairs(d, lora, p.h, p.u_d, P, st))
+        launch_lora_a(d, slots, table, experts, x, lora, p.u_gu, p.h, p.u_d, p.status, T, 1, st);
     if (umma) EDG_CUDA_TRY(launch_umma_down(p, max_tiles, st));
     else if (small) grouped_down_kernel<1><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);
     else grouped_down_kernel<8><<<dim3(max_tiles, d->H / 256), G_WARPS * 32, sm_d, st>>>(p);

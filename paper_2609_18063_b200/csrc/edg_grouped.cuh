@@ -44,4 +44,8 @@ cudaError_t launch_umma_down(const GroupedParams& p, int max_tiles, cudaStream_t
 bool grouped_stream_supported(const edg_layer_desc& d);
 int32_t run_grouped_stream(const edg_layer_desc* d, const GroupedParams& g, float* o_part, uint8_t* xt, int max_tiles, cudaStream_t st);
 
+// adapter projections for many tokens / pairs on the tensor cores (one shared adapter); false = shape not covered
+bool launch_lora_ax_tokens(const edg_layer_desc* d, const void* x, const edg_lora* lora, float* u_gu, int T, cudaStream_t st);
+bool launch_lora_adh_pairs(const edg_layer_desc* d, const edg_lora* lora, const float* h, float* u_d, int P, cudaStream_t st);
+
 }  // namespace edg
