@@ -79,6 +79,7 @@ __host__ __device__ inline RecordLayout record_layout(int H, int I, int group) {
 // delivered, reducers finished -- one set per ring slot).
 constexpr int kPairWords = 64;         // words behind the logits of a ring slot: 32 (expert, gate) pairs, the routing itself
 constexpr int kHandoffRing = 128;      // ring slots shared by chained batch-1 layer-steps in flight
+constexpr int kDepWords = 16;           // words per ring slot of the dependent chain: 4 sums of squares, 4 "rows written" flags, a counter
 constexpr size_t kCtrlBytes = 4096;    // control block: status word at 0, then the ring's counters
 constexpr size_t kCtrlCounters = 64;                               // [ring][4] arrivals per block of output rows
 constexpr size_t kCtrlHead = kCtrlCounters + kHandoffRing * 16;    // [ring] head rows delivered
@@ -122,7 +123,7 @@ inline WorkspaceLayout workspace_layout(const edg_layer_desc& d, int T) {
     W.u_d = round_up(W.h + (size_t)T * d.K * d.I * sizeof(float), 256);
     W.logits = round_up(W.u_d + (size_t)T * d.K * r * sizeof(float), 256);
     W.dep = round_up(W.logits + (size_t)kHandoffRing * (d.E + kPairWords) * sizeof(float), 256);
-    W.partial = round_up(W.dep + (size_t)kHandoffRing * 8 * sizeof(float), 256);
+    W.partial = round_up(W.dep + (size_t)kHandoffRing * kDepWords * sizeof(float), 256);
     const size_t one_set = (size_t)kDownSlices * (d.K + 1) * d.H * sizeof(float);   // K routed experts and the shared expert
     W.lone_bytes = W.partial + one_set;
     size_t end = round_up(W.partial + (size_t)kHandoffRing * one_set, 256);

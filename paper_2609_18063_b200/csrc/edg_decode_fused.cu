@@ -150,7 +150,7 @@ struct FusedParams {
     int stale;                    // -1, or a ring slot whose unread logits this (unchained) call clears
     int32_t* inds_mirror;         // [K] copy of inds_next in mapped pinned host memory, or null
     uint16_t* x_next;             // [H] bf16 or null: bf16(rmsnorm(x + y)), the next layer-step's hidden state in a dependent chain
-    float* dep_ws;                // [kRing][8]: per ring slot, kC partial sums of squares and (word 4) the "x_next is written" flag
+    float* dep_ws;                // [kRing][kDepWords]: per ring slot, kC partial sums of squares, (words 4..7) the reducers' "my rows of x_next are written" flags, (word 8) a counter
     int32_t* norm_cnt;            // [kRing] reducers that have delivered their sum of squares
     float eps;
     int head_extra;               // CTAs behind those of the experts that evaluate the head and nothing else (0: the first CTAs of the grid do)
@@ -423,7 +423,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
     // A step that produces the next hidden state clears its "written" flag before it releases the
     // next kernel, which may start polling it at once.
     if (p.x_next != nullptr && blockIdx.x == 0 && tid == 0) {
-        st_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + 4, 0u);
+        for (int c = 0; c < kC; ++c) st_relaxed_gpu_u32(p.dep_ws + p.ring * kDepWords + 4 + c, 0u);
         __threadfence();
     }
     if (tid == 0) pdl_launch_dependents();
@@ -729,18 +729,22 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
         // ---- a dependent step: everything that does not need the hidden state is on its way; now
         //      wait (bounded) until the step before this one has written it
         if (p.dep_wait >= 0) {
-            if (tid == 0) {
-                const float* flag = p.dep_ws + p.dep_wait * 8 + 4;
+            if (warp == 0) {
+                // one flag per reducer of the step before (its rows of the state are written): lane c polls flag c
+                const float* flag = p.dep_ws + p.dep_wait * kDepWords + 4 + (lane < kC ? lane : 0);
                 uint32_t it = 0, v = 0;
+                bool all = false;
                 do {
                     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-                    if (v == 0u) __nanosleep(40);
-                } while (v == 0u && ++it < kSpinLimit);
-                if (v == 0u) {                         // never seen: the previous kernel's end is always sufficient
+                    all = __all_sync(0xFFFFFFFFu, v != 0u);
+                    if (!all) __nanosleep(40);
+                } while (!all && ++it < kSpinLimit);
+                if (!all && lane == 0) {               // never seen: the previous kernel's end is always sufficient
                     atomicExch(p.status, EDG_E_TIMEOUT);
                     pdl_wait_prior_grid();
                 }
-                trace_mark(p, 20);
+                __syncwarp();
+                if (lane == 0) trace_mark(p, 20);
             }
             __syncthreads();
             convert_x();
@@ -1257,14 +1261,14 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
             //      sums are there -- the reducers are running CTAs that publish before they wait --, adds
             //      them in a fixed order and normalises the rows it still holds in registers.  The last one
             //      to have written its rows raises the flag the next step waits for.
-            int32_t* norm_done = reinterpret_cast<int32_t*>(p.dep_ws + p.ring * 8 + 5);
+            int32_t* norm_done = reinterpret_cast<int32_t*>(p.dep_ws + p.ring * kDepWords + 8);
             ss = warp_sum(ss);
             if (lane == 0) s_red[warp] = ss;
             __syncthreads();
             if (tid == 0) {
                 float tot = 0.f;
                 for (int w = 0; w < kFW; ++w) tot += s_red[w];
-                st_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + crank, __float_as_uint(tot));
+                st_relaxed_gpu_u32(p.dep_ws + p.ring * kDepWords + crank, __float_as_uint(tot));
                 int seen = atom_add_acq_rel_gpu(&p.norm_cnt[p.ring], 1) + 1;
                 uint32_t it = 0;
                 while (seen < kC && ++it < kSpinLimit) {
@@ -1273,7 +1277,7 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 }
                 if (seen < kC) atomicExch(p.status, EDG_E_TIMEOUT);
                 float all = 0.f;
-                for (int c = 0; c < kC; ++c) all += __uint_as_float(ld_relaxed_gpu_u32(p.dep_ws + p.ring * 8 + c));
+                for (int c = 0; c < kC; ++c) all += __uint_as_float(ld_relaxed_gpu_u32(p.dep_ws + p.ring * kDepWords + c));
                 s_red[kFW] = rsqrtf(all / (float)p.H + p.eps);
             }
             __syncthreads();
@@ -1286,11 +1290,15 @@ __global__ void __launch_bounds__(kFW * 32, 4) fused_layer_kernel(const __grid_c
                 store_out<bf16_t>(xn, 3, yv.w * inv);
             }
             __syncthreads();                      // this CTA's rows of the next state are written
-            if (tid == 0 && atom_add_acq_rel_gpu(norm_done, 1) == kC - 1) {
-                st_relaxed_gpu(p.norm_cnt + p.ring, 0);
-                st_relaxed_gpu(norm_done, 0);
-                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.dep_ws + p.ring * 8 + 4), "r"(1u) : "memory");
+            if (tid == 0) {
+                // (the release covers the rows every thread of this CTA wrote before the barrier)
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.dep_ws + p.ring * kDepWords + 4 + crank), "r"(1u) : "memory");
                 trace_stamp(p, 21);
+                // off the critical path: the last reducer past the exchange of sums resets its counters
+                if (atom_add_acq_rel_gpu(norm_done, 1) == kC - 1) {
+                    st_relaxed_gpu(p.norm_cnt + p.ring, 0);
+                    st_relaxed_gpu(norm_done, 0);
+                }
             }
         }
         if (p.flag_in >= 0) {

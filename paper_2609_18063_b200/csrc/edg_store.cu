@@ -632,7 +632,7 @@ static int32_t layer_decode(edg_store* s, int32_t layer, const void* x,
             const edg::WorkspaceLayout W = edg::workspace_layout(s->d, 1);
             EDG_CUDA_TRY(cudaMemsetAsync(w8 + edg::kCtrlCounters, 0, edg::kCtrlBytes - edg::kCtrlCounters, st));
             EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.logits, 0xFF, (size_t)edg::kHandoffRing * (s->d.E + edg::kPairWords) * sizeof(float), st));
-            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.dep, 0, (size_t)edg::kHandoffRing * 8 * sizeof(float), st));
+            EDG_CUDA_TRY(cudaMemsetAsync(w8 + W.dep, 0, (size_t)edg::kHandoffRing * edg::kDepWords * sizeof(float), st));
             s->ring_ws = workspace;
             s->ring_next = 0;
             s->pub_slot = -1;
